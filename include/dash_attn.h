@@ -1,0 +1,166 @@
+/*
+ * dash_attn.h -- C ABI of the DashAttention forward pass for NVIDIA B200 (sm_100a).
+ *
+ * The forward pass has three stages (paper Section 3):
+ *   Stage 0  chunk summaries          kbar_c = softmax(<qbar, k_t>/sqrt(d))-weighted mean of the B keys
+ *                                     of chunk c                                   (Eq. 3, Algorithm 1)
+ *   Stage 1  alpha-entmax routing     x = gamma (alpha-1) <q, kbar_c>/sqrt(d) over the chunks before the
+ *                                     query's own; per head tau with sum [x-tau]_+^(1/(alpha-1)) = 1;
+ *                                     group weight w = mean over the GQA group; support = {w > 0};
+ *                                     bias d_c = (log w_c - mean log w)/sigma
+ *                                                         (Eq. 2, Eq. 4, Algorithm 2, Proposition 1)
+ *   Stage 2  softmax attention over the tokens of the routed chunks plus the causal part of the
+ *            query's own chunk, logits <q,k>/sqrt(d) + d_c (0 on the own chunk)
+ *                                                         (Eq. 7, Proposition 1, Algorithm 3)
+ *
+ * Conventions
+ *   - Every pointer is DEVICE memory unless its comment says "host".  The caller owns every buffer;
+ *     the library allocates nothing, keeps no state between calls and launches only on `stream`.
+ *   - Calls are asynchronous: they return after enqueueing.  Argument errors are detected on the host
+ *     before anything is enqueued and are returned synchronously.  Problems only a kernel can see
+ *     (a bounded wait that ran out, a capacity overrun) are written to a status word at the start of
+ *     the workspace; dash_attn_last_status() synchronises the stream and returns it.
+ *   - Tensors are strided: stride arrays give element strides of (batch, token, head); the head_dim
+ *     axis is contiguous.  Base pointers must be 16-byte aligned, strides multiples of 8 elements.
+ *   - 0-based positions.  Chunk of token j is j / block.  T_s = seq_kv / block complete chunks have
+ *     summaries; T_a = ceil(seq_kv / block) chunks exist; W = ceil(T_a / 32) mask words per row.
+ *   - Query head h uses KV head h / (h_q / h_kv) (Section 3.2).
+ *   - Only causal = 1 (the paper's setting) is implemented; causal = 0 returns DASH_ERR_UNSUPPORTED.
+ *
+ * Routing outputs (Stage 1 -> Stage 2)
+ *   mask     uint32 [batch, h_kv, seq_q, W]: bit (c & 31) of word (c >> 5) is set iff chunk c is
+ *            attended by that row: the routed chunks and the row's own chunk (Algorithm 2, last step).
+ *   count    int32 [batch, h_kv, seq_q]: number of routed chunks (own chunk not counted).
+ *   blk_idx, blk_bias   compact per-row lists, ascending chunk index, own chunk excluded.  The list of
+ *            row (b, r, i) starts at entry dash_attn_list_offset(p, b, r, i) and holds count entries;
+ *            its region has room for every candidate chunk of the row, so regions never overlap:
+ *              prefill: offset = (b*h_kv + r) * R + block*c*(c-1)/2 + (i % block)*c,  c = i / block,
+ *                       with the candidate count of a row in the incomplete tail chunk clamped to T_s,
+ *                       R = sum over rows of their candidate counts;
+ *              decode : offset = (b*h_kv + r) * T_s.
+ */
+#ifndef DASH_ATTN_H_
+#define DASH_ATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  DASH_OK = 0,
+  DASH_ERR_INVALID_ARG = -1, /* null pointer, non-positive size, bad stride/alignment, struct_size mismatch */
+  DASH_ERR_UNSUPPORTED = -2, /* valid request outside what is built (head_dim, block, non-causal, ...) */
+  DASH_ERR_WORKSPACE = -3,   /* workspace null, misaligned or smaller than dash_attn_workspace_bytes() */
+  DASH_ERR_CAPACITY = -4,    /* device side: a list or queue overran its region */
+  DASH_ERR_CUDA = -5,        /* a CUDA runtime / driver call failed */
+  DASH_ERR_ARCH = -6,        /* the current device is not compute capability 10.x */
+  DASH_ERR_TIMEOUT = -7      /* device side: a bounded wait (mbarrier) ran out; results are invalid */
+} dash_status;
+
+typedef enum { DASH_F32 = 0, DASH_BF16 = 1 } dash_dtype;
+
+/* Problem statement (Section 3, "Problem setup and notation"; Algorithms 1-3 inputs). */
+typedef struct dash_params {
+  uint32_t struct_size; /* sizeof(dash_params); checked */
+  int32_t batch;
+  int32_t seq_q;        /* prefill: n (must equal seq_kv); decode: 1 */
+  int32_t seq_kv;       /* prefill: n; decode: capacity of the KV cache in tokens */
+  int32_t h_q, h_kv;    /* h_q % h_kv == 0 */
+  int32_t head_dim;     /* 64 or 128 */
+  int32_t block;        /* chunk size B: 16, 32, 64 or 128 */
+  int32_t dtype;        /* dash_dtype of Q, K, V, O */
+  int32_t causal;       /* 1 */
+  float alpha;          /* > 1; 1.25, 1.5 and 2 have integer exponents and take the fast path */
+  float gamma;          /* Stage-1 temperature multiplying the chunk logit (Eq. 4) */
+  float sigma;          /* prior strength of Eq. 8, > 0 */
+  int32_t reserved;     /* 0 */
+  const int32_t* q_to_kv; /* host, h_q entries, or NULL for h / (h_q/h_kv); only that map is accepted */
+  int64_t q_stride[3], k_stride[3], v_stride[3], o_stride[3]; /* elements: batch, token, head */
+} dash_params;
+
+/* Bytes of workspace that select / fwd_prefill / fwd_decode / attend_* need for these parameters
+ * (0 if the parameters are invalid).  The workspace must be 256-byte aligned.  Its first 256 bytes
+ * hold the status word; the rest is scratch whose contents mean nothing between calls. */
+size_t dash_attn_workspace_bytes(const dash_params* p);
+
+/* Entries the blk_idx / blk_bias lists need, and where a row's region starts (see top of file).
+ * Both return -1 for invalid parameters or indices. */
+int64_t dash_attn_list_capacity(const dash_params* p);
+int64_t dash_attn_list_offset(const dash_params* p, int32_t b, int32_t kv_head, int32_t row);
+
+/* Stage 0 (Eq. 3, Algorithm 1).  Writes the summaries of chunks [first_block, first_block+num_blocks)
+ * of every (batch, KV head) into Kbar, fp32 [batch, h_kv, T_s, head_dim] (T_s = seq_kv / block).
+ *   K       keys, dtype p->dtype, strides p->k_stride.
+ *   qbar    summary queries, fp32, [h_kv, head_dim] when qbar_chunk_stride == 0, else entry (c, r) at
+ *           qbar + c*qbar_chunk_stride + r*head_dim; NULL = zero query = mean pooling.
+ *   kv_len  int32 [batch] valid tokens per sequence, or NULL for seq_kv; chunks that are not complete
+ *           within kv_len are left untouched.
+ * num_blocks < 0 means "to the end".  A summary depends only on its own chunk, so a cache can be
+ * extended by calling this for the chunks that completed since the last call. */
+int dash_attn_block_summaries(const dash_params* p, const void* K, const float* qbar,
+                              int64_t qbar_chunk_stride, const int32_t* kv_len, int32_t first_block,
+                              int32_t num_blocks, float* Kbar, void* stream);
+
+/* Stage 1 (Eq. 2, Eq. 4, Algorithm 2, Proposition 1).  For every (batch, KV head, query row):
+ * chunk logits against Kbar, the entmax threshold of every query head of the group, the group-averaged
+ * weights, the support, and the bias of Proposition 1.
+ *   Q        queries; prefill [batch, seq_q, h_q, d] by p->q_stride; decode: token stride unused.
+ *   Kbar     fp32 [batch, h_kv, T_s, head_dim].
+ *   kv_len   decode only (NULL = seq_kv): the query of sequence b sits at kv_len[b]-1 and its candidates
+ *            are the chunks before that position's own chunk.  Must be NULL for prefill.
+ *   mask, count, blk_idx, blk_bias   outputs described at the top of the file; blk_idx may be NULL.
+ *   tau      optional fp32 [batch, h_q, seq_q] thresholds (in the scaled units of x), NULL to skip;
+ *            rows without candidates get 0.
+ * A chunk is in the support iff max over the group's heads of (x - tau) > 0. */
+int dash_attn_select(const dash_params* p, const void* Q, const float* Kbar, const int32_t* kv_len,
+                     uint32_t* mask, int32_t* count, int32_t* blk_idx, float* blk_bias, float* tau,
+                     void* workspace, size_t workspace_bytes, void* stream);
+
+/* Stage 2 alone, prefill (Eq. 7 in the form of Proposition 1, Algorithm 3): online-softmax attention of
+ * every row over the chunks its mask marks, adding blk_bias to the logits of routed chunks and applying
+ * the causal mask inside the row's own chunk.  mask / blk_bias in the layout dash_attn_select writes
+ * (any mask obeying it is accepted, e.g. a random one).  O has dtype p->dtype, strides p->o_stride. */
+int dash_attn_attend_prefill(const dash_params* p, const void* Q, const void* K, const void* V,
+                             const uint32_t* mask, const float* blk_bias, void* O, void* workspace,
+                             size_t workspace_bytes, void* stream);
+
+/* Stage 2 alone, decode: one query row per sequence at position kv_len[b]-1, the routed chunk list split
+ * across thread blocks along KV and merged (Section 3.5, split-KV variant). */
+int dash_attn_attend_decode(const dash_params* p, const void* Q, const void* Kcache, const void* Vcache,
+                            const int32_t* kv_len, const int32_t* count, const int32_t* blk_idx,
+                            const float* blk_bias, void* O, void* workspace, size_t workspace_bytes,
+                            void* stream);
+
+/* Whole prefill forward: Stage 0 (skipped when Kbar is given), Stage 1, Stage 2.
+ *   qbar / qbar_chunk_stride as in dash_attn_block_summaries (used only when Kbar == NULL).
+ *   Kbar      NULL: summaries are computed into the workspace; else used as given.
+ *   mask_out  optional uint32 [batch, h_kv, seq_q, W]; NULL keeps the mask in the workspace. */
+int dash_attn_fwd_prefill(const dash_params* p, const void* Q, const void* K, const void* V,
+                          const float* qbar, int64_t qbar_chunk_stride, const float* Kbar, void* O,
+                          uint32_t* mask_out, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Whole decode step: Stage 1 for the one new row of every sequence against the summary cache, then the
+ * split-KV Stage 2 over the selected chunks of the KV cache.  Kbar must hold the summaries of every chunk
+ * that is complete within kv_len[b]-1 tokens (dash_attn_block_summaries keeps it up to date). */
+int dash_attn_fwd_decode(const dash_params* p, const void* Q, const void* Kcache, const void* Vcache,
+                         const float* Kbar, const int32_t* kv_len, void* O, void* workspace,
+                         size_t workspace_bytes, void* stream);
+
+/* Zeroes the status word (enqueued on stream).  Call once after allocating a workspace. */
+int dash_attn_reset_status(void* workspace, void* stream);
+
+/* Synchronises `stream` and returns the workspace's status word (DASH_OK or a device-side error). */
+int dash_attn_last_status(const void* workspace, void* stream);
+
+/* Number of kernel launches this library has enqueued in this process (for launch accounting). */
+int64_t dash_attn_launch_count(void);
+
+const char* dash_attn_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DASH_ATTN_H_ */

@@ -1,0 +1,298 @@
+// C ABI of the DashAttention library: argument validation, workspace carving and stage dispatch.
+// Every operation is defined in include/dash_attn.h; kernels live in the sibling translation units.
+#include <atomic>
+#include <cmath>
+#include <cstring>
+
+#include "common.cuh"
+
+namespace dash {
+
+static std::atomic<long long> g_launches{0};
+void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+
+static inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+struct WorkspaceLayout {
+  size_t status, kbar, mask, count, blk_idx, blk_bias, partials, total;
+};
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+static int check_strides(const long long* s, int dtype) {
+  const int mult = dtype == DASH_BF16 ? 8 : 4;
+  for (int k = 0; k < 3; ++k)
+    if (s[k] < 0 || s[k] % mult != 0) return 0;
+  return 1;
+}
+
+// Validates p and fills the derived description.  Returns a dash_status.
+static int make_dims(const dash_params* p, Dims* dm) {
+  if (!p) return DASH_ERR_INVALID_ARG;
+  if (p->struct_size != sizeof(dash_params)) return DASH_ERR_INVALID_ARG;
+  if (p->batch <= 0 || p->seq_q <= 0 || p->seq_kv <= 0 || p->h_q <= 0 || p->h_kv <= 0) return DASH_ERR_INVALID_ARG;
+  if (p->batch > 65535 || p->h_kv > 65535) return DASH_ERR_INVALID_ARG;
+  if (p->h_q % p->h_kv != 0) return DASH_ERR_INVALID_ARG;
+  if (p->dtype != DASH_F32 && p->dtype != DASH_BF16) return DASH_ERR_INVALID_ARG;
+  if (!(p->alpha > 1.f) || !(p->gamma > 0.f) || !(p->sigma > 0.f)) return DASH_ERR_INVALID_ARG;
+  if (!std::isfinite(p->alpha) || !std::isfinite(p->gamma) || !std::isfinite(p->sigma)) return DASH_ERR_INVALID_ARG;
+  if (p->reserved != 0) return DASH_ERR_INVALID_ARG;
+  if (p->seq_q != p->seq_kv && p->seq_q != 1) return DASH_ERR_INVALID_ARG;
+  const int g_q = p->h_q / p->h_kv;
+  if (p->q_to_kv) {
+    for (int h = 0; h < p->h_q; ++h)
+      if (p->q_to_kv[h] != h / g_q) return DASH_ERR_UNSUPPORTED;
+  }
+  if (p->head_dim != 64 && p->head_dim != 128) return DASH_ERR_UNSUPPORTED;
+  if (p->block != 16 && p->block != 32 && p->block != 64 && p->block != 128) return DASH_ERR_UNSUPPORTED;
+  if (g_q != 1 && g_q != 2 && g_q != 4 && g_q != 8 && g_q != 16) return DASH_ERR_UNSUPPORTED;
+  if (p->causal != 1) return DASH_ERR_UNSUPPORTED;
+  if (!check_strides((const long long*)p->q_stride, p->dtype) || !check_strides((const long long*)p->k_stride, p->dtype) ||
+      !check_strides((const long long*)p->v_stride, p->dtype) || !check_strides((const long long*)p->o_stride, p->dtype))
+    return DASH_ERR_INVALID_ARG;
+
+  std::memset(dm, 0, sizeof(*dm));
+  dm->batch = p->batch; dm->seq_q = p->seq_q; dm->seq_kv = p->seq_kv;
+  dm->h_q = p->h_q; dm->h_kv = p->h_kv; dm->d = p->head_dim; dm->B = p->block; dm->g_q = g_q;
+  dm->dtype = p->dtype;
+  dm->T_s = p->seq_kv / p->block;
+  dm->T_a = (p->seq_kv + p->block - 1) / p->block;
+  dm->W = (dm->T_a + 31) / 32;
+  dm->decode = (p->seq_q == 1 && p->seq_kv != 1) ? 1 : 0;
+  dm->e = 1.f / (p->alpha - 1.f);
+  dm->e_int = p->alpha == 2.f ? 1 : p->alpha == 1.5f ? 2 : p->alpha == 1.25f ? 4 : 0;
+  dm->sm_scale = 1.f / std::sqrt((float)p->head_dim);
+  dm->x_scale = (float)((double)p->gamma * ((double)p->alpha - 1.0) / std::sqrt((double)p->head_dim));
+  dm->inv_sigma = 1.f / p->sigma;
+  for (int k = 0; k < 3; ++k) {
+    dm->qs[k] = p->q_stride[k]; dm->ks[k] = p->k_stride[k]; dm->vs[k] = p->v_stride[k]; dm->os[k] = p->o_stride[k];
+  }
+  if (dm->decode) {
+    dm->list_rows = dm->T_s;
+  } else {
+    Dims tmp = *dm;
+    const long long n = p->seq_q;
+    const long long c = n / p->block;
+    dm->list_rows = (long long)p->block * c * (c - 1) / 2 + (n % p->block) * c;
+    (void)tmp;
+  }
+  if (select_smem_bytes(*dm, nullptr) == 0) return DASH_ERR_UNSUPPORTED;  // score rows do not fit on chip
+  return DASH_OK;
+}
+
+static WorkspaceLayout layout(const Dims& dm) {
+  WorkspaceLayout w;
+  size_t off = 0;
+  w.status = off; off += 256;
+  w.kbar = off; off += align256((size_t)dm.batch * dm.h_kv * (size_t)max(dm.T_s, 1) * dm.d * sizeof(float));
+  w.mask = off; off += align256((size_t)dm.batch * dm.h_kv * (size_t)dm.seq_q * dm.W * sizeof(uint32_t));
+  w.count = off; off += align256((size_t)dm.batch * dm.h_kv * (size_t)dm.seq_q * sizeof(int));
+  const size_t cap = (size_t)dm.batch * dm.h_kv * (size_t)(dm.list_rows > 0 ? dm.list_rows : 1);
+  w.blk_idx = off; off += align256(cap * sizeof(int));
+  w.blk_bias = off; off += align256(cap * sizeof(float));
+  w.partials = off; off += align256(dm.decode ? decode_partial_bytes(dm) : 0);
+  w.total = off;
+  return w;
+}
+
+static int check_device() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return DASH_ERR_CUDA;
+  static int cached[64];  // 0 unknown, 1 ok, 2 wrong architecture
+  if (dev >= 0 && dev < 64 && cached[dev]) return cached[dev] == 1 ? DASH_OK : DASH_ERR_ARCH;
+  int major = 0;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return DASH_ERR_CUDA;
+  if (dev >= 0 && dev < 64) cached[dev] = major == 10 ? 1 : 2;
+  return major == 10 ? DASH_OK : DASH_ERR_ARCH;
+}
+
+static int check_workspace(const Dims& dm, void* ws, size_t bytes, WorkspaceLayout* out) {
+  if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255) != 0) return DASH_ERR_WORKSPACE;
+  *out = layout(dm);
+  if (bytes < out->total) return DASH_ERR_WORKSPACE;
+  return DASH_OK;
+}
+
+template <typename T> static T* at(void* ws, size_t off) { return reinterpret_cast<T*>(static_cast<char*>(ws) + off); }
+
+static int cuda_status(cudaError_t e) { return e == cudaSuccess ? DASH_OK : DASH_ERR_CUDA; }
+
+static int run_attend_prefill(const Dims& dm, const void* Q, const void* K, const void* V, const uint32_t* mask,
+                              const float* blk_bias, void* O, StatusBlock* sb, cudaStream_t st) {
+  if (prefill_sm100_supported(dm)) return cuda_status(launch_attend_prefill_sm100(dm, Q, K, V, mask, blk_bias, O, sb, st));
+  return cuda_status(launch_attend_prefill_generic(dm, Q, K, V, mask, blk_bias, O, st));
+}
+
+}  // namespace dash
+
+using namespace dash;
+
+extern "C" {
+
+size_t dash_attn_workspace_bytes(const dash_params* p) {
+  Dims dm;
+  if (make_dims(p, &dm) != DASH_OK) return 0;
+  return layout(dm).total;
+}
+
+int64_t dash_attn_list_capacity(const dash_params* p) {
+  Dims dm;
+  if (make_dims(p, &dm) != DASH_OK) return -1;
+  return (int64_t)dm.batch * dm.h_kv * dm.list_rows;
+}
+
+int64_t dash_attn_list_offset(const dash_params* p, int32_t b, int32_t kv_head, int32_t row) {
+  Dims dm;
+  if (make_dims(p, &dm) != DASH_OK) return -1;
+  if (b < 0 || b >= dm.batch || kv_head < 0 || kv_head >= dm.h_kv || row < 0 || row >= dm.seq_q) return -1;
+  return ((int64_t)b * dm.h_kv + kv_head) * dm.list_rows + list_row_offset(dm, row);
+}
+
+int dash_attn_block_summaries(const dash_params* p, const void* K, const float* qbar, int64_t qbar_chunk_stride,
+                              const int32_t* kv_len, int32_t first_block, int32_t num_blocks, float* Kbar,
+                              void* stream) {
+  Dims dm;
+  int rc = make_dims(p, &dm);
+  if (rc != DASH_OK) return rc;
+  if (!K || !Kbar || !aligned16(K) || !aligned16(Kbar)) return DASH_ERR_INVALID_ARG;
+  if (qbar && (!aligned16(qbar) || qbar_chunk_stride < 0 || qbar_chunk_stride % 4 != 0)) return DASH_ERR_INVALID_ARG;
+  if (first_block < 0 || first_block > dm.T_s) return DASH_ERR_INVALID_ARG;
+  if (num_blocks < 0) num_blocks = dm.T_s - first_block;
+  if (first_block + num_blocks > dm.T_s) return DASH_ERR_INVALID_ARG;
+  if ((rc = check_device()) != DASH_OK) return rc;
+  return cuda_status(launch_summaries(dm, K, qbar, qbar_chunk_stride, kv_len, first_block, num_blocks, Kbar,
+                                      (cudaStream_t)stream));
+}
+
+int dash_attn_select(const dash_params* p, const void* Q, const float* Kbar, const int32_t* kv_len, uint32_t* mask,
+                     int32_t* count, int32_t* blk_idx, float* blk_bias, float* tau, void* workspace,
+                     size_t workspace_bytes, void* stream) {
+  Dims dm;
+  int rc = make_dims(p, &dm);
+  if (rc != DASH_OK) return rc;
+  if (!Q || !Kbar || !mask || !count || !blk_bias) return DASH_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(Kbar)) return DASH_ERR_INVALID_ARG;
+  if (!dm.decode && kv_len) return DASH_ERR_INVALID_ARG;
+  WorkspaceLayout wl;
+  if ((rc = check_workspace(dm, workspace, workspace_bytes, &wl)) != DASH_OK) return rc;
+  if ((rc = check_device()) != DASH_OK) return rc;
+  return cuda_status(launch_select(dm, Q, Kbar, kv_len, mask, count, blk_idx, blk_bias, tau,
+                                   at<StatusBlock>(workspace, wl.status), (cudaStream_t)stream));
+}
+
+int dash_attn_attend_prefill(const dash_params* p, const void* Q, const void* K, const void* V, const uint32_t* mask,
+                             const float* blk_bias, void* O, void* workspace, size_t workspace_bytes, void* stream) {
+  Dims dm;
+  int rc = make_dims(p, &dm);
+  if (rc != DASH_OK) return rc;
+  if (dm.decode) return DASH_ERR_INVALID_ARG;
+  if (!Q || !K || !V || !mask || !blk_bias || !O) return DASH_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O)) return DASH_ERR_INVALID_ARG;
+  WorkspaceLayout wl;
+  if ((rc = check_workspace(dm, workspace, workspace_bytes, &wl)) != DASH_OK) return rc;
+  if ((rc = check_device()) != DASH_OK) return rc;
+  return run_attend_prefill(dm, Q, K, V, mask, blk_bias, O, at<StatusBlock>(workspace, wl.status), (cudaStream_t)stream);
+}
+
+int dash_attn_attend_decode(const dash_params* p, const void* Q, const void* Kcache, const void* Vcache,
+                            const int32_t* kv_len, const int32_t* count, const int32_t* blk_idx,
+                            const float* blk_bias, void* O, void* workspace, size_t workspace_bytes, void* stream) {
+  Dims dm;
+  int rc = make_dims(p, &dm);
+  if (rc != DASH_OK) return rc;
+  if (!dm.decode) return DASH_ERR_INVALID_ARG;
+  if (!Q || !Kcache || !Vcache || !count || !blk_idx || !blk_bias || !O) return DASH_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(Kcache) || !aligned16(Vcache) || !aligned16(O)) return DASH_ERR_INVALID_ARG;
+  WorkspaceLayout wl;
+  if ((rc = check_workspace(dm, workspace, workspace_bytes, &wl)) != DASH_OK) return rc;
+  if ((rc = check_device()) != DASH_OK) return rc;
+  return cuda_status(launch_attend_decode(dm, Q, Kcache, Vcache, kv_len, count, blk_idx, blk_bias, O,
+                                          at<float>(workspace, wl.partials), (cudaStream_t)stream));
+}
+
+int dash_attn_fwd_prefill(const dash_params* p, const void* Q, const void* K, const void* V, const float* qbar,
+                          int64_t qbar_chunk_stride, const float* Kbar, void* O, uint32_t* mask_out, void* workspace,
+                          size_t workspace_bytes, void* stream) {
+  Dims dm;
+  int rc = make_dims(p, &dm);
+  if (rc != DASH_OK) return rc;
+  if (dm.decode) return DASH_ERR_INVALID_ARG;
+  if (!Q || !K || !V || !O) return DASH_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O)) return DASH_ERR_INVALID_ARG;
+  if (Kbar && !aligned16(Kbar)) return DASH_ERR_INVALID_ARG;
+  if (qbar && (!aligned16(qbar) || qbar_chunk_stride < 0 || qbar_chunk_stride % 4 != 0)) return DASH_ERR_INVALID_ARG;
+  WorkspaceLayout wl;
+  if ((rc = check_workspace(dm, workspace, workspace_bytes, &wl)) != DASH_OK) return rc;
+  if ((rc = check_device()) != DASH_OK) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  StatusBlock* sb = at<StatusBlock>(workspace, wl.status);
+  const float* kb = Kbar;
+  if (!kb) {
+    float* kbw = at<float>(workspace, wl.kbar);
+    if ((rc = cuda_status(launch_summaries(dm, K, qbar, qbar_chunk_stride, nullptr, 0, dm.T_s, kbw, st))) != DASH_OK) return rc;
+    kb = kbw;
+  }
+  uint32_t* mask = mask_out ? mask_out : at<uint32_t>(workspace, wl.mask);
+  float* bias = at<float>(workspace, wl.blk_bias);
+  if ((rc = cuda_status(launch_select(dm, Q, kb, nullptr, mask, at<int>(workspace, wl.count), nullptr, bias, nullptr,
+                                      sb, st))) != DASH_OK)
+    return rc;
+  return run_attend_prefill(dm, Q, K, V, mask, bias, O, sb, st);
+}
+
+int dash_attn_fwd_decode(const dash_params* p, const void* Q, const void* Kcache, const void* Vcache,
+                         const float* Kbar, const int32_t* kv_len, void* O, void* workspace, size_t workspace_bytes,
+                         void* stream) {
+  Dims dm;
+  int rc = make_dims(p, &dm);
+  if (rc != DASH_OK) return rc;
+  if (!dm.decode) return DASH_ERR_INVALID_ARG;
+  if (!Q || !Kcache || !Vcache || !Kbar || !O) return DASH_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(Kcache) || !aligned16(Vcache) || !aligned16(Kbar) || !aligned16(O))
+    return DASH_ERR_INVALID_ARG;
+  WorkspaceLayout wl;
+  if ((rc = check_workspace(dm, workspace, workspace_bytes, &wl)) != DASH_OK) return rc;
+  if ((rc = check_device()) != DASH_OK) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  StatusBlock* sb = at<StatusBlock>(workspace, wl.status);
+  int* count = at<int>(workspace, wl.count);
+  int* idx = at<int>(workspace, wl.blk_idx);
+  float* bias = at<float>(workspace, wl.blk_bias);
+  if ((rc = cuda_status(launch_select(dm, Q, Kbar, kv_len, at<uint32_t>(workspace, wl.mask), count, idx, bias, nullptr,
+                                      sb, st))) != DASH_OK)
+    return rc;
+  return cuda_status(launch_attend_decode(dm, Q, Kcache, Vcache, kv_len, count, idx, bias, O,
+                                          at<float>(workspace, wl.partials), st));
+}
+
+int dash_attn_reset_status(void* workspace, void* stream) {
+  if (!workspace) return DASH_ERR_WORKSPACE;
+  return cuda_status(cudaMemsetAsync(workspace, 0, 256, (cudaStream_t)stream));
+}
+
+int dash_attn_last_status(const void* workspace, void* stream) {
+  if (!workspace) return DASH_ERR_WORKSPACE;
+  int st = 0;
+  if (cudaMemcpyAsync(&st, workspace, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream) != cudaSuccess)
+    return DASH_ERR_CUDA;
+  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return DASH_ERR_CUDA;
+  return st;
+}
+
+int64_t dash_attn_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char* dash_attn_strerror(int status) {
+  switch (status) {
+    case DASH_OK: return "ok";
+    case DASH_ERR_INVALID_ARG: return "invalid argument";
+    case DASH_ERR_UNSUPPORTED: return "unsupported configuration";
+    case DASH_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case DASH_ERR_CAPACITY: return "device-side capacity overrun";
+    case DASH_ERR_CUDA: return "CUDA call failed";
+    case DASH_ERR_ARCH: return "device is not compute capability 10.x";
+    case DASH_ERR_TIMEOUT: return "device-side bounded wait ran out";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

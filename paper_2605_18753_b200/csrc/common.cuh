@@ -1,0 +1,121 @@
+// Shared declarations of the DashAttention CUDA library (internal; the public ABI is include/dash_attn.h).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "dash_attn.h"
+
+namespace dash {
+
+// Derived problem description handed to kernels by value.
+struct Dims {
+  int batch, seq_q, seq_kv, h_q, h_kv, d, B, g_q;
+  int dtype;    // dash_dtype of Q, K, V, O
+  int T_s;      // complete chunks (those with summaries): seq_kv / B
+  int T_a;      // all chunks: ceil(seq_kv / B)
+  int W;        // mask words per row: ceil(T_a / 32)
+  int decode;   // 1: one query row per sequence at kv_len[b]-1
+  int e_int;    // 1/(alpha-1) when it is 1, 2 or 4 (alpha = 2, 1.5, 1.25); 0 otherwise
+  float e;      // 1/(alpha-1)
+  float x_scale;   // gamma (alpha-1) / sqrt(d): chunk logit scale (Algorithm 2, step 1)
+  float sm_scale;  // 1 / sqrt(d): token logit scale (Eq. 1)
+  float inv_sigma;
+  long long qs[3], ks[3], vs[3], os[3];
+  long long list_rows;  // list entries per (batch, KV head)
+};
+
+// Start of row i's list region inside its (batch, KV head) slab.
+__host__ __device__ inline long long list_row_offset(const Dims& dm, int i) {
+  if (dm.decode) return 0;
+  long long c = i / dm.B;
+  return (long long)dm.B * c * (c - 1) / 2 + (long long)(i % dm.B) * c;
+}
+
+// Workspace: 256-byte header (status word first), then regions carved by the host.
+struct StatusBlock {
+  int status;        // dash_status written by kernels (first error wins)
+  int detail;        // where it happened (kernel-specific code)
+  unsigned int tile_counter;  // persistent-kernel work queue
+  int pad[61];
+};
+static_assert(sizeof(StatusBlock) == 256, "status block is the first 256 bytes of the workspace");
+
+__device__ inline void report_error(StatusBlock* sb, int status, int detail) {
+  if (atomicCAS(&sb->status, 0, status) == 0) sb->detail = detail;
+}
+
+template <typename T> __device__ inline float to_f32(T v);
+template <> __device__ inline float to_f32<float>(float v) { return v; }
+template <> __device__ inline float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+template <typename T> __device__ inline T from_f32(float v);
+template <> __device__ inline float from_f32<float>(float v) { return v; }
+template <> __device__ inline __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+// Load 4 consecutive elements as float4 (pointer 8-byte aligned for bf16, 16 for fp32).
+__device__ inline float4 load4(const float* p) { return *reinterpret_cast<const float4*>(p); }
+__device__ inline float4 load4(const __nv_bfloat16* p) {
+  uint2 u = *reinterpret_cast<const uint2*>(p);
+  __nv_bfloat162 a = *reinterpret_cast<__nv_bfloat162*>(&u.x);
+  __nv_bfloat162 b = *reinterpret_cast<__nv_bfloat162*>(&u.y);
+  float2 fa = __bfloat1622float2(a), fb = __bfloat1622float2(b);
+  return make_float4(fa.x, fa.y, fb.x, fb.y);
+}
+__device__ inline void store4(float* p, float4 v) { *reinterpret_cast<float4*>(p) = v; }
+__device__ inline void store4(__nv_bfloat16* p, float4 v) {
+  __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b = __floats2bfloat162_rn(v.z, v.w);
+  uint2 u;
+  u.x = *reinterpret_cast<unsigned int*>(&a);
+  u.y = *reinterpret_cast<unsigned int*>(&b);
+  *reinterpret_cast<uint2*>(p) = u;
+}
+
+__device__ inline float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ inline float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// m^e for the integer exponents of alpha = 2, 1.5, 1.25; powf otherwise.  m >= 0.
+__device__ inline float pow_e(float m, int e_int, float e) {
+  if (e_int == 1) return m;
+  if (e_int == 2) return m * m;
+  if (e_int == 4) { float s = m * m; return s * s; }
+  return m > 0.f ? __powf(m, e) : 0.f;
+}
+// m^(e-1)
+__device__ inline float pow_em1(float m, int e_int, float e) {
+  if (e_int == 1) return m > 0.f ? 1.f : 0.f;
+  if (e_int == 2) return m;
+  if (e_int == 4) return m * m * m;
+  return m > 0.f ? __powf(m, e - 1.f) : 0.f;
+}
+
+void count_launch();
+
+// Launchers (one per translation unit).  All return a cudaError_t from the launch.
+cudaError_t launch_summaries(const Dims& dm, const void* K, const float* qbar, long long qbar_chunk_stride,
+                             const int* kv_len, int first_block, int num_blocks, float* Kbar, cudaStream_t st);
+size_t select_smem_bytes(const Dims& dm, int* tq_out);
+cudaError_t launch_select(const Dims& dm, const void* Q, const float* Kbar, const int* kv_len, uint32_t* mask,
+                          int* count, int* blk_idx, float* blk_bias, float* tau, StatusBlock* sb, cudaStream_t st);
+cudaError_t launch_attend_prefill_generic(const Dims& dm, const void* Q, const void* K, const void* V,
+                                          const uint32_t* mask, const float* blk_bias, void* O, cudaStream_t st);
+int decode_num_splits(const Dims& dm);
+size_t decode_partial_bytes(const Dims& dm);
+cudaError_t launch_attend_decode(const Dims& dm, const void* Q, const void* K, const void* V, const int* kv_len,
+                                 const int* count, const int* blk_idx, const float* blk_bias, void* O,
+                                 float* partials, cudaStream_t st);
+bool prefill_sm100_supported(const Dims& dm);
+cudaError_t launch_attend_prefill_sm100(const Dims& dm, const void* Q, const void* K, const void* V,
+                                        const uint32_t* mask, const float* blk_bias, void* O, StatusBlock* sb,
+                                        cudaStream_t st);
+
+}  // namespace dash

@@ -67,12 +67,12 @@ WORKLOADS = {
                            rho=0.72, shift=2.0),
     # C3: prefill 64K at ~75 % and ~90 %
     "prefill_64k_s75": Workload("prefill_64k_s75", "prefill", 1, 65536, 32, 8, 128, 64, 1.5, "bf16", "planted",
-                                rho=0.72, shift=1.9),
+                                rho=0.72, shift=1.49),
     "prefill_64k_s90": Workload("prefill_64k_s90", "prefill", 1, 65536, 32, 8, 128, 64, 1.5, "bf16", "planted",
-                                rho=0.72, shift=2.8),
+                                rho=0.72, shift=1.95),
     # C4: decode, batch 16, 131072-token cache, ~90 %
     "decode_128k": Workload("decode_128k", "decode", 16, 131072, 32, 8, 128, 64, 1.5, "bf16", "planted",
-                            rho=0.72, shift=1.4),
+                            rho=0.72, shift=1.42),
     # C5: alpha sweep base point (block and alpha are varied by the caller)
     "sweep_32k": Workload("sweep_32k", "prefill", 2, 32768, 32, 8, 128, 64, 1.5, "bf16", "planted",
                           rho=0.72, shift=2.0),

@@ -1,0 +1,319 @@
+"""GPU parity: every stage of the CUDA library, through the C ABI, against the float64 oracle on the same
+seeded inputs.  Integer outputs (mask, count, lists) must match exactly except for chunks whose oracle
+margin is within 1e-4 of the entmax threshold; floating outputs within the stated tolerances."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import dash_oracle as orc
+from paper_2605_18753_b200 import binding as B
+from paper_2605_18753_b200 import synth
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _wl(**kw):
+    base = dict(name="t", kind="prefill", batch=1, seq=512, h_q=4, h_kv=2, head_dim=64, block=16, alpha=1.5,
+                dtype="bf16", recipe="planted", gamma=1.0, sigma=10.0, rho=0.72, shift=2.0, n_planted=3, seed=0)
+    base.update(kw)
+    return synth.Workload(**base)
+
+
+# ------------------------------------------------------------------ Stage 0
+
+@pytest.mark.parametrize("dtype,d,Bk,n,mode", [
+    ("bf16", 128, 64, 1000, "none"), ("bf16", 128, 64, 1000, "head"), ("bf16", 64, 16, 200, "chunk"),
+    ("f32", 64, 64, 1024, "none"), ("f32", 128, 128, 700, "head"), ("bf16", 128, 32, 96, "chunk"),
+])
+def test_block_summaries(dtype, d, Bk, n, mode):
+    w = _wl(seq=n, head_dim=d, block=Bk, dtype=dtype, h_q=6, h_kv=3, batch=2)
+    inp = synth.make_prefill_inputs(w, DEV)
+    K = inp["K"]
+    T_s = n // Bk
+    qbar = None
+    stride = 0
+    if mode == "head":
+        qbar = torch.randn(3, d, device=DEV, generator=torch.Generator(DEV).manual_seed(5)) * 2
+    elif mode == "chunk":
+        qbar = torch.randn(T_s, 3, d, device=DEV, generator=torch.Generator(DEV).manual_seed(6)) * 2
+        stride = 3 * d
+    O = torch.empty_like(inp["Q"])
+    p = B.params_for_prefill(inp["Q"], K, inp["V"], O, block=Bk, alpha=1.5)
+    kbar = torch.full((2, 3, T_s, d), float("nan"), device=DEV)
+    B.dash_attn_block_summaries(p, K, kbar, qbar, stride)
+    got = kbar.cpu().double().numpy()
+    for bb in range(2):
+        want = orc.block_summaries(H.to_np64(K[bb]), Bk, None if qbar is None else H.to_np64(qbar))
+        err = np.abs(got[bb].transpose(1, 0, 2) - want)
+        assert err.max() <= 2e-6 * max(1.0, np.abs(want).max()), err.max()
+
+
+def test_block_summaries_incremental_and_kv_len():
+    w = _wl(seq=640, head_dim=128, block=64, h_q=2, h_kv=2, batch=2)
+    inp = synth.make_prefill_inputs(w, DEV)
+    p = B.params_for_prefill(inp["Q"], inp["K"], inp["V"], torch.empty_like(inp["Q"]), block=64, alpha=1.5)
+    full = torch.zeros(2, 2, 10, 128, device=DEV)
+    B.dash_attn_block_summaries(p, inp["K"], full)
+    part = torch.full_like(full, -7.0)
+    kv_len = torch.tensor([640, 200], dtype=torch.int32, device=DEV)
+    B.dash_attn_block_summaries(p, inp["K"], part, kv_len=kv_len, first_block=2, num_blocks=5)
+    assert torch.equal(part[0, :, 2:7], full[0, :, 2:7]) and (part[0, :, :2] == -7).all() and (part[0, :, 7:] == -7).all()
+    assert torch.equal(part[1, :, 2:3], full[1, :, 2:3]) and (part[1, :, 3:] == -7).all()   # chunk 3 incomplete at 200
+
+
+# ------------------------------------------------------------------ Stage 1
+
+def _run_select(w, inp, with_idx=True):
+    Q, K, V = inp["Q"], inp["K"], inp["V"]
+    O = torch.empty_like(Q)
+    p = B.params_for_prefill(Q, K, V, O, block=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma)
+    kbar = B.alloc_kbar(p)
+    B.dash_attn_block_summaries(p, K, kbar)
+    ws = B.alloc_workspace(p)
+    rt = B.alloc_routing(p, with_tau=True)
+    for t in rt.values():
+        if t is not None:
+            t.fill_(-1 if t.dtype != torch.float32 else float("nan"))
+    B.dash_attn_select(p, Q, kbar, rt["mask"], rt["count"], rt["blk_idx"] if with_idx else None, rt["blk_bias"], ws,
+                       tau=rt["tau"])
+    assert B.dash_attn_last_status(ws) == 0
+    return p, kbar, ws, rt
+
+
+def _check_select(w, inp, p, rt, rows, kv_heads=None):
+    ora = H.oracle_prefill_rows(inp["Q"], inp["K"], inp["V"], B=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma,
+                                rows=rows, kv_heads=kv_heads)
+    mask = rt["mask"].cpu().numpy().view(np.uint32)
+    count = rt["count"].cpu().numpy()
+    idx = rt["blk_idx"].cpu().numpy()
+    bias = rt["blk_bias"].cpu().numpy()
+    tau = rt["tau"].cpu().numpy()
+    g_q = w.h_q // w.h_kv
+    n_border = n_diff = 0
+    clean_rows = {}
+    for (b, r, i), (ro, o) in ora.items():
+        off = B.dash_attn_list_offset(p, b, r, i)
+        nb, nd, clean = H.compare_routing(ro, i // w.block, mask[b, r, i], int(count[b, r, i]), bias[off:], idx[off:],
+                                          w.sigma, 1.0 / (w.alpha - 1.0))
+        n_border += nb
+        n_diff += nd
+        clean_rows[(b, r, i)] = clean
+        if ro.n_cand:
+            terr = np.abs(tau[b, r * g_q:(r + 1) * g_q, i] - ro.tau).max()
+            assert terr <= 1e-5 * max(1.0, np.abs(ro.x).max()), (i, terr)
+    return ora, clean_rows, n_border, n_diff
+
+
+@pytest.mark.parametrize("kw", [
+    dict(), dict(alpha=2.0), dict(alpha=1.25, gamma=2.0), dict(alpha=1.75, gamma=1.5),
+    dict(h_q=8, h_kv=2, head_dim=128, block=32, seq=1000), dict(h_q=2, h_kv=2, block=64, seq=777),
+    dict(h_q=16, h_kv=1, head_dim=128, block=64, seq=1500, batch=2), dict(dtype="f32", seq=300, gamma=3.0),
+    dict(h_q=8, h_kv=1, head_dim=64, block=128, seq=1100), dict(seq=15), dict(seq=16), dict(seq=17),
+])
+def test_select_matches_oracle(kw):
+    w = _wl(**kw)
+    inp = synth.make_prefill_inputs(w, DEV)
+    p, kbar, ws, rt = _run_select(w, inp)
+    rows = sorted(set(list(range(0, w.seq, 7)) + [w.seq - 1] + list(range(min(w.seq, 3 * w.block)))))
+    ora, clean, nb, nd = _check_select(w, inp, p, rt, rows)
+    sizes = [v[0].support.size for v in ora.values()]
+    if w.seq > 4 * w.block:
+        assert max(sizes) >= 2
+    assert nd <= nb
+
+
+def test_select_tiny_configs_and_sparsity_regimes():
+    """C1 (gamma=1: every visible chunk routed) and C1' (gamma=512: the threshold prunes), fp32."""
+    for name in ("tiny", "tiny_g512"):
+        w = synth.workload(name)
+        inp = synth.make_prefill_inputs(w, DEV)
+        p, kbar, ws, rt = _run_select(w, inp)
+        ora, clean, nb, nd = _check_select(w, inp, p, rt, range(w.seq))
+        sup = [v[0].support.size for v in ora.values()]
+        vis = [i // w.block for (_, _, i) in ora.keys()]
+        s = orc.block_sparsity(sup, vis)
+        assert (s == 0.0) if name == "tiny" else (0.3 < s < 0.6)
+
+
+def test_select_without_block_index_list_and_determinism():
+    w = _wl(seq=900, h_q=8, h_kv=2, head_dim=128, block=64)
+    inp = synth.make_prefill_inputs(w, DEV)
+    p, kbar, ws, rt1 = _run_select(w, inp, with_idx=True)
+    p, kbar, ws, rt2 = _run_select(w, inp, with_idx=False)
+    assert torch.equal(rt1["mask"], rt2["mask"]) and torch.equal(rt1["count"], rt2["count"])
+    assert torch.equal(rt1["tau"], rt2["tau"])
+    assert (rt2["blk_idx"] == -1).all()
+
+
+# ------------------------------------------------------------------ Stage 2 (prefill)
+
+def _gather_O(O, keys, g_q):
+    On = O.float().cpu().double().numpy()
+    return np.stack([On[b, i, r * g_q:(r + 1) * g_q] for (b, r, i) in keys])
+
+
+@pytest.mark.parametrize("kw", [
+    dict(), dict(dtype="f32"), dict(h_q=8, h_kv=2, head_dim=128, block=64, seq=1000, sigma=1.0),
+    dict(h_q=4, h_kv=4, head_dim=128, block=32, seq=333, alpha=2.0), dict(seq=17), dict(seq=5),
+    dict(h_q=16, h_kv=1, head_dim=128, block=128, seq=700, alpha=1.25, gamma=2.0),
+])
+def test_attend_prefill_with_oracle_lists(kw):
+    """Stage 2 alone, fed the oracle's own routing: no exclusions, every row must match."""
+    w = _wl(**kw)
+    inp = synth.make_prefill_inputs(w, DEV)
+    Q, K, V = inp["Q"], inp["K"], inp["V"]
+    O = torch.full_like(Q, float("nan"))
+    p = B.params_for_prefill(Q, K, V, O, block=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma)
+    ora = H.oracle_prefill_rows(Q, K, V, B=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma, rows=range(w.seq))
+    mask, count, idx, bias = H.routing_to_abi(ora, p, B.dash_attn_list_offset)
+    ws = B.alloc_workspace(p)
+    B.dash_attn_attend_prefill(p, Q, K, V, mask, bias, O, ws)
+    assert B.dash_attn_last_status(ws) == 0
+    keys = list(ora.keys())
+    want = np.stack([ora[k][1] for k in keys])
+    H.check_outputs(_gather_O(O, keys, w.h_q // w.h_kv), want, Q.dtype, "attend_prefill")
+
+
+@pytest.mark.parametrize("name,sigmas", [("tiny", (10.0, 1.0, 1e8)), ("tiny_g512", (10.0, 1e8))])
+def test_fwd_prefill_tiny_fp32(name, sigmas):
+    for sigma in sigmas:
+        w = synth.workload(name, sigma=sigma)
+        _fwd_prefill_case(w, rows=range(w.seq))
+
+
+@pytest.mark.parametrize("kw", [
+    dict(seq=1024, h_q=8, h_kv=2, head_dim=128, block=64),
+    dict(seq=1024, h_q=8, h_kv=2, head_dim=128, block=64, sigma=1e8),
+    dict(seq=2000, h_q=4, h_kv=1, head_dim=128, block=128, alpha=2.0, batch=2),
+    dict(seq=600, h_q=4, h_kv=2, head_dim=64, block=32, alpha=1.25, gamma=2.0),
+    dict(seq=1500, h_q=32, h_kv=2, head_dim=128, block=64, seed=1),
+    dict(seq=1111, h_q=2, h_kv=2, head_dim=128, block=64, seed=2),
+])
+def test_fwd_prefill_small(kw):
+    w = _wl(**kw)
+    rows = sorted(set(list(range(0, w.seq, 5)) + [w.seq - 1, w.seq - 2] + list(range(min(w.seq, 2 * w.block)))))
+    _fwd_prefill_case(w, rows)
+
+
+def _fwd_prefill_case(w, rows, kv_heads=None, min_clean=0.9):
+    inp = synth.make_prefill_inputs(w, DEV)
+    Q, K, V = inp["Q"], inp["K"], inp["V"]
+    O = torch.full_like(Q, float("nan"))
+    p = B.params_for_prefill(Q, K, V, O, block=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma)
+    ws = B.alloc_workspace(p)
+    T_a = (w.seq + w.block - 1) // w.block
+    mask = torch.empty(w.batch, w.h_kv, w.seq, (T_a + 31) // 32, dtype=torch.int32, device=DEV)
+    B.dash_attn_fwd_prefill(p, Q, K, V, O, ws, mask_out=mask)
+    assert B.dash_attn_last_status(ws) == 0
+    assert torch.isfinite(O.float()).all()
+    ora = H.oracle_prefill_rows(Q, K, V, B=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma, rows=rows,
+                                kv_heads=kv_heads)
+    mk = mask.cpu().numpy().view(np.uint32)
+    keys = []
+    n_excluded = 0
+    for (b, r, i), (ro, o) in ora.items():
+        want = orc.pack_mask_words(ro.support, i // w.block, mk.shape[-1])
+        if np.array_equal(mk[b, r, i], want):
+            # rows holding a member or non-member inside the borderline band are compared on the mask only:
+            # at finite sigma their bias (log of a near-zero weight) is ill-conditioned by construction
+            if ro.n_cand and (np.abs(ro.margin) <= H.BORDERLINE).any():
+                n_excluded += 1
+            else:
+                keys.append((b, r, i))
+        else:
+            got = {c for c in range(T_a) if (int(mk[b, r, i, c >> 5]) >> (c & 31)) & 1}
+            diff = got ^ (set(int(c) for c in ro.support) | {i // w.block})
+            border = set(int(c) for c in np.nonzero(np.abs(ro.margin) <= H.BORDERLINE)[0])
+            assert diff <= border, (b, r, i, sorted(diff))
+            n_excluded += 1
+    assert len(keys) >= min_clean * len(ora), (len(keys), len(ora), n_excluded)
+    want = np.stack([ora[k][1] for k in keys])
+    return H.check_outputs(_gather_O(O, keys, w.h_q // w.h_kv), want, Q.dtype, f"fwd_prefill {w.name}")
+
+
+def test_fwd_prefill_8k_config_sampled_rows():
+    """The 8K prefill workload at full size, in the configuration the benchmark times; the oracle computes a
+    seeded sample of rows (first/last rows of chunks, rows after planted chunks, two whole tiles)."""
+    w = synth.workload("prefill_8k")
+    rng = np.random.default_rng(0)
+    rows = set(rng.integers(0, w.seq, 96).tolist()) | {0, 63, 64, 65, 127, 128, w.seq - 1, w.seq - 64, w.seq - 65}
+    rows |= set(range(4096, 4096 + 32)) | set(range(8000, 8032))
+    for sigma in (10.0, 1e8):
+        _fwd_prefill_case(w.with_(sigma=sigma), sorted(rows), kv_heads=[0, 5])
+
+
+# ------------------------------------------------------------------ decode
+
+def _decode_case(w, kv_len, use_lists_from_oracle=False):
+    inp = synth.make_decode_inputs(w, DEV, kv_len=kv_len)
+    Q, Kc, Vc, lens = inp["Q"], inp["K"], inp["V"], inp["kv_len"]
+    O = torch.full_like(Q, float("nan"))
+    p = B.params_for_decode(Q, Kc, Vc, O, block=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma)
+    kbar = B.alloc_kbar(p)
+    kbar.fill_(float("nan"))
+    B.dash_attn_block_summaries(p, Kc, kbar, kv_len=lens)
+    ws = B.alloc_workspace(p)
+    ora = orc.forward_decode(H.to_np64(Q), H.to_np64(Kc), H.to_np64(Vc), lens.cpu().numpy(), B=w.block, alpha=w.alpha,
+                             gamma=w.gamma, sigma=w.sigma)
+    if use_lists_from_oracle:
+        mask, count, idx, bias = H.routing_to_abi({(b, r, 0): rt for (b, r), rt in ora["routing"].items()}, p,
+                                                  B.dash_attn_list_offset)
+        B.dash_attn_attend_decode(p, Q, Kc, Vc, lens, count, idx, bias, O, ws)
+        assert B.dash_attn_last_status(ws) == 0
+        H.check_outputs(O.float().cpu().double().numpy(), ora["O"], Q.dtype, "attend_decode")
+        return
+    # Stage 1 alone on the decode row, then the whole step
+    rt = B.alloc_routing(p, with_tau=True)
+    B.dash_attn_select(p, Q, kbar, rt["mask"], rt["count"], rt["blk_idx"], rt["blk_bias"], ws, tau=rt["tau"], kv_len=lens)
+    mask = rt["mask"].cpu().numpy().view(np.uint32)
+    count = rt["count"].cpu().numpy()
+    idx = rt["blk_idx"].cpu().numpy()
+    bias = rt["blk_bias"].cpu().numpy()
+    clean = np.ones((w.batch, w.h_kv), dtype=bool)
+    for (b, r), ro in ora["routing"].items():
+        off = B.dash_attn_list_offset(p, b, r, 0)
+        L = int(lens[b])
+        nb, nd, ok = H.compare_routing(ro, (L - 1) // w.block, mask[b, r, 0], int(count[b, r, 0]), bias[off:], idx[off:],
+                                       w.sigma, 1.0 / (w.alpha - 1.0))
+        clean[b, r] = ok and not (ro.n_cand and (np.abs(ro.margin) <= H.BORDERLINE).any())
+    B.dash_attn_fwd_decode(p, Q, Kc, Vc, kbar, lens, O, ws)
+    assert B.dash_attn_last_status(ws) == 0
+    got = O.float().cpu().double().numpy()
+    g_q = w.h_q // w.h_kv
+    sel = np.repeat(clean, g_q, axis=1)
+    assert sel.mean() >= 0.8
+    H.check_outputs(got[sel], ora["O"][sel], Q.dtype, "fwd_decode")
+
+
+@pytest.mark.parametrize("kw,kv_len", [
+    (dict(kind="decode", batch=3, seq=2000, h_q=8, h_kv=2, head_dim=128, block=64), [2000, 1, 777]),
+    (dict(kind="decode", batch=2, seq=1024, h_q=4, h_kv=4, head_dim=64, block=32, alpha=2.0), [1024, 65]),
+    (dict(kind="decode", batch=2, seq=4096, h_q=16, h_kv=1, head_dim=128, block=128, alpha=1.25, gamma=2.0), [4095, 129]),
+    (dict(kind="decode", batch=1, seq=3000, h_q=2, h_kv=2, head_dim=128, block=64, dtype="f32"), [2999]),
+])
+def test_decode_matches_oracle(kw, kv_len):
+    w = _wl(**kw)
+    _decode_case(w, kv_len, use_lists_from_oracle=True)
+    _decode_case(w, kv_len)
+
+
+def test_decode_equals_last_prefill_row_on_gpu():
+    w = _wl(seq=1000, h_q=8, h_kv=2, head_dim=128, block=64)
+    inp = synth.make_prefill_inputs(w, DEV)
+    Q, K, V = inp["Q"], inp["K"], inp["V"]
+    O = torch.empty_like(Q)
+    p = B.params_for_prefill(Q, K, V, O, block=64, alpha=1.5)
+    ws = B.alloc_workspace(p)
+    B.dash_attn_fwd_prefill(p, Q, K, V, O, ws)
+    q1 = Q[:, -1].contiguous()
+    o1 = torch.empty_like(q1)
+    pd = B.params_for_decode(q1, K, V, o1, block=64, alpha=1.5)
+    kbar = B.alloc_kbar(pd)
+    B.dash_attn_block_summaries(pd, K, kbar)
+    wsd = B.alloc_workspace(pd)
+    B.dash_attn_fwd_decode(pd, q1, K, V, kbar, None, o1, wsd)
+    assert (o1.float() - O[:, -1].float()).abs().max().item() <= 2e-2
