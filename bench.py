@@ -1,0 +1,381 @@
+#!/usr/bin/env python
+"""Benchmark of the DashAttention forward pass (prefill 8K workload by default).
+
+    python bench.py --gpus N --steps K --warmup W [--workload NAME] [--impl reference]
+
+A step is one pass of the whole hot path (Stage 0 summaries, Stage 1 routing, Stage 2 attention) over one
+batch of seeded synthetic input through the C-ABI library.  Prints ONE JSON line (rank 0).
+Multi-GPU: every rank runs its own batch (different seed), no collective on the data path (weak scaling).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+METRIC = "dashattention_prefill_fwd_effective_tflops"
+UNIT = "TFLOP/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        d["_source"] = "measured"
+        return d
+    d = dict(FALLBACK_PEAKS)
+    d["_source"] = "fallback"
+    return d
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks / throttle reasons of one GPU while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.samples, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.samples.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for s in self.samples:
+            f = [x.strip() for x in s.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for k, nm in enumerate(names):
+                if f[3 + k].lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def selected_flops_from_count(count: torch.Tensor, B: int, d: int, g_q: int) -> float:
+    """4 d g_q sum_rows (B |S_i| + (i mod B) + 1) from the routed-chunk counts [b, h_kv, n]."""
+    b, h_kv, n = count.shape
+    diag = (torch.arange(n, device=count.device) % B + 1).to(torch.float64)
+    tok = count.to(torch.float64) * B + diag[None, None, :]
+    return float(4.0 * d * g_q * tok.sum().item())
+
+
+def sparsity_from_count(count: torch.Tensor, B: int) -> float:
+    n = count.shape[-1]
+    vis = (torch.arange(n, device=count.device) // B).to(torch.float64)
+    return float(1.0 - (count.to(torch.float64) + 1).sum().item() / ((vis + 1).sum().item() * count.shape[0] * count.shape[1]))
+
+
+def time_oracle_sample(w, inp, budget_s: float = 15.0):
+    """Times the oracle (as it stands, one thread) on a seeded sample of rows of the workload.
+    Returns (TFLOP/s on selected FLOPs, rows done, seconds)."""
+    from oracle import dash_oracle as orc
+    from threadpoolctl import threadpool_limits
+    Qn = inp["Q"][0].cpu().double().numpy()
+    Kn = inp["K"][0].cpu().double().numpy()
+    Vn = inp["V"][0].cpu().double().numpy()
+    rng = np.random.default_rng(0)
+    g_q = w.h_q // w.h_kv
+    flops, rows = 0.0, 0
+    with threadpool_limits(limits=1):
+        t0 = time.perf_counter()
+        Kbar = orc.block_summaries(Kn, w.block)
+        while time.perf_counter() - t0 < budget_s:
+            i = int(rng.integers(0, w.seq))
+            r = int(rng.integers(0, w.h_kv))
+            rt, _ = orc.forward_row(Qn, Kn, Vn, Kbar, i, r, B=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma)
+            flops += 4.0 * w.head_dim * g_q * (w.block * rt.support.size + (i % w.block) + 1)
+            rows += 1
+        dt = time.perf_counter() - t0
+    return flops / dt / 1e12, rows, dt
+
+
+def run_reference(args, w):
+    """The oracle timed on the host cores: each step is a bounded sample of the workload's rows."""
+    from paper_2605_18753_b200 import synth
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    inp = synth.make_prefill_inputs(w.with_(batch=1), "cpu")
+    per_step = max(2.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
+    vals, rows = [], 0
+    for s in range(args.warmup + args.steps):
+        v, r, dt = time_oracle_sample(w, inp, per_step)
+        if s >= args.warmup:
+            vals.append(v); rows += r
+    value = float(np.mean(vals))
+    sample = f"{rows} random (row, KV head) pairs of {w.name} in {args.steps} steps of {per_step:.0f} s, whole oracle row each"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": per_step * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, **{k: getattr(w, k) for k in ("batch", "seq", "h_q", "h_kv", "head_dim", "block", "alpha", "gamma", "sigma")}},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="prefill_8k")
+    ap.add_argument("--no-extras", action="store_true", help="skip the SDPA / decode / long-context side measurements")
+    ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    from paper_2605_18753_b200 import synth
+    w = synth.workload(args.workload)
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    from paper_2605_18753_b200 import binding as B
+    B.lib()  # fails loudly when the CUDA library is missing: there is no other path
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+    peaks = load_peaks()
+
+    # every rank owns an independent batch of the workload (seed = rank): shards need no exchange
+    wr = w.with_(seed=w.seed + rank)
+    inp = synth.make_prefill_inputs(wr, dev)
+    Q, K, V = inp["Q"], inp["K"], inp["V"]
+    O = torch.empty_like(Q)
+    p = B.params_for_prefill(Q, K, V, O, block=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma)
+    ws = B.alloc_workspace(p, dev)
+    rt = B.alloc_routing(p, dev)
+    kbar = B.alloc_kbar(p, dev)
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
+    g_q = w.h_q // w.h_kv
+
+    def step():
+        B.dash_attn_fwd_prefill(p, Q, K, V, O, ws)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        flush.fill_(1)
+        step()
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    n0 = B.dash_attn_launch_count()
+    barrier()
+    t_wall = time.perf_counter()
+    for s in range(args.steps):
+        flush.fill_(s & 0xFF)               # evict L2 between timed iterations (outside the event bracket)
+        ev[s][0].record()
+        step()
+        ev[s][1].record()
+    barrier()
+    t_wall = time.perf_counter() - t_wall
+    launches = B.dash_attn_launch_count() - n0
+    clocks = sampler.stop()
+    assert B.dash_attn_last_status(ws) == 0, "device-side error reported by the library"
+    step_ms = [a.elapsed_time(b) for a, b in ev]
+    ms = float(np.mean(step_ms))
+    if dist is not None:
+        t = torch.tensor([ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+
+    # per-stage timing (same steps, stages called one by one through the C ABI) and workload statistics
+    stage_ms = {"summaries": [], "select": [], "attend": []}
+    for s in range(args.steps):
+        flush.fill_(s & 0xFF)
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+        e[0].record()
+        B.dash_attn_block_summaries(p, K, kbar)
+        e[1].record()
+        B.dash_attn_select(p, Q, kbar, rt["mask"], rt["count"], None, rt["blk_bias"], ws)
+        e[2].record()
+        B.dash_attn_attend_prefill(p, Q, K, V, rt["mask"], rt["blk_bias"], O, ws)
+        e[3].record()
+        torch.cuda.synchronize()
+        for k, name in enumerate(("summaries", "select", "attend")):
+            stage_ms[name].append(e[k].elapsed_time(e[k + 1]))
+    stage_ms = {k: float(np.mean(v)) for k, v in stage_ms.items()}
+    f_sel = selected_flops_from_count(rt["count"], w.block, w.head_dim, g_q)
+    sparsity = sparsity_from_count(rt["count"], w.block)
+    f_dense = 4.0 * w.head_dim * w.h_q * w.batch * w.seq * (w.seq + 1) / 2.0
+    if dist is not None:
+        t = torch.tensor([f_sel], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.SUM)
+        f_total = float(t.item())
+    else:
+        f_total = f_sel
+    value = f_total / (ms * 1e-3) / 1e12
+
+    # end to end: pinned host inputs -> device, forward, output -> pinned host, all inside the timed region
+    hQ, hK, hV = (t.cpu().pin_memory() for t in (Q, K, V))
+    hO = torch.empty_like(hQ).pin_memory()
+    dQ, dK, dV, dO = (torch.empty_like(t) for t in (Q, K, V, O))
+    pe = B.params_for_prefill(dQ, dK, dV, dO, block=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma)
+
+    def e2e_step():
+        dQ.copy_(hQ, non_blocking=True); dK.copy_(hK, non_blocking=True); dV.copy_(hV, non_blocking=True)
+        B.dash_attn_fwd_prefill(pe, dQ, dK, dV, dO, ws)
+        hO.copy_(dO, non_blocking=True)
+
+    for _ in range(3):
+        e2e_step()
+    barrier()
+    a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(args.steps):
+        e2e_step()
+    b_.record()
+    barrier()
+    e2e_ms = a.elapsed_time(b_) / args.steps
+    if dist is not None:
+        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    h2d = sum(t.numel() * t.element_size() for t in (hQ, hK, hV))
+    d2h = hO.numel() * hO.element_size()
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peak_tf = float(peaks["bf16_tflops"])
+    achieved = f_sel / (stage_ms["attend"] * 1e-3) / 1e12
+    roofline = {"bound": "tensor", "kernel": "attend_prefill (Stage 2)", "achieved": achieved, "peak": peak_tf,
+                "unit": "TFLOP/s", "frac": achieved / peak_tf, "peak_source": f"{peaks['_source']} bf16 burst",
+                "traffic": None}
+    extras = {"fwd_ms": ms, "stage_ms": stage_ms, "block_sparsity": sparsity, "selected_tflop": f_sel / 1e12,
+              "dense_causal_tflop": f_dense / 1e12, "wall_s_timed_region": t_wall}
+
+    cpu_val, cpu_rows, cpu_dt = time_oracle_sample(w, {k: v for k, v in inp.items()}, args.cpu_seconds)
+    cpu_baseline = {"value": cpu_val, "unit": UNIT, "cores": 1, "kind": "oracle",
+                    "sample": f"{cpu_rows} random (row, KV head) pairs of {w.name}, whole oracle row each, {cpu_dt:.1f} s"}
+
+    if not args.no_extras:
+        try:
+            extras.update(side_measurements(B, synth, w, Q, K, V, dev, peaks))
+        except Exception as ex:  # side numbers never break the contract line
+            extras["side_error"] = repr(ex)
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
+            "config": {"workload": w.name, "batch_per_gpu": w.batch, "seq": w.seq, "h_q": w.h_q, "h_kv": w.h_kv,
+                       "head_dim": w.head_dim, "block": w.block, "alpha": w.alpha, "gamma": w.gamma, "sigma": w.sigma,
+                       "rho": w.rho, "shift": w.shift, "l2": "256 MiB buffer written between timed iterations",
+                       "parallelism": f"independent batches x{world}"},
+            "clocks": clocks,
+            "e2e": {"value": f_total / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+            "gpu_launches": int(launches),
+            "roofline": roofline, "cpu_baseline": cpu_baseline, "extras": extras}
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def side_measurements(B, synth, w, Q, K, V, dev, peaks) -> dict:
+    """Context numbers beside the contract line: dense SDPA on the same tensors and the decode workload."""
+    out = {}
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
+
+    def timed(fn, iters=10, warm=3):
+        for _ in range(warm):
+            fn()
+        ts = []
+        for k in range(iters):
+            flush.fill_(k)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); fn(); b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        return float(np.mean(ts))
+
+    q, k, v = (t.transpose(1, 2) for t in (Q, K, V))
+    sd = lambda: torch.nn.functional.scaled_dot_product_attention(q, k, v, is_causal=True, enable_gqa=True)
+    out["sdpa_dense_ms"] = timed(sd)
+
+    # decode workload: batch 16, 131072-token cache, ~90 % sparsity
+    wd = synth.workload("decode_128k")
+    di = synth.make_decode_inputs(wd, dev)
+    qd, Kc, Vc, lens = di["Q"], di["K"], di["V"], di["kv_len"]
+    od = torch.empty_like(qd)
+    pd = B.params_for_decode(qd, Kc, Vc, od, block=wd.block, alpha=wd.alpha, gamma=wd.gamma, sigma=wd.sigma)
+    kbar = B.alloc_kbar(pd, dev)
+    out["decode_summaries_ms"] = timed(lambda: B.dash_attn_block_summaries(pd, Kc, kbar, kv_len=lens), iters=3, warm=1)
+    wsd = B.alloc_workspace(pd, dev)
+    rt = B.alloc_routing(pd, dev)
+    B.dash_attn_select(pd, qd, kbar, rt["mask"], rt["count"], rt["blk_idx"], rt["blk_bias"], wsd, kv_len=lens)
+    cnt = rt["count"].to(torch.float64)
+    g = wd.batch * wd.h_kv
+    diag = ((lens.to(torch.float64) - 1) % wd.block + 1).sum().item() * wd.h_kv
+    kv_bytes = (cnt.sum().item() * wd.block + diag) * wd.head_dim * 2 * 2
+    kbar_bytes = g * ((wd.seq - 1) // wd.block) * wd.head_dim * 4
+    t_sel = timed(lambda: B.dash_attn_select(pd, qd, kbar, rt["mask"], rt["count"], rt["blk_idx"], rt["blk_bias"], wsd, kv_len=lens))
+    t_att = timed(lambda: B.dash_attn_attend_decode(pd, qd, Kc, Vc, lens, rt["count"], rt["blk_idx"], rt["blk_bias"], od, wsd))
+    t_all = timed(lambda: B.dash_attn_fwd_decode(pd, qd, Kc, Vc, kbar, lens, od, wsd))
+    hbm = float(peaks["hbm_gbs"])
+    out["decode"] = {"workload": wd.name, "fwd_ms": t_all, "select_ms": t_sel, "attend_ms": t_att,
+                     "block_sparsity": float(1.0 - (cnt + 1).sum().item() / (g * ((wd.seq - 1) // wd.block + 1))),
+                     "bytes_touched": kv_bytes + kbar_bytes,
+                     "hbm_gbs_fwd": (kv_bytes + kbar_bytes) / (t_all * 1e-3) / 1e9,
+                     "hbm_gbs_attend_kv_only": kv_bytes / (t_att * 1e-3) / 1e9,
+                     "hbm_frac_fwd": (kv_bytes + kbar_bytes) / (t_all * 1e-3) / 1e9 / hbm,
+                     "hbm_peak_gbs": hbm}
+    kd = Kc.transpose(1, 2); vd = Vc.transpose(1, 2); q1 = qd[:, :, None, :]
+    out["decode"]["sdpa_dense_ms"] = timed(lambda: torch.nn.functional.scaled_dot_product_attention(q1, kd, vd, enable_gqa=True), iters=5)
+    return out
+
+
+if __name__ == "__main__":
+    main()

@@ -70,11 +70,9 @@ static int make_dims(const dash_params* p, Dims* dm) {
   if (dm->decode) {
     dm->list_rows = dm->T_s;
   } else {
-    Dims tmp = *dm;
     const long long n = p->seq_q;
     const long long c = n / p->block;
     dm->list_rows = (long long)p->block * c * (c - 1) / 2 + (n % p->block) * c;
-    (void)tmp;
   }
   if (select_smem_bytes(*dm, nullptr) == 0) return DASH_ERR_UNSUPPORTED;  // score rows do not fit on chip
   return DASH_OK;
@@ -154,7 +152,8 @@ int dash_attn_block_summaries(const dash_params* p, const void* K, const float* 
   Dims dm;
   int rc = make_dims(p, &dm);
   if (rc != DASH_OK) return rc;
-  if (!K || !Kbar || !aligned16(K) || !aligned16(Kbar)) return DASH_ERR_INVALID_ARG;
+  if (!K || !aligned16(K)) return DASH_ERR_INVALID_ARG;
+  if (dm.T_s > 0 && (!Kbar || !aligned16(Kbar))) return DASH_ERR_INVALID_ARG;  // no complete chunk: nothing to write
   if (qbar && (!aligned16(qbar) || qbar_chunk_stride < 0 || qbar_chunk_stride % 4 != 0)) return DASH_ERR_INVALID_ARG;
   if (first_block < 0 || first_block > dm.T_s) return DASH_ERR_INVALID_ARG;
   if (num_blocks < 0) num_blocks = dm.T_s - first_block;
@@ -170,8 +169,8 @@ int dash_attn_select(const dash_params* p, const void* Q, const float* Kbar, con
   Dims dm;
   int rc = make_dims(p, &dm);
   if (rc != DASH_OK) return rc;
-  if (!Q || !Kbar || !mask || !count || !blk_bias) return DASH_ERR_INVALID_ARG;
-  if (!aligned16(Q) || !aligned16(Kbar)) return DASH_ERR_INVALID_ARG;
+  if (!Q || !mask || !count || !aligned16(Q)) return DASH_ERR_INVALID_ARG;
+  if (dm.T_s > 0 && (!Kbar || !aligned16(Kbar) || !blk_bias)) return DASH_ERR_INVALID_ARG;
   if (!dm.decode && kv_len) return DASH_ERR_INVALID_ARG;
   WorkspaceLayout wl;
   if ((rc = check_workspace(dm, workspace, workspace_bytes, &wl)) != DASH_OK) return rc;
@@ -186,7 +185,8 @@ int dash_attn_attend_prefill(const dash_params* p, const void* Q, const void* K,
   int rc = make_dims(p, &dm);
   if (rc != DASH_OK) return rc;
   if (dm.decode) return DASH_ERR_INVALID_ARG;
-  if (!Q || !K || !V || !mask || !blk_bias || !O) return DASH_ERR_INVALID_ARG;
+  if (!Q || !K || !V || !mask || !O) return DASH_ERR_INVALID_ARG;
+  if (dm.T_s > 0 && !blk_bias) return DASH_ERR_INVALID_ARG;
   if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O)) return DASH_ERR_INVALID_ARG;
   WorkspaceLayout wl;
   if ((rc = check_workspace(dm, workspace, workspace_bytes, &wl)) != DASH_OK) return rc;
@@ -201,7 +201,8 @@ int dash_attn_attend_decode(const dash_params* p, const void* Q, const void* Kca
   int rc = make_dims(p, &dm);
   if (rc != DASH_OK) return rc;
   if (!dm.decode) return DASH_ERR_INVALID_ARG;
-  if (!Q || !Kcache || !Vcache || !count || !blk_idx || !blk_bias || !O) return DASH_ERR_INVALID_ARG;
+  if (!Q || !Kcache || !Vcache || !count || !O) return DASH_ERR_INVALID_ARG;
+  if (dm.T_s > 0 && (!blk_idx || !blk_bias)) return DASH_ERR_INVALID_ARG;
   if (!aligned16(Q) || !aligned16(Kcache) || !aligned16(Vcache) || !aligned16(O)) return DASH_ERR_INVALID_ARG;
   WorkspaceLayout wl;
   if ((rc = check_workspace(dm, workspace, workspace_bytes, &wl)) != DASH_OK) return rc;
@@ -247,9 +248,9 @@ int dash_attn_fwd_decode(const dash_params* p, const void* Q, const void* Kcache
   int rc = make_dims(p, &dm);
   if (rc != DASH_OK) return rc;
   if (!dm.decode) return DASH_ERR_INVALID_ARG;
-  if (!Q || !Kcache || !Vcache || !Kbar || !O) return DASH_ERR_INVALID_ARG;
-  if (!aligned16(Q) || !aligned16(Kcache) || !aligned16(Vcache) || !aligned16(Kbar) || !aligned16(O))
-    return DASH_ERR_INVALID_ARG;
+  if (!Q || !Kcache || !Vcache || !O) return DASH_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(Kcache) || !aligned16(Vcache) || !aligned16(O)) return DASH_ERR_INVALID_ARG;
+  if (dm.T_s > 0 && (!Kbar || !aligned16(Kbar))) return DASH_ERR_INVALID_ARG;
   WorkspaceLayout wl;
   if ((rc = check_workspace(dm, workspace, workspace_bytes, &wl)) != DASH_OK) return rc;
   if ((rc = check_device()) != DASH_OK) return rc;
