@@ -1,13 +1,472 @@
-// Stage 2, prefill, tensor-core path for sm_100a (placeholder until the tcgen05 kernel lands).
+// Stage 2, prefill, tensor-core path for sm_100a (Eq. 7 in the form of Proposition 1; Algorithm 3).
+//
+// Tile: one (batch, KV head) and TQ = 128/g_q consecutive query tokens; the 128 rows of the MMA tile are
+// (token, head-of-group) pairs, token-major.  A tile never straddles a chunk, so its rows share the own
+// chunk; it walks the UNION of its rows' routed chunks in ascending order, 64 KV tokens per step, own
+// chunk last.  A row that did not route a chunk gets bias -inf for that step (probability exactly 0), so
+// every row still attends to its own selection only.
+//
+// Warp roles (192 threads, two blocks per SM so one block's softmax overlaps the other's MMAs):
+//   warps 0-3  softmax: S (TMEM) -> registers, logit = S/sqrt(d) + bias, causal mask inside the own chunk,
+//              online softmax with a lazily moved row maximum, P (bf16) -> shared memory, rescale of the O
+//              accumulator in TMEM when the maximum moved, final O / l -> global.
+//   warp 4     producer: OR of the tile's mask words = union list; per step the TMA loads of the K and V
+//              tiles (128-byte swizzle, no multicast) and the per-token bias of the step (each lane walks
+//              its token's compact bias list with a cursor).
+//   warp 5     MMA issuer: S = Q K^T (M128 N64 K128) into one of two TMEM buffers, O += P V (M128 N128 K64),
+//              tcgen05.commit to the mbarriers that release the stages; owns the TMEM allocation.
+// Every wait is bounded; a wait that runs out raises DASH_ERR_TIMEOUT in the status word and every role
+// leaves its loop, frees TMEM and returns.
+#include <cuda.h>
+
 #include "common.cuh"
+#include "sm100_ptx.cuh"
 
 namespace dash {
 
-bool prefill_sm100_supported(const Dims&) { return false; }
+namespace {
 
-cudaError_t launch_attend_prefill_sm100(const Dims&, const void*, const void*, const void*, const uint32_t*,
-                                        const float*, void*, StatusBlock*, cudaStream_t) {
-  return cudaErrorNotSupported;
+constexpr int NKV = 64;           // KV tokens per step
+constexpr int KST = 2, VST = 2;   // ring depths
+constexpr int PF_THREADS = 192;
+constexpr int HD = 128;           // head_dim
+constexpr uint32_t TMEM_COLS = 256;  // S0 [0,64), S1 [64,128), O [128,256)
+constexpr float RESCALE_LOG2 = 8.f;  // the running maximum is moved only when it grew by more than this
+
+constexpr uint32_t Q_BYTES = 128 * HD * 2;           // 32 KiB: two 128x64 K-major regions
+constexpr uint32_t KV_TILE_BYTES = NKV * HD * 2;     // 16 KiB: two 64x64 regions
+constexpr uint32_t P_BYTES = 128 * NKV * 2;          // 16 KiB
+constexpr uint32_t OFF_Q = 0;
+constexpr uint32_t OFF_K = OFF_Q + Q_BYTES;
+constexpr uint32_t OFF_V = OFF_K + KST * KV_TILE_BYTES;
+constexpr uint32_t OFF_P = OFF_V + VST * KV_TILE_BYTES;
+constexpr uint32_t OFF_MISC = OFF_P + P_BYTES;
+constexpr int MAX_TQ = 64;
+struct Misc {
+  unsigned long long bar[16];
+  uint32_t tmem_base;
+  int n_steps;
+  int abort_flag;
+  int kvbase[VST];
+  float bias[VST][MAX_TQ];
+};
+constexpr uint32_t PF_SMEM = OFF_MISC + sizeof(Misc);
+static_assert(PF_SMEM <= 115712, "two blocks per SM need <= 113 KiB each");
+
+enum Bar { Q_FULL = 0, META, K_FULL = 2, K_EMPTY = 4, V_FULL = 6, V_EMPTY = 8, S_FULL = 10, S_EMPTY = 12, P_FULL = 14,
+           P_EMPTY = 15 };
+
+struct PrefillArgs {
+  Dims dm;
+  int TQ;            // tokens per tile
+  int n_tiles;       // tiles per (batch, KV head)
+  const uint32_t* mask;
+  const float* blk_bias;
+  __nv_bfloat16* O;
+  StatusBlock* sb;
+};
+
+__global__ void __launch_bounds__(PF_THREADS, 2)
+attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                            const __grid_constant__ CUtensorMap tmV, PrefillArgs a) {
+  extern __shared__ __align__(1024) uint8_t smem[];
+  Misc* misc = reinterpret_cast<Misc*>(smem + OFF_MISC);
+  const Dims& dm = a.dm;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t sbase = ptx::smem_u32(smem);
+  auto bar = [&](int i) { return ptx::smem_u32(&misc->bar[i]); };
+  volatile int* abort_flag = &misc->abort_flag;
+
+  const int groups = dm.batch * dm.h_kv;
+  const int tile = a.n_tiles - 1 - (int)(blockIdx.x / groups);  // late (long) tiles first
+  const int grp = (int)(blockIdx.x % groups);
+  const int b = grp / dm.h_kv, r = grp % dm.h_kv;
+  const int TQ = a.TQ, g_q = dm.g_q;
+  const int i0 = tile * TQ;
+  const int c_own = i0 / dm.B;
+  const int sub_per_blk = dm.B / NKV;                 // 64-token steps per chunk (1 or 2)
+  const int own_steps = (i0 % dm.B) / NKV + 1;        // steps of the own chunk the tile can see
+
+  if (tid == 0) {
+    if ((sbase & 1023u) != 0u) {
+      report_error(a.sb, DASH_ERR_CUDA, 100);
+      misc->abort_flag = 1;
+    } else {
+      misc->abort_flag = 0;
+    }
+    ptx::mbar_init(bar(Q_FULL), 1);
+    ptx::mbar_init(bar(META), 1);
+    for (int s = 0; s < 2; ++s) {
+      ptx::mbar_init(bar(K_FULL + s), 1);
+      ptx::mbar_init(bar(K_EMPTY + s), 1);
+      ptx::mbar_init(bar(V_FULL + s), 1);
+      ptx::mbar_init(bar(V_EMPTY + s), 1);
+      ptx::mbar_init(bar(S_FULL + s), 1);
+      ptx::mbar_init(bar(S_EMPTY + s), 128);
+    }
+    ptx::mbar_init(bar(P_FULL), 128);
+    ptx::mbar_init(bar(P_EMPTY), 1);
+    ptx::fence_barrier_init();
+  }
+  if (warp == 5) {
+    ptx::tmem_alloc(ptx::smem_u32(&misc->tmem_base), TMEM_COLS);
+    ptx::tmem_relinquish();
+    ptx::tc_fence_before();
+  }
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem = misc->tmem_base;
+
+  if (warp == 4) {
+    // =========================== producer ===========================
+    if (lane == 0) {
+      ptx::prefetch_tensormap(&tmQ);
+      ptx::prefetch_tensormap(&tmK);
+      ptx::prefetch_tensormap(&tmV);
+      ptx::mbar_arrive_expect_tx(bar(Q_FULL), Q_BYTES);
+      ptx::tma_load_4d(sbase + OFF_Q, &tmQ, bar(Q_FULL), 0, r * g_q, i0, b);
+      ptx::tma_load_4d(sbase + OFF_Q + Q_BYTES / 2, &tmQ, bar(Q_FULL), 64, r * g_q, i0, b);
+    }
+    // union of the tile's mask words (lane t owns tokens t, t+32)
+    const int n_words = (c_own >> 5) + 1;
+    const long long row0 = ((long long)b * dm.h_kv + r) * dm.seq_q;
+    const uint32_t own_word_keep = (c_own & 31) == 31 ? 0xffffffffu : ((2u << (c_own & 31)) - 1u);
+    int total = 0;
+    for (int w = 0; w < n_words; ++w) {
+      uint32_t u = 0;
+      for (int t = lane; t < TQ; t += 32)
+        if (i0 + t < dm.seq_q) u |= a.mask[(row0 + i0 + t) * dm.W + w];
+      u = __reduce_or_sync(0xffffffffu, u);
+      if (w == n_words - 1) u = (u & own_word_keep) | (1u << (c_own & 31));  // own chunk: always, and last
+      total += __popc(u);
+    }
+    // the own chunk is always in the union (its bit is set in every row); it contributes own_steps steps
+    const int n_steps = (total - 1) * sub_per_blk + own_steps;
+    if (lane == 0) {
+      misc->n_steps = n_steps;
+      ptx::mbar_arrive(bar(META));
+    }
+    // per-lane cursors into the compact bias lists of this lane's tokens
+    int cursor[2] = {0, 0};
+    long long loff[2];
+    uint32_t roww[2] = {0u, 0u};
+    for (int q = 0; q < 2; ++q) {
+      const int t = lane + 32 * q;
+      const int i = min(i0 + t, dm.seq_q - 1);
+      loff[q] = ((long long)b * dm.h_kv + r) * dm.list_rows + list_row_offset(dm, i);
+    }
+    int j = 0;
+    bool ok = true;
+    for (int w = 0; w < n_words && ok; ++w) {
+      uint32_t u = 0;
+      for (int q = 0; q < 2; ++q) {
+        const int t = lane + 32 * q;
+        roww[q] = (t < TQ && i0 + t < dm.seq_q) ? a.mask[(row0 + i0 + t) * dm.W + w] : 0u;
+        u |= roww[q];
+      }
+      u = __reduce_or_sync(0xffffffffu, u);
+      if (w == n_words - 1) u = (u & own_word_keep) | (1u << (c_own & 31));
+      while (u && ok) {
+        const int bit = __ffs(u) - 1;
+        u &= u - 1;
+        const int c = w * 32 + bit;
+        const bool own = (c == c_own);
+        float bv[2];
+        for (int q = 0; q < 2; ++q) {
+          bv[q] = -INFINITY;
+          if (own) {
+            bv[q] = 0.f;
+          } else if ((roww[q] >> bit) & 1u) {
+            bv[q] = a.blk_bias[loff[q] + cursor[q]];
+            ++cursor[q];
+          }
+        }
+        const int nsub = own ? own_steps : sub_per_blk;
+        for (int sub = 0; sub < nsub && ok; ++sub, ++j) {
+          const int ks = j % KST, vs = j % VST;
+          const int kv0 = c * dm.B + sub * NKV;
+          ok = ptx::mbar_wait(bar(K_EMPTY + ks), ((j / KST) & 1) ^ 1, abort_flag);
+          if (!ok) break;
+          if (lane == 0) {
+            ptx::mbar_arrive_expect_tx(bar(K_FULL + ks), KV_TILE_BYTES);
+            ptx::tma_load_4d(sbase + OFF_K + ks * KV_TILE_BYTES, &tmK, bar(K_FULL + ks), 0, r, kv0, b);
+            ptx::tma_load_4d(sbase + OFF_K + ks * KV_TILE_BYTES + KV_TILE_BYTES / 2, &tmK, bar(K_FULL + ks), 64, r, kv0, b);
+          }
+          ok = ptx::mbar_wait(bar(V_EMPTY + vs), ((j / VST) & 1) ^ 1, abort_flag);
+          if (!ok) break;
+          for (int q = 0; q < 2; ++q) {
+            const int t = lane + 32 * q;
+            if (t < TQ) misc->bias[vs][t] = bv[q];
+          }
+          if (lane == 0) misc->kvbase[vs] = kv0;
+          __syncwarp();
+          if (lane == 0) {
+            ptx::mbar_arrive_expect_tx(bar(V_FULL + vs), KV_TILE_BYTES);
+            ptx::tma_load_4d(sbase + OFF_V + vs * KV_TILE_BYTES, &tmV, bar(V_FULL + vs), 0, r, kv0, b);
+            ptx::tma_load_4d(sbase + OFF_V + vs * KV_TILE_BYTES + KV_TILE_BYTES / 2, &tmV, bar(V_FULL + vs), 64, r, kv0, b);
+          }
+        }
+      }
+    }
+    if (!ok && lane == 0) {
+      // a wait ran out: let the copies already issued land (bounded) before the block retires
+      for (int s = 0; s < 2; ++s) {
+        for (int k = 0; k < 200000 && !ptx::mbar_try_wait(bar(K_FULL + s), 0) && !ptx::mbar_try_wait(bar(K_FULL + s), 1); ++k) {}
+        for (int k = 0; k < 200000 && !ptx::mbar_try_wait(bar(V_FULL + s), 0) && !ptx::mbar_try_wait(bar(V_FULL + s), 1); ++k) {}
+      }
+    }
+  } else if (warp == 5) {
+    // =========================== MMA issuer ===========================
+    if (lane == 0) {
+      bool ok = ptx::mbar_wait(bar(META), 0, abort_flag);
+      const int n_steps = ok ? misc->n_steps : 0;
+      ok = ok && ptx::mbar_wait(bar(Q_FULL), 0, abort_flag);
+      constexpr uint32_t IDESC_QK = ptx::idesc_bf16_f32(128, NKV, false, false);
+      constexpr uint32_t IDESC_PV = ptx::idesc_bf16_f32(128, HD, false, true);
+      auto issue_qk = [&](int j) -> bool {
+        const int ks = j % KST, buf = j & 1;
+        if (!ptx::mbar_wait(bar(K_FULL + ks), (j / KST) & 1, abort_flag)) return false;
+        if (!ptx::mbar_wait(bar(S_EMPTY + buf), ((j >> 1) & 1) ^ 1, abort_flag)) return false;
+        ptx::tc_fence_after();
+        const uint32_t qa = sbase + OFF_Q, ka = sbase + OFF_K + ks * KV_TILE_BYTES;
+#pragma unroll
+        for (int k = 0; k < HD / 16; ++k) {
+          const uint32_t koff = (k & 3) * 32;  // 16 bf16 = 32 bytes inside the 128-byte swizzle row
+          const uint64_t ad = ptx::smem_desc_sw128(qa + (k >> 2) * (Q_BYTES / 2) + koff, 16, 1024);
+          const uint64_t bd = ptx::smem_desc_sw128(ka + (k >> 2) * (KV_TILE_BYTES / 2) + koff, 16, 1024);
+          ptx::mma_bf16_ss(tmem + buf * NKV, ad, bd, IDESC_QK, k > 0 ? 1u : 0u);
+        }
+        ptx::mma_commit(bar(S_FULL + buf));
+        ptx::mma_commit(bar(K_EMPTY + ks));
+        return true;
+      };
+      if (ok && n_steps > 0) ok = issue_qk(0);
+      for (int j = 0; j < n_steps && ok; ++j) {
+        if (j + 1 < n_steps) ok = issue_qk(j + 1);
+        if (!ok) break;
+        const int vs = j % VST;
+        ok = ptx::mbar_wait(bar(V_FULL + vs), (j / VST) & 1, abort_flag) &&
+             ptx::mbar_wait(bar(P_FULL), j & 1, abort_flag);
+        if (!ok) break;
+        ptx::tc_fence_after();
+        const uint32_t pa = sbase + OFF_P, va = sbase + OFF_V + vs * KV_TILE_BYTES;
+#pragma unroll
+        for (int k = 0; k < NKV / 16; ++k) {
+          const uint64_t ad = ptx::smem_desc_sw128(pa + k * 32, 16, 1024);
+          // V is [kv token][d]: MN-major B operand; 64-wide d blocks are KV_TILE_BYTES/2 apart
+          const uint64_t bd = ptx::smem_desc_sw128(va + k * 16 * 128, KV_TILE_BYTES / 2, 1024);
+          ptx::mma_bf16_ss(tmem + 2 * NKV, ad, bd, IDESC_PV, (j > 0 || k > 0) ? 1u : 0u);
+        }
+        ptx::mma_commit(bar(V_EMPTY + vs));
+        ptx::mma_commit(bar(P_EMPTY));
+      }
+    }
+    __syncwarp();
+  } else {
+    // =========================== softmax / epilogue ===========================
+    const int m = tid;                       // tile row = TMEM lane
+    const int t = m / g_q, hh = m % g_q;     // token in tile, head in group
+    const int i_row = i0 + t;
+    const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+    const float c1 = dm.sm_scale * 1.4426950408889634f;
+    bool ok = ptx::mbar_wait(bar(META), 0, abort_flag);
+    const int n_steps = ok ? misc->n_steps : 0;
+    float m_used = -INFINITY, l = 0.f;
+    uint8_t* prow = smem + OFF_P + m * 128;
+
+    for (int j = 0; j < n_steps && ok; ++j) {
+      const int vs = j % VST, buf = j & 1;
+      ok = ptx::mbar_wait(bar(V_FULL + vs), (j / VST) & 1, abort_flag);   // bias / kvbase of the step visible
+      if (!ok) break;
+      const float bias = misc->bias[vs][t];
+      const int kv0 = misc->kvbase[vs];
+      ok = ptx::mbar_wait(bar(S_FULL + buf), (j >> 1) & 1, abort_flag);
+      if (!ok) break;
+      ptx::tc_fence_after();
+      uint32_t sreg[64];
+      {
+        uint32_t* lo = sreg;
+        uint32_t* hi = sreg + 32;
+        DASH_TMEM_LD32(lo, lane_addr + buf * NKV);
+        DASH_TMEM_LD32(hi, lane_addr + buf * NKV + 32);
+      }
+      ptx::tmem_wait_ld();
+      ptx::tc_fence_before();
+      ptx::mbar_arrive(bar(S_EMPTY + buf));
+
+      const bool selected = bias > -INFINITY;
+      const float b2 = bias * 1.4426950408889634f;
+      const int n_vis = min(NKV, i_row - kv0 + 1);   // causal: KV token kv0 + c visible iff c < n_vis
+      float mloc = -INFINITY;
+      if (selected) {
+#pragma unroll
+        for (int c = 0; c < NKV; ++c) {
+          float x = fmaf(__uint_as_float(sreg[c]), c1, b2);
+          x = (c < n_vis) ? x : -INFINITY;
+          sreg[c] = __float_as_uint(x);
+          mloc = fmaxf(mloc, x);
+        }
+      }
+      float corr = 1.f;
+      bool moved = false;
+      if (mloc > m_used + RESCALE_LOG2 || (m_used == -INFINITY && mloc > -INFINITY)) {
+        corr = exp2f(m_used - mloc);   // 0 when nothing was accumulated yet
+        m_used = mloc;
+        moved = true;
+      }
+      l *= corr;
+      uint32_t packed[32];
+      if (selected && m_used > -INFINITY) {
+        float ls = 0.f;
+#pragma unroll
+        for (int c = 0; c < NKV; c += 2) {
+          const float p0 = exp2f(__uint_as_float(sreg[c]) - m_used);
+          const float p1 = exp2f(__uint_as_float(sreg[c + 1]) - m_used);
+          ls += p0 + p1;
+          __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
+          packed[c >> 1] = *reinterpret_cast<uint32_t*>(&h);
+        }
+        l += ls;
+      } else {
+#pragma unroll
+        for (int c = 0; c < 32; ++c) packed[c] = 0u;
+      }
+
+      // P buffer free and O stable once the previous step's PV has completed
+      ok = ptx::mbar_wait(bar(P_EMPTY), (j & 1) ^ 1, abort_flag);
+      if (!ok) break;
+      ptx::tc_fence_after();
+      if (j > 0 && __any_sync(0xffffffffu, moved)) {
+        // rescale this row of the accumulator: O *= 2^(m_old - m_new)
+#pragma unroll 1
+        for (int q = 0; q < HD / 32; ++q) {
+          uint32_t o[32];
+          DASH_TMEM_LD32(o, lane_addr + 2 * NKV + q * 32);
+          ptx::tmem_wait_ld();
+#pragma unroll
+          for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * corr);
+          DASH_TMEM_ST32(lane_addr + 2 * NKV + q * 32, o);
+        }
+        ptx::tmem_wait_st();
+      }
+      // P row -> shared memory, K-major with the 128-byte swizzle (16-byte chunk q of row m sits at q ^ (m & 7))
+#pragma unroll
+      for (int q = 0; q < 8; ++q) {
+        uint4 v = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+        *reinterpret_cast<uint4*>(prow + ((q ^ (m & 7)) << 4)) = v;
+      }
+      ptx::fence_proxy_async_smem();
+      ptx::tc_fence_before();
+      ptx::mbar_arrive(bar(P_FULL));
+    }
+
+    // epilogue: O / l -> global (row m is 128 contiguous bf16 of token i_row, head r*g_q + hh)
+    if (ok && n_steps > 0) ok = ptx::mbar_wait(bar(P_EMPTY), (n_steps - 1) & 1, abort_flag);
+    if (ok && n_steps > 0) {
+      ptx::tc_fence_after();
+      const float inv = l > 0.f ? 1.f / l : 0.f;
+      __nv_bfloat16* op = a.O + (long long)b * dm.os[0] + (long long)i_row * dm.os[1] + (long long)(r * g_q + hh) * dm.os[2];
+#pragma unroll 1
+      for (int q = 0; q < HD / 32; ++q) {
+        uint32_t o[32];
+        DASH_TMEM_LD32(o, lane_addr + 2 * NKV + q * 32);
+        ptx::tmem_wait_ld();
+        if (i_row < dm.seq_q) {
+#pragma unroll
+          for (int c = 0; c < 32; c += 8) {
+            uint4 v;
+            __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(o[c]) * inv, __uint_as_float(o[c + 1]) * inv);
+            __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(o[c + 2]) * inv, __uint_as_float(o[c + 3]) * inv);
+            __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(o[c + 4]) * inv, __uint_as_float(o[c + 5]) * inv);
+            __nv_bfloat162 h3 = __floats2bfloat162_rn(__uint_as_float(o[c + 6]) * inv, __uint_as_float(o[c + 7]) * inv);
+            v.x = *reinterpret_cast<uint32_t*>(&h0); v.y = *reinterpret_cast<uint32_t*>(&h1);
+            v.z = *reinterpret_cast<uint32_t*>(&h2); v.w = *reinterpret_cast<uint32_t*>(&h3);
+            *reinterpret_cast<uint4*>(op + q * 32 + c) = v;
+          }
+        }
+      }
+    }
+    ptx::tc_fence_before();
+  }
+
+  __syncthreads();
+  if (warp == 5) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem, TMEM_COLS);
+  }
+  if (tid == 0 && misc->abort_flag) report_error(a.sb, DASH_ERR_TIMEOUT, 101);
+}
+
+// ---------------------------------------------------------------- host side
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// [batch, tokens, heads, 128] bf16 tensor with element strides s[3]; box = 64 x box_heads x box_tokens x 1.
+bool make_map(CUtensorMap* out, const void* base, long long tokens, int heads, int batch, const long long* s,
+              int box_heads, int box_tokens) {
+  EncodeTiledFn enc = get_encode();
+  if (!enc) return false;
+  cuuint64_t dims[4] = {(cuuint64_t)HD, (cuuint64_t)heads, (cuuint64_t)tokens, (cuuint64_t)batch};
+  // a size-1 dimension may come with stride 0; any positive multiple of 16 bytes is accepted there
+  auto st = [](long long e) { return (cuuint64_t)((e > 0 ? e : 8) * 2); };
+  cuuint64_t strides[3] = {st(s[2]), st(s[1]), st(s[0])};
+  cuuint32_t box[4] = {64u, (cuuint32_t)box_heads, (cuuint32_t)box_tokens, 1u};
+  cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+  return enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+bool prefill_sm100_supported(const Dims& dm) {
+  if (dm.decode || dm.dtype != DASH_BF16 || dm.d != HD) return false;
+  if (dm.B != 64 && dm.B != 128) return false;
+  const int tq = 128 / dm.g_q;
+  if (dm.g_q < 2 || tq > MAX_TQ || tq > dm.B) return false;
+  if (dm.os[2] % 8 != 0 || dm.os[1] % 8 != 0) return false;
+  return get_encode() != nullptr;
+}
+
+cudaError_t launch_attend_prefill_sm100(const Dims& dm, const void* Q, const void* K, const void* V,
+                                        const uint32_t* mask, const float* blk_bias, void* O, StatusBlock* sb,
+                                        cudaStream_t st) {
+  PrefillArgs a;
+  a.dm = dm;
+  a.TQ = 128 / dm.g_q;
+  a.n_tiles = (dm.seq_q + a.TQ - 1) / a.TQ;
+  a.mask = mask;
+  a.blk_bias = blk_bias;
+  a.O = (__nv_bfloat16*)O;
+  a.sb = sb;
+  CUtensorMap tq, tk, tv;
+  if (!make_map(&tq, Q, dm.seq_q, dm.h_q, dm.batch, dm.qs, dm.g_q, a.TQ)) return cudaErrorInvalidValue;
+  if (!make_map(&tk, K, dm.seq_kv, dm.h_kv, dm.batch, dm.ks, 1, NKV)) return cudaErrorInvalidValue;
+  if (!make_map(&tv, V, dm.seq_kv, dm.h_kv, dm.batch, dm.vs, 1, NKV)) return cudaErrorInvalidValue;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(attend_prefill_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PF_SMEM);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  const long long blocks = (long long)a.n_tiles * dm.batch * dm.h_kv;
+  attend_prefill_sm100_kernel<<<(unsigned)blocks, PF_THREADS, PF_SMEM, st>>>(tq, tk, tv, a);
+  count_launch();
+  return cudaGetLastError();
 }
 
 }  // namespace dash
