@@ -58,7 +58,7 @@ size_t select_smem_bytes(const Dims& dm, int* tq_out) {
 // RPT rows x CPT chunks per thread; CX = 64/CPT threads along chunks, RY = 256/CX along rows.
 template <typename T, int D, int RPT, int CPT>
 __global__ void __launch_bounds__(SEL_THREADS)
-select_kernel(Dims dm, int TQ, int xs_stride, const T* __restrict__ Q, const float* __restrict__ Kbar,
+select_kernel(Dims dm, int TQ, int xs_stride, int token_base, const T* __restrict__ Q, const float* __restrict__ Kbar,
               const int* __restrict__ kv_len, uint32_t* __restrict__ mask, int* __restrict__ count,
               int* __restrict__ blk_idx, float* __restrict__ blk_bias, float* __restrict__ tau_out) {
   constexpr int CX = SEL_CT / CPT;
@@ -85,7 +85,7 @@ select_kernel(Dims dm, int TQ, int xs_stride, const T* __restrict__ Q, const flo
     c_own = (L - 1) / dm.B;
     n_cand = min(c_own, dm.T_s);
   } else {
-    i0 = tile * TQ;
+    i0 = token_base + tile * TQ;
     c_own = i0 / dm.B;
     n_cand = min(c_own, dm.T_s);
   }
@@ -249,7 +249,7 @@ select_kernel(Dims dm, int TQ, int xs_stride, const T* __restrict__ Q, const flo
 }
 
 template <typename T, int D, int RPT, int CPT>
-static cudaError_t launch_one(const Dims& dm, const SelectPlan& pl, const void* Q, const float* Kbar,
+static cudaError_t launch_one(const Dims& dm, const SelectPlan& pl, int token_base, const void* Q, const float* Kbar,
                               const int* kv_len, uint32_t* mask, int* count, int* blk_idx, float* blk_bias,
                               float* tau, cudaStream_t st) {
   auto kern = select_kernel<T, D, RPT, CPT>;
@@ -259,36 +259,46 @@ static cudaError_t launch_one(const Dims& dm, const SelectPlan& pl, const void* 
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  const int tiles = dm.decode ? 1 : (dm.seq_q + pl.TQ - 1) / pl.TQ;
+  const int tiles = dm.decode ? 1 : (dm.seq_q - token_base + pl.TQ - 1) / pl.TQ;
   dim3 grid(tiles, dm.h_kv, dm.batch);
-  kern<<<grid, SEL_THREADS, pl.smem, st>>>(dm, pl.TQ, pl.xs_stride, (const T*)Q, Kbar, kv_len, mask, count,
+  kern<<<grid, SEL_THREADS, pl.smem, st>>>(dm, pl.TQ, pl.xs_stride, token_base, (const T*)Q, Kbar, kv_len, mask, count,
                                             blk_idx, blk_bias, tau);
   count_launch();
   return cudaGetLastError();
 }
 
 template <typename T, int D>
-static cudaError_t launch_rows(const Dims& dm, const SelectPlan& pl, const void* Q, const float* Kbar,
+static cudaError_t launch_rows(const Dims& dm, const SelectPlan& pl, int token_base, const void* Q, const float* Kbar,
                                const int* kv_len, uint32_t* mask, int* count, int* blk_idx, float* blk_bias,
                                float* tau, cudaStream_t st) {
   switch (pl.r_pad) {
-    case 32: return launch_one<T, D, 2, 4>(dm, pl, Q, Kbar, kv_len, mask, count, blk_idx, blk_bias, tau, st);
-    case 16: return launch_one<T, D, 1, 4>(dm, pl, Q, Kbar, kv_len, mask, count, blk_idx, blk_bias, tau, st);
-    case 8:  return launch_one<T, D, 1, 2>(dm, pl, Q, Kbar, kv_len, mask, count, blk_idx, blk_bias, tau, st);
-    default: return launch_one<T, D, 1, 1>(dm, pl, Q, Kbar, kv_len, mask, count, blk_idx, blk_bias, tau, st);
+    case 32: return launch_one<T, D, 2, 4>(dm, pl, token_base, Q, Kbar, kv_len, mask, count, blk_idx, blk_bias, tau, st);
+    case 16: return launch_one<T, D, 1, 4>(dm, pl, token_base, Q, Kbar, kv_len, mask, count, blk_idx, blk_bias, tau, st);
+    case 8:  return launch_one<T, D, 1, 2>(dm, pl, token_base, Q, Kbar, kv_len, mask, count, blk_idx, blk_bias, tau, st);
+    default: return launch_one<T, D, 1, 1>(dm, pl, token_base, Q, Kbar, kv_len, mask, count, blk_idx, blk_bias, tau, st);
   }
 }
 
 cudaError_t launch_select(const Dims& dm, const void* Q, const float* Kbar, const int* kv_len, uint32_t* mask,
-                          int* count, int* blk_idx, float* blk_bias, float* tau, StatusBlock*, cudaStream_t st) {
+                          int* count, int* blk_idx, float* blk_bias, float* tau, void* scratch, StatusBlock* sb,
+                          cudaStream_t st) {
+  // bf16 prefill rows whose candidates fit in tensor memory go to the tcgen05 kernel; everything else
+  // (fp32, decode, very long rows) to the CUDA-core kernel below
+  int token_base = 0;
+  const int tc_tokens = scratch ? select_sm100_token_limit(dm) : 0;
+  if (tc_tokens > 0) {
+    cudaError_t e = launch_select_sm100(dm, tc_tokens, Q, Kbar, scratch, mask, count, blk_idx, blk_bias, tau, sb, st);
+    if (e != cudaSuccess || tc_tokens >= dm.seq_q) return e;
+    token_base = tc_tokens;
+  }
   SelectPlan pl;
   if (!plan_select(dm, &pl)) return cudaErrorInvalidConfiguration;
   if (dm.dtype == DASH_BF16) {
-    if (dm.d == 128) return launch_rows<__nv_bfloat16, 128>(dm, pl, Q, Kbar, kv_len, mask, count, blk_idx, blk_bias, tau, st);
-    return launch_rows<__nv_bfloat16, 64>(dm, pl, Q, Kbar, kv_len, mask, count, blk_idx, blk_bias, tau, st);
+    if (dm.d == 128) return launch_rows<__nv_bfloat16, 128>(dm, pl, token_base, Q, Kbar, kv_len, mask, count, blk_idx, blk_bias, tau, st);
+    return launch_rows<__nv_bfloat16, 64>(dm, pl, token_base, Q, Kbar, kv_len, mask, count, blk_idx, blk_bias, tau, st);
   }
-  if (dm.d == 128) return launch_rows<float, 128>(dm, pl, Q, Kbar, kv_len, mask, count, blk_idx, blk_bias, tau, st);
-  return launch_rows<float, 64>(dm, pl, Q, Kbar, kv_len, mask, count, blk_idx, blk_bias, tau, st);
+  if (dm.d == 128) return launch_rows<float, 128>(dm, pl, token_base, Q, Kbar, kv_len, mask, count, blk_idx, blk_bias, tau, st);
+  return launch_rows<float, 64>(dm, pl, token_base, Q, Kbar, kv_len, mask, count, blk_idx, blk_bias, tau, st);
 }
 
 }  // namespace dash

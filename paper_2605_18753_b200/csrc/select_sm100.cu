@@ -1,0 +1,414 @@
+// Stage 1 on tensor cores for sm_100a (Eq. 2, Eq. 4, Algorithm 2, Proposition 1), bf16 queries, head_dim 128.
+//
+// Tile = the 128 (token, head-of-group) rows of TQ = 128/g_q consecutive tokens of one (batch, KV head);
+// they share their candidate chunks.  The whole score tile X[128 rows][n_cand <= 512 chunks] is produced by
+// tcgen05.mma into tensor memory and never leaves the SM (Algorithm 2 writes it to HBM).  The fp32
+// summaries are split beforehand into three bf16 planes (hi + mid + lo = the fp32 value exactly), so that
+// Q (exact in bf16) times the three planes, accumulated in fp32, carries fp32-class accuracy: the support
+// must match a float64 evaluation except within 1e-4 of the threshold.
+//
+// Each of the 128 solver threads owns one row = one TMEM lane, so the threshold search needs no
+// cross-thread reduction: a pass streams the row out of tensor memory 32 columns at a time.  tau is found
+// by Newton's method from max(x) - 1 (f convex and decreasing: monotone from below, finite for alpha = 2).
+// The GQA group's heads sit in adjacent lanes; the group weights, the 32-chunk mask words, log w, mu and the
+// compact bias lists are formed through a small shared-memory exchange tile, one warp-synchronous step per
+// 32 chunks.  Waits are bounded as in the Stage 2 kernel.
+#include <cuda.h>
+
+#include "common.cuh"
+#include "sm100_ptx.cuh"
+
+namespace dash {
+
+namespace {
+
+constexpr int SC = 64;               // candidate chunks per MMA block / staged summary tile
+constexpr int HD = 128;
+constexpr int SEL_TC_THREADS = 192;
+constexpr uint32_t Q_BYTES = 128 * HD * 2;            // 32 KiB
+constexpr uint32_t PLANE_BYTES = SC * HD * 2;         // 16 KiB per plane per stage
+constexpr uint32_t STAGE_BYTES = 3 * PLANE_BYTES;     // hi, mid, lo
+constexpr int XCH_STRIDE = 33;
+constexpr uint32_t XCH_BYTES = 128 * XCH_STRIDE * 4;
+constexpr int MAX_NEWTON = 64, MAX_NEWTON_GENERIC = 400;
+
+struct MiscS {
+  unsigned long long bar[8];
+  uint32_t tmem_base;
+  int abort_flag;
+};
+enum BarS { Q_FULL = 0, X_FULL = 1, KB_FULL = 2, KB_EMPTY = 4 };
+
+template <int NST> struct SmemPlan {
+  static constexpr uint32_t OFF_Q = 0;
+  static constexpr uint32_t OFF_KB = Q_BYTES;
+  static constexpr uint32_t OFF_XCH = OFF_KB + NST * STAGE_BYTES;
+  static constexpr uint32_t OFF_MISC = OFF_XCH + ((XCH_BYTES + 127) / 128) * 128;
+  static constexpr uint32_t TOTAL = OFF_MISC + sizeof(MiscS);
+};
+
+struct SelectTcArgs {
+  Dims dm;
+  int TQ, n_tiles;        // tiles [0, n_tiles) of every (batch, KV head) are handled here
+  uint32_t tmem_cols;     // power of two >= 32 covering the widest tile
+  long long plane_rows;   // rows of one bf16 plane = batch * h_kv * T_s
+  uint32_t* mask;
+  int* count;
+  int* blk_idx;
+  float* blk_bias;
+  float* tau;
+  StatusBlock* sb;
+};
+
+__global__ void kbar_split_kernel(const float* __restrict__ kbar, __nv_bfloat16* __restrict__ planes, long long n) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const float x = kbar[i];
+  const __nv_bfloat16 hi = __float2bfloat16_rn(x);
+  const float r1 = x - __bfloat162float(hi);
+  const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+  const float r2 = r1 - __bfloat162float(mid);
+  planes[i] = hi;
+  planes[n + i] = mid;
+  planes[2 * n + i] = __float2bfloat16_rn(r2);
+}
+
+template <int NST>
+__global__ void __launch_bounds__(SEL_TC_THREADS)
+select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKB, SelectTcArgs a) {
+  using SP = SmemPlan<NST>;
+  extern __shared__ __align__(1024) uint8_t smem[];
+  MiscS* misc = reinterpret_cast<MiscS*>(smem + SP::OFF_MISC);
+  float* xch = reinterpret_cast<float*>(smem + SP::OFF_XCH);
+  const Dims& dm = a.dm;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t sbase = ptx::smem_u32(smem);
+  auto bar = [&](int i) { return ptx::smem_u32(&misc->bar[i]); };
+  volatile int* abort_flag = &misc->abort_flag;
+
+  const int groups = dm.batch * dm.h_kv;
+  const int tile = a.n_tiles - 1 - (int)(blockIdx.x / groups);
+  const int grp = (int)(blockIdx.x % groups);
+  const int b = grp / dm.h_kv, r = grp % dm.h_kv;
+  const int TQ = a.TQ, g_q = dm.g_q;
+  const int i0 = tile * TQ;
+  const int c_own = i0 / dm.B;
+  const int n_cand = min(c_own, dm.T_s);
+  const int n_blk = (n_cand + SC - 1) / SC;
+
+  if (tid == 0) {
+    misc->abort_flag = 0;
+    if ((sbase & 1023u) != 0u) {
+      report_error(a.sb, DASH_ERR_CUDA, 200);
+      misc->abort_flag = 1;
+    }
+    ptx::mbar_init(bar(Q_FULL), 1);
+    ptx::mbar_init(bar(X_FULL), 1);
+    for (int s = 0; s < 2; ++s) {
+      ptx::mbar_init(bar(KB_FULL + s), 1);
+      ptx::mbar_init(bar(KB_EMPTY + s), 1);
+    }
+    ptx::fence_barrier_init();
+  }
+  if (warp == 5) {
+    ptx::tmem_alloc(ptx::smem_u32(&misc->tmem_base), a.tmem_cols);
+    ptx::tmem_relinquish();
+    ptx::tc_fence_before();
+  }
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem = misc->tmem_base;
+
+  if (warp == 4) {
+    // ---------------- producer: Q tile, then the three planes of every 64-chunk block of summaries
+    if (lane == 0 && n_cand > 0) {
+      ptx::prefetch_tensormap(&tmQ);
+      ptx::prefetch_tensormap(&tmKB);
+      ptx::mbar_arrive_expect_tx(bar(Q_FULL), Q_BYTES);
+      ptx::tma_load_4d(sbase + SP::OFF_Q, &tmQ, bar(Q_FULL), 0, r * g_q, i0, b);
+      ptx::tma_load_4d(sbase + SP::OFF_Q + Q_BYTES / 2, &tmQ, bar(Q_FULL), 64, r * g_q, i0, b);
+      const long long row0 = ((long long)b * dm.h_kv + r) * dm.T_s;
+      bool ok = true;
+      for (int cb = 0; cb < n_blk && ok; ++cb) {
+        const int s = cb % NST;
+        ok = ptx::mbar_wait(bar(KB_EMPTY + s), ((cb / NST) & 1) ^ 1, abort_flag);
+        if (!ok) break;
+        ptx::mbar_arrive_expect_tx(bar(KB_FULL + s), STAGE_BYTES);
+        for (int pl = 0; pl < 3; ++pl) {
+          const uint32_t dst = sbase + SP::OFF_KB + s * STAGE_BYTES + pl * PLANE_BYTES;
+          const int row = (int)(pl * a.plane_rows + row0 + (long long)cb * SC);
+          ptx::tma_load_4d(dst, &tmKB, bar(KB_FULL + s), 0, row, 0, 0);
+          ptx::tma_load_4d(dst + PLANE_BYTES / 2, &tmKB, bar(KB_FULL + s), 64, row, 0, 0);
+        }
+      }
+      if (!ok) {
+        for (int s = 0; s < NST; ++s)
+          for (int k = 0; k < 200000 && !ptx::mbar_try_wait(bar(KB_FULL + s), 0) && !ptx::mbar_try_wait(bar(KB_FULL + s), 1); ++k) {}
+      }
+    }
+  } else if (warp == 5) {
+    // ---------------- MMA issuer: X[:, cb*64 .. +64) = Q Kbar_hi^T + Q Kbar_mid^T + Q Kbar_lo^T
+    if (lane == 0 && n_cand > 0) {
+      constexpr uint32_t IDESC = ptx::idesc_bf16_f32(128, SC, false, false);
+      bool ok = ptx::mbar_wait(bar(Q_FULL), 0, abort_flag);
+      for (int cb = 0; cb < n_blk && ok; ++cb) {
+        const int s = cb % NST;
+        ok = ptx::mbar_wait(bar(KB_FULL + s), (cb / NST) & 1, abort_flag);
+        if (!ok) break;
+        ptx::tc_fence_after();
+        const uint32_t qa = sbase + SP::OFF_Q;
+#pragma unroll
+        for (int pl = 0; pl < 3; ++pl) {
+          const uint32_t ka = sbase + SP::OFF_KB + s * STAGE_BYTES + pl * PLANE_BYTES;
+#pragma unroll
+          for (int k = 0; k < HD / 16; ++k) {
+            const uint32_t koff = (k & 3) * 32;
+            const uint64_t ad = ptx::smem_desc_sw128(qa + (k >> 2) * (Q_BYTES / 2) + koff, 16, 1024);
+            const uint64_t bd = ptx::smem_desc_sw128(ka + (k >> 2) * (PLANE_BYTES / 2) + koff, 16, 1024);
+            ptx::mma_bf16_ss(tmem + cb * SC, ad, bd, IDESC, (pl > 0 || k > 0) ? 1u : 0u);
+          }
+        }
+        ptx::mma_commit(bar(KB_EMPTY + s));
+      }
+      if (ok) ptx::mma_commit(bar(X_FULL));
+    }
+    __syncwarp();
+  } else {
+    // ---------------- solver: thread = row = TMEM lane
+    const int m = tid;
+    const int t = m / g_q, hh = m % g_q;
+    const int i = i0 + t;
+    const bool row_valid = i < dm.seq_q;
+    const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+    const int e_int = dm.e_int;
+    const float e = dm.e, xs = dm.x_scale;
+    const int n_chunks = (n_cand + 31) / 32;
+    bool ok = true;
+    float tau = 0.f;
+    if (n_cand > 0) {
+      ok = ptx::mbar_wait(bar(X_FULL), 0, abort_flag);
+      ptx::tc_fence_after();
+    }
+    if (ok && n_cand > 0) {
+      // pass 0: row maximum
+      float mx = -INFINITY;
+      for (int k = 0; k < n_chunks; ++k) {
+        uint32_t v[32];
+        DASH_TMEM_LD32(v, lane_addr + k * 32);
+        ptx::tmem_wait_ld();
+        const int lim = n_cand - k * 32;
+#pragma unroll
+        for (int c = 0; c < 32; ++c) mx = fmaxf(mx, c < lim ? __uint_as_float(v[c]) : -INFINITY);
+      }
+      mx *= xs;
+      tau = mx - 1.f;
+      bool done = false;
+      const int max_it = e_int ? MAX_NEWTON : MAX_NEWTON_GENERIC;
+      for (int it = 0; it < max_it; ++it) {
+        float f = 0.f, g = 0.f;
+        for (int k = 0; k < n_chunks; ++k) {
+          uint32_t v[32];
+          DASH_TMEM_LD32(v, lane_addr + k * 32);
+          ptx::tmem_wait_ld();
+          const int lim = n_cand - k * 32;
+#pragma unroll
+          for (int c = 0; c < 32; ++c) {
+            float mm = fmaxf(fmaf(__uint_as_float(v[c]), xs, -tau), 0.f);
+            mm = c < lim ? mm : 0.f;
+            f += pow_e(mm, e_int, e);
+            g += pow_em1(mm, e_int, e);
+          }
+        }
+        if (!done) {
+          f -= 1.f;
+          if (!(f > 0.f)) {
+            done = true;
+          } else {
+            const float nt = tau + f / (e * g);
+            if (!(nt > tau)) done = true; else tau = nt;
+          }
+        }
+        if (__all_sync(0xffffffffu, done)) break;
+      }
+    }
+    if (ok && row_valid && a.tau) a.tau[((long long)b * dm.h_q + r * g_q + hh) * dm.seq_q + i] = tau;
+
+    // ---------------- group weights, mask words, log w, compact lists (warp-synchronous, 32 chunks a step)
+    const long long row_id = ((long long)b * dm.h_kv + r) * dm.seq_q + i;
+    const long long loff = ((long long)b * dm.h_kv + r) * dm.list_rows + list_row_offset(dm, min(i, dm.seq_q - 1));
+    uint32_t* mrow = a.mask + row_id * dm.W;
+    float* xw = xch + (size_t)warp * 32 * XCH_STRIDE;        // this warp's 32 rows
+    const int lrow = lane;                                     // row inside the warp's slab
+    const int grow0 = (lane / g_q) * g_q;                      // first row of this token's group in the slab
+    const float log_gq = logf((float)g_q);
+    float slog = 0.f;
+    int nsel = 0;
+    if (ok) {
+      for (int k = 0; k < n_chunks; ++k) {
+        uint32_t v[32];
+        DASH_TMEM_LD32(v, lane_addr + k * 32);
+        ptx::tmem_wait_ld();
+        const int lim = n_cand - k * 32;
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+          float mm = fmaxf(fmaf(__uint_as_float(v[c]), xs, -tau), 0.f);
+          xw[lrow * XCH_STRIDE + c] = c < lim ? mm : 0.f;
+        }
+        __syncwarp();
+        uint32_t bits = 0;
+        float lw_own[32 / 2];      // at most 32/g_q <= 16 columns per thread
+        int n_own = 0;
+        for (int c = hh; c < 32; c += g_q, ++n_own) {
+          float mstar = 0.f;
+          for (int h2 = 0; h2 < g_q; ++h2) mstar = fmaxf(mstar, xw[(grow0 + h2) * XCH_STRIDE + c]);
+          float lw = 0.f;
+          if (mstar > 0.f) {
+            const float inv = 1.f / mstar;
+            float s = 0.f;
+            for (int h2 = 0; h2 < g_q; ++h2) s += pow_e(xw[(grow0 + h2) * XCH_STRIDE + c] * inv, e_int, e);
+            lw = e * logf(mstar) + logf(s) - log_gq;
+            bits |= 1u << c;
+            slog += lw;
+          }
+          lw_own[n_own] = lw;
+        }
+        for (int o = 1; o < g_q; o <<= 1) bits |= __shfl_xor_sync(0xffffffffu, bits, o);
+        if (row_valid) {
+          int q = 0;
+          for (int c = hh; c < 32; c += g_q, ++q) {
+            if ((bits >> c) & 1u) {
+              const long long pos = loff + nsel + __popc(bits & ((1u << c) - 1u));
+              a.blk_bias[pos] = lw_own[q];
+              if (a.blk_idx) a.blk_idx[pos] = k * 32 + c;
+            }
+          }
+          if (hh == 0) mrow[k] = bits | (((c_own >> 5) == k) ? (1u << (c_own & 31)) : 0u);
+        }
+        nsel += __popc(bits);
+        __syncwarp();
+      }
+      for (int o = 1; o < g_q; o <<= 1) slog += __shfl_xor_sync(0xffffffffu, slog, o);
+      if (row_valid) {
+        if (hh == 0) {
+          for (int j = n_chunks; j < dm.W; ++j) mrow[j] = ((c_own >> 5) == j) ? (1u << (c_own & 31)) : 0u;
+          a.count[row_id] = nsel;
+        }
+        if (nsel > 0) {
+          const float mu = slog / (float)nsel;
+          for (int p = hh; p < nsel; p += g_q) a.blk_bias[loff + p] = (a.blk_bias[loff + p] - mu) * dm.inv_sigma;
+        }
+      }
+    }
+    ptx::tc_fence_before();
+  }
+
+  __syncthreads();
+  if (warp == 5) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem, a.tmem_cols);
+  }
+  if (tid == 0 && misc->abort_flag) report_error(a.sb, DASH_ERR_TIMEOUT, 201);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+bool encode4(CUtensorMap* out, const void* base, const cuuint64_t* dims, const cuuint64_t* strides_bytes,
+             const cuuint32_t* box) {
+  EncodeTiledFn enc = get_encode();
+  if (!enc) return false;
+  cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+  return enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides_bytes, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+// Tokens [0, select_sm100_token_limit) can be routed by the tensor-core kernel (0: not applicable).
+int select_sm100_token_limit(const Dims& dm) {
+  if (dm.decode || dm.dtype != DASH_BF16 || dm.d != HD || dm.T_s < 1) return 0;
+  const int tq = 128 / dm.g_q;
+  if (dm.g_q < 2 || tq > dm.B) return 0;
+  if (get_encode() == nullptr) return 0;
+  const long long lim = (long long)(512 + 1) * dm.B;   // tiles whose own chunk index is <= 512 have <= 512 candidates
+  return (int)(lim < dm.seq_q ? lim : dm.seq_q);
+}
+
+size_t select_sm100_scratch_bytes(const Dims& dm) {
+  return (size_t)3 * dm.batch * dm.h_kv * (size_t)(dm.T_s > 0 ? dm.T_s : 1) * dm.d * sizeof(__nv_bfloat16);
+}
+
+cudaError_t launch_select_sm100(const Dims& dm, int token_limit, const void* Q, const float* Kbar, void* planes,
+                                uint32_t* mask, int* count, int* blk_idx, float* blk_bias, float* tau,
+                                StatusBlock* sb, cudaStream_t st) {
+  const long long plane_rows = (long long)dm.batch * dm.h_kv * dm.T_s;
+  const long long n = plane_rows * dm.d;
+  kbar_split_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(Kbar, (__nv_bfloat16*)planes, n);
+  count_launch();
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+
+  SelectTcArgs a;
+  a.dm = dm;
+  a.TQ = 128 / dm.g_q;
+  a.n_tiles = (token_limit + a.TQ - 1) / a.TQ;
+  a.plane_rows = plane_rows;
+  a.mask = mask; a.count = count; a.blk_idx = blk_idx; a.blk_bias = blk_bias; a.tau = tau; a.sb = sb;
+  const int max_cand = min(dm.T_s, (token_limit - 1) / dm.B);
+  uint32_t cols = 32;
+  while ((int)cols < ((max_cand + SC - 1) / SC) * SC) cols <<= 1;
+  a.tmem_cols = cols;
+
+  CUtensorMap tq, tkb;
+  {
+    cuuint64_t dims[4] = {(cuuint64_t)HD, (cuuint64_t)dm.h_q, (cuuint64_t)dm.seq_q, (cuuint64_t)dm.batch};
+    auto sb2 = [](long long el) { return (cuuint64_t)((el > 0 ? el : 8) * 2); };
+    cuuint64_t strides[3] = {sb2(dm.qs[2]), sb2(dm.qs[1]), sb2(dm.qs[0])};
+    cuuint32_t box[4] = {64u, (cuuint32_t)dm.g_q, (cuuint32_t)a.TQ, 1u};
+    if (!encode4(&tq, Q, dims, strides, box)) return cudaErrorInvalidValue;
+  }
+  {
+    cuuint64_t dims[4] = {(cuuint64_t)HD, (cuuint64_t)(3 * plane_rows), 1, 1};
+    cuuint64_t strides[3] = {(cuuint64_t)HD * 2, (cuuint64_t)(3 * plane_rows) * HD * 2, (cuuint64_t)(3 * plane_rows) * HD * 2};
+    cuuint32_t box[4] = {64u, (cuuint32_t)SC, 1u, 1u};
+    if (!encode4(&tkb, planes, dims, strides, box)) return cudaErrorInvalidValue;
+  }
+  const long long blocks = (long long)a.n_tiles * dm.batch * dm.h_kv;
+  if (cols <= 256) {
+    auto kern = select_sm100_kernel<1>;
+    static bool configured = false;
+    if (!configured) {
+      e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemPlan<1>::TOTAL);
+      if (e != cudaSuccess) return e;
+      configured = true;
+    }
+    kern<<<(unsigned)blocks, SEL_TC_THREADS, SmemPlan<1>::TOTAL, st>>>(tq, tkb, a);
+  } else {
+    auto kern = select_sm100_kernel<2>;
+    static bool configured = false;
+    if (!configured) {
+      e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemPlan<2>::TOTAL);
+      if (e != cudaSuccess) return e;
+      configured = true;
+    }
+    kern<<<(unsigned)blocks, SEL_TC_THREADS, SmemPlan<2>::TOTAL, st>>>(tq, tkb, a);
+  }
+  count_launch();
+  return cudaGetLastError();
+}
+
+}  // namespace dash
