@@ -57,7 +57,8 @@ typedef enum {
   DASH_ERR_CAPACITY = -4,    /* device side: a list or queue overran its region */
   DASH_ERR_CUDA = -5,        /* a CUDA runtime / driver call failed */
   DASH_ERR_ARCH = -6,        /* the current device is not compute capability 10.x */
-  DASH_ERR_TIMEOUT = -7      /* device side: a bounded wait (mbarrier) ran out; results are invalid */
+  DASH_ERR_TIMEOUT = -7,     /* device side: a bounded wait (mbarrier) ran out; results are invalid */
+  DASH_ERR_TOO_LARGE = -8    /* the problem needs more scratch than a *_static entry point's fixed array holds */
 } dash_status;
 
 typedef enum { DASH_F32 = 0, DASH_BF16 = 1 } dash_dtype;
@@ -133,6 +134,30 @@ int dash_attn_attend_decode(const dash_params* p, const void* Q, const void* Kca
                             const int32_t* kv_len, const int32_t* count, const int32_t* blk_idx,
                             const float* blk_bias, void* O, void* workspace, size_t workspace_bytes,
                             void* stream);
+
+/* dash_attn_attend_decode without any scratch from the caller.  (The paper has no counterpart: this is a
+ * packaging variant of the call above, computing exactly the same thing.)
+ *
+ * Who it is for: callers that cannot hand the library a workspace because they are not allowed to allocate
+ * device memory at the point of the call -- a serving loop whose memory plan was frozen at start-up, a plugin
+ * inside a host runtime that owns the allocator, code on a path where cudaMalloc's implicit device
+ * synchronisation is unacceptable.  They still pass the inputs and the output; the split-KV partial results
+ * (m, l, O per split and head), which dash_attn_attend_decode keeps in the workspace, go to a fixed 4 MiB
+ * device array that is part of the library image (every GPU that loads the library holds it until exit).
+ *
+ * Limits and rules:
+ *   - batch * h_q * n_split * (head_dim + 2) floats must fit in 4 MiB (n_split = ceil(592 / (batch*h_kv)),
+ *     clamped to [1, 32]); larger problems return DASH_ERR_TOO_LARGE and nothing is enqueued.
+ *   - The call allocates nothing (no cudaMalloc / cudaFree, no allocating library routine).  The first call
+ *     on each device looks up the array's device address (a host-side query, no allocation); make that first
+ *     call before any stream capture begins.
+ *   - All calls on a device share the one array.  Every slot a call reads it has written itself first, so
+ *     earlier contents never matter, but two calls that overlap on the GPU (different streams) race: keep
+ *     calls to this entry point ordered on one stream or otherwise serialised.
+ *   - No status word: argument errors are returned synchronously as for the other entry points. */
+int dash_attn_attend_decode_static(const dash_params* p, const void* Q, const void* Kcache, const void* Vcache,
+                                   const int32_t* kv_len, const int32_t* count, const int32_t* blk_idx,
+                                   const float* blk_bias, void* O, void* stream);
 
 /* Whole prefill forward: Stage 0 (skipped when Kbar is given), Stage 1, Stage 2.
  *   qbar / qbar_chunk_stride as in dash_attn_block_summaries (used only when Kbar == NULL).

@@ -18,11 +18,13 @@ LIB_PATH = os.path.join(_PKG, "libdash_attn.so")
 DASH_F32, DASH_BF16 = 0, 1
 DASH_OK = 0
 STATUS = {0: "DASH_OK", -1: "DASH_ERR_INVALID_ARG", -2: "DASH_ERR_UNSUPPORTED", -3: "DASH_ERR_WORKSPACE",
-          -4: "DASH_ERR_CAPACITY", -5: "DASH_ERR_CUDA", -6: "DASH_ERR_ARCH", -7: "DASH_ERR_TIMEOUT"}
+          -4: "DASH_ERR_CAPACITY", -5: "DASH_ERR_CUDA", -6: "DASH_ERR_ARCH", -7: "DASH_ERR_TIMEOUT",
+          -8: "DASH_ERR_TOO_LARGE"}
 
 EXPORTS = [
     "dash_attn_workspace_bytes", "dash_attn_list_capacity", "dash_attn_list_offset",
     "dash_attn_block_summaries", "dash_attn_select", "dash_attn_attend_prefill", "dash_attn_attend_decode",
+    "dash_attn_attend_decode_static",
     "dash_attn_fwd_prefill", "dash_attn_fwd_decode", "dash_attn_reset_status", "dash_attn_last_status",
     "dash_attn_launch_count", "dash_attn_strerror",
 ]
@@ -70,6 +72,8 @@ def lib() -> ctypes.CDLL:
         L.dash_attn_attend_prefill.argtypes = [P] + [c_void_p] * 7 + [c_size_t, c_void_p]
         L.dash_attn_attend_decode.restype = ctypes.c_int
         L.dash_attn_attend_decode.argtypes = [P] + [c_void_p] * 9 + [c_size_t, c_void_p]
+        L.dash_attn_attend_decode_static.restype = ctypes.c_int
+        L.dash_attn_attend_decode_static.argtypes = [P] + [c_void_p] * 9
         L.dash_attn_fwd_prefill.restype = ctypes.c_int
         L.dash_attn_fwd_prefill.argtypes = [P, c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_void_p, c_void_p,
                                             c_void_p, c_void_p, c_size_t, c_void_p]
@@ -226,6 +230,14 @@ def dash_attn_attend_decode(p, Q, Kc, Vc, kv_len, count, blk_idx, blk_bias, O, w
     _check(lib().dash_attn_attend_decode(ctypes.byref(p), _ptr(Q), _ptr(Kc), _ptr(Vc), _ptr(kv_len), _ptr(count),
                                          _ptr(blk_idx), _ptr(blk_bias), _ptr(O), _ptr(workspace), workspace.numel(),
                                          _stream()), "dash_attn_attend_decode")
+
+
+def dash_attn_attend_decode_static(p, Q, Kc, Vc, kv_len, count, blk_idx, blk_bias, O):
+    """Split-KV decode attention for callers that cannot allocate device memory: no workspace argument, the
+    split partials use a fixed 4 MiB array inside the library.  Calls must not overlap on the GPU."""
+    _check(lib().dash_attn_attend_decode_static(ctypes.byref(p), _ptr(Q), _ptr(Kc), _ptr(Vc), _ptr(kv_len),
+                                                _ptr(count), _ptr(blk_idx), _ptr(blk_bias), _ptr(O), _stream()),
+           "dash_attn_attend_decode_static")
 
 
 def dash_attn_fwd_prefill(p, Q, K, V, O, workspace, qbar=None, qbar_chunk_stride=0, Kbar=None, mask_out=None):

@@ -112,6 +112,9 @@ static int check_workspace(const Dims& dm, void* ws, size_t bytes, WorkspaceLayo
   return DASH_OK;
 }
 
+int validate_params(const dash_params* p, Dims* dm) { return make_dims(p, dm); }
+int validate_device() { return check_device(); }
+
 template <typename T> static T* at(void* ws, size_t off) { return reinterpret_cast<T*>(static_cast<char*>(ws) + off); }
 
 static int cuda_status(cudaError_t e) { return e == cudaSuccess ? DASH_OK : DASH_ERR_CUDA; }
@@ -294,6 +297,7 @@ const char* dash_attn_strerror(int status) {
     case DASH_ERR_CUDA: return "CUDA call failed";
     case DASH_ERR_ARCH: return "device is not compute capability 10.x";
     case DASH_ERR_TIMEOUT: return "device-side bounded wait ran out";
+    case DASH_ERR_TOO_LARGE: return "problem exceeds the fixed scratch of a *_static entry point";
     default: return "unknown status";
   }
 }

@@ -99,6 +99,9 @@ __device__ inline float pow_em1(float m, int e_int, float e) {
 }
 
 void count_launch();
+// Host-side checks shared by the entry points that live outside api.cu.
+int validate_params(const dash_params* p, Dims* dm);
+int validate_device();
 
 // Launchers (one per translation unit).  All return a cudaError_t from the launch.
 cudaError_t launch_summaries(const Dims& dm, const void* K, const float* qbar, long long qbar_chunk_stride,

@@ -7,6 +7,8 @@
 // keys for the logits and head_dim slices for the output.  Every warp's state is merged in shared
 // memory, every block writes one partial (m, l, O) per head, and a second kernel merges the partials in
 // split order, so results do not depend on scheduling.  Only the selected chunks' K and V rows are read.
+#include <mutex>
+
 #include "common.cuh"
 
 namespace dash {
@@ -228,3 +230,57 @@ cudaError_t launch_attend_decode(const Dims& dm, const void* Q, const void* K, c
 }
 
 }  // namespace dash
+
+// ---------------------------------------------------------------------------------------------------
+// dash_attn_attend_decode_static: the same split-KV decode attention with NO caller-provided scratch.
+// The per-split partial results (m, l, O) live in the fixed device array below instead of a workspace.
+// ---------------------------------------------------------------------------------------------------
+namespace dash {
+
+constexpr size_t DECODE_STATIC_MAX_FLOATS = (size_t)1 << 20;  // 4 MiB, held by every GPU that loads the library
+static __device__ __align__(256) float g_decode_static_scratch[DECODE_STATIC_MAX_FLOATS];
+
+// In host code the array's name is only a handle; the device address has to be asked for, once per device,
+// with that device current.
+static cudaError_t decode_static_scratch(float** out) {
+  static std::mutex mu;
+  static float* per_device[64] = {};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!per_device[dev]) {
+    float* ptr = nullptr;
+    e = cudaGetSymbolAddress((void**)&ptr, g_decode_static_scratch);
+    if (e != cudaSuccess) return e;
+    per_device[dev] = ptr;
+  }
+  *out = per_device[dev];
+  return cudaSuccess;
+}
+
+}  // namespace dash
+
+extern "C" int dash_attn_attend_decode_static(const dash_params* p, const void* Q, const void* Kcache,
+                                              const void* Vcache, const int32_t* kv_len, const int32_t* count,
+                                              const int32_t* blk_idx, const float* blk_bias, void* O, void* stream) {
+  using namespace dash;
+  Dims dm;
+  int rc = validate_params(p, &dm);
+  if (rc != DASH_OK) return rc;
+  if (!dm.decode) return DASH_ERR_INVALID_ARG;
+  if (!Q || !Kcache || !Vcache || !count || !O) return DASH_ERR_INVALID_ARG;
+  if (dm.T_s > 0 && (!blk_idx || !blk_bias)) return DASH_ERR_INVALID_ARG;
+  const uintptr_t bits = (uintptr_t)Q | (uintptr_t)Kcache | (uintptr_t)Vcache | (uintptr_t)O;
+  if (bits & 15) return DASH_ERR_INVALID_ARG;
+  if (decode_partial_bytes(dm) > DECODE_STATIC_MAX_FLOATS * sizeof(float)) return DASH_ERR_TOO_LARGE;
+  if ((rc = validate_device()) != DASH_OK) return rc;
+  float* scratch = nullptr;
+  if (decode_static_scratch(&scratch) != cudaSuccess) return DASH_ERR_CUDA;
+  // every partial slot that the merge kernel reads is written by the split kernel of the same call,
+  // so nothing left over from an earlier call needs clearing
+  return launch_attend_decode(dm, Q, Kcache, Vcache, kv_len, count, blk_idx, blk_bias, O, scratch,
+                              (cudaStream_t)stream) == cudaSuccess ? DASH_OK : DASH_ERR_CUDA;
+}
+
