@@ -294,19 +294,21 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
       ptx::tc_fence_before();
       ptx::mbar_arrive(bar(S_EMPTY + buf));
 
+      // logit (log2 domain) = s*c1 + b2; c1 > 0, so the row maximum can be taken on the raw scores
       const bool selected = bias > -INFINITY;
       const float b2 = bias * 1.4426950408889634f;
-      const int n_vis = min(NKV, i_row - kv0 + 1);   // causal: KV token kv0 + c visible iff c < n_vis
-      float mloc = -INFINITY;
+      const int n_vis = i_row - kv0 + 1;             // causal: KV token kv0 + c visible iff c < n_vis
+      float mr = -INFINITY;
       if (selected) {
+        if (n_vis < NKV) {                           // only inside the own chunk
 #pragma unroll
-        for (int c = 0; c < NKV; ++c) {
-          float x = fmaf(__uint_as_float(sreg[c]), c1, b2);
-          x = (c < n_vis) ? x : -INFINITY;
-          sreg[c] = __float_as_uint(x);
-          mloc = fmaxf(mloc, x);
+          for (int c = 0; c < NKV; ++c)
+            if (c >= n_vis) sreg[c] = 0xff800000u;   // -inf
         }
+#pragma unroll
+        for (int c = 0; c < NKV; ++c) mr = fmaxf(mr, __uint_as_float(sreg[c]));
       }
+      const float mloc = fmaf(mr, c1, b2);           // -inf when not selected
       float corr = 1.f;
       bool moved = false;
       if (mloc > m_used + RESCALE_LOG2 || (m_used == -INFINITY && mloc > -INFINITY)) {
@@ -316,17 +318,19 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
       }
       l *= corr;
       uint32_t packed[32];
-      if (selected && m_used > -INFINITY) {
-        float ls = 0.f;
+      if (selected) {
+        const float off = b2 - m_used;
+        float ls0 = 0.f, ls1 = 0.f;
 #pragma unroll
         for (int c = 0; c < NKV; c += 2) {
-          const float p0 = exp2f(__uint_as_float(sreg[c]) - m_used);
-          const float p1 = exp2f(__uint_as_float(sreg[c + 1]) - m_used);
-          ls += p0 + p1;
+          const float p0 = exp2f(fmaf(__uint_as_float(sreg[c]), c1, off));
+          const float p1 = exp2f(fmaf(__uint_as_float(sreg[c + 1]), c1, off));
+          ls0 += p0;
+          ls1 += p1;
           __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
           packed[c >> 1] = *reinterpret_cast<uint32_t*>(&h);
         }
-        l += ls;
+        l += ls0 + ls1;
       } else {
 #pragma unroll
         for (int c = 0; c < 32; ++c) packed[c] = 0u;

@@ -67,9 +67,9 @@ WORKLOADS = {
                            rho=0.72, shift=2.0),
     # C3: prefill 64K at ~75 % and ~90 %
     "prefill_64k_s75": Workload("prefill_64k_s75", "prefill", 1, 65536, 32, 8, 128, 64, 1.5, "bf16", "planted",
-                                rho=0.72, shift=1.49),
+                                rho=0.72, shift=1.56),
     "prefill_64k_s90": Workload("prefill_64k_s90", "prefill", 1, 65536, 32, 8, 128, 64, 1.5, "bf16", "planted",
-                                rho=0.72, shift=1.95),
+                                rho=0.72, shift=2.10),
     # C4: decode, batch 16, 131072-token cache, ~90 %
     "decode_128k": Workload("decode_128k", "decode", 16, 131072, 32, 8, 128, 64, 1.5, "bf16", "planted",
                             rho=0.72, shift=1.42),
