@@ -26,8 +26,10 @@ namespace dash {
 
 namespace {
 
+constexpr bool P_TMEM = true;     // P (bf16) reaches the PV MMA through tensor memory (over the S columns), not smem
+constexpr bool QK_FIRST = true;   // issue S of step j+1 before PV of step j even if its K tile has to be waited for
 constexpr int NKV = 64;           // KV tokens per step
-constexpr int KST = 2, VST = 2;   // ring depths
+constexpr int KST = 3, VST = 2;   // ring depths
 constexpr int PF_THREADS = 192;
 constexpr int HD = 128;           // head_dim
 constexpr uint32_t TMEM_COLS = 256;  // S0 [0,64), S1 [64,128), O [128,256)
@@ -35,15 +37,17 @@ constexpr float RESCALE_LOG2 = 8.f;  // the running maximum is moved only when i
 
 constexpr uint32_t Q_BYTES = 128 * HD * 2;           // 32 KiB: two 128x64 K-major regions
 constexpr uint32_t KV_TILE_BYTES = NKV * HD * 2;     // 16 KiB: two 64x64 regions
-constexpr uint32_t P_BYTES = 128 * NKV * 2;          // 16 KiB
+constexpr uint32_t P_BYTES = P_TMEM ? 0 : 128 * NKV * 2;   // 16 KiB when P goes through shared memory
 constexpr uint32_t OFF_Q = 0;
 constexpr uint32_t OFF_K = OFF_Q + Q_BYTES;
 constexpr uint32_t OFF_V = OFF_K + KST * KV_TILE_BYTES;
 constexpr uint32_t OFF_P = OFF_V + VST * KV_TILE_BYTES;
 constexpr uint32_t OFF_MISC = OFF_P + P_BYTES;
 constexpr int MAX_TQ = 64;
+enum Bar { Q_FULL = 0, META, S_FULL = 2, S_EMPTY = 4, P_FULL = 6, P_EMPTY = 8, V_FULL = 9, V_EMPTY = 9 + VST,
+           K_FULL = 9 + 2 * VST, K_EMPTY = 9 + 2 * VST + KST, N_BARS = 9 + 2 * VST + 2 * KST };
 struct Misc {
-  unsigned long long bar[16];
+  unsigned long long bar[N_BARS];
   uint32_t tmem_base;
   int n_steps;
   int abort_flag;
@@ -53,8 +57,6 @@ struct Misc {
 constexpr uint32_t PF_SMEM = OFF_MISC + sizeof(Misc);
 static_assert(PF_SMEM <= 115712, "two blocks per SM need <= 113 KiB each");
 
-enum Bar { Q_FULL = 0, META, K_FULL = 2, K_EMPTY = 4, V_FULL = 6, V_EMPTY = 8, S_FULL = 10, S_EMPTY = 12, P_FULL = 14,
-           P_EMPTY = 15 };
 
 struct PrefillArgs {
   Dims dm;
@@ -97,14 +99,21 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
     ptx::mbar_init(bar(Q_FULL), 1);
     ptx::mbar_init(bar(META), 1);
     for (int s = 0; s < 2; ++s) {
-      ptx::mbar_init(bar(K_FULL + s), 1);
-      ptx::mbar_init(bar(K_EMPTY + s), 1);
-      ptx::mbar_init(bar(V_FULL + s), 1);
-      ptx::mbar_init(bar(V_EMPTY + s), 1);
       ptx::mbar_init(bar(S_FULL + s), 1);
       ptx::mbar_init(bar(S_EMPTY + s), 128);
     }
+    for (int s = 0; s < KST; ++s) {
+      ptx::mbar_init(bar(K_FULL + s), 1);
+      ptx::mbar_init(bar(K_EMPTY + s), 1);
+    }
+    for (int s = 0; s < VST; ++s) {
+      ptx::mbar_init(bar(V_FULL + s), 1);
+      ptx::mbar_init(bar(V_EMPTY + s), 1);
+    }
+    // two P_FULL barriers (step parity): the softmax warps may finish step j+1 before the MMA thread has
+    // looked at step j, and a single barrier's phase bit cannot tell j from j+2
     ptx::mbar_init(bar(P_FULL), 128);
+    ptx::mbar_init(bar(P_FULL + 1), 128);
     ptx::mbar_init(bar(P_EMPTY), 1);
     ptx::fence_barrier_init();
   }
@@ -146,74 +155,122 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
       misc->n_steps = n_steps;
       ptx::mbar_arrive(bar(META));
     }
-    // per-lane cursors into the compact bias lists of this lane's tokens
+    // per-lane cursors into the compact bias lists of this lane's tokens (lane t owns tokens t and t+32)
     int cursor[2] = {0, 0};
     long long loff[2];
-    uint32_t roww[2] = {0u, 0u};
     for (int q = 0; q < 2; ++q) {
       const int t = lane + 32 * q;
       const int i = min(i0 + t, dm.seq_q - 1);
       loff[q] = ((long long)b * dm.h_kv + r) * dm.list_rows + list_row_offset(dm, i);
     }
-    int j = 0;
-    bool ok = true;
-    for (int w = 0; w < n_words && ok; ++w) {
-      uint32_t u = 0;
+    auto load_rows = [&](int w, uint32_t* rw) {
       for (int q = 0; q < 2; ++q) {
         const int t = lane + 32 * q;
-        roww[q] = (t < TQ && i0 + t < dm.seq_q) ? a.mask[(row0 + i0 + t) * dm.W + w] : 0u;
-        u |= roww[q];
+        rw[q] = (t < TQ && i0 + t < dm.seq_q) ? a.mask[(row0 + i0 + t) * dm.W + w] : 0u;
       }
-      u = __reduce_or_sync(0xffffffffu, u);
+    };
+    auto union_of = [&](int w, const uint32_t* rw) -> uint32_t {
+      uint32_t u = __reduce_or_sync(0xffffffffu, rw[0] | rw[1]);
       if (w == n_words - 1) u = (u & own_word_keep) | (1u << (c_own & 31));
-      while (u && ok) {
-        const int bit = __ffs(u) - 1;
-        u &= u - 1;
-        const int c = w * 32 + bit;
-        const bool own = (c == c_own);
-        float bv[2];
+      return u;
+    };
+    // Bias list entries are consumed in order, so every lane keeps the next 4..8 entries of each of its
+    // rows in registers (two groups of four; the second group is loading while the first is consumed).
+    // A dependent global read per step would otherwise put a DRAM latency on every step of the walk.
+    float bq[2][4], bn[2][4];
+    int taken[2] = {0, 0};                 // entries of the current group already handed out
+    const int row_cap = c_own;             // list entries a row can hold (= its candidate count)
+    auto load_group = [&](int q, int first, float* dst) {
+#pragma unroll
+      for (int k = 0; k < 4; ++k) dst[k] = (first + k < row_cap) ? __ldg(a.blk_bias + loff[q] + first + k) : 0.f;
+    };
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+      load_group(q, 0, bq[q]);
+      load_group(q, 4, bn[q]);
+    }
+    auto take = [&](int q) -> float {
+      const int k = taken[q];
+      const float v = k == 0 ? bq[q][0] : k == 1 ? bq[q][1] : k == 2 ? bq[q][2] : bq[q][3];
+      ++cursor[q];
+      if (++taken[q] == 4) {
+        taken[q] = 0;
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) bq[q][kk] = bn[q][kk];
+        load_group(q, cursor[q] + 4, bn[q]);
+      }
+      return v;
+    };
+    // The walk is a generator of (chunk, per-token bias) pairs; mask words are read one word ahead.
+    struct Blk { int c; float bv[2]; };
+    int w = 0;
+    uint32_t rw[2], rw_n[2] = {0u, 0u};
+    load_rows(0, rw);
+    uint32_t u = union_of(0, rw);
+    if (n_words > 1) load_rows(1, rw_n);
+    auto pop = [&](Blk& out) -> bool {
+      while (u == 0u) {
+        if (++w >= n_words) return false;
+        rw[0] = rw_n[0]; rw[1] = rw_n[1];
+        u = union_of(w, rw);
+        if (w + 1 < n_words) load_rows(w + 1, rw_n);
+      }
+      const int bit = __ffs(u) - 1;
+      u &= u - 1;
+      out.c = w * 32 + bit;
+#pragma unroll
+      for (int q = 0; q < 2; ++q) {
+        out.bv[q] = -INFINITY;
+        if (out.c == c_own) {
+          out.bv[q] = 0.f;
+        } else if ((rw[q] >> bit) & 1u) {
+          out.bv[q] = take(q);
+        }
+      }
+      return true;
+    };
+    int j = 0, ks = 0, kph = 1, vs = 0, vph = 1;   // ring slots and the parity to wait for on the empty barriers
+    bool ok = true;
+    Blk cur, nxt;
+    bool has = pop(nxt);
+    while (has && ok) {
+      cur = nxt;
+      has = pop(nxt);
+      const int nsub = (cur.c == c_own) ? own_steps : sub_per_blk;
+      for (int sub = 0; sub < nsub && ok; ++sub, ++j) {
+        const int kv0 = cur.c * dm.B + sub * NKV;
+        ok = ptx::mbar_wait(bar(K_EMPTY + ks), kph, abort_flag);
+        if (!ok) break;
+        if (lane == 0) {
+          const uint32_t dst = sbase + OFF_K + ks * KV_TILE_BYTES;
+          ptx::mbar_arrive_expect_tx(bar(K_FULL + ks), KV_TILE_BYTES);
+          ptx::tma_load_4d(dst, &tmK, bar(K_FULL + ks), 0, r, kv0, b);
+          ptx::tma_load_4d(dst + KV_TILE_BYTES / 2, &tmK, bar(K_FULL + ks), 64, r, kv0, b);
+        }
+        if (++ks == KST) { ks = 0; kph ^= 1; }
+        ok = ptx::mbar_wait(bar(V_EMPTY + vs), vph, abort_flag);
+        if (!ok) break;
         for (int q = 0; q < 2; ++q) {
-          bv[q] = -INFINITY;
-          if (own) {
-            bv[q] = 0.f;
-          } else if ((roww[q] >> bit) & 1u) {
-            bv[q] = a.blk_bias[loff[q] + cursor[q]];
-            ++cursor[q];
-          }
+          const int t = lane + 32 * q;
+          if (t < TQ) misc->bias[vs][t] = cur.bv[q];
         }
-        const int nsub = own ? own_steps : sub_per_blk;
-        for (int sub = 0; sub < nsub && ok; ++sub, ++j) {
-          const int ks = j % KST, vs = j % VST;
-          const int kv0 = c * dm.B + sub * NKV;
-          ok = ptx::mbar_wait(bar(K_EMPTY + ks), ((j / KST) & 1) ^ 1, abort_flag);
-          if (!ok) break;
-          if (lane == 0) {
-            ptx::mbar_arrive_expect_tx(bar(K_FULL + ks), KV_TILE_BYTES);
-            ptx::tma_load_4d(sbase + OFF_K + ks * KV_TILE_BYTES, &tmK, bar(K_FULL + ks), 0, r, kv0, b);
-            ptx::tma_load_4d(sbase + OFF_K + ks * KV_TILE_BYTES + KV_TILE_BYTES / 2, &tmK, bar(K_FULL + ks), 64, r, kv0, b);
-          }
-          ok = ptx::mbar_wait(bar(V_EMPTY + vs), ((j / VST) & 1) ^ 1, abort_flag);
-          if (!ok) break;
-          for (int q = 0; q < 2; ++q) {
-            const int t = lane + 32 * q;
-            if (t < TQ) misc->bias[vs][t] = bv[q];
-          }
-          if (lane == 0) misc->kvbase[vs] = kv0;
-          __syncwarp();
-          if (lane == 0) {
-            ptx::mbar_arrive_expect_tx(bar(V_FULL + vs), KV_TILE_BYTES);
-            ptx::tma_load_4d(sbase + OFF_V + vs * KV_TILE_BYTES, &tmV, bar(V_FULL + vs), 0, r, kv0, b);
-            ptx::tma_load_4d(sbase + OFF_V + vs * KV_TILE_BYTES + KV_TILE_BYTES / 2, &tmV, bar(V_FULL + vs), 64, r, kv0, b);
-          }
+        if (lane == 0) misc->kvbase[vs] = kv0;
+        __syncwarp();
+        if (lane == 0) {
+          const uint32_t dst = sbase + OFF_V + vs * KV_TILE_BYTES;
+          ptx::mbar_arrive_expect_tx(bar(V_FULL + vs), KV_TILE_BYTES);
+          ptx::tma_load_4d(dst, &tmV, bar(V_FULL + vs), 0, r, kv0, b);
+          ptx::tma_load_4d(dst + KV_TILE_BYTES / 2, &tmV, bar(V_FULL + vs), 64, r, kv0, b);
         }
+        if (++vs == VST) { vs = 0; vph ^= 1; }
       }
     }
     if (!ok && lane == 0) {
       // a wait ran out: let the copies already issued land (bounded) before the block retires
-      for (int s = 0; s < 2; ++s) {
+      for (int s = 0; s < KST; ++s)
         for (int k = 0; k < 200000 && !ptx::mbar_try_wait(bar(K_FULL + s), 0) && !ptx::mbar_try_wait(bar(K_FULL + s), 1); ++k) {}
+      for (int s = 0; s < VST; ++s)
         for (int k = 0; k < 200000 && !ptx::mbar_try_wait(bar(V_FULL + s), 0) && !ptx::mbar_try_wait(bar(V_FULL + s), 1); ++k) {}
-      }
     }
   } else if (warp == 5) {
     // =========================== MMA issuer ===========================
@@ -223,42 +280,63 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
       ok = ok && ptx::mbar_wait(bar(Q_FULL), 0, abort_flag);
       constexpr uint32_t IDESC_QK = ptx::idesc_bf16_f32(128, NKV, false, false);
       constexpr uint32_t IDESC_PV = ptx::idesc_bf16_f32(128, HD, false, true);
+      // Descriptors differ only in the 14-bit start-address field (16-byte units, no carry into the next
+      // field): build them once, then a single add per MMA keeps the issuing thread's instruction stream short.
+      const uint64_t qd0 = ptx::smem_desc_sw128(sbase + OFF_Q, 16, 1024);
+      const uint64_t kd0 = ptx::smem_desc_sw128(sbase + OFF_K, 16, 1024);
+      const uint64_t vd0 = ptx::smem_desc_sw128(sbase + OFF_V, KV_TILE_BYTES / 2, 1024);
+      const uint64_t pd0 = ptx::smem_desc_sw128(sbase + OFF_P, 16, 1024);
+      int ks_q = 0, kph_q = 0;   // ring slot / phase of the next QK
       auto issue_qk = [&](int j) -> bool {
-        const int ks = j % KST, buf = j & 1;
-        if (!ptx::mbar_wait(bar(K_FULL + ks), (j / KST) & 1, abort_flag)) return false;
-        if (!ptx::mbar_wait(bar(S_EMPTY + buf), ((j >> 1) & 1) ^ 1, abort_flag)) return false;
+        const int buf = j & 1;
+        if (!ptx::mbar_wait(bar(K_FULL + ks_q), kph_q, abort_flag)) return false;
+        // with P in tensor memory the S/P buffer is recycled in MMA issue order (PV of step j-2 precedes this QK)
+        if (!P_TMEM && !ptx::mbar_wait(bar(S_EMPTY + buf), ((j >> 1) & 1) ^ 1, abort_flag)) return false;
         ptx::tc_fence_after();
-        const uint32_t qa = sbase + OFF_Q, ka = sbase + OFF_K + ks * KV_TILE_BYTES;
+        const uint64_t kd = kd0 + (uint64_t)((ks_q * KV_TILE_BYTES) >> 4);
+        const uint32_t d_tmem = tmem + buf * NKV;
 #pragma unroll
         for (int k = 0; k < HD / 16; ++k) {
-          const uint32_t koff = (k & 3) * 32;  // 16 bf16 = 32 bytes inside the 128-byte swizzle row
-          const uint64_t ad = ptx::smem_desc_sw128(qa + (k >> 2) * (Q_BYTES / 2) + koff, 16, 1024);
-          const uint64_t bd = ptx::smem_desc_sw128(ka + (k >> 2) * (KV_TILE_BYTES / 2) + koff, 16, 1024);
-          ptx::mma_bf16_ss(tmem + buf * NKV, ad, bd, IDESC_QK, k > 0 ? 1u : 0u);
+          // 16 bf16 = 32 bytes inside the 128-byte swizzle row; the second 64 columns live in the next region
+          const uint64_t ad = qd0 + (uint64_t)(((k >> 2) * (Q_BYTES / 2) + (k & 3) * 32) >> 4);
+          const uint64_t bd = kd + (uint64_t)(((k >> 2) * (KV_TILE_BYTES / 2) + (k & 3) * 32) >> 4);
+          ptx::mma_bf16_ss(d_tmem, ad, bd, IDESC_QK, k > 0 ? 1u : 0u);
         }
         ptx::mma_commit(bar(S_FULL + buf));
-        ptx::mma_commit(bar(K_EMPTY + ks));
+        ptx::mma_commit(bar(K_EMPTY + ks_q));
+        if (++ks_q == KST) { ks_q = 0; kph_q ^= 1; }
         return true;
       };
       if (ok && n_steps > 0) ok = issue_qk(0);
+      int vs = 0, vph = 0;
       for (int j = 0; j < n_steps && ok; ++j) {
-        if (j + 1 < n_steps) ok = issue_qk(j + 1);
+        // S of the next step first (its K tile is normally resident), then this step's PV
+        bool qk_done = j + 1 >= n_steps;
+        if (!qk_done && (QK_FIRST || ptx::mbar_try_wait(bar(K_FULL + ks_q), kph_q))) {
+          ok = issue_qk(j + 1);
+          qk_done = true;
+        }
         if (!ok) break;
-        const int vs = j % VST;
-        ok = ptx::mbar_wait(bar(V_FULL + vs), (j / VST) & 1, abort_flag) &&
-             ptx::mbar_wait(bar(P_FULL), j & 1, abort_flag);
+        const int pbuf = j & 1;
+        ok = ptx::mbar_wait(bar(V_FULL + vs), vph, abort_flag) &&
+             ptx::mbar_wait(bar(P_FULL + pbuf), (j >> 1) & 1, abort_flag);
         if (!ok) break;
         ptx::tc_fence_after();
-        const uint32_t pa = sbase + OFF_P, va = sbase + OFF_V + vs * KV_TILE_BYTES;
+        // V is [kv token][d]: MN-major B operand; 64-wide d blocks are KV_TILE_BYTES/2 apart; 16 tokens = 2048 bytes
+        const uint64_t vd = vd0 + (uint64_t)((vs * KV_TILE_BYTES) >> 4);
+        const uint32_t p_tmem = tmem + pbuf * NKV;
 #pragma unroll
         for (int k = 0; k < NKV / 16; ++k) {
-          const uint64_t ad = ptx::smem_desc_sw128(pa + k * 32, 16, 1024);
-          // V is [kv token][d]: MN-major B operand; 64-wide d blocks are KV_TILE_BYTES/2 apart
-          const uint64_t bd = ptx::smem_desc_sw128(va + k * 16 * 128, KV_TILE_BYTES / 2, 1024);
-          ptx::mma_bf16_ss(tmem + 2 * NKV, ad, bd, IDESC_PV, (j > 0 || k > 0) ? 1u : 0u);
+          const uint64_t bd = vd + (uint64_t)((k * 16 * 128) >> 4);
+          if (P_TMEM)  // A = P from tensor memory: 16 bf16 per K step = 8 packed columns
+            ptx::mma_bf16_ts(tmem + 2 * NKV, p_tmem + k * 8, bd, IDESC_PV, (j > 0 || k > 0) ? 1u : 0u);
+          else
+            ptx::mma_bf16_ss(tmem + 2 * NKV, pd0 + (uint64_t)((k * 32) >> 4), bd, IDESC_PV, (j > 0 || k > 0) ? 1u : 0u);
         }
         ptx::mma_commit(bar(V_EMPTY + vs));
         ptx::mma_commit(bar(P_EMPTY));
+        if (++vs == VST) { vs = 0; vph ^= 1; }
+        if (!qk_done) ok = issue_qk(j + 1);
       }
     }
     __syncwarp();
@@ -274,12 +352,14 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
     float m_used = -INFINITY, l = 0.f;
     uint8_t* prow = smem + OFF_P + m * 128;
 
+    int vs = 0, vph = 0;
     for (int j = 0; j < n_steps && ok; ++j) {
-      const int vs = j % VST, buf = j & 1;
-      ok = ptx::mbar_wait(bar(V_FULL + vs), (j / VST) & 1, abort_flag);   // bias / kvbase of the step visible
+      const int buf = j & 1;
+      ok = ptx::mbar_wait(bar(V_FULL + vs), vph, abort_flag);   // bias / kvbase of the step visible
       if (!ok) break;
       const float bias = misc->bias[vs][t];
       const int kv0 = misc->kvbase[vs];
+      if (++vs == VST) { vs = 0; vph ^= 1; }
       ok = ptx::mbar_wait(bar(S_FULL + buf), (j >> 1) & 1, abort_flag);
       if (!ok) break;
       ptx::tc_fence_after();
@@ -291,8 +371,10 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
         DASH_TMEM_LD32(hi, lane_addr + buf * NKV + 32);
       }
       ptx::tmem_wait_ld();
-      ptx::tc_fence_before();
-      ptx::mbar_arrive(bar(S_EMPTY + buf));
+      if (!P_TMEM) {
+        ptx::tc_fence_before();
+        ptx::mbar_arrive(bar(S_EMPTY + buf));
+      }
 
       // logit (log2 domain) = s*c1 + b2; c1 > 0, so the row maximum can be taken on the raw scores
       const bool selected = bias > -INFINITY;
@@ -306,7 +388,12 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
             if (c >= n_vis) sreg[c] = 0xff800000u;   // -inf
         }
 #pragma unroll
-        for (int c = 0; c < NKV; ++c) mr = fmaxf(mr, __uint_as_float(sreg[c]));
+        for (int c = 0; c < 8; ++c) {   // eight independent chains, then a tree
+          float a = __uint_as_float(sreg[c]);
+#pragma unroll
+          for (int k = 8; k < NKV; k += 8) a = fmaxf(a, __uint_as_float(sreg[c + k]));
+          mr = fmaxf(mr, a);
+        }
       }
       const float mloc = fmaf(mr, c1, b2);           // -inf when not selected
       float corr = 1.f;
@@ -320,27 +407,29 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
       uint32_t packed[32];
       if (selected) {
         const float off = b2 - m_used;
-        float ls0 = 0.f, ls1 = 0.f;
+        float lsum[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int c = 0; c < NKV; c += 2) {
           const float p0 = exp2f(fmaf(__uint_as_float(sreg[c]), c1, off));
           const float p1 = exp2f(fmaf(__uint_as_float(sreg[c + 1]), c1, off));
-          ls0 += p0;
-          ls1 += p1;
+          lsum[(c >> 1) & 7] += p0 + p1;
           __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
           packed[c >> 1] = *reinterpret_cast<uint32_t*>(&h);
         }
-        l += ls0 + ls1;
+        l += ((lsum[0] + lsum[1]) + (lsum[2] + lsum[3])) + ((lsum[4] + lsum[5]) + (lsum[6] + lsum[7]));
       } else {
 #pragma unroll
         for (int c = 0; c < 32; ++c) packed[c] = 0u;
       }
 
-      // P buffer free and O stable once the previous step's PV has completed
-      ok = ptx::mbar_wait(bar(P_EMPTY), (j & 1) ^ 1, abort_flag);
-      if (!ok) break;
-      ptx::tc_fence_after();
-      if (j > 0 && __any_sync(0xffffffffu, moved)) {
+      // O is stable (and the shared-memory P buffer free) once the previous step's PV has completed
+      const bool fix = j > 0 && __any_sync(0xffffffffu, moved);
+      if (!P_TMEM || fix) {
+        ok = ptx::mbar_wait(bar(P_EMPTY), (j & 1) ^ 1, abort_flag);
+        if (!ok) break;
+        ptx::tc_fence_after();
+      }
+      if (fix) {
         // rescale this row of the accumulator: O *= 2^(m_old - m_new)
 #pragma unroll 1
         for (int q = 0; q < HD / 32; ++q) {
@@ -351,17 +440,23 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
           for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * corr);
           DASH_TMEM_ST32(lane_addr + 2 * NKV + q * 32, o);
         }
+        if (!P_TMEM) ptx::tmem_wait_st();
+      }
+      if (P_TMEM) {
+        // P row -> the first 32 columns of this step's S buffer (two bf16 per column)
+        DASH_TMEM_ST32(lane_addr + buf * NKV, packed);
         ptx::tmem_wait_st();
-      }
-      // P row -> shared memory, K-major with the 128-byte swizzle (16-byte chunk q of row m sits at q ^ (m & 7))
+      } else {
+        // P row -> shared memory, K-major with the 128-byte swizzle (16-byte chunk q of row m sits at q ^ (m & 7))
 #pragma unroll
-      for (int q = 0; q < 8; ++q) {
-        uint4 v = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
-        *reinterpret_cast<uint4*>(prow + ((q ^ (m & 7)) << 4)) = v;
+        for (int q = 0; q < 8; ++q) {
+          uint4 v = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+          *reinterpret_cast<uint4*>(prow + ((q ^ (m & 7)) << 4)) = v;
+        }
+        ptx::fence_proxy_async_smem();
       }
-      ptx::fence_proxy_async_smem();
       ptx::tc_fence_before();
-      ptx::mbar_arrive(bar(P_FULL));
+      ptx::mbar_arrive(bar(P_FULL + (j & 1)));
     }
 
     // epilogue: O / l -> global (row m is 128 contiguous bf16 of token i_row, head r*g_q + hh)
