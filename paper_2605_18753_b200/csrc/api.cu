@@ -212,8 +212,9 @@ int dash_attn_attend_decode(const dash_params* p, const void* Q, const void* Kca
   WorkspaceLayout wl;
   if ((rc = check_workspace(dm, workspace, workspace_bytes, &wl)) != DASH_OK) return rc;
   if ((rc = check_device()) != DASH_OK) return rc;
-  return cuda_status(launch_attend_decode(dm, Q, Kcache, Vcache, kv_len, count, blk_idx, blk_bias, O,
-                                          at<float>(workspace, wl.partials), (cudaStream_t)stream));
+  return cuda_status(launch_attend_decode_ex(dm, Q, Kcache, Vcache, kv_len, count, blk_idx, blk_bias, O,
+                                             at<float>(workspace, wl.partials), at<StatusBlock>(workspace, wl.status),
+                                             (cudaStream_t)stream));
 }
 
 int dash_attn_fwd_prefill(const dash_params* p, const void* Q, const void* K, const void* V, const float* qbar,
@@ -267,8 +268,8 @@ int dash_attn_fwd_decode(const dash_params* p, const void* Q, const void* Kcache
   if ((rc = cuda_status(launch_select(dm, Q, Kbar, kv_len, at<uint32_t>(workspace, wl.mask), count, idx, bias, nullptr,
                                       at<void>(workspace, wl.planes), sb, st))) != DASH_OK)
     return rc;
-  return cuda_status(launch_attend_decode(dm, Q, Kcache, Vcache, kv_len, count, idx, bias, O,
-                                          at<float>(workspace, wl.partials), st));
+  return cuda_status(launch_attend_decode_ex(dm, Q, Kcache, Vcache, kv_len, count, idx, bias, O,
+                                             at<float>(workspace, wl.partials), sb, st));
 }
 
 int dash_attn_reset_status(void* workspace, void* stream) {

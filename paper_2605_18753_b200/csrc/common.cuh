@@ -43,6 +43,7 @@ struct StatusBlock {
 static_assert(sizeof(StatusBlock) == 256, "status block is the first 256 bytes of the workspace");
 
 __device__ inline void report_error(StatusBlock* sb, int status, int detail) {
+  if (!sb) return;
   if (atomicCAS(&sb->status, 0, status) == 0) sb->detail = detail;
 }
 
@@ -122,6 +123,13 @@ size_t decode_partial_bytes(const Dims& dm);
 cudaError_t launch_attend_decode(const Dims& dm, const void* Q, const void* K, const void* V, const int* kv_len,
                                  const int* count, const int* blk_idx, const float* blk_bias, void* O,
                                  float* partials, cudaStream_t st);
+cudaError_t launch_attend_decode_ex(const Dims& dm, const void* Q, const void* K, const void* V, const int* kv_len,
+                                    const int* count, const int* blk_idx, const float* blk_bias, void* O,
+                                    float* partials, StatusBlock* sb, cudaStream_t st);
+int decode_sm100_min_splits(const Dims& dm);
+cudaError_t launch_decode_sm100(const Dims& dm, int n_split, const void* Q, const void* K, const void* V,
+                                const int* kv_len, const int* count, const int* blk_idx, const float* blk_bias,
+                                float* partials, StatusBlock* sb, cudaStream_t st);
 bool prefill_sm100_supported(const Dims& dm);
 cudaError_t launch_attend_prefill_sm100(const Dims& dm, const void* Q, const void* K, const void* V,
                                         const uint32_t* mask, const float* blk_bias, void* O, StatusBlock* sb,

@@ -17,10 +17,16 @@ constexpr int DEC_WARPS = 4;
 constexpr int DEC_TARGET_BLOCKS = 148 * 4;
 constexpr int DEC_MAX_SPLITS = 32;
 
+static bool decode_use_sm100(const Dims& dm) {
+  const int need = decode_sm100_min_splits(dm);
+  return need > 0 && need <= DEC_MAX_SPLITS;
+}
+
 int decode_num_splits(const Dims& dm) {
   const int groups = dm.batch * dm.h_kv;
   int s = (DEC_TARGET_BLOCKS + groups - 1) / groups;
   if (s < 1) s = 1;
+  if (decode_use_sm100(dm)) s = max(s, decode_sm100_min_splits(dm));  // a block owns at most 512 sub-blocks there
   if (s > DEC_MAX_SPLITS) s = DEC_MAX_SPLITS;
   return s;
 }
@@ -216,6 +222,27 @@ static cudaError_t launch_dec(const Dims& dm, const void* Q, const void* K, cons
   decode_merge_kernel<T, D><<<(unsigned)((rows + 3) / 4), 128, 0, st>>>(dm, ns, partials, (T*)O);
   count_launch();
   return cudaGetLastError();
+}
+
+template <typename T, int D>
+static cudaError_t launch_merge(const Dims& dm, int ns, const float* partials, void* O, cudaStream_t st) {
+  const long long rows = (long long)dm.batch * dm.h_q;
+  decode_merge_kernel<T, D><<<(unsigned)((rows + 3) / 4), 128, 0, st>>>(dm, ns, partials, (T*)O);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_attend_decode_ex(const Dims& dm, const void* Q, const void* K, const void* V, const int* kv_len,
+                                    const int* count, const int* blk_idx, const float* blk_bias, void* O,
+                                    float* partials, StatusBlock* sb, cudaStream_t st) {
+  if (decode_use_sm100(dm)) {
+    // bf16, head_dim 128, chunks of 64 or 128: TMA-fed tensor-core split kernel, then the common merge
+    const int ns = decode_num_splits(dm);
+    cudaError_t e = launch_decode_sm100(dm, ns, Q, K, V, kv_len, count, blk_idx, blk_bias, partials, sb, st);
+    if (e != cudaSuccess) return e;
+    return launch_merge<__nv_bfloat16, 128>(dm, ns, partials, O, st);
+  }
+  return launch_attend_decode(dm, Q, K, V, kv_len, count, blk_idx, blk_bias, O, partials, st);
 }
 
 cudaError_t launch_attend_decode(const Dims& dm, const void* Q, const void* K, const void* V, const int* kv_len,
