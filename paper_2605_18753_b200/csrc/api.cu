@@ -14,7 +14,7 @@ void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
 static inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 struct WorkspaceLayout {
-  size_t status, kbar, mask, count, blk_idx, blk_bias, partials, planes, total;
+  size_t status, kbar, mask, count, blk_idx, blk_bias, partials, planes, xscratch, total;
 };
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
@@ -90,6 +90,7 @@ static WorkspaceLayout layout(const Dims& dm) {
   w.blk_bias = off; off += align256(cap * sizeof(float));
   w.partials = off; off += align256(dm.decode ? decode_partial_bytes(dm) : 0);
   w.planes = off; off += align256(select_sm100_token_limit(dm) > 0 ? select_sm100_scratch_bytes(dm) : 0);
+  w.xscratch = off; off += align256(select_decode_scratch_bytes(dm));
   w.total = off;
   return w;
 }
@@ -180,7 +181,7 @@ int dash_attn_select(const dash_params* p, const void* Q, const float* Kbar, con
   if ((rc = check_workspace(dm, workspace, workspace_bytes, &wl)) != DASH_OK) return rc;
   if ((rc = check_device()) != DASH_OK) return rc;
   return cuda_status(launch_select(dm, Q, Kbar, kv_len, mask, count, blk_idx, blk_bias, tau,
-                                   at<void>(workspace, wl.planes), at<StatusBlock>(workspace, wl.status),
+                                   at<void>(workspace, wl.planes), at<float>(workspace, wl.xscratch), at<StatusBlock>(workspace, wl.status),
                                    (cudaStream_t)stream));
 }
 
@@ -242,7 +243,7 @@ int dash_attn_fwd_prefill(const dash_params* p, const void* Q, const void* K, co
   uint32_t* mask = mask_out ? mask_out : at<uint32_t>(workspace, wl.mask);
   float* bias = at<float>(workspace, wl.blk_bias);
   if ((rc = cuda_status(launch_select(dm, Q, kb, nullptr, mask, at<int>(workspace, wl.count), nullptr, bias, nullptr,
-                                      at<void>(workspace, wl.planes), sb, st))) != DASH_OK)
+                                      at<void>(workspace, wl.planes), at<float>(workspace, wl.xscratch), sb, st))) != DASH_OK)
     return rc;
   return run_attend_prefill(dm, Q, K, V, mask, bias, O, sb, st);
 }
@@ -266,7 +267,7 @@ int dash_attn_fwd_decode(const dash_params* p, const void* Q, const void* Kcache
   int* idx = at<int>(workspace, wl.blk_idx);
   float* bias = at<float>(workspace, wl.blk_bias);
   if ((rc = cuda_status(launch_select(dm, Q, Kbar, kv_len, at<uint32_t>(workspace, wl.mask), count, idx, bias, nullptr,
-                                      at<void>(workspace, wl.planes), sb, st))) != DASH_OK)
+                                      at<void>(workspace, wl.planes), at<float>(workspace, wl.xscratch), sb, st))) != DASH_OK)
     return rc;
   return cuda_status(launch_attend_decode_ex(dm, Q, Kcache, Vcache, kv_len, count, idx, bias, O,
                                              at<float>(workspace, wl.partials), sb, st));

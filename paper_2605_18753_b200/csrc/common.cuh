@@ -109,8 +109,13 @@ cudaError_t launch_summaries(const Dims& dm, const void* K, const float* qbar, l
                              const int* kv_len, int first_block, int num_blocks, float* Kbar, cudaStream_t st);
 size_t select_smem_bytes(const Dims& dm, int* tq_out);
 cudaError_t launch_select(const Dims& dm, const void* Q, const float* Kbar, const int* kv_len, uint32_t* mask,
-                          int* count, int* blk_idx, float* blk_bias, float* tau, void* scratch, StatusBlock* sb,
-                          cudaStream_t st);
+                          int* count, int* blk_idx, float* blk_bias, float* tau, void* scratch, float* xscratch,
+                          StatusBlock* sb, cudaStream_t st);
+size_t select_decode_scratch_bytes(const Dims& dm);
+bool select_decode_supported(const Dims& dm);
+cudaError_t launch_select_decode(const Dims& dm, const void* Q, const float* Kbar, const int* kv_len, uint32_t* mask,
+                                 int* count, int* blk_idx, float* blk_bias, float* tau, float* scratch,
+                                 cudaStream_t st);
 int select_sm100_token_limit(const Dims& dm);
 size_t select_sm100_scratch_bytes(const Dims& dm);
 cudaError_t launch_select_sm100(const Dims& dm, int token_limit, const void* Q, const float* Kbar, void* planes,

@@ -280,8 +280,11 @@ static cudaError_t launch_rows(const Dims& dm, const SelectPlan& pl, int token_b
 }
 
 cudaError_t launch_select(const Dims& dm, const void* Q, const float* Kbar, const int* kv_len, uint32_t* mask,
-                          int* count, int* blk_idx, float* blk_bias, float* tau, void* scratch, StatusBlock* sb,
-                          cudaStream_t st) {
+                          int* count, int* blk_idx, float* blk_bias, float* tau, void* scratch, float* xscratch,
+                          StatusBlock* sb, cudaStream_t st) {
+  // decode: streaming score kernel + per-(batch, KV head) routing kernel
+  if (dm.decode && xscratch && select_decode_supported(dm))
+    return launch_select_decode(dm, Q, Kbar, kv_len, mask, count, blk_idx, blk_bias, tau, xscratch, st);
   // bf16 prefill rows whose candidates fit in tensor memory go to the tcgen05 kernel; everything else
   // (fp32, decode, very long rows) to the CUDA-core kernel below
   int token_base = 0;

@@ -1,0 +1,288 @@
+// Stage 1 for decode (Eq. 2, Eq. 4, Algorithm 2, Proposition 1): one query row per sequence.
+//
+// Decode routing is HBM-bound on the summary cache (every candidate's kbar row is read once per step and
+// per KV head), so it is split in two kernels:
+//   decode_scores_kernel  many thread blocks per (batch, KV head) stream kbar with fully coalesced 512-byte
+//                         row reads (one warp per row, four rows in flight per warp) and write the scaled
+//                         chunk logits x = gamma(alpha-1) <q, kbar_c>/sqrt(d) of the g_q heads to a small
+//                         fp32 scratch (b * h_q * T_s floats, stays in L2);
+//   decode_route_kernel   one thread block per (batch, KV head) loads its g_q logit rows into shared memory,
+//                         finds tau per head (Newton from max-1: monotone from below on the convex f),
+//                         forms the group weights, mask words, log w, mu and the compact (chunk, bias) list.
+#include "common.cuh"
+
+namespace dash {
+
+namespace {
+
+constexpr int SC_WARPS = 8;
+constexpr int SC_ROWS_PER_BLOCK = 256;   // summary rows one thread block scores
+constexpr int RT_THREADS = 256;
+constexpr int RT_MAX_NEWTON = 64, RT_MAX_NEWTON_GENERIC = 400;
+
+// Sum V values held by every lane across the warp with V-1+... shuffles (halving exchange): after the
+// call lane 0..V-1 ... we only need the totals in ONE lane per value, so the classic butterfly that halves
+// the number of live values per step is used; value v ends up (fully reduced) in lane (v * 32 / V) for V | 32.
+template <int V>
+__device__ __forceinline__ void warp_reduce_many(float (&x)[V], int lane) {
+#pragma unroll
+  for (int width = 16, live = V; width >= 1; width >>= 1) {
+    if (live > 1) {
+      // exchange halves: lanes with bit `width` clear keep the lower half of the live values, others the upper
+      const bool upper = (lane & width) != 0;
+      const int half = live / 2;
+#pragma unroll
+      for (int k = 0; k < V / 2; ++k) {
+        if (k < half) {
+          const float mine = upper ? x[k + half] : x[k];
+          const float give = upper ? x[k] : x[k + half];
+          x[k] = mine + __shfl_xor_sync(0xffffffffu, give, width);
+        }
+      }
+      live = half;
+    } else {
+      x[0] += __shfl_xor_sync(0xffffffffu, x[0], width);
+    }
+  }
+}
+
+template <typename T, int D, int G>
+__global__ void __launch_bounds__(SC_WARPS * 32)
+decode_scores_kernel(Dims dm, const T* __restrict__ Q, const float* __restrict__ Kbar, const int* __restrict__ kv_len,
+                     float* __restrict__ xs) {
+  constexpr int VPL = D / 32;   // floats per lane of one summary row
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int r = blockIdx.y, b = blockIdx.z;
+  int L = kv_len ? kv_len[b] : dm.seq_kv;
+  L = max(1, min(L, dm.seq_kv));
+  const int n_cand = min((L - 1) / dm.B, dm.T_s);
+  const int c_begin = blockIdx.x * SC_ROWS_PER_BLOCK;
+  const int c_end = min(n_cand, c_begin + SC_ROWS_PER_BLOCK);
+  if (c_begin >= c_end) return;
+
+  float q[G][VPL];
+#pragma unroll
+  for (int g = 0; g < G; ++g) {
+    const T* qp = Q + (long long)b * dm.qs[0] + (long long)(r * G + g) * dm.qs[2] + lane * VPL;
+#pragma unroll
+    for (int v = 0; v < VPL; ++v) q[g][v] = to_f32<T>(qp[v]) * dm.x_scale;
+  }
+  const float* kb = Kbar + ((long long)b * dm.h_kv + r) * dm.T_s * D + lane * VPL;
+  float* xo = xs + ((long long)b * dm.h_kv + r) * G * dm.T_s;
+
+  constexpr int RB = (G <= 8) ? 4 : 2;        // rows per iteration: RB * G values reduced together (<= 32)
+  for (int c0 = c_begin + warp * RB; c0 < c_end; c0 += SC_WARPS * RB) {
+    float kv[RB][VPL];
+#pragma unroll
+    for (int u = 0; u < RB; ++u) {
+      const int c = min(c0 + u, c_end - 1);
+      if constexpr (VPL == 4) {
+        const float4 f = *reinterpret_cast<const float4*>(kb + (long long)c * D);
+        kv[u][0] = f.x; kv[u][1] = f.y; kv[u][2] = f.z; kv[u][3] = f.w;
+      } else {
+        const float2 f = *reinterpret_cast<const float2*>(kb + (long long)c * D);
+        kv[u][0] = f.x; kv[u][1] = f.y;
+      }
+    }
+    float part[RB * G];
+#pragma unroll
+    for (int u = 0; u < RB; ++u)
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+        float s = 0.f;
+#pragma unroll
+        for (int v = 0; v < VPL; ++v) s = fmaf(q[g][v], kv[u][v], s);
+        part[u * G + g] = s;
+      }
+    warp_reduce_many<RB * G>(part, lane);
+    // value v = u*G + g is complete in lane v * (32 / (RB*G)) as part[0]
+    constexpr int STRIDE = 32 / (RB * G);
+    if (lane % STRIDE == 0) {
+      const int v = lane / STRIDE, u = v / G, g = v % G;
+      if (c0 + u < c_end) xo[(long long)g * dm.T_s + c0 + u] = part[0];
+    }
+  }
+}
+
+__global__ void __launch_bounds__(RT_THREADS)
+decode_route_kernel(Dims dm, const float* __restrict__ xs, const int* __restrict__ kv_len, uint32_t* __restrict__ mask,
+                    int* __restrict__ count, int* __restrict__ blk_idx, float* __restrict__ blk_bias,
+                    float* __restrict__ tau_out) {
+  extern __shared__ __align__(16) float sm[];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int r = blockIdx.x, b = blockIdx.y;
+  const int G = dm.g_q;
+  int L = kv_len ? kv_len[b] : dm.seq_kv;
+  L = max(1, min(L, dm.seq_kv));
+  const int c_own = (L - 1) / dm.B;
+  const int n_cand = min(c_own, dm.T_s);
+  const int stride = ((n_cand + 31) / 32) * 32 + 32;
+  float* X = sm;                                 // [G][stride]
+  float* taus = X + (size_t)G * stride;          // [G]
+  float* wsum = taus + 32;                       // per-word sum of log w   [W]
+  int* wcnt = reinterpret_cast<int*>(wsum + dm.W);   // per-word popcount / exclusive prefix [W + 1]
+  const long long grp = (long long)b * dm.h_kv + r;
+  const float* xg = xs + grp * G * dm.T_s;
+  for (int idx = tid; idx < G * n_cand; idx += RT_THREADS) {
+    const int g = idx / n_cand, c = idx % n_cand;
+    X[(size_t)g * stride + c] = xg[(long long)g * dm.T_s + c];
+  }
+  __syncthreads();
+
+  const int e_int = dm.e_int;
+  const float e = dm.e;
+  for (int g = warp; g < G; g += RT_THREADS / 32) {
+    const float* x = X + (size_t)g * stride;
+    float tau = 0.f;
+    if (n_cand > 0) {
+      float mx = -INFINITY;
+      for (int c = lane; c < n_cand; c += 32) mx = fmaxf(mx, x[c]);
+      mx = warp_max(mx);
+      tau = mx - 1.f;
+      const int max_it = e_int ? RT_MAX_NEWTON : RT_MAX_NEWTON_GENERIC;
+      for (int it = 0; it < max_it; ++it) {
+        float f = 0.f, gsum = 0.f;
+        for (int c = lane; c < n_cand; c += 32) {
+          const float m = x[c] - tau;
+          if (m > 0.f) { f += pow_e(m, e_int, e); gsum += pow_em1(m, e_int, e); }
+        }
+        f = warp_sum(f) - 1.f;
+        gsum = warp_sum(gsum);
+        if (!(f > 0.f)) break;
+        const float nt = tau + f / (e * gsum);
+        if (!(nt > tau)) break;
+        tau = nt;
+      }
+    }
+    if (lane == 0) {
+      taus[g] = tau;
+      if (tau_out) tau_out[(long long)b * dm.h_q + r * G + g] = tau;
+    }
+  }
+  __syncthreads();
+
+  // pass 1: one warp per 32-chunk mask word: support bits, log w (stashed over head 0's logits)
+  const float log_gq = logf((float)G);
+  uint32_t* mrow = mask + grp * dm.W;
+  for (int j = warp; j < dm.W; j += RT_THREADS / 32) {
+    const int c = j * 32 + lane;
+    bool sel = false;
+    float lw = INFINITY;
+    if (c < n_cand) {
+      float mstar = 0.f;
+      for (int g = 0; g < G; ++g) mstar = fmaxf(mstar, X[(size_t)g * stride + c] - taus[g]);
+      if (mstar > 0.f) {
+        sel = true;
+        const float inv = 1.f / mstar;
+        float s = 0.f;
+        for (int g = 0; g < G; ++g) s += pow_e(fmaxf(X[(size_t)g * stride + c] - taus[g], 0.f) * inv, e_int, e);
+        lw = e * logf(mstar) + logf(s) - log_gq;
+      }
+    }
+    const uint32_t word = __ballot_sync(0xffffffffu, sel);
+    const float ls = warp_sum(sel ? lw : 0.f);
+    if (c < n_cand) X[c] = lw;                      // +inf marks "not routed"
+    if (lane == 0) {
+      mrow[j] = word | (((c_own >> 5) == j) ? (1u << (c_own & 31)) : 0u);
+      wsum[j] = ls;
+      wcnt[j] = __popc(word);
+    }
+  }
+  __syncthreads();
+  // exclusive prefix of the per-word counts and the total of log w (W <= a few hundred: one warp)
+  if (warp == 0) {
+    int base = 0;
+    float tot = 0.f;
+    for (int j0 = 0; j0 < dm.W; j0 += 32) {
+      const int j = j0 + lane;
+      const int v = j < dm.W ? wcnt[j] : 0;
+      const float sv = j < dm.W ? wsum[j] : 0.f;
+      int incl = v;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+      }
+      if (j < dm.W) wcnt[j] = base + incl - v;
+      base += __shfl_sync(0xffffffffu, incl, 31);
+      tot += warp_sum(sv);
+    }
+    if (lane == 0) {
+      wcnt[dm.W] = base;
+      wsum[0] = tot;
+      count[grp] = base;
+    }
+  }
+  __syncthreads();
+  const int nsel = wcnt[dm.W];
+  if (nsel > 0) {
+    const float mu = wsum[0] / (float)nsel;
+    const long long loff = grp * dm.list_rows;
+    for (int j = warp; j * 32 < n_cand; j += RT_THREADS / 32) {
+      const int c = j * 32 + lane;
+      const float lw = (c < n_cand) ? X[c] : INFINITY;
+      const bool sel = lw < INFINITY;
+      const uint32_t word = __ballot_sync(0xffffffffu, sel);
+      if (sel) {
+        const long long pos = loff + wcnt[j] + __popc(word & ((1u << lane) - 1u));
+        blk_bias[pos] = (lw - mu) * dm.inv_sigma;
+        if (blk_idx) blk_idx[pos] = c;
+      }
+    }
+  }
+}
+
+}  // namespace
+
+size_t select_decode_scratch_bytes(const Dims& dm) {
+  return dm.decode ? (size_t)dm.batch * dm.h_q * (size_t)(dm.T_s > 0 ? dm.T_s : 1) * sizeof(float) : 0;
+}
+
+static size_t route_smem(const Dims& dm) {
+  const int stride = ((dm.T_s + 31) / 32) * 32 + 32;
+  return ((size_t)dm.g_q * stride + 32 + dm.W + dm.W + 1 + 8) * sizeof(float);
+}
+
+bool select_decode_supported(const Dims& dm) { return dm.decode && route_smem(dm) <= 200 * 1024; }
+
+cudaError_t launch_select_decode(const Dims& dm, const void* Q, const float* Kbar, const int* kv_len, uint32_t* mask,
+                                 int* count, int* blk_idx, float* blk_bias, float* tau, float* scratch,
+                                 cudaStream_t st) {
+  const int blocks_x = (dm.T_s + SC_ROWS_PER_BLOCK - 1) / SC_ROWS_PER_BLOCK;
+  if (blocks_x > 0) {
+    dim3 grid(blocks_x, dm.h_kv, dm.batch);
+#define DASH_SC(T, D, G) decode_scores_kernel<T, D, G><<<grid, SC_WARPS * 32, 0, st>>>(dm, (const T*)Q, Kbar, kv_len, scratch)
+#define DASH_SC_G(T, D)                                \
+  switch (dm.g_q) {                                    \
+    case 1: DASH_SC(T, D, 1); break;                   \
+    case 2: DASH_SC(T, D, 2); break;                   \
+    case 4: DASH_SC(T, D, 4); break;                   \
+    case 8: DASH_SC(T, D, 8); break;                   \
+    case 16: DASH_SC(T, D, 16); break;                 \
+    default: return cudaErrorInvalidValue;             \
+  }
+    if (dm.dtype == DASH_BF16) {
+      if (dm.d == 128) { DASH_SC_G(__nv_bfloat16, 128) } else { DASH_SC_G(__nv_bfloat16, 64) }
+    } else {
+      if (dm.d == 128) { DASH_SC_G(float, 128) } else { DASH_SC_G(float, 64) }
+    }
+#undef DASH_SC_G
+#undef DASH_SC
+    count_launch();
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+  const size_t smem = route_smem(dm);
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(decode_route_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  decode_route_kernel<<<dim3(dm.h_kv, dm.batch), RT_THREADS, smem, st>>>(dm, scratch, kv_len, mask, count, blk_idx,
+                                                                       blk_bias, tau);
+  count_launch();
+  return cudaGetLastError();
+}
+
+}  // namespace dash
