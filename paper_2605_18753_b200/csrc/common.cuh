@@ -99,6 +99,11 @@ __device__ inline float pow_em1(float m, int e_int, float e) {
   return m > 0.f ? __powf(m, e - 1.f) : 0.f;
 }
 
+// Newton on f(tau) = sum [x - tau]_+^e - 1 stops once f <= this: the sum itself carries about 1e-6 of fp32
+// rounding noise, and f'(tau) <= -1 at the root for every alpha > 1 (sum m^e = 1 implies sum m^(e-1) >= 1), so the
+// threshold is then within 4e-6 of the root; iterating on noise only burns passes.
+constexpr float NEWTON_F_TOL = 4e-6f;
+
 void count_launch();
 // Host-side checks shared by the entry points that live outside api.cu.
 int validate_params(const dash_params* p, Dims* dm);

@@ -178,7 +178,7 @@ select_kernel(Dims dm, int TQ, int xs_stride, int token_base, const T* __restric
           }
           f = warp_sum(f) - 1.f;
           g = warp_sum(g);
-          if (!(f > 0.f)) break;
+          if (!(f > NEWTON_F_TOL)) break;
           const float nt = tau + f / (e * g);
           if (!(nt > tau)) break;
           tau = nt;

@@ -148,7 +148,7 @@ decode_route_kernel(Dims dm, const float* __restrict__ xs, const int* __restrict
         }
         f = warp_sum(f) - 1.f;
         gsum = warp_sum(gsum);
-        if (!(f > 0.f)) break;
+        if (!(f > NEWTON_F_TOL)) break;
         const float nt = tau + f / (e * gsum);
         if (!(nt > tau)) break;
         tau = nt;

@@ -221,7 +221,7 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         }
         if (!done) {
           f -= 1.f;
-          if (!(f > 0.f)) {
+          if (!(f > NEWTON_F_TOL)) {
             done = true;
           } else {
             const float nt = tau + f / (e * g);
