@@ -73,8 +73,8 @@ __global__ void kbar_split_kernel(const float* __restrict__ kbar, __nv_bfloat16*
   planes[2 * n + i] = __float2bfloat16_rn(r2);
 }
 
-template <int NST>
-__global__ void __launch_bounds__(SEL_TC_THREADS)
+template <int NST, int G>
+__global__ void __launch_bounds__(SEL_TC_THREADS, NST == 1 ? 2 : 1)
 select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKB, SelectTcArgs a) {
   using SP = SmemPlan<NST>;
   extern __shared__ __align__(1024) uint8_t smem[];
@@ -90,7 +90,8 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   const int tile = a.n_tiles - 1 - (int)(blockIdx.x / groups);
   const int grp = (int)(blockIdx.x % groups);
   const int b = grp / dm.h_kv, r = grp % dm.h_kv;
-  const int TQ = a.TQ, g_q = dm.g_q;
+  const int TQ = a.TQ;
+  constexpr int g_q = G;
   const int i0 = tile * TQ;
   const int c_own = i0 / dm.B;
   const int n_cand = min(c_own, dm.T_s);
@@ -189,8 +190,80 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       ok = ptx::mbar_wait(bar(X_FULL), 0, abort_flag);
       ptx::tc_fence_after();
     }
-    if (ok && n_cand > 0) {
-      // pass 0: row maximum
+    // Newton on f(tau) = sum [x - tau]_+^e - 1, convex and decreasing.  From the left of the root the iterates
+    // rise monotonically and never pass it; from the right one step lands on the left.  The start is the root
+    // of the same equation with every candidate taken as active (closed form for alpha = 2 and 1.5), clamped to
+    // max - 1 <= tau* < max, which saves the slow first halvings of a start at max - 1.
+    const int max_it = e_int ? MAX_NEWTON : MAX_NEWTON_GENERIC;
+    auto start_tau = [&](float mx, float s1, float s2) -> float {   // s1, s2: sums of (x - mx), (x - mx)^2
+      const float n = (float)n_cand;
+      float t = -1.f;
+      if (e_int == 1) {
+        t = (s1 - 1.f) / n;
+      } else if (e_int == 2) {
+        const float mean = s1 / n, ss = s2 - s1 * mean;
+        if (ss < 1.f) t = mean - sqrtf((1.f - ss) / n);
+      }
+      return mx + fminf(fmaxf(t, -1.f), -1e-6f);
+    };
+    auto newton_step = [&](float f, float g, bool& done) {
+      if (done) return;
+      f -= 1.f;
+      if (fabsf(f) <= NEWTON_F_TOL || !(g > 0.f)) { done = true; return; }
+      const float nt = tau + f / (e * g);
+      if (nt == tau) done = true; else tau = nt;
+    };
+    float xr[4][32];                               // the whole row, when it has at most 128 candidates
+    const bool in_regs = n_chunks <= 4;
+    if (ok && n_cand > 0 && in_regs) {
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        if (k < n_chunks) {
+          uint32_t v[32];
+          DASH_TMEM_LD32(v, lane_addr + k * 32);
+          ptx::tmem_wait_ld();
+          const int lim = n_cand - k * 32;
+#pragma unroll
+          for (int c = 0; c < 32; ++c) xr[k][c] = c < lim ? __uint_as_float(v[c]) * xs : -INFINITY;
+        } else {
+#pragma unroll
+          for (int c = 0; c < 32; ++c) xr[k][c] = -INFINITY;
+        }
+      }
+      float mx = -INFINITY;
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+#pragma unroll
+        for (int c = 0; c < 32; ++c) mx = fmaxf(mx, xr[k][c]);
+      float s1 = 0.f, s2 = 0.f;
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+          const float y = xr[k][c] > -INFINITY ? xr[k][c] - mx : 0.f;
+          s1 += y;
+          s2 = fmaf(y, y, s2);
+        }
+      tau = start_tau(mx, s1, s2);
+      bool done = false;
+      for (int it = 0; it < max_it; ++it) {
+        float f[4] = {0.f, 0.f, 0.f, 0.f}, g[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          if (k < n_chunks) {
+#pragma unroll
+            for (int c = 0; c < 32; ++c) {
+              const float mm = fmaxf(xr[k][c] - tau, 0.f);
+              f[c & 3] += pow_e(mm, e_int, e);
+              g[c & 3] += pow_em1(mm, e_int, e);
+            }
+          }
+        }
+        newton_step((f[0] + f[1]) + (f[2] + f[3]), (g[0] + g[1]) + (g[2] + g[3]), done);
+        if (__all_sync(0xffffffffu, done)) break;
+      }
+    } else if (ok && n_cand > 0) {
+      // longer rows stream from tensor memory every pass
       float mx = -INFINITY;
       for (int k = 0; k < n_chunks; ++k) {
         uint32_t v[32];
@@ -201,11 +274,23 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         for (int c = 0; c < 32; ++c) mx = fmaxf(mx, c < lim ? __uint_as_float(v[c]) : -INFINITY);
       }
       mx *= xs;
-      tau = mx - 1.f;
+      float s1 = 0.f, s2 = 0.f;
+      for (int k = 0; k < n_chunks; ++k) {
+        uint32_t v[32];
+        DASH_TMEM_LD32(v, lane_addr + k * 32);
+        ptx::tmem_wait_ld();
+        const int lim = n_cand - k * 32;
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+          const float y = c < lim ? fmaf(__uint_as_float(v[c]), xs, -mx) : 0.f;
+          s1 += y;
+          s2 = fmaf(y, y, s2);
+        }
+      }
+      tau = start_tau(mx, s1, s2);
       bool done = false;
-      const int max_it = e_int ? MAX_NEWTON : MAX_NEWTON_GENERIC;
       for (int it = 0; it < max_it; ++it) {
-        float f = 0.f, g = 0.f;
+        float f[4] = {0.f, 0.f, 0.f, 0.f}, g[4] = {0.f, 0.f, 0.f, 0.f};
         for (int k = 0; k < n_chunks; ++k) {
           uint32_t v[32];
           DASH_TMEM_LD32(v, lane_addr + k * 32);
@@ -215,88 +300,126 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           for (int c = 0; c < 32; ++c) {
             float mm = fmaxf(fmaf(__uint_as_float(v[c]), xs, -tau), 0.f);
             mm = c < lim ? mm : 0.f;
-            f += pow_e(mm, e_int, e);
-            g += pow_em1(mm, e_int, e);
+            f[c & 3] += pow_e(mm, e_int, e);
+            g[c & 3] += pow_em1(mm, e_int, e);
           }
         }
-        if (!done) {
-          f -= 1.f;
-          if (!(f > NEWTON_F_TOL)) {
-            done = true;
-          } else {
-            const float nt = tau + f / (e * g);
-            if (!(nt > tau)) done = true; else tau = nt;
-          }
-        }
+        newton_step((f[0] + f[1]) + (f[2] + f[3]), (g[0] + g[1]) + (g[2] + g[3]), done);
         if (__all_sync(0xffffffffu, done)) break;
       }
     }
     if (ok && row_valid && a.tau) a.tau[((long long)b * dm.h_q + r * g_q + hh) * dm.seq_q + i] = tau;
 
-    // ---------------- group weights, mask words, log w, compact lists (warp-synchronous, 32 chunks a step)
+    // ---------------- group weights, mask words, log w, compact lists
+    // The g_q heads of a token sit in g_q adjacent lanes.  Per 32-chunk step every lane raises its own margins
+    // to the power e and the group sums them with a halving exchange (log2(g_q) rounds of shuffles), after
+    // which lane j of the group owns the sums of 32/g_q contiguous chunks: w = sum / g_q, bit = (sum > 0),
+    // log w = log(sum) - log(g_q).  log w (or +inf) is parked in the lane's own TMEM columns (the scores there
+    // are spent), so the second sweep, which needs mu = mean log w, writes the final biases straight into the
+    // compact list: no read-modify-write of global memory.
+    constexpr int OWN = 32 / G;                                  // chunks a lane owns per step
+    const int own0 = [&] {                                       // first owned chunk: bit k of hh picks a half
+      int base = 0, width = 32;
+#pragma unroll
+      for (int o = 1; o < G; o <<= 1) { width >>= 1; if (hh & o) base += width; }
+      return base;
+    }();
     const long long row_id = ((long long)b * dm.h_kv + r) * dm.seq_q + i;
     const long long loff = ((long long)b * dm.h_kv + r) * dm.list_rows + list_row_offset(dm, min(i, dm.seq_q - 1));
     uint32_t* mrow = a.mask + row_id * dm.W;
-    float* xw = xch + (size_t)warp * 32 * XCH_STRIDE;        // this warp's 32 rows
-    const int lrow = lane;                                     // row inside the warp's slab
-    const int grow0 = (lane / g_q) * g_q;                      // first row of this token's group in the slab
-    const float log_gq = logf((float)g_q);
+    const float log_gq = logf((float)G);
     float slog = 0.f;
     int nsel = 0;
+    auto group_sums = [&](float (&pe)[32]) {
+      // after the call pe[0 .. OWN) hold the group sums of chunks own0 .. own0+OWN
+      int live = 32;
+#pragma unroll
+      for (int o = 1; o < G; o <<= 1) {
+        const bool upper = (hh & o) != 0;
+        const int half = live / 2;
+#pragma unroll
+        for (int c = 0; c < 16; ++c) {
+          if (c < half) {
+            const float mine = upper ? pe[c + half] : pe[c];
+            const float give = upper ? pe[c] : pe[c + half];
+            pe[c] = mine + __shfl_xor_sync(0xffffffffu, give, o);
+          }
+        }
+        live = half;
+      }
+    };
     if (ok) {
       for (int k = 0; k < n_chunks; ++k) {
-        uint32_t v[32];
-        DASH_TMEM_LD32(v, lane_addr + k * 32);
-        ptx::tmem_wait_ld();
-        const int lim = n_cand - k * 32;
+        float pe[32];
+        if (in_regs) {
 #pragma unroll
-        for (int c = 0; c < 32; ++c) {
-          float mm = fmaxf(fmaf(__uint_as_float(v[c]), xs, -tau), 0.f);
-          xw[lrow * XCH_STRIDE + c] = c < lim ? mm : 0.f;
-        }
-        __syncwarp();
-        uint32_t bits = 0;
-        float lw_own[32 / 2];      // at most 32/g_q <= 16 columns per thread
-        int n_own = 0;
-        for (int c = hh; c < 32; c += g_q, ++n_own) {
-          float mstar = 0.f;
-          for (int h2 = 0; h2 < g_q; ++h2) mstar = fmaxf(mstar, xw[(grow0 + h2) * XCH_STRIDE + c]);
-          float lw = 0.f;
-          if (mstar > 0.f) {
-            const float inv = 1.f / mstar;
-            float s = 0.f;
-            for (int h2 = 0; h2 < g_q; ++h2) s += pow_e(xw[(grow0 + h2) * XCH_STRIDE + c] * inv, e_int, e);
-            lw = e * logf(mstar) + logf(s) - log_gq;
-            bits |= 1u << c;
-            slog += lw;
+          for (int kk = 0; kk < 4; ++kk)
+            if (kk == k) {
+#pragma unroll
+              for (int c = 0; c < 32; ++c) pe[c] = pow_e(fmaxf(xr[kk][c] - tau, 0.f), e_int, e);
+            }
+        } else {
+          uint32_t v[32];
+          DASH_TMEM_LD32(v, lane_addr + k * 32);
+          ptx::tmem_wait_ld();
+          const int lim = n_cand - k * 32;
+#pragma unroll
+          for (int c = 0; c < 32; ++c) {
+            const float mm = fmaxf(fmaf(__uint_as_float(v[c]), xs, -tau), 0.f);
+            pe[c] = c < lim ? pow_e(mm, e_int, e) : 0.f;
           }
-          lw_own[n_own] = lw;
         }
-        for (int o = 1; o < g_q; o <<= 1) bits |= __shfl_xor_sync(0xffffffffu, bits, o);
+        group_sums(pe);
+        uint32_t bits = 0;
+        uint32_t lwv[32];
+#pragma unroll
+        for (int c = 0; c < 32; ++c) lwv[c] = 0x7f800000u;        // +inf: not routed
+#pragma unroll
+        for (int q = 0; q < OWN; ++q) {
+          if (pe[q] > 0.f) {
+            const float lw = __logf(pe[q]) - log_gq;
+            lwv[q] = __float_as_uint(lw);
+            slog += lw;
+            bits |= 1u << (own0 + q);
+          }
+        }
+#pragma unroll
+        for (int o = 1; o < G; o <<= 1) bits |= __shfl_xor_sync(0xffffffffu, bits, o);
+        DASH_TMEM_ST32(lane_addr + k * 32, lwv);                 // slot q of this lane = chunk own0 + q of step k
+        if (row_valid && hh == 0) mrow[k] = bits | (((c_own >> 5) == k) ? (1u << (c_own & 31)) : 0u);
+        nsel += __popc(bits);
+      }
+      ptx::tmem_wait_st();
+#pragma unroll
+      for (int o = 1; o < G; o <<= 1) slog += __shfl_xor_sync(0xffffffffu, slog, o);
+      if (row_valid && hh == 0) {
+        for (int j = n_chunks; j < dm.W; ++j) mrow[j] = ((c_own >> 5) == j) ? (1u << (c_own & 31)) : 0u;
+        a.count[row_id] = nsel;
+      }
+      const float mu = nsel > 0 ? slog / (float)nsel : 0.f;
+      int base = 0;
+      for (int k = 0; k < n_chunks; ++k) {
+        uint32_t lwv[32];
+        DASH_TMEM_LD32(lwv, lane_addr + k * 32);
+        ptx::tmem_wait_ld();
+        uint32_t bits = 0;
+#pragma unroll
+        for (int q = 0; q < OWN; ++q)
+          if (lwv[q] != 0x7f800000u) bits |= 1u << (own0 + q);
+#pragma unroll
+        for (int o = 1; o < G; o <<= 1) bits |= __shfl_xor_sync(0xffffffffu, bits, o);
         if (row_valid) {
-          int q = 0;
-          for (int c = hh; c < 32; c += g_q, ++q) {
-            if ((bits >> c) & 1u) {
-              const long long pos = loff + nsel + __popc(bits & ((1u << c) - 1u));
-              a.blk_bias[pos] = lw_own[q];
+#pragma unroll
+          for (int q = 0; q < OWN; ++q) {
+            if (lwv[q] != 0x7f800000u) {
+              const int c = own0 + q;
+              const long long pos = loff + base + __popc(bits & ((1u << c) - 1u));
+              a.blk_bias[pos] = (__uint_as_float(lwv[q]) - mu) * dm.inv_sigma;
               if (a.blk_idx) a.blk_idx[pos] = k * 32 + c;
             }
           }
-          if (hh == 0) mrow[k] = bits | (((c_own >> 5) == k) ? (1u << (c_own & 31)) : 0u);
         }
-        nsel += __popc(bits);
-        __syncwarp();
-      }
-      for (int o = 1; o < g_q; o <<= 1) slog += __shfl_xor_sync(0xffffffffu, slog, o);
-      if (row_valid) {
-        if (hh == 0) {
-          for (int j = n_chunks; j < dm.W; ++j) mrow[j] = ((c_own >> 5) == j) ? (1u << (c_own & 31)) : 0u;
-          a.count[row_id] = nsel;
-        }
-        if (nsel > 0) {
-          const float mu = slog / (float)nsel;
-          for (int p = hh; p < nsel; p += g_q) a.blk_bias[loff + p] = (a.blk_bias[loff + p] - mu) * dm.inv_sigma;
-        }
+        base += __popc(bits);
       }
     }
     ptx::tc_fence_before();
@@ -388,25 +511,28 @@ cudaError_t launch_select_sm100(const Dims& dm, int token_limit, const void* Q, 
     if (!encode4(&tkb, planes, dims, strides, box)) return cudaErrorInvalidValue;
   }
   const long long blocks = (long long)a.n_tiles * dm.batch * dm.h_kv;
-  if (cols <= 256) {
-    auto kern = select_sm100_kernel<1>;
-    static bool configured = false;
-    if (!configured) {
-      e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemPlan<1>::TOTAL);
-      if (e != cudaSuccess) return e;
-      configured = true;
-    }
-    kern<<<(unsigned)blocks, SEL_TC_THREADS, SmemPlan<1>::TOTAL, st>>>(tq, tkb, a);
-  } else {
-    auto kern = select_sm100_kernel<2>;
-    static bool configured = false;
-    if (!configured) {
-      e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemPlan<2>::TOTAL);
-      if (e != cudaSuccess) return e;
-      configured = true;
-    }
-    kern<<<(unsigned)blocks, SEL_TC_THREADS, SmemPlan<2>::TOTAL, st>>>(tq, tkb, a);
+#define DASH_SEL_TC(NSTV, GV)                                                                                      \
+  {                                                                                                                 \
+    auto kern = select_sm100_kernel<NSTV, GV>;                                                                      \
+    static bool configured = false;                                                                                 \
+    if (!configured) {                                                                                              \
+      e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemPlan<NSTV>::TOTAL);           \
+      if (e != cudaSuccess) return e;                                                                               \
+      configured = true;                                                                                            \
+    }                                                                                                               \
+    kern<<<(unsigned)blocks, SEL_TC_THREADS, SmemPlan<NSTV>::TOTAL, st>>>(tq, tkb, a);                              \
   }
+#define DASH_SEL_TC_G(NSTV)                    \
+  switch (dm.g_q) {                            \
+    case 2: DASH_SEL_TC(NSTV, 2); break;       \
+    case 4: DASH_SEL_TC(NSTV, 4); break;       \
+    case 8: DASH_SEL_TC(NSTV, 8); break;       \
+    case 16: DASH_SEL_TC(NSTV, 16); break;     \
+    default: return cudaErrorInvalidValue;     \
+  }
+  if (cols <= 256) { DASH_SEL_TC_G(1) } else { DASH_SEL_TC_G(2) }
+#undef DASH_SEL_TC_G
+#undef DASH_SEL_TC
   count_launch();
   return cudaGetLastError();
 }
