@@ -12,7 +12,6 @@ from __future__ import annotations
 import argparse
 import json
 import os
-import subprocess
 import sys
 import threading
 import time
@@ -42,50 +41,53 @@ def load_peaks():
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks / throttle reasons of one GPU while the timed region runs."""
-    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    """Samples SM clock and throttle reasons of one GPU through NVML (read-only) while the timed region runs."""
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
 
-    def __init__(self, index: int):
-        self.index, self.samples, self.proc = index, [], None
+    def __init__(self, index: int, period_s: float = 0.002):
+        self.index, self.period, self.sm, self.reasons = index, period_s, [], set()
+        self.max_mhz, self._stop, self.thread, self.err = None, threading.Event(), None, None
+        self._ready = threading.Event()
+
+    def _run(self):
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+            phys = self.index
+            if vis:
+                try:
+                    phys = int(vis.split(",")[self.index])
+                except (ValueError, IndexError):
+                    phys = self.index
+            h = pynvml.nvmlDeviceGetHandleByIndex(phys)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+            self._ready.set()
+            while not self._stop.is_set():
+                self.sm.append(float(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)))
+                mask = int(pynvml.nvmlDeviceGetCurrentClocksEventReasons(h))
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+                time.sleep(self.period)
+        except Exception as ex:  # pragma: no cover
+            self.err = repr(ex)
+            self._ready.set()
 
     def start(self):
-        try:
-            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
-                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-            self.t = threading.Thread(target=self._read, daemon=True)
-            self.t.start()
-        except Exception:
-            self.proc = None
-
-    def _read(self):
-        for line in self.proc.stdout:
-            self.samples.append(line.strip())
+        self.thread = threading.Thread(target=self._run, daemon=True)
+        self.thread.start()
+        self._ready.wait(timeout=10)      # NVML is initialised before the timed region begins
 
     def stop(self) -> dict:
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            pass
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for s in self.samples:
-            f = [x.strip() for x in s.split(",")]
-            if len(f) < 7:
-                continue
-            try:
-                sm.append(float(f[0])); mx.append(float(f[1]))
-            except ValueError:
-                continue
-            for k, nm in enumerate(names):
-                if f[3 + k].lower().startswith("active"):
-                    reasons.add(nm)
-        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+        self._stop.set()
+        if self.thread is not None:
+            self.thread.join(timeout=5)
+        out = {"sm_mhz": float(np.median(self.sm)) if self.sm else None, "sm_max_mhz": self.max_mhz,
+               "reasons": sorted(self.reasons), "samples": len(self.sm)}
+        if self.err:
+            out["error"] = self.err
+        return out
 
 
 def selected_flops_from_count(count: torch.Tensor, B: int, d: int, g_q: int) -> float:
@@ -94,6 +96,30 @@ def selected_flops_from_count(count: torch.Tensor, B: int, d: int, g_q: int) -> 
     diag = (torch.arange(n, device=count.device) % B + 1).to(torch.float64)
     tok = count.to(torch.float64) * B + diag[None, None, :]
     return float(4.0 * d * g_q * tok.sum().item())
+
+
+def executed_flops_from_mask(mask: torch.Tensor, w) -> tuple:
+    """FLOPs the Stage-2 tensor-core kernel executes: it walks, per tile of 128/g_q tokens, the UNION of the
+    rows' routed chunks in 64-token steps, each step costing 4*128*128*64 FLOPs whatever the rows select."""
+    b, h_kv, n, W = mask.shape
+    g_q = w.h_q // w.h_kv
+    tq = max(1, 128 // g_q)
+    if n % tq != 0 or tq > w.block:
+        return float("nan"), 0
+    steps = 0
+    sub = max(1, w.block // 64)
+    for bb in range(b):                                    # one sequence at a time bounds the temporary
+        m = mask[bb].view(h_kv, n // tq, tq, W)
+        u = m[:, :, 0, :].clone()
+        for t in range(1, tq):
+            u |= m[:, :, t, :]
+        bits = torch.zeros(u.shape[:2], dtype=torch.int64, device=mask.device)
+        for k in range(32):
+            bits += ((u >> k) & 1).sum(dim=-1)
+        own_first = (torch.arange(n // tq, device=mask.device) * tq) % w.block   # offset of the tile in its own chunk
+        own_steps = own_first // 64 + 1
+        steps += int(((bits - 1) * sub + own_steps[None, :]).sum().item())
+    return float(steps) * 4.0 * 128 * 128 * 64, steps
 
 
 def sparsity_from_count(count: torch.Tensor, B: int) -> float:
@@ -154,7 +180,7 @@ def run_reference(args, w):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="prefill_8k")
@@ -202,12 +228,12 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    sampler = ClockSampler(local)
+    sampler.start()
     for _ in range(args.warmup):
         flush.fill_(1)
         step()
     barrier()
-    sampler = ClockSampler(local)
-    sampler.start()
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
     n0 = B.dash_attn_launch_count()
     barrier()
@@ -220,14 +246,9 @@ def main():
     barrier()
     t_wall = time.perf_counter() - t_wall
     launches = B.dash_attn_launch_count() - n0
-    clocks = sampler.stop()
     assert B.dash_attn_last_status(ws) == 0, "device-side error reported by the library"
     step_ms = [a.elapsed_time(b) for a, b in ev]
-    ms = float(np.mean(step_ms))
-    if dist is not None:
-        t = torch.tensor([ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms_local = float(np.mean(step_ms))
 
     # per-stage timing (same steps, stages called one by one through the C ABI) and workload statistics
     stage_ms = {"summaries": [], "select": [], "attend": []}
@@ -245,16 +266,14 @@ def main():
         for k, name in enumerate(("summaries", "select", "attend")):
             stage_ms[name].append(e[k].elapsed_time(e[k + 1]))
     stage_ms = {k: float(np.mean(v)) for k, v in stage_ms.items()}
+    clocks = sampler.stop()      # sampled from before the warm-up to after the per-stage pass (both under load)
     f_sel = selected_flops_from_count(rt["count"], w.block, w.head_dim, g_q)
     sparsity = sparsity_from_count(rt["count"], w.block)
     f_dense = 4.0 * w.head_dim * w.h_q * w.batch * w.seq * (w.seq + 1) / 2.0
-    if dist is not None:
-        t = torch.tensor([f_sel], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.SUM)
-        f_total = float(t.item())
-    else:
-        f_total = f_sel
+    from paper_2605_18753_b200.shard import combine_timing
+    ms, f_total = combine_timing(ms_local, f_sel, device=dev)      # max over ranks, sum over ranks
     value = f_total / (ms * 1e-3) / 1e12
+    executed, n_steps_total = executed_flops_from_mask(rt["mask"], w)
 
     # end to end: pinned host inputs -> device, forward, output -> pinned host, all inside the timed region
     hQ, hK, hV = (t.cpu().pin_memory() for t in (Q, K, V))
@@ -276,11 +295,7 @@ def main():
         e2e_step()
     b_.record()
     barrier()
-    e2e_ms = a.elapsed_time(b_) / args.steps
-    if dist is not None:
-        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms, _ = combine_timing(a.elapsed_time(b_) / args.steps, 0.0, device=dev)
     h2d = sum(t.numel() * t.element_size() for t in (hQ, hK, hV))
     d2h = hO.numel() * hO.element_size()
 
@@ -295,6 +310,8 @@ def main():
                 "unit": "TFLOP/s", "frac": achieved / peak_tf, "peak_source": f"{peaks['_source']} bf16 burst",
                 "traffic": None}
     extras = {"fwd_ms": ms, "stage_ms": stage_ms, "block_sparsity": sparsity, "selected_tflop": f_sel / 1e12,
+              "executed_tflop": executed / 1e12, "union_inflation": executed / f_sel, "tile_steps": n_steps_total,
+              "stage2_executed_tflops": executed / (stage_ms["attend"] * 1e-3) / 1e12,
               "dense_causal_tflop": f_dense / 1e12, "wall_s_timed_region": t_wall}
 
     cpu_val, cpu_rows, cpu_dt = time_oracle_sample(w, {k: v for k, v in inp.items()}, args.cpu_seconds)
@@ -319,6 +336,8 @@ def main():
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "gpu_launches": int(launches),
             "roofline": roofline, "cpu_baseline": cpu_baseline, "extras": extras}
+    line["roofline"]["note"] = ("achieved = selected-token FLOPs / Stage-2 kernel time; the kernel executes "
+                                "union_inflation x that many FLOPs (extras.stage2_executed_tflops)")
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
