@@ -30,7 +30,7 @@ constexpr bool P_TMEM = true;     // P (bf16) reaches the PV MMA through tensor 
 constexpr bool QK_FIRST = true;   // issue S of step j+1 before PV of step j even if its K tile has to be waited for
 constexpr int NKV = 64;           // KV tokens per step
 constexpr int KST = 3, VST = 2;   // ring depths
-constexpr int PF_THREADS = 192;
+constexpr int PF_THREADS = 224;   // 4 softmax warps, K producer, MMA issuer, V/bias producer
 constexpr int HD = 128;           // head_dim
 constexpr uint32_t TMEM_COLS = 256;  // S0 [0,64), S1 [64,128), O [128,256)
 constexpr float RESCALE_LOG2 = 8.f;  // the running maximum is moved only when it grew by more than this
@@ -126,9 +126,12 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
   ptx::tc_fence_after();
   const uint32_t tmem = misc->tmem_base;
 
-  if (warp == 4) {
-    // =========================== producer ===========================
-    if (lane == 0) {
+  if (warp == 4 || warp == 6) {
+    // =========================== producers ===========================
+    // Two warps walk the same union list: warp 4 feeds the K ring (and loads Q), warp 6 feeds the V ring and
+    // the per-token bias of each step.  Split like this, a full V ring never holds back the next K tile.
+    const bool do_k = (warp == 4), do_v = (warp == 6);
+    if (lane == 0 && do_k) {
       ptx::prefetch_tensormap(&tmQ);
       ptx::prefetch_tensormap(&tmK);
       ptx::prefetch_tensormap(&tmV);
@@ -151,7 +154,7 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
     }
     // the own chunk is always in the union (its bit is set in every row); it contributes own_steps steps
     const int n_steps = (total - 1) * sub_per_blk + own_steps;
-    if (lane == 0) {
+    if (lane == 0 && do_k) {
       misc->n_steps = n_steps;
       ptx::mbar_arrive(bar(META));
     }
@@ -186,8 +189,13 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
     };
 #pragma unroll
     for (int q = 0; q < 2; ++q) {
-      load_group(q, 0, bq[q]);
-      load_group(q, 4, bn[q]);
+      if (do_v) {
+        load_group(q, 0, bq[q]);
+        load_group(q, 4, bn[q]);
+      } else {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) bq[q][k] = bn[q][k] = 0.f;
+      }
     }
     auto take = [&](int q) -> float {
       const int k = taken[q];
@@ -223,7 +231,7 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
         out.bv[q] = -INFINITY;
         if (out.c == c_own) {
           out.bv[q] = 0.f;
-        } else if ((rw[q] >> bit) & 1u) {
+        } else if (do_v && ((rw[q] >> bit) & 1u)) {
           out.bv[q] = take(q);
         }
       }
@@ -239,15 +247,18 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
       const int nsub = (cur.c == c_own) ? own_steps : sub_per_blk;
       for (int sub = 0; sub < nsub && ok; ++sub, ++j) {
         const int kv0 = cur.c * dm.B + sub * NKV;
-        ok = ptx::mbar_wait(bar(K_EMPTY + ks), kph, abort_flag);
-        if (!ok) break;
-        if (lane == 0) {
-          const uint32_t dst = sbase + OFF_K + ks * KV_TILE_BYTES;
-          ptx::mbar_arrive_expect_tx(bar(K_FULL + ks), KV_TILE_BYTES);
-          ptx::tma_load_4d(dst, &tmK, bar(K_FULL + ks), 0, r, kv0, b);
-          ptx::tma_load_4d(dst + KV_TILE_BYTES / 2, &tmK, bar(K_FULL + ks), 64, r, kv0, b);
+        if (do_k) {
+          ok = ptx::mbar_wait(bar(K_EMPTY + ks), kph, abort_flag);
+          if (!ok) break;
+          if (lane == 0) {
+            const uint32_t dst = sbase + OFF_K + ks * KV_TILE_BYTES;
+            ptx::mbar_arrive_expect_tx(bar(K_FULL + ks), KV_TILE_BYTES);
+            ptx::tma_load_4d(dst, &tmK, bar(K_FULL + ks), 0, r, kv0, b);
+            ptx::tma_load_4d(dst + KV_TILE_BYTES / 2, &tmK, bar(K_FULL + ks), 64, r, kv0, b);
+          }
+          if (++ks == KST) { ks = 0; kph ^= 1; }
+          continue;
         }
-        if (++ks == KST) { ks = 0; kph ^= 1; }
         ok = ptx::mbar_wait(bar(V_EMPTY + vs), vph, abort_flag);
         if (!ok) break;
         for (int q = 0; q < 2; ++q) {
@@ -267,9 +278,9 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
     }
     if (!ok && lane == 0) {
       // a wait ran out: let the copies already issued land (bounded) before the block retires
-      for (int s = 0; s < KST; ++s)
+      for (int s = 0; s < KST && do_k; ++s)
         for (int k = 0; k < 200000 && !ptx::mbar_try_wait(bar(K_FULL + s), 0) && !ptx::mbar_try_wait(bar(K_FULL + s), 1); ++k) {}
-      for (int s = 0; s < VST; ++s)
+      for (int s = 0; s < VST && do_v; ++s)
         for (int k = 0; k < 200000 && !ptx::mbar_try_wait(bar(V_FULL + s), 0) && !ptx::mbar_try_wait(bar(V_FULL + s), 1); ++k) {}
     }
   } else if (warp == 5) {
