@@ -33,11 +33,12 @@ constexpr uint32_t XCH_BYTES = 128 * XCH_STRIDE * 4;
 constexpr int MAX_NEWTON = 64, MAX_NEWTON_GENERIC = 400;
 
 struct MiscS {
-  unsigned long long bar[8];
+  unsigned long long bar[16];
   uint32_t tmem_base;
   int abort_flag;
 };
-enum BarS { Q_FULL = 0, X_FULL = 1, KB_FULL = 2, KB_EMPTY = 4 };
+enum BarS { Q_FULL = 0, X_FULL = 1, KB_FULL = 2, KB_EMPTY = 4, XBAR = 6 };   // XBAR: [warp 0..3][parity]
+constexpr int CLUSTER_COLS = 512;      // candidates one block of a cluster holds in tensor memory
 
 template <int NST> struct SmemPlan {
   static constexpr uint32_t OFF_Q = 0;
@@ -49,7 +50,7 @@ template <int NST> struct SmemPlan {
 
 struct SelectTcArgs {
   Dims dm;
-  int TQ, n_tiles;        // tiles [0, n_tiles) of every (batch, KV head) are handled here
+  int TQ, tile_base, n_tiles;   // tiles [tile_base, tile_base + n_tiles) of every (batch, KV head) are handled here
   uint32_t tmem_cols;     // power of two >= 32 covering the widest tile
   long long plane_rows;   // rows of one bf16 plane = batch * h_kv * T_s
   uint32_t* mask;
@@ -73,7 +74,7 @@ __global__ void kbar_split_kernel(const float* __restrict__ kbar, __nv_bfloat16*
   planes[2 * n + i] = __float2bfloat16_rn(r2);
 }
 
-template <int NST, int G>
+template <int NST, int G, int CS>
 __global__ void __launch_bounds__(SEL_TC_THREADS, NST == 1 ? 2 : 1)
 select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKB, SelectTcArgs a) {
   using SP = SmemPlan<NST>;
@@ -86,16 +87,22 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   auto bar = [&](int i) { return ptx::smem_u32(&misc->bar[i]); };
   volatile int* abort_flag = &misc->abort_flag;
 
+  // A cluster of CS blocks shares one tile: block `cr` holds candidates [cr*512, cr*512 + 512) of all 128 rows
+  // and the per-row partial sums meet through distributed shared memory (CS = 1: a plain block).
+  const int cr = CS > 1 ? (int)ptx::cluster_ctarank() : 0;
+  const int cid = (int)(blockIdx.x / CS);
   const int groups = dm.batch * dm.h_kv;
-  const int tile = a.n_tiles - 1 - (int)(blockIdx.x / groups);
-  const int grp = (int)(blockIdx.x % groups);
+  const int tile = a.tile_base + a.n_tiles - 1 - cid / groups;
+  const int grp = cid % groups;
   const int b = grp / dm.h_kv, r = grp % dm.h_kv;
   const int TQ = a.TQ;
   constexpr int g_q = G;
   const int i0 = tile * TQ;
   const int c_own = i0 / dm.B;
-  const int n_cand = min(c_own, dm.T_s);
-  const int n_blk = (n_cand + SC - 1) / SC;
+  const int n_cand = min(c_own, dm.T_s);                       // candidates of the tile's rows
+  const int c_lo = cr * CLUSTER_COLS;                          // first candidate this block holds
+  const int n_loc = CS > 1 ? max(0, min(CLUSTER_COLS, n_cand - c_lo)) : n_cand;
+  const int n_blk = (n_loc + SC - 1) / SC;
 
   if (tid == 0) {
     misc->abort_flag = 0;
@@ -109,6 +116,7 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       ptx::mbar_init(bar(KB_FULL + s), 1);
       ptx::mbar_init(bar(KB_EMPTY + s), 1);
     }
+    for (int s = 0; s < 8; ++s) ptx::mbar_init(bar(XBAR + s), CS * 32);
     ptx::fence_barrier_init();
   }
   if (warp == 5) {
@@ -117,18 +125,19 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     ptx::tc_fence_before();
   }
   __syncthreads();
+  if (CS > 1) ptx::cluster_sync_all();     // every block's barriers exist before anybody arrives on them remotely
   ptx::tc_fence_after();
   const uint32_t tmem = misc->tmem_base;
 
   if (warp == 4) {
     // ---------------- producer: Q tile, then the three planes of every 64-chunk block of summaries
-    if (lane == 0 && n_cand > 0) {
+    if (lane == 0 && n_loc > 0) {
       ptx::prefetch_tensormap(&tmQ);
       ptx::prefetch_tensormap(&tmKB);
       ptx::mbar_arrive_expect_tx(bar(Q_FULL), Q_BYTES);
       ptx::tma_load_4d(sbase + SP::OFF_Q, &tmQ, bar(Q_FULL), 0, r * g_q, i0, b);
       ptx::tma_load_4d(sbase + SP::OFF_Q + Q_BYTES / 2, &tmQ, bar(Q_FULL), 64, r * g_q, i0, b);
-      const long long row0 = ((long long)b * dm.h_kv + r) * dm.T_s;
+      const long long row0 = ((long long)b * dm.h_kv + r) * dm.T_s + c_lo;
       bool ok = true;
       for (int cb = 0; cb < n_blk && ok; ++cb) {
         const int s = cb % NST;
@@ -149,7 +158,7 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     }
   } else if (warp == 5) {
     // ---------------- MMA issuer: X[:, cb*64 .. +64) = Q Kbar_hi^T + Q Kbar_mid^T + Q Kbar_lo^T
-    if (lane == 0 && n_cand > 0) {
+    if (lane == 0 && n_loc > 0) {
       constexpr uint32_t IDESC = ptx::idesc_bf16_f32(128, SC, false, false);
       bool ok = ptx::mbar_wait(bar(Q_FULL), 0, abort_flag);
       for (int cb = 0; cb < n_blk && ok; ++cb) {
@@ -183,13 +192,43 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
     const int e_int = dm.e_int;
     const float e = dm.e, xs = dm.x_scale;
-    const int n_chunks = (n_cand + 31) / 32;
+    const int n_chunks = (n_loc + 31) / 32;
     bool ok = true;
     float tau = 0.f;
-    if (n_cand > 0) {
+    if (n_loc > 0) {
       ok = ptx::mbar_wait(bar(X_FULL), 0, abort_flag);
       ptx::tc_fence_after();
     }
+    // Cluster all-reduce of two floats per row: every thread writes its pair into slot [parity][its rank][row]
+    // of every block, arrives (release, cluster scope) on every block's per-warp barrier, waits on its own and
+    // reads the CS pairs back in rank order, so all blocks see bit-identical results and take the same branches.
+    int xround = 0;
+    float xa[CS], xb[CS];
+    auto exchange = [&](float va, float vb) -> bool {
+      if constexpr (CS == 1) {
+        xa[0] = va; xb[0] = vb;
+        return true;
+      } else {
+        const int par = xround & 1;
+        float2* xbuf = reinterpret_cast<float2*>(smem + SP::OFF_XCH);          // [2][CS][128]
+        const uint32_t slot = ptx::smem_u32(&xbuf[(par * CS + cr) * 128 + m]);
+        const uint32_t mybar = bar(XBAR + warp * 2 + par);
+#pragma unroll
+        for (int pr = 0; pr < CS; ++pr) ptx::st_cluster_f32x2(ptx::map_to_rank(slot, pr), va, vb);
+#pragma unroll
+        for (int pr = 0; pr < CS; ++pr) ptx::mbar_arrive_cluster(ptx::map_to_rank(mybar, pr));
+        if (!ptx::mbar_wait_cluster(mybar, (xround >> 1) & 1, abort_flag)) return false;
+#pragma unroll
+        for (int pr = 0; pr < CS; ++pr) {
+          const float2 v = xbuf[(par * CS + pr) * 128 + m];
+          xa[pr] = v.x; xb[pr] = v.y;
+        }
+        ++xround;
+        return true;
+      }
+    };
+    auto xsum_a = [&]() { float v = xa[0]; for (int pr = 1; pr < CS; ++pr) v += xa[pr]; return v; };
+    auto xsum_b = [&]() { float v = xb[0]; for (int pr = 1; pr < CS; ++pr) v += xb[pr]; return v; };
     // Newton on f(tau) = sum [x - tau]_+^e - 1, convex and decreasing.  From the left of the root the iterates
     // rise monotonically and never pass it; from the right one step lands on the left.  The start is the root
     // of the same equation with every candidate taken as active (closed form for alpha = 2 and 1.5), clamped to
@@ -214,7 +253,7 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       if (nt == tau) done = true; else tau = nt;
     };
     float xr[4][32];                               // the whole row, when it has at most 128 candidates
-    const bool in_regs = n_chunks <= 4;
+    const bool in_regs = CS == 1 && n_chunks <= 4;
     if (ok && n_cand > 0 && in_regs) {
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
@@ -263,23 +302,25 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         if (__all_sync(0xffffffffu, done)) break;
       }
     } else if (ok && n_cand > 0) {
-      // longer rows stream from tensor memory every pass
+      // longer rows stream from tensor memory every pass (and, in a cluster, meet the other blocks' partial sums)
       float mx = -INFINITY;
       for (int k = 0; k < n_chunks; ++k) {
         uint32_t v[32];
         DASH_TMEM_LD32(v, lane_addr + k * 32);
         ptx::tmem_wait_ld();
-        const int lim = n_cand - k * 32;
+        const int lim = n_loc - k * 32;
 #pragma unroll
         for (int c = 0; c < 32; ++c) mx = fmaxf(mx, c < lim ? __uint_as_float(v[c]) : -INFINITY);
       }
       mx *= xs;
+      ok = exchange(mx, 0.f);
+      for (int pr = 0; pr < CS; ++pr) mx = fmaxf(mx, xa[pr]);
       float s1 = 0.f, s2 = 0.f;
       for (int k = 0; k < n_chunks; ++k) {
         uint32_t v[32];
         DASH_TMEM_LD32(v, lane_addr + k * 32);
         ptx::tmem_wait_ld();
-        const int lim = n_cand - k * 32;
+        const int lim = n_loc - k * 32;
 #pragma unroll
         for (int c = 0; c < 32; ++c) {
           const float y = c < lim ? fmaf(__uint_as_float(v[c]), xs, -mx) : 0.f;
@@ -287,15 +328,16 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           s2 = fmaf(y, y, s2);
         }
       }
-      tau = start_tau(mx, s1, s2);
+      ok = ok && exchange(s1, s2);
+      tau = start_tau(mx, xsum_a(), xsum_b());
       bool done = false;
-      for (int it = 0; it < max_it; ++it) {
+      for (int it = 0; it < max_it && ok; ++it) {
         float f[4] = {0.f, 0.f, 0.f, 0.f}, g[4] = {0.f, 0.f, 0.f, 0.f};
         for (int k = 0; k < n_chunks; ++k) {
           uint32_t v[32];
           DASH_TMEM_LD32(v, lane_addr + k * 32);
           ptx::tmem_wait_ld();
-          const int lim = n_cand - k * 32;
+          const int lim = n_loc - k * 32;
 #pragma unroll
           for (int c = 0; c < 32; ++c) {
             float mm = fmaxf(fmaf(__uint_as_float(v[c]), xs, -tau), 0.f);
@@ -304,11 +346,13 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             g[c & 3] += pow_em1(mm, e_int, e);
           }
         }
-        newton_step((f[0] + f[1]) + (f[2] + f[3]), (g[0] + g[1]) + (g[2] + g[3]), done);
+        ok = exchange((f[0] + f[1]) + (f[2] + f[3]), (g[0] + g[1]) + (g[2] + g[3]));
+        if (!ok) break;
+        newton_step(xsum_a(), xsum_b(), done);
         if (__all_sync(0xffffffffu, done)) break;
       }
     }
-    if (ok && row_valid && a.tau) a.tau[((long long)b * dm.h_q + r * g_q + hh) * dm.seq_q + i] = tau;
+    if (ok && row_valid && a.tau && cr == 0) a.tau[((long long)b * dm.h_q + r * g_q + hh) * dm.seq_q + i] = tau;
 
     // ---------------- group weights, mask words, log w, compact lists
     // The g_q heads of a token sit in g_q adjacent lanes.  Per 32-chunk step every lane raises its own margins
@@ -362,7 +406,7 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           uint32_t v[32];
           DASH_TMEM_LD32(v, lane_addr + k * 32);
           ptx::tmem_wait_ld();
-          const int lim = n_cand - k * 32;
+          const int lim = n_loc - k * 32;
 #pragma unroll
           for (int c = 0; c < 32; ++c) {
             const float mm = fmaxf(fmaf(__uint_as_float(v[c]), xs, -tau), 0.f);
@@ -386,19 +430,30 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 #pragma unroll
         for (int o = 1; o < G; o <<= 1) bits |= __shfl_xor_sync(0xffffffffu, bits, o);
         DASH_TMEM_ST32(lane_addr + k * 32, lwv);                 // slot q of this lane = chunk own0 + q of step k
-        if (row_valid && hh == 0) mrow[k] = bits | (((c_own >> 5) == k) ? (1u << (c_own & 31)) : 0u);
+        if (row_valid && hh == 0) {
+          const int wj = cr * (CLUSTER_COLS / 32) + k;         // mask word of this step
+          mrow[wj] = bits | (((c_own >> 5) == wj) ? (1u << (c_own & 31)) : 0u);
+        }
         nsel += __popc(bits);
       }
       ptx::tmem_wait_st();
 #pragma unroll
       for (int o = 1; o < G; o <<= 1) slog += __shfl_xor_sync(0xffffffffu, slog, o);
-      if (row_valid && hh == 0) {
-        for (int j = n_chunks; j < dm.W; ++j) mrow[j] = ((c_own >> 5) == j) ? (1u << (c_own & 31)) : 0u;
-        a.count[row_id] = nsel;
+      // counts and sums of log w of the other blocks: total for mu, lower ranks for the list position
+      ok = exchange((float)nsel, slog);
+      int nsel_all = 0, base = 0;
+      float slog_all = 0.f;
+      for (int pr = 0; pr < CS; ++pr) {
+        nsel_all += (int)xa[pr];
+        slog_all += xb[pr];
+        if (pr < cr) base += (int)xa[pr];
       }
-      const float mu = nsel > 0 ? slog / (float)nsel : 0.f;
-      int base = 0;
-      for (int k = 0; k < n_chunks; ++k) {
+      if (row_valid && hh == 0 && cr == 0) {
+        for (int j = (n_cand + 31) / 32; j < dm.W; ++j) mrow[j] = ((c_own >> 5) == j) ? (1u << (c_own & 31)) : 0u;
+        a.count[row_id] = nsel_all;
+      }
+      const float mu = nsel_all > 0 ? slog_all / (float)nsel_all : 0.f;
+      for (int k = 0; k < n_chunks && ok; ++k) {
         uint32_t lwv[32];
         DASH_TMEM_LD32(lwv, lane_addr + k * 32);
         ptx::tmem_wait_ld();
@@ -415,7 +470,7 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
               const int c = own0 + q;
               const long long pos = loff + base + __popc(bits & ((1u << c) - 1u));
               a.blk_bias[pos] = (__uint_as_float(lwv[q]) - mu) * dm.inv_sigma;
-              if (a.blk_idx) a.blk_idx[pos] = k * 32 + c;
+              if (a.blk_idx) a.blk_idx[pos] = c_lo + k * 32 + c;
             }
           }
         }
@@ -431,6 +486,7 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     ptx::tmem_dealloc(tmem, a.tmem_cols);
   }
   if (tid == 0 && misc->abort_flag) report_error(a.sb, DASH_ERR_TIMEOUT, 201);
+  if (CS > 1) ptx::cluster_sync_all();     // nobody leaves while a peer may still write into its shared memory
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -461,18 +517,58 @@ bool encode4(CUtensorMap* out, const void* base, const cuuint64_t* dims, const c
 
 }  // namespace
 
-// Tokens [0, select_sm100_token_limit) can be routed by the tensor-core kernel (0: not applicable).
+// Tokens [0, select_sm100_token_limit) can be routed by the tensor-core kernel (0: not applicable).  A block
+// holds 512 candidates per row in tensor memory; clusters of 2 or 4 blocks extend that to 1024 / 2048.
 int select_sm100_token_limit(const Dims& dm) {
   if (dm.decode || dm.dtype != DASH_BF16 || dm.d != HD || dm.T_s < 1) return 0;
   const int tq = 128 / dm.g_q;
   if (dm.g_q < 2 || tq > dm.B) return 0;
   if (get_encode() == nullptr) return 0;
-  const long long lim = (long long)(512 + 1) * dm.B;   // tiles whose own chunk index is <= 512 have <= 512 candidates
+  const long long lim = (long long)(4 * CLUSTER_COLS + 1) * dm.B;   // own chunk index <= 2048
   return (int)(lim < dm.seq_q ? lim : dm.seq_q);
 }
 
 size_t select_sm100_scratch_bytes(const Dims& dm) {
   return (size_t)3 * dm.batch * dm.h_kv * (size_t)(dm.T_s > 0 ? dm.T_s : 1) * dm.d * sizeof(__nv_bfloat16);
+}
+
+template <int NST, int G, int CS>
+static cudaError_t launch_band(const CUtensorMap& tq, const CUtensorMap& tkb, const SelectTcArgs& a, long long clusters,
+                               cudaStream_t st) {
+  auto kern = select_sm100_kernel<NST, G, CS>;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemPlan<NST>::TOTAL);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(clusters * CS));
+  cfg.blockDim = dim3(SEL_TC_THREADS);
+  cfg.dynamicSmemBytes = SmemPlan<NST>::TOTAL;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = CS;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tq, tkb, a);
+  count_launch();
+  return e;
+}
+
+template <int NST, int CS>
+static cudaError_t launch_band_g(const Dims& dm, const CUtensorMap& tq, const CUtensorMap& tkb, const SelectTcArgs& a,
+                                 long long clusters, cudaStream_t st) {
+  switch (dm.g_q) {
+    case 2: return launch_band<NST, 2, CS>(tq, tkb, a, clusters, st);
+    case 4: return launch_band<NST, 4, CS>(tq, tkb, a, clusters, st);
+    case 8: return launch_band<NST, 8, CS>(tq, tkb, a, clusters, st);
+    case 16: return launch_band<NST, 16, CS>(tq, tkb, a, clusters, st);
+    default: return cudaErrorInvalidValue;
+  }
 }
 
 cudaError_t launch_select_sm100(const Dims& dm, int token_limit, const void* Q, const float* Kbar, void* planes,
@@ -488,13 +584,8 @@ cudaError_t launch_select_sm100(const Dims& dm, int token_limit, const void* Q, 
   SelectTcArgs a;
   a.dm = dm;
   a.TQ = 128 / dm.g_q;
-  a.n_tiles = (token_limit + a.TQ - 1) / a.TQ;
   a.plane_rows = plane_rows;
   a.mask = mask; a.count = count; a.blk_idx = blk_idx; a.blk_bias = blk_bias; a.tau = tau; a.sb = sb;
-  const int max_cand = min(dm.T_s, (token_limit - 1) / dm.B);
-  uint32_t cols = 32;
-  while ((int)cols < ((max_cand + SC - 1) / SC) * SC) cols <<= 1;
-  a.tmem_cols = cols;
 
   CUtensorMap tq, tkb;
   {
@@ -510,31 +601,35 @@ cudaError_t launch_select_sm100(const Dims& dm, int token_limit, const void* Q, 
     cuuint32_t box[4] = {64u, (cuuint32_t)SC, 1u, 1u};
     if (!encode4(&tkb, planes, dims, strides, box)) return cudaErrorInvalidValue;
   }
-  const long long blocks = (long long)a.n_tiles * dm.batch * dm.h_kv;
-#define DASH_SEL_TC(NSTV, GV)                                                                                      \
-  {                                                                                                                 \
-    auto kern = select_sm100_kernel<NSTV, GV>;                                                                      \
-    static bool configured = false;                                                                                 \
-    if (!configured) {                                                                                              \
-      e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemPlan<NSTV>::TOTAL);           \
-      if (e != cudaSuccess) return e;                                                                               \
-      configured = true;                                                                                            \
-    }                                                                                                               \
-    kern<<<(unsigned)blocks, SEL_TC_THREADS, SmemPlan<NSTV>::TOTAL, st>>>(tq, tkb, a);                              \
+  // Bands of tiles by candidate count: <= 512 one block per tile, <= 1024 clusters of 2, <= 2048 clusters of 4.
+  // Tiles are TQ tokens; a tile's candidate count is its own chunk index i0 / B.
+  const int groups = dm.batch * dm.h_kv;
+  const int total_tiles = (token_limit + a.TQ - 1) / a.TQ;
+  auto tiles_up_to = [&](long long max_cand) -> int {      // tiles whose own chunk index is <= max_cand
+    const long long tokens = (max_cand + 1) * dm.B;
+    const long long t = (tokens + a.TQ - 1) / a.TQ;
+    return (int)(t < total_tiles ? t : total_tiles);
+  };
+  const int t1 = tiles_up_to(CLUSTER_COLS), t2 = tiles_up_to(2 * CLUSTER_COLS), t3 = total_tiles;
+  // widest bands first: they are the long-running ones
+  if (t3 > t2) {
+    a.tile_base = t2; a.n_tiles = t3 - t2; a.tmem_cols = 512;
+    if ((e = launch_band_g<2, 4>(dm, tq, tkb, a, (long long)a.n_tiles * groups, st)) != cudaSuccess) return e;
   }
-#define DASH_SEL_TC_G(NSTV)                    \
-  switch (dm.g_q) {                            \
-    case 2: DASH_SEL_TC(NSTV, 2); break;       \
-    case 4: DASH_SEL_TC(NSTV, 4); break;       \
-    case 8: DASH_SEL_TC(NSTV, 8); break;       \
-    case 16: DASH_SEL_TC(NSTV, 16); break;     \
-    default: return cudaErrorInvalidValue;     \
+  if (t2 > t1) {
+    a.tile_base = t1; a.n_tiles = t2 - t1; a.tmem_cols = 512;
+    if ((e = launch_band_g<2, 2>(dm, tq, tkb, a, (long long)a.n_tiles * groups, st)) != cudaSuccess) return e;
   }
-  if (cols <= 256) { DASH_SEL_TC_G(1) } else { DASH_SEL_TC_G(2) }
-#undef DASH_SEL_TC_G
-#undef DASH_SEL_TC
-  count_launch();
-  return cudaGetLastError();
+  {
+    a.tile_base = 0; a.n_tiles = t1;
+    const int max_cand = min(dm.T_s, (int)(((long long)t1 * a.TQ - 1) / dm.B));
+    uint32_t cols = 32;
+    while ((int)cols < ((max_cand + SC - 1) / SC) * SC) cols <<= 1;
+    a.tmem_cols = cols;
+    if (cols <= 256) e = launch_band_g<1, 1>(dm, tq, tkb, a, (long long)a.n_tiles * groups, st);
+    else e = launch_band_g<2, 1>(dm, tq, tkb, a, (long long)a.n_tiles * groups, st);
+  }
+  return e;
 }
 
 }  // namespace dash

@@ -113,14 +113,16 @@ def _check_select(w, inp, p, rt, rows, kv_heads=None):
     dict(h_q=8, h_kv=2, head_dim=128, block=32, seq=1000), dict(h_q=2, h_kv=2, block=64, seq=777),
     dict(h_q=16, h_kv=1, head_dim=128, block=64, seq=1500, batch=2), dict(dtype="f32", seq=300, gamma=3.0),
     dict(h_q=8, h_kv=1, head_dim=64, block=128, seq=1100), dict(seq=15), dict(seq=16), dict(seq=17),
-    dict(h_q=8, h_kv=1, head_dim=128, block=16, seq=9000),      # rows beyond 512 candidates: both Stage-1 kernels
+    dict(h_q=8, h_kv=1, head_dim=128, block=16, seq=9000),      # rows beyond 512 candidates: clusters of two blocks
+    dict(h_q=16, h_kv=1, head_dim=128, block=16, seq=17000, n_planted=6),   # beyond 1024: clusters of four
     dict(h_q=4, h_kv=2, head_dim=128, block=64, seq=2100, alpha=2.0), dict(h_q=32, h_kv=2, head_dim=128, block=32, seq=700),
 ])
 def test_select_matches_oracle(kw):
     w = _wl(**kw)
     inp = synth.make_prefill_inputs(w, DEV)
     p, kbar, ws, rt = _run_select(w, inp)
-    rows = sorted(set(list(range(0, w.seq, 7)) + [w.seq - 1] + list(range(min(w.seq, 3 * w.block)))))
+    step = 7 if w.seq < 12000 else 41
+    rows = sorted(set(list(range(0, w.seq, step)) + [w.seq - 1] + list(range(min(w.seq, 3 * w.block)))))
     ora, clean, nb, nd = _check_select(w, inp, p, rt, rows)
     sizes = [v[0].support.size for v in ora.values()]
     if w.seq > 4 * w.block:
