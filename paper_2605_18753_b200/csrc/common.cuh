@@ -104,6 +104,47 @@ __device__ inline float pow_em1(float m, int e_int, float e) {
 // threshold is then within 4e-6 of the root; iterating on noise only burns passes.
 constexpr float NEWTON_F_TOL = 4e-6f;
 
+// Newton step for the threshold, taken on h(tau) = F(tau)^(1/e) - 1 with F = sum [x - tau]_+^e (G = sum [x - tau]_+^(e-1)):
+// tau += (F - F^(1-1/e)) / G.  h has the root of F - 1 and is convex and decreasing like it (it is the e-norm of the
+// positive parts, minus one), so the iterates still rise monotonically from the left and one step from the right
+// lands on the left; but h is close to linear far from the root, where a step on F - 1 only gains a factor
+// 1 - 1/e of the distance, so the same tolerance is reached in about half the passes.  Near the root the two steps
+// agree to first order ((F - 1) / (e G)).
+__device__ inline float newton_delta(float F, float G, int e_int, float e) {
+  if (e_int == 1) return (F - 1.f) / G;
+  if (e < 1.f) return (F - 1.f) / (e * G);              // alpha > 2: h is no norm, keep the step on F - 1
+  if (e_int == 2) return (F - sqrtf(F)) / G;
+  if (e_int == 4) return (F - F * rsqrtf(sqrtf(F))) / G;    // F^(3/4)
+  return (F - __powf(F, 1.f - 1.f / e)) / G;
+}
+
+// ---- chained launches (programmatic dependent launch).  The kernels of one forward pass run back to back on one
+// stream, each consuming what the previous one wrote.  Launched through launch_chained, a kernel's thread blocks
+// may become resident while the previous kernel drains; chain_wait() then holds them until that kernel has
+// completed and its writes are visible, so it must come before the first global access (reads of the previous
+// kernel's output and writes to anything it may still read alike).  chain_release() lets the NEXT kernel's blocks
+// start arriving once every block of this grid has called it.  Without the launch attribute both are no-ops.
+#ifdef __CUDACC__
+__device__ __forceinline__ void chain_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void chain_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_chained(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                  Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+#endif
+
 void count_launch();
 // Host-side checks shared by the entry points that live outside api.cu.
 int validate_params(const dash_params* p, Dims* dm);

@@ -51,6 +51,8 @@ decode_split_kernel(Dims dm, int n_split, const T* __restrict__ Q, const T* __re
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int split = blockIdx.x, r = blockIdx.y, b = blockIdx.z;
 
+  chain_wait();
+  chain_release();
   int L = kv_len ? kv_len[b] : dm.seq_kv;
   L = max(1, min(L, dm.seq_kv));
   const int c_own = (L - 1) / dm.B;
@@ -176,6 +178,8 @@ __global__ void decode_merge_kernel(Dims dm, int n_split, const float* __restric
   const int lane = threadIdx.x & 31;
   const long long bh = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (bh >= (long long)dm.batch * dm.h_q) return;
+  chain_wait();
+  chain_release();
   const float* p = partials + bh * n_split * (D + 2);
   float M = -INFINITY;
   for (int s = 0; s < n_split; ++s) M = fmaxf(M, p[s * (D + 2)]);
@@ -203,9 +207,10 @@ static cudaError_t launch_dec(const Dims& dm, const void* Q, const void* K, cons
                               float* partials, cudaStream_t st) {
   const int ns = decode_num_splits(dm);
   dim3 grid(ns, dm.h_kv, dm.batch);
-#define DASH_DEC(G)                                                                                          \
-  decode_split_kernel<T, D, G><<<grid, DEC_WARPS * 32, 0, st>>>(dm, ns, (const T*)Q, (const T*)K, (const T*)V, \
-                                                                 kv_len, count, blk_idx, blk_bias, partials)
+  cudaError_t e = cudaSuccess;
+#define DASH_DEC(G)                                                                                              \
+  e = launch_chained(decode_split_kernel<T, D, G>, grid, dim3(DEC_WARPS * 32), 0, st, dm, ns, (const T*)Q,       \
+                     (const T*)K, (const T*)V, kv_len, count, blk_idx, blk_bias, partials)
   switch (dm.g_q) {
     case 1: DASH_DEC(1); break;
     case 2: DASH_DEC(2); break;
@@ -216,20 +221,21 @@ static cudaError_t launch_dec(const Dims& dm, const void* Q, const void* K, cons
   }
 #undef DASH_DEC
   count_launch();
-  cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   const long long rows = (long long)dm.batch * dm.h_q;
-  decode_merge_kernel<T, D><<<(unsigned)((rows + 3) / 4), 128, 0, st>>>(dm, ns, partials, (T*)O);
+  e = launch_chained(decode_merge_kernel<T, D>, dim3((unsigned)((rows + 3) / 4)), dim3(128), 0, st, dm, ns,
+                     (const float*)partials, (T*)O);
   count_launch();
-  return cudaGetLastError();
+  return e;
 }
 
 template <typename T, int D>
 static cudaError_t launch_merge(const Dims& dm, int ns, const float* partials, void* O, cudaStream_t st) {
   const long long rows = (long long)dm.batch * dm.h_q;
-  decode_merge_kernel<T, D><<<(unsigned)((rows + 3) / 4), 128, 0, st>>>(dm, ns, partials, (T*)O);
+  cudaError_t e = launch_chained(decode_merge_kernel<T, D>, dim3((unsigned)((rows + 3) / 4)), dim3(128), 0, st, dm, ns,
+                                 partials, (T*)O);
   count_launch();
-  return cudaGetLastError();
+  return e;
 }
 
 cudaError_t launch_attend_decode_ex(const Dims& dm, const void* Q, const void* K, const void* V, const int* kv_len,

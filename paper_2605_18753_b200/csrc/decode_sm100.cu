@@ -92,19 +92,6 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   const int split = blockIdx.x, r = blockIdx.y, b = blockIdx.z;
   const int n_split = a.n_split;
 
-  int L = a.kv_len ? a.kv_len[b] : dm.seq_kv;
-  L = max(1, min(L, dm.seq_kv));
-  const int c_own = (L - 1) / dm.B;
-  const long long grp = (long long)b * dm.h_kv + r;
-  const int spb = dm.B / SUB;                                   // sub-blocks per routed chunk
-  const int n_routed_sub = a.count[grp] * spb;
-  const int own_tokens = L - c_own * dm.B;                       // 1 .. B
-  const int n_items = n_routed_sub + (own_tokens + SUB - 1) / SUB;
-  const int per = (n_items + n_split - 1) / n_split;
-  const int lo = min(n_items, split * per), hi = min(n_items, lo + per);
-  const int n_own = hi - lo;                                     // <= MAX_RANGE by the host's choice of n_split
-  const int n_steps = (n_own + 1) / 2;
-
   if (tid == 0) {
     misc->abort_flag = 0;
     if ((sbase & 1023u) != 0u) {
@@ -136,6 +123,23 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem = misc->tmem_base;
+
+  // barriers and tensor memory are set up; everything below reads what the routing kernels wrote
+  chain_wait();
+  chain_release();
+  int L = a.kv_len ? a.kv_len[b] : dm.seq_kv;
+  L = max(1, min(L, dm.seq_kv));
+  const int c_own = (L - 1) / dm.B;
+  const long long grp = (long long)b * dm.h_kv + r;
+  const int spb = dm.B / SUB;                                   // sub-blocks per routed chunk
+  const int n_routed_sub = a.count[grp] * spb;
+  const int own_tokens = L - c_own * dm.B;                       // 1 .. B
+  const int n_items = n_routed_sub + (own_tokens + SUB - 1) / SUB;
+  const int per = (n_items + n_split - 1) / n_split;
+  const int lo = min(n_items, split * per), hi = min(n_items, lo + per);
+  const int n_own = hi - lo;                                     // <= MAX_RANGE by the host's choice of n_split
+  const int n_steps = (n_own + 1) / 2;
+
   const long long loff = grp * dm.list_rows;
 
   if (warp == 4) {
@@ -425,6 +429,7 @@ cudaError_t launch_decode_sm100(const Dims& dm, int n_split, const void* Q, cons
   CUtensorMap tk, tv;
   if (!make_kv_map(&tk, K, dm, dm.ks) || !make_kv_map(&tv, V, dm, dm.vs)) return cudaErrorInvalidValue;
   dim3 grid(n_split, dm.h_kv, dm.batch);
+  cudaError_t le = cudaSuccess;
 #define DASH_DEC_TC(G)                                                                                          \
   {                                                                                                             \
     static bool configured = false;                                                                             \
@@ -434,7 +439,7 @@ cudaError_t launch_decode_sm100(const Dims& dm, int n_split, const void* Q, cons
       if (e != cudaSuccess) return e;                                                                           \
       configured = true;                                                                                        \
     }                                                                                                           \
-    decode_sm100_kernel<G><<<grid, DEC_THREADS, DEC_SMEM, st>>>(tk, tv, a);                                     \
+    le = launch_chained(decode_sm100_kernel<G>, grid, dim3(DEC_THREADS), DEC_SMEM, st, tk, tv, a);              \
   }
   switch (dm.g_q) {
     case 1: DASH_DEC_TC(1); break;
@@ -446,7 +451,7 @@ cudaError_t launch_decode_sm100(const Dims& dm, int n_split, const void* Q, cons
   }
 #undef DASH_DEC_TC
   count_launch();
-  return cudaGetLastError();
+  return le;
 }
 
 }  // namespace dash

@@ -179,7 +179,7 @@ select_kernel(Dims dm, int TQ, int xs_stride, int token_base, const T* __restric
           f = warp_sum(f) - 1.f;
           g = warp_sum(g);
           if (!(f > NEWTON_F_TOL)) break;
-          const float nt = tau + f / (e * g);
+          const float nt = tau + newton_delta(f + 1.f, g, e_int, e);
           if (!(nt > tau)) break;
           tau = nt;
         }

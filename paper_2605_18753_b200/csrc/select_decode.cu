@@ -6,9 +6,12 @@
 //                         row reads (one warp per row, four rows in flight per warp) and write the scaled
 //                         chunk logits x = gamma(alpha-1) <q, kbar_c>/sqrt(d) of the g_q heads to a small
 //                         fp32 scratch (b * h_q * T_s floats, stays in L2);
-//   decode_route_kernel   one thread block per (batch, KV head) loads its g_q logit rows into shared memory,
-//                         finds tau per head (Newton from max-1: monotone from below on the convex f),
-//                         forms the group weights, mask words, log w, mu and the compact (chunk, bias) list.
+//   decode_route_kernel   one thread block of 32 warps per (batch, KV head) loads its g_q logit rows into shared
+//                         memory, finds tau per head (Newton from max - 1: monotone from below; a team of
+//                         32 / g_q warps per head), then forms the group weights, mask words, log w, mu and
+//                         the compact (chunk, bias) list.
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace dash {
@@ -17,7 +20,7 @@ namespace {
 
 constexpr int SC_WARPS = 8;
 constexpr int SC_ROWS_PER_BLOCK = 256;   // summary rows one thread block scores
-constexpr int RT_THREADS = 256;
+constexpr int RT_THREADS = 1024;
 constexpr int RT_MAX_NEWTON = 64, RT_MAX_NEWTON_GENERIC = 400;
 
 // Sum V values held by every lane across the warp with V-1+... shuffles (halving exchange): after the
@@ -53,6 +56,8 @@ decode_scores_kernel(Dims dm, const T* __restrict__ Q, const float* __restrict__
   constexpr int VPL = D / 32;   // floats per lane of one summary row
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int r = blockIdx.y, b = blockIdx.z;
+  chain_wait();
+  chain_release();
   int L = kv_len ? kv_len[b] : dm.seq_kv;
   L = max(1, min(L, dm.seq_kv));
   const int n_cand = min((L - 1) / dm.B, dm.T_s);
@@ -104,57 +109,132 @@ decode_scores_kernel(Dims dm, const T* __restrict__ Q, const float* __restrict__
   }
 }
 
+// Row pitch of the logits in decode_route_kernel's shared memory (host and device agree through this helper).
+__host__ __device__ inline int route_stride(int n) { return ((n + 31) / 32) * 32 + 32; }
+
+template <int G>
 __global__ void __launch_bounds__(RT_THREADS)
 decode_route_kernel(Dims dm, const float* __restrict__ xs, const int* __restrict__ kv_len, uint32_t* __restrict__ mask,
                     int* __restrict__ count, int* __restrict__ blk_idx, float* __restrict__ blk_bias,
                     float* __restrict__ tau_out) {
   extern __shared__ __align__(16) float sm[];
+  constexpr int NW = RT_THREADS / 32;
+  static_assert(NW == 32, "one lane per warp segment in the Newton phase");
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int r = blockIdx.x, b = blockIdx.y;
-  const int G = dm.g_q;
+  chain_wait();
+  chain_release();
   int L = kv_len ? kv_len[b] : dm.seq_kv;
   L = max(1, min(L, dm.seq_kv));
   const int c_own = (L - 1) / dm.B;
   const int n_cand = min(c_own, dm.T_s);
-  const int stride = ((n_cand + 31) / 32) * 32 + 32;
-  float* X = sm;                                 // [G][stride]
-  float* taus = X + (size_t)G * stride;          // [G]
-  float* wsum = taus + 32;                       // per-word sum of log w   [W]
+  const int stride = route_stride(n_cand);
+  float* X = sm;                                 // [G][stride] all logits of the group
+  float* taus = X + (size_t)G * stride;          // [G] (32 floats reserved)
+  float2* part = reinterpret_cast<float2*>(taus + 32);   // [2][G][warps per team] partial (F, G) sums; 8-byte aligned:
+                                                 // the offset G * stride + 32 is a multiple of 32 floats
+  float* wsum = taus + 32 + 4 * NW;              // per-word sum of log w   [W]
   int* wcnt = reinterpret_cast<int*>(wsum + dm.W);   // per-word popcount / exclusive prefix [W + 1]
+  float* red = reinterpret_cast<float*>(wcnt + dm.W + 1);   // [NW][G] per-warp maxima
   const long long grp = (long long)b * dm.h_kv + r;
   const float* xg = xs + grp * G * dm.T_s;
-  for (int idx = tid; idx < G * n_cand; idx += RT_THREADS) {
-    const int g = idx / n_cand, c = idx % n_cand;
-    X[(size_t)g * stride + c] = xg[(long long)g * dm.T_s + c];
+
+  // ---- logits -> shared memory, row maxima
+  float mx[G];
+#pragma unroll
+  for (int g = 0; g < G; ++g) {
+    mx[g] = -INFINITY;
+    for (int c = tid; c < n_cand; c += RT_THREADS) {
+      const float x = xg[(long long)g * dm.T_s + c];
+      X[(size_t)g * stride + c] = x;
+      mx[g] = fmaxf(mx[g], x);
+    }
+  }
+  // maxima through the integer warp reduction (one instruction instead of five shuffles): floats map to
+  // signed integers of the same order by flipping the magnitude bits of the negative ones
+  auto f2ord = [](float f) { const int i = __float_as_int(f); return i ^ ((i >> 31) & 0x7fffffff); };
+  auto ord2f = [](int i) { return __int_as_float(i ^ ((i >> 31) & 0x7fffffff)); };
+#pragma unroll
+  for (int g = 0; g < G; ++g) {
+    const int m = __reduce_max_sync(0xffffffffu, f2ord(mx[g]));
+    if (lane == 0) red[warp * G + g] = ord2f(m);
   }
   __syncthreads();
+#pragma unroll
+  for (int g = 0; g < G; ++g) mx[g] = ord2f(__reduce_max_sync(0xffffffffu, f2ord(red[lane * G + g])));
 
+  // ---- tau per head (Newton from max - 1, monotone from below): a team of warps per head; a team's warps each
+  // sum their share of the row, meet at the team's named barrier and all apply the same update.
   const int e_int = dm.e_int;
   const float e = dm.e;
-  for (int g = warp; g < G; g += RT_THREADS / 32) {
+  {
+    // Shuffles retire one warp per clock per SM, so the 2 x 5 of a warp sum times 32 warps would dominate a pass:
+    // about four warps in all do the iteration (one per head from g_q = 4 up), each lane walking its share of the
+    // row with eight independent accumulators; the other warps wait at the block barrier below.
+    constexpr int NWH = G >= 4 ? 1 : 4 / G;       // warps per team
+    constexpr int TEAM = NWH * 32;
+    const int g = min(warp / NWH, G - 1), sw = warp % NWH;
+    const bool in_team = warp < G * NWH;
+    static_assert(2 * G * NWH * 2 <= 4 * NW, "partial-sum buffers fit their reservation");
     const float* x = X + (size_t)g * stride;
     float tau = 0.f;
-    if (n_cand > 0) {
-      float mx = -INFINITY;
-      for (int c = lane; c < n_cand; c += 32) mx = fmaxf(mx, x[c]);
-      mx = warp_max(mx);
-      tau = mx - 1.f;
-      const int max_it = e_int ? RT_MAX_NEWTON : RT_MAX_NEWTON_GENERIC;
+#pragma unroll
+    for (int k = 0; k < G; ++k) if (k == g) tau = mx[k] - 1.f;
+    // the exponent is a compile-time constant inside the loop (alpha = 2, 1.5, 1.25 -> 1, 2, 4; 0 = powf)
+    auto newton = [&](auto ei_tag) {
+      constexpr int EI = decltype(ei_tag)::value;
+      const int max_it = EI ? RT_MAX_NEWTON : RT_MAX_NEWTON_GENERIC;
       for (int it = 0; it < max_it; ++it) {
-        float f = 0.f, gsum = 0.f;
-        for (int c = lane; c < n_cand; c += 32) {
-          const float m = x[c] - tau;
-          if (m > 0.f) { f += pow_e(m, e_int, e); gsum += pow_em1(m, e_int, e); }
+        float F[8], Gs[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) F[u] = Gs[u] = 0.f;
+        int c = sw * 32 + lane;
+        for (; c + 7 * TEAM < n_cand; c += 8 * TEAM) {
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+            const float m = fmaxf(x[c + u * TEAM] - tau, 0.f);
+            F[u] += pow_e(m, EI, e);
+            Gs[u] += pow_em1(m, EI, e);
+          }
         }
-        f = warp_sum(f) - 1.f;
-        gsum = warp_sum(gsum);
-        if (!(f > NEWTON_F_TOL)) break;
-        const float nt = tau + f / (e * gsum);
+        for (; c < n_cand; c += TEAM) {
+          const float m = fmaxf(x[c] - tau, 0.f);
+          F[0] += pow_e(m, EI, e);
+          Gs[0] += pow_em1(m, EI, e);
+        }
+        const float Fw = warp_sum(((F[0] + F[1]) + (F[2] + F[3])) + ((F[4] + F[5]) + (F[6] + F[7])));
+        const float Gw = warp_sum(((Gs[0] + Gs[1]) + (Gs[2] + Gs[3])) + ((Gs[4] + Gs[5]) + (Gs[6] + Gs[7])));
+        float2 t = make_float2(Fw, Gw);
+        if constexpr (NWH > 1) {
+          float2* pp = part + ((it & 1) * G + g) * NWH;
+          if (lane == 0) pp[sw] = t;
+          asm volatile("bar.sync %0, %1;" ::"r"(1 + g), "r"(TEAM) : "memory");
+          // every thread of the team forms the same totals (fixed order) and takes the same step; the other
+          // buffer is written next pass, and this one only after the whole team has passed the next barrier
+          t = pp[lane % NWH];
+#pragma unroll
+          for (int o = 1; o < NWH; o <<= 1) {
+            t.x += __shfl_xor_sync(0xffffffffu, t.x, o);
+            t.y += __shfl_xor_sync(0xffffffffu, t.y, o);
+          }
+        }
+        if (!(t.x - 1.f > NEWTON_F_TOL)) break;
+        const float nt = tau + newton_delta(t.x, t.y, EI, e);
         if (!(nt > tau)) break;
         tau = nt;
       }
+    };
+    if (n_cand > 0 && in_team) {
+      switch (e_int) {
+        case 1: newton(std::integral_constant<int, 1>{}); break;
+        case 2: newton(std::integral_constant<int, 2>{}); break;
+        case 4: newton(std::integral_constant<int, 4>{}); break;
+        default: newton(std::integral_constant<int, 0>{}); break;
+      }
+    } else {
+      tau = 0.f;
     }
-    if (lane == 0) {
+    if (in_team && sw == 0 && lane == 0) {
       taus[g] = tau;
       if (tau_out) tau_out[(long long)b * dm.h_q + r * G + g] = tau;
     }
@@ -239,8 +319,9 @@ size_t select_decode_scratch_bytes(const Dims& dm) {
 }
 
 static size_t route_smem(const Dims& dm) {
-  const int stride = ((dm.T_s + 31) / 32) * 32 + 32;
-  return ((size_t)dm.g_q * stride + 32 + dm.W + dm.W + 1 + 8) * sizeof(float);
+  // logits, taus, per-word sums and counts, per-warp maxima, two buffers of per-warp (F, G) partials
+  return ((size_t)dm.g_q * route_stride(dm.T_s) + 32 + dm.W + dm.W + 1 + 8 + (size_t)(RT_THREADS / 32) * dm.g_q +
+          4 * (RT_THREADS / 32) + 8) * sizeof(float);
 }
 
 bool select_decode_supported(const Dims& dm) { return dm.decode && route_smem(dm) <= 200 * 1024; }
@@ -251,7 +332,9 @@ cudaError_t launch_select_decode(const Dims& dm, const void* Q, const float* Kba
   const int blocks_x = (dm.T_s + SC_ROWS_PER_BLOCK - 1) / SC_ROWS_PER_BLOCK;
   if (blocks_x > 0) {
     dim3 grid(blocks_x, dm.h_kv, dm.batch);
-#define DASH_SC(T, D, G) decode_scores_kernel<T, D, G><<<grid, SC_WARPS * 32, 0, st>>>(dm, (const T*)Q, Kbar, kv_len, scratch)
+    cudaError_t le = cudaSuccess;
+#define DASH_SC(T, D, G) \
+  le = launch_chained(decode_scores_kernel<T, D, G>, grid, dim3(SC_WARPS * 32), 0, st, dm, (const T*)Q, Kbar, kv_len, scratch)
 #define DASH_SC_G(T, D)                                \
   switch (dm.g_q) {                                    \
     case 1: DASH_SC(T, D, 1); break;                   \
@@ -269,20 +352,33 @@ cudaError_t launch_select_decode(const Dims& dm, const void* Q, const float* Kba
 #undef DASH_SC_G
 #undef DASH_SC
     count_launch();
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
+    if (le != cudaSuccess) return le;
   }
   const size_t smem = route_smem(dm);
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(decode_route_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-    if (e != cudaSuccess) return e;
-    configured = true;
+  cudaError_t re = cudaSuccess;
+#define DASH_RT(G)                                                                                                  \
+  {                                                                                                                 \
+    static bool configured = false;                                                                                 \
+    if (!configured) {                                                                                              \
+      cudaError_t e = cudaFuncSetAttribute(decode_route_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize,     \
+                                           200 * 1024);                                                             \
+      if (e != cudaSuccess) return e;                                                                               \
+      configured = true;                                                                                            \
+    }                                                                                                               \
+    re = launch_chained(decode_route_kernel<G>, dim3(dm.h_kv, dm.batch), dim3(RT_THREADS), smem, st, dm,           \
+                        (const float*)scratch, kv_len, mask, count, blk_idx, blk_bias, tau);                       \
   }
-  decode_route_kernel<<<dim3(dm.h_kv, dm.batch), RT_THREADS, smem, st>>>(dm, scratch, kv_len, mask, count, blk_idx,
-                                                                       blk_bias, tau);
+  switch (dm.g_q) {
+    case 1: DASH_RT(1) break;
+    case 2: DASH_RT(2) break;
+    case 4: DASH_RT(4) break;
+    case 8: DASH_RT(8) break;
+    case 16: DASH_RT(16) break;
+    default: return cudaErrorInvalidValue;
+  }
+#undef DASH_RT
   count_launch();
-  return cudaGetLastError();
+  return re;
 }
 
 }  // namespace dash

@@ -229,8 +229,9 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     };
     auto xsum_a = [&]() { float v = xa[0]; for (int pr = 1; pr < CS; ++pr) v += xa[pr]; return v; };
     auto xsum_b = [&]() { float v = xb[0]; for (int pr = 1; pr < CS; ++pr) v += xb[pr]; return v; };
-    // Newton on f(tau) = sum [x - tau]_+^e - 1, convex and decreasing.  From the left of the root the iterates
-    // rise monotonically and never pass it; from the right one step lands on the left.  The start is the root
+    // Newton on f(tau) = sum [x - tau]_+^e - 1 (steps taken on f^(1/e), see newton_delta), convex and decreasing.
+    // From the left of the root the iterates rise monotonically and never pass it; from the right one step lands
+    // on the left.  The start is the root
     // of the same equation with every candidate taken as active (closed form for alpha = 2 and 1.5), clamped to
     // max - 1 <= tau* < max, which saves the slow first halvings of a start at max - 1.
     const int max_it = e_int ? MAX_NEWTON : MAX_NEWTON_GENERIC;
@@ -247,9 +248,8 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     };
     auto newton_step = [&](float f, float g, bool& done) {
       if (done) return;
-      f -= 1.f;
-      if (fabsf(f) <= NEWTON_F_TOL || !(g > 0.f)) { done = true; return; }
-      const float nt = tau + f / (e * g);
+      if (fabsf(f - 1.f) <= NEWTON_F_TOL || !(g > 0.f)) { done = true; return; }
+      const float nt = tau + newton_delta(f, g, e_int, e);
       if (nt == tau) done = true; else tau = nt;
     };
     float xr[4][32];                               // the whole row, when it has at most 128 candidates
