@@ -85,14 +85,14 @@ __device__ inline float warp_max(float v) {
 }
 
 // m^e for the integer exponents of alpha = 2, 1.5, 1.25; powf otherwise.  m >= 0.
-__device__ inline float pow_e(float m, int e_int, float e) {
+__device__ __forceinline__ float pow_e(float m, int e_int, float e) {
   if (e_int == 1) return m;
   if (e_int == 2) return m * m;
   if (e_int == 4) { float s = m * m; return s * s; }
   return m > 0.f ? __powf(m, e) : 0.f;
 }
 // m^(e-1)
-__device__ inline float pow_em1(float m, int e_int, float e) {
+__device__ __forceinline__ float pow_em1(float m, int e_int, float e) {
   if (e_int == 1) return m > 0.f ? 1.f : 0.f;
   if (e_int == 2) return m;
   if (e_int == 4) return m * m * m;
@@ -110,7 +110,7 @@ constexpr float NEWTON_F_TOL = 4e-6f;
 // lands on the left; but h is close to linear far from the root, where a step on F - 1 only gains a factor
 // 1 - 1/e of the distance, so the same tolerance is reached in about half the passes.  Near the root the two steps
 // agree to first order ((F - 1) / (e G)).
-__device__ inline float newton_delta(float F, float G, int e_int, float e) {
+__device__ __forceinline__ float newton_delta(float F, float G, int e_int, float e) {
   if (e_int == 1) return (F - 1.f) / G;
   if (e < 1.f) return (F - 1.f) / (e * G);              // alpha > 2: h is no norm, keep the step on F - 1
   if (e_int == 2) return (F - sqrtf(F)) / G;

@@ -131,9 +131,9 @@ decode_route_kernel(Dims dm, const float* __restrict__ xs, const int* __restrict
   const int stride = route_stride(n_cand);
   float* X = sm;                                 // [G][stride] all logits of the group
   float* taus = X + (size_t)G * stride;          // [G] (32 floats reserved)
-  float2* part = reinterpret_cast<float2*>(taus + 32);   // [2][G][warps per team] partial (F, G) sums; 8-byte aligned:
-                                                 // the offset G * stride + 32 is a multiple of 32 floats
-  float* wsum = taus + 32 + 4 * NW;              // per-word sum of log w   [W]
+  float2* part = reinterpret_cast<float2*>(taus + 32);   // [RT_THREADS] per-lane (F, G) partials + [G] control words;
+                                                 // 8-byte aligned: the offset G * stride + 32 is a multiple of 32 floats
+  float* wsum = taus + 32 + 2 * RT_THREADS + 32; // per-word sum of log w   [W]
   int* wcnt = reinterpret_cast<int*>(wsum + dm.W);   // per-word popcount / exclusive prefix [W + 1]
   float* red = reinterpret_cast<float*>(wcnt + dm.W + 1);   // [NW][G] per-warp maxima
   const long long grp = (long long)b * dm.h_kv + r;
@@ -163,19 +163,19 @@ decode_route_kernel(Dims dm, const float* __restrict__ xs, const int* __restrict
 #pragma unroll
   for (int g = 0; g < G; ++g) mx[g] = ord2f(__reduce_max_sync(0xffffffffu, f2ord(red[lane * G + g])));
 
-  // ---- tau per head (Newton from max - 1, monotone from below): a team of warps per head; a team's warps each
-  // sum their share of the row, meet at the team's named barrier and all apply the same update.
+  // ---- tau per head (Newton from max - 1, monotone from below).  Shuffles retire one warp per clock per SM, so
+  // warp sums in all 32 warps would dominate a pass.  Instead the warps form g_q teams, one per head: every lane
+  // sums its few logits and stores the pair (F, G) unreduced; after the team's named barrier the team's first
+  // warp adds the columns, does the one warp sum, takes the Newton step and publishes (tau, done).
   const int e_int = dm.e_int;
   const float e = dm.e;
   {
-    // Shuffles retire one warp per clock per SM, so the 2 x 5 of a warp sum times 32 warps would dominate a pass:
-    // about four warps in all do the iteration (one per head from g_q = 4 up), each lane walking its share of the
-    // row with eight independent accumulators; the other warps wait at the block barrier below.
-    constexpr int NWH = G >= 4 ? 1 : 4 / G;       // warps per team
+    constexpr int NWH = G <= 8 ? NW / G : 1;      // warps per team (named barriers 1..8); one warp per head beyond
     constexpr int TEAM = NWH * 32;
     const int g = min(warp / NWH, G - 1), sw = warp % NWH;
     const bool in_team = warp < G * NWH;
-    static_assert(2 * G * NWH * 2 <= 4 * NW, "partial-sum buffers fit their reservation");
+    float2* pt = part + (size_t)g * TEAM;         // this team's [TEAM] lane partials
+    float2* ctrl = part + (size_t)G * TEAM + g;   // (tau, continue?) of this team
     const float* x = X + (size_t)g * stride;
     float tau = 0.f;
 #pragma unroll
@@ -184,11 +184,22 @@ decode_route_kernel(Dims dm, const float* __restrict__ xs, const int* __restrict
     auto newton = [&](auto ei_tag) {
       constexpr int EI = decltype(ei_tag)::value;
       const int max_it = EI ? RT_MAX_NEWTON : RT_MAX_NEWTON_GENERIC;
+      // a lane's first eight logits stay in registers over the passes (all of them up to 8 * TEAM candidates)
+      float xr[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int c = sw * 32 + lane + u * TEAM;
+        xr[u] = c < n_cand ? x[c] : -INFINITY;
+      }
       for (int it = 0; it < max_it; ++it) {
         float F[8], Gs[8];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) F[u] = Gs[u] = 0.f;
-        int c = sw * 32 + lane;
+        for (int u = 0; u < 8; ++u) {
+          const float m = fmaxf(xr[u] - tau, 0.f);
+          F[u] = pow_e(m, EI, e);
+          Gs[u] = pow_em1(m, EI, e);
+        }
+        int c = sw * 32 + lane + 8 * TEAM;
         for (; c + 7 * TEAM < n_cand; c += 8 * TEAM) {
 #pragma unroll
           for (int u = 0; u < 8; ++u) {
@@ -197,31 +208,49 @@ decode_route_kernel(Dims dm, const float* __restrict__ xs, const int* __restrict
             Gs[u] += pow_em1(m, EI, e);
           }
         }
-        for (; c < n_cand; c += TEAM) {
-          const float m = fmaxf(x[c] - tau, 0.f);
-          F[0] += pow_e(m, EI, e);
-          Gs[0] += pow_em1(m, EI, e);
-        }
-        const float Fw = warp_sum(((F[0] + F[1]) + (F[2] + F[3])) + ((F[4] + F[5]) + (F[6] + F[7])));
-        const float Gw = warp_sum(((Gs[0] + Gs[1]) + (Gs[2] + Gs[3])) + ((Gs[4] + Gs[5]) + (Gs[6] + Gs[7])));
-        float2 t = make_float2(Fw, Gw);
-        if constexpr (NWH > 1) {
-          float2* pp = part + ((it & 1) * G + g) * NWH;
-          if (lane == 0) pp[sw] = t;
-          asm volatile("bar.sync %0, %1;" ::"r"(1 + g), "r"(TEAM) : "memory");
-          // every thread of the team forms the same totals (fixed order) and takes the same step; the other
-          // buffer is written next pass, and this one only after the whole team has passed the next barrier
-          t = pp[lane % NWH];
 #pragma unroll
-          for (int o = 1; o < NWH; o <<= 1) {
-            t.x += __shfl_xor_sync(0xffffffffu, t.x, o);
-            t.y += __shfl_xor_sync(0xffffffffu, t.y, o);
+        for (int u = 0; u < 8; ++u) {
+          if (c < n_cand) {
+            const float m = fmaxf(x[c] - tau, 0.f);
+            F[u] += pow_e(m, EI, e);
+            Gs[u] += pow_em1(m, EI, e);
+          }
+          c += TEAM;
+        }
+        float2 t = make_float2(((F[0] + F[1]) + (F[2] + F[3])) + ((F[4] + F[5]) + (F[6] + F[7])),
+                               ((Gs[0] + Gs[1]) + (Gs[2] + Gs[3])) + ((Gs[4] + Gs[5]) + (Gs[6] + Gs[7])));
+        bool go = true;
+        if constexpr (NWH > 1) {
+          pt[sw * 32 + lane] = t;
+          asm volatile("bar.sync %0, %1;" ::"r"(1 + g), "r"(TEAM) : "memory");
+          if (sw == 0) {
+#pragma unroll
+            for (int k = 1; k < NWH; ++k) {
+              const float2 o = pt[k * 32 + lane];
+              t.x += o.x;
+              t.y += o.y;
+            }
           }
         }
-        if (!(t.x - 1.f > NEWTON_F_TOL)) break;
-        const float nt = tau + newton_delta(t.x, t.y, EI, e);
-        if (!(nt > tau)) break;
-        tau = nt;
+        if (NWH == 1 || sw == 0) {
+          t.x = warp_sum(t.x);
+          t.y = warp_sum(t.y);
+          go = t.x - 1.f > NEWTON_F_TOL;
+          if (go) {
+            const float nt = tau + newton_delta(t.x, t.y, EI, e);
+            go = nt > tau;
+            if (go) tau = nt;
+          }
+          if (NWH > 1 && lane == 0) *ctrl = make_float2(tau, go ? 1.f : 0.f);
+        }
+        if constexpr (NWH > 1) {
+          // the partials are rewritten only after this barrier, the control word only after the next pass's first
+          asm volatile("bar.sync %0, %1;" ::"r"(1 + g), "r"(TEAM) : "memory");
+          const float2 cw = *ctrl;
+          tau = cw.x;
+          go = cw.y != 0.f;
+        }
+        if (!go) break;
       }
     };
     if (n_cand > 0 && in_team) {
@@ -319,9 +348,9 @@ size_t select_decode_scratch_bytes(const Dims& dm) {
 }
 
 static size_t route_smem(const Dims& dm) {
-  // logits, taus, per-word sums and counts, per-warp maxima, two buffers of per-warp (F, G) partials
-  return ((size_t)dm.g_q * route_stride(dm.T_s) + 32 + dm.W + dm.W + 1 + 8 + (size_t)(RT_THREADS / 32) * dm.g_q +
-          4 * (RT_THREADS / 32) + 8) * sizeof(float);
+  // logits, taus, per-lane (F, G) partials and control words, per-word sums and counts, per-warp maxima
+  return ((size_t)dm.g_q * route_stride(dm.T_s) + 32 + 2 * RT_THREADS + 32 + dm.W + dm.W + 1 + 8 +
+          (size_t)(RT_THREADS / 32) * dm.g_q) * sizeof(float);
 }
 
 bool select_decode_supported(const Dims& dm) { return dm.decode && route_smem(dm) <= 200 * 1024; }
