@@ -22,6 +22,8 @@ attend_prefill_generic_kernel(Dims dm, const T* __restrict__ Q, const T* __restr
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const long long gw = (long long)blockIdx.x * AG_WARPS + warp;
   const long long total = (long long)dm.batch * dm.seq_q * dm.h_q;
+  chain_wait();
+  chain_release();
   if (gw >= total) return;
   const int h = (int)(gw % dm.h_q);
   const int i = dm.seq_q - 1 - (int)((gw / dm.h_q) % dm.seq_q);  // long rows first
@@ -103,9 +105,10 @@ cudaError_t launch_attend_prefill_generic(const Dims& dm, const void* Q, const v
                                           const uint32_t* mask, const float* blk_bias, void* O, cudaStream_t st) {
   const long long total = (long long)dm.batch * dm.seq_q * dm.h_q;
   const unsigned grid = (unsigned)((total + AG_WARPS - 1) / AG_WARPS);
+  cudaError_t le = cudaSuccess;
 #define DASH_LAUNCH_AG(T, D)                                                                                    \
-  attend_prefill_generic_kernel<T, D><<<grid, AG_WARPS * 32, 0, st>>>(dm, (const T*)Q, (const T*)K, (const T*)V, \
-                                                                      mask, blk_bias, (T*)O)
+  le = launch_chained(attend_prefill_generic_kernel<T, D>, dim3(grid), dim3(AG_WARPS * 32), 0, st, dm,          \
+                      (const T*)Q, (const T*)K, (const T*)V, mask, blk_bias, (T*)O)
   if (dm.dtype == DASH_BF16) {
     if (dm.d == 128) DASH_LAUNCH_AG(__nv_bfloat16, 128); else DASH_LAUNCH_AG(__nv_bfloat16, 64);
   } else {
@@ -113,7 +116,7 @@ cudaError_t launch_attend_prefill_generic(const Dims& dm, const void* Q, const v
   }
 #undef DASH_LAUNCH_AG
   count_launch();
-  return cudaGetLastError();
+  return le;
 }
 
 }  // namespace dash

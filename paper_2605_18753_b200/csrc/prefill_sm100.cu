@@ -125,6 +125,9 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem = misc->tmem_base;
+  // barriers and tensor memory are set up; from here on the kernel reads what the routing kernels wrote
+  chain_wait();
+  chain_release();
 
   if (warp == 4 || warp == 6) {
     // =========================== producers ===========================
@@ -574,9 +577,10 @@ cudaError_t launch_attend_prefill_sm100(const Dims& dm, const void* Q, const voi
     configured = true;
   }
   const long long blocks = (long long)a.n_tiles * dm.batch * dm.h_kv;
-  attend_prefill_sm100_kernel<<<(unsigned)blocks, PF_THREADS, PF_SMEM, st>>>(tq, tk, tv, a);
+  cudaError_t le = launch_chained(attend_prefill_sm100_kernel, dim3((unsigned)blocks), dim3(PF_THREADS), PF_SMEM, st, tq,
+                                  tk, tv, a);
   count_launch();
-  return cudaGetLastError();
+  return le;
 }
 
 }  // namespace dash

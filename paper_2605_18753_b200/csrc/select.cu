@@ -76,6 +76,8 @@ select_kernel(Dims dm, int TQ, int xs_stride, int token_base, const T* __restric
   const int r = blockIdx.y, b = blockIdx.z;
   const int g_q = dm.g_q;
   const int rows = TQ * g_q;
+  chain_wait();
+  chain_release();
 
   int i0, c_own, n_cand;
   if (dm.decode) {
@@ -261,10 +263,10 @@ static cudaError_t launch_one(const Dims& dm, const SelectPlan& pl, int token_ba
   }
   const int tiles = dm.decode ? 1 : (dm.seq_q - token_base + pl.TQ - 1) / pl.TQ;
   dim3 grid(tiles, dm.h_kv, dm.batch);
-  kern<<<grid, SEL_THREADS, pl.smem, st>>>(dm, pl.TQ, pl.xs_stride, token_base, (const T*)Q, Kbar, kv_len, mask, count,
-                                            blk_idx, blk_bias, tau);
+  cudaError_t le = launch_chained(kern, grid, dim3(SEL_THREADS), pl.smem, st, dm, pl.TQ, pl.xs_stride, token_base,
+                                  (const T*)Q, Kbar, kv_len, mask, count, blk_idx, blk_bias, tau);
   count_launch();
-  return cudaGetLastError();
+  return le;
 }
 
 template <typename T, int D>

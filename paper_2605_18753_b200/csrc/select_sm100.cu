@@ -63,6 +63,8 @@ struct SelectTcArgs {
 
 __global__ void kbar_split_kernel(const float* __restrict__ kbar, __nv_bfloat16* __restrict__ planes, long long n) {
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  chain_wait();
+  chain_release();
   if (i >= n) return;
   const float x = kbar[i];
   const __nv_bfloat16 hi = __float2bfloat16_rn(x);
@@ -128,6 +130,9 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   if (CS > 1) ptx::cluster_sync_all();     // every block's barriers exist before anybody arrives on them remotely
   ptx::tc_fence_after();
   const uint32_t tmem = misc->tmem_base;
+  // barriers and tensor memory are set up; from here on the kernel reads the planes the previous kernel wrote
+  chain_wait();
+  chain_release();
 
   if (warp == 4) {
     // ---------------- producer: Q tile, then the three planes of every 64-chunk block of summaries
@@ -547,13 +552,15 @@ static cudaError_t launch_band(const CUtensorMap& tq, const CUtensorMap& tkb, co
   cfg.blockDim = dim3(SEL_TC_THREADS);
   cfg.dynamicSmemBytes = SmemPlan<NST>::TOTAL;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = CS;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // see launch_chained
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tq, tkb, a);
   count_launch();
   return e;
@@ -576,9 +583,9 @@ cudaError_t launch_select_sm100(const Dims& dm, int token_limit, const void* Q, 
                                 StatusBlock* sb, cudaStream_t st) {
   const long long plane_rows = (long long)dm.batch * dm.h_kv * dm.T_s;
   const long long n = plane_rows * dm.d;
-  kbar_split_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(Kbar, (__nv_bfloat16*)planes, n);
+  cudaError_t e = launch_chained(kbar_split_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, st, Kbar,
+                                 (__nv_bfloat16*)planes, n);
   count_launch();
-  cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
 
   SelectTcArgs a;

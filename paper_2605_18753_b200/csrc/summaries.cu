@@ -20,6 +20,8 @@ summaries_kernel(Dims dm, const T* __restrict__ K, const float* __restrict__ qba
   const int lane = threadIdx.x & 31;
   const long long warp = (long long)blockIdx.x * SUM_WARPS + (threadIdx.x >> 5);
   const long long total = (long long)dm.batch * dm.h_kv * num_blocks;
+  chain_wait();       // before any exit: the kernel behind this one relies on it having outlasted its predecessor
+  chain_release();
   if (warp >= total) return;
   const int c = first_block + (int)(warp % num_blocks);
   const int r = (int)((warp / num_blocks) % dm.h_kv);
@@ -106,9 +108,10 @@ cudaError_t launch_summaries(const Dims& dm, const void* K, const float* qbar, l
   const long long total = (long long)dm.batch * dm.h_kv * num_blocks;
   const unsigned grid = (unsigned)((total + SUM_WARPS - 1) / SUM_WARPS);
   const dim3 block(SUM_WARPS * 32);
-#define DASH_LAUNCH_SUM(T, D)                                                                         \
-  summaries_kernel<T, D><<<grid, block, 0, st>>>(dm, (const T*)K, qbar, qbar_chunk_stride, kv_len,    \
-                                                 first_block, num_blocks, Kbar)
+  cudaError_t le = cudaSuccess;
+#define DASH_LAUNCH_SUM(T, D)                                                                               \
+  le = launch_chained(summaries_kernel<T, D>, dim3(grid), block, 0, st, dm, (const T*)K, qbar,              \
+                      qbar_chunk_stride, kv_len, first_block, num_blocks, Kbar)
   if (dm.B % SUM_UNROLL != 0) return cudaErrorInvalidValue;
   if (dm.dtype == DASH_BF16) {
     if (dm.d == 128) DASH_LAUNCH_SUM(__nv_bfloat16, 128); else DASH_LAUNCH_SUM(__nv_bfloat16, 64);
@@ -116,7 +119,7 @@ cudaError_t launch_summaries(const Dims& dm, const void* K, const float* qbar, l
     if (dm.d == 128) DASH_LAUNCH_SUM(float, 128); else DASH_LAUNCH_SUM(float, 64);
   }
   count_launch();
-  return cudaGetLastError();
+  return le;
 #undef DASH_LAUNCH_SUM
 }
 
