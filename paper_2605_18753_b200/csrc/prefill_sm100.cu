@@ -26,10 +26,9 @@ namespace dash {
 
 namespace {
 
-constexpr bool P_TMEM = true;     // P (bf16) reaches the PV MMA through tensor memory (over the S columns), not smem
-constexpr bool QK_FIRST = true;   // issue S of step j+1 before PV of step j even if its K tile has to be waited for
 constexpr int NKV = 64;           // KV tokens per step
-constexpr int KST = 3, VST = 2;   // ring depths
+constexpr int KST = 2, VST = 2;   // ring depths: stage = step parity, like the S/P buffers, so that the two
+                                  // MMA completion barriers of a step also release its K and V stages
 constexpr int PF_THREADS = 224;   // 4 softmax warps, K producer, MMA issuer, V/bias producer
 constexpr int HD = 128;           // head_dim
 constexpr uint32_t TMEM_COLS = 256;  // S0 [0,64), S1 [64,128), O [128,256)
@@ -37,15 +36,16 @@ constexpr float RESCALE_LOG2 = 8.f;  // the running maximum is moved only when i
 
 constexpr uint32_t Q_BYTES = 128 * HD * 2;           // 32 KiB: two 128x64 K-major regions
 constexpr uint32_t KV_TILE_BYTES = NKV * HD * 2;     // 16 KiB: two 64x64 regions
-constexpr uint32_t P_BYTES = P_TMEM ? 0 : 128 * NKV * 2;   // 16 KiB when P goes through shared memory
 constexpr uint32_t OFF_Q = 0;
 constexpr uint32_t OFF_K = OFF_Q + Q_BYTES;
 constexpr uint32_t OFF_V = OFF_K + KST * KV_TILE_BYTES;
-constexpr uint32_t OFF_P = OFF_V + VST * KV_TILE_BYTES;
-constexpr uint32_t OFF_MISC = OFF_P + P_BYTES;
+constexpr uint32_t OFF_MISC = OFF_V + VST * KV_TILE_BYTES;
 constexpr int MAX_TQ = 64;
-enum Bar { Q_FULL = 0, META, S_FULL = 2, S_EMPTY = 4, P_FULL = 6, P_EMPTY = 8, V_FULL = 9, V_EMPTY = 9 + VST,
-           K_FULL = 9 + 2 * VST, K_EMPTY = 9 + 2 * VST + KST, N_BARS = 9 + 2 * VST + 2 * KST };
+// S_FULL[j&1]: QK of step j complete (S readable; K stage j&1 reusable).  PV_DONE[j&1]: PV of step j complete (O stable;
+// S/P buffer and V stage j&1 reusable).  Every tcgen05.commit and every barrier test costs the issuing thread as
+// much as an MMA, so each product signals exactly one barrier and the producers listen to the same ones.
+enum Bar { Q_FULL = 0, META, S_FULL = 2, PV_DONE = 4, P_FULL = 6, V_FULL = 8, K_FULL = 10, N_BARS = 12 };
+static_assert(KST == 2 && VST == 2, "stage = step parity");
 struct Misc {
   unsigned long long bar[N_BARS];
   uint32_t tmem_base;
@@ -100,21 +100,14 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
     ptx::mbar_init(bar(META), 1);
     for (int s = 0; s < 2; ++s) {
       ptx::mbar_init(bar(S_FULL + s), 1);
-      ptx::mbar_init(bar(S_EMPTY + s), 128);
-    }
-    for (int s = 0; s < KST; ++s) {
+      ptx::mbar_init(bar(PV_DONE + s), 1);
       ptx::mbar_init(bar(K_FULL + s), 1);
-      ptx::mbar_init(bar(K_EMPTY + s), 1);
-    }
-    for (int s = 0; s < VST; ++s) {
       ptx::mbar_init(bar(V_FULL + s), 1);
-      ptx::mbar_init(bar(V_EMPTY + s), 1);
     }
     // two P_FULL barriers (step parity): the softmax warps may finish step j+1 before the MMA thread has
     // looked at step j, and a single barrier's phase bit cannot tell j from j+2
     ptx::mbar_init(bar(P_FULL), 128);
     ptx::mbar_init(bar(P_FULL + 1), 128);
-    ptx::mbar_init(bar(P_EMPTY), 1);
     ptx::fence_barrier_init();
   }
   if (warp == 5) {
@@ -128,6 +121,10 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
   // barriers and tensor memory are set up; from here on the kernel reads what the routing kernels wrote
   chain_wait();
   chain_release();
+  // a workspace whose status word already holds an error makes every role leave at its first wait: after one
+  // block's wait has run out, the rest of the grid retires in microseconds instead of a wait limit each
+  if (a.sb && *reinterpret_cast<volatile int*>(&a.sb->status) != 0) *abort_flag = 1;
+  __syncthreads();
 
   if (warp == 4 || warp == 6) {
     // =========================== producers ===========================
@@ -240,7 +237,7 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
       }
       return true;
     };
-    int j = 0, ks = 0, kph = 1, vs = 0, vph = 1;   // ring slots and the parity to wait for on the empty barriers
+    int j = 0;
     bool ok = true;
     Blk cur, nxt;
     bool has = pop(nxt);
@@ -250,19 +247,20 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
       const int nsub = (cur.c == c_own) ? own_steps : sub_per_blk;
       for (int sub = 0; sub < nsub && ok; ++sub, ++j) {
         const int kv0 = cur.c * dm.B + sub * NKV;
+        const int st = j & 1, prev_ph = ((j >> 1) - 1) & 1;   // stage, and the phase of step j-2 on the completion barriers
         if (do_k) {
-          ok = ptx::mbar_wait(bar(K_EMPTY + ks), kph, abort_flag);
+          if (j >= 2) ok = ptx::mbar_wait(bar(S_FULL + st), prev_ph, abort_flag);   // QK of step j-2 has read the stage
           if (!ok) break;
           if (lane == 0) {
-            const uint32_t dst = sbase + OFF_K + ks * KV_TILE_BYTES;
-            ptx::mbar_arrive_expect_tx(bar(K_FULL + ks), KV_TILE_BYTES);
-            ptx::tma_load_4d(dst, &tmK, bar(K_FULL + ks), 0, r, kv0, b);
-            ptx::tma_load_4d(dst + KV_TILE_BYTES / 2, &tmK, bar(K_FULL + ks), 64, r, kv0, b);
+            const uint32_t dst = sbase + OFF_K + st * KV_TILE_BYTES;
+            ptx::mbar_arrive_expect_tx(bar(K_FULL + st), KV_TILE_BYTES);
+            ptx::tma_load_4d(dst, &tmK, bar(K_FULL + st), 0, r, kv0, b);
+            ptx::tma_load_4d(dst + KV_TILE_BYTES / 2, &tmK, bar(K_FULL + st), 64, r, kv0, b);
           }
-          if (++ks == KST) { ks = 0; kph ^= 1; }
           continue;
         }
-        ok = ptx::mbar_wait(bar(V_EMPTY + vs), vph, abort_flag);
+        const int vs = st;
+        if (j >= 2) ok = ptx::mbar_wait(bar(PV_DONE + st), prev_ph, abort_flag);     // PV of step j-2 has read the stage
         if (!ok) break;
         for (int q = 0; q < 2; ++q) {
           const int t = lane + 32 * q;
@@ -276,7 +274,6 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
           ptx::tma_load_4d(dst, &tmV, bar(V_FULL + vs), 0, r, kv0, b);
           ptx::tma_load_4d(dst + KV_TILE_BYTES / 2, &tmV, bar(V_FULL + vs), 64, r, kv0, b);
         }
-        if (++vs == VST) { vs = 0; vph ^= 1; }
       }
     }
     if (!ok && lane == 0) {
@@ -288,6 +285,8 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
     }
   } else if (warp == 5) {
     // =========================== MMA issuer ===========================
+    // Per step: S_{j+1} = Q K_{j+1}^T (needs only its K tile), then O += P_j V_j.  V_FULL is not tested here: the
+    // softmax threads wait for it (the step's bias arrives with it) before they arrive on P_FULL.
     if (lane == 0) {
       bool ok = ptx::mbar_wait(bar(META), 0, abort_flag);
       const int n_steps = ok ? misc->n_steps : 0;
@@ -299,15 +298,12 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
       const uint64_t qd0 = ptx::smem_desc_sw128(sbase + OFF_Q, 16, 1024);
       const uint64_t kd0 = ptx::smem_desc_sw128(sbase + OFF_K, 16, 1024);
       const uint64_t vd0 = ptx::smem_desc_sw128(sbase + OFF_V, KV_TILE_BYTES / 2, 1024);
-      const uint64_t pd0 = ptx::smem_desc_sw128(sbase + OFF_P, 16, 1024);
-      int ks_q = 0, kph_q = 0;   // ring slot / phase of the next QK
       auto issue_qk = [&](int j) -> bool {
         const int buf = j & 1;
-        if (!ptx::mbar_wait(bar(K_FULL + ks_q), kph_q, abort_flag)) return false;
-        // with P in tensor memory the S/P buffer is recycled in MMA issue order (PV of step j-2 precedes this QK)
-        if (!P_TMEM && !ptx::mbar_wait(bar(S_EMPTY + buf), ((j >> 1) & 1) ^ 1, abort_flag)) return false;
+        if (!ptx::mbar_wait(bar(K_FULL + buf), (j >> 1) & 1, abort_flag)) return false;
+        // the S/P buffer is recycled in MMA issue order (PV of step j-2 precedes this QK)
         ptx::tc_fence_after();
-        const uint64_t kd = kd0 + (uint64_t)((ks_q * KV_TILE_BYTES) >> 4);
+        const uint64_t kd = kd0 + (uint64_t)((buf * KV_TILE_BYTES) >> 4);
         const uint32_t d_tmem = tmem + buf * NKV;
 #pragma unroll
         for (int k = 0; k < HD / 16; ++k) {
@@ -317,40 +313,26 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
           ptx::mma_bf16_ss(d_tmem, ad, bd, IDESC_QK, k > 0 ? 1u : 0u);
         }
         ptx::mma_commit(bar(S_FULL + buf));
-        ptx::mma_commit(bar(K_EMPTY + ks_q));
-        if (++ks_q == KST) { ks_q = 0; kph_q ^= 1; }
         return true;
       };
       if (ok && n_steps > 0) ok = issue_qk(0);
-      int vs = 0, vph = 0;
       for (int j = 0; j < n_steps && ok; ++j) {
-        // S of the next step first (its K tile is normally resident), then this step's PV
-        bool qk_done = j + 1 >= n_steps;
-        if (!qk_done && (QK_FIRST || ptx::mbar_try_wait(bar(K_FULL + ks_q), kph_q))) {
-          ok = issue_qk(j + 1);
-          qk_done = true;
-        }
+        if (j + 1 < n_steps) ok = issue_qk(j + 1);
         if (!ok) break;
-        const int pbuf = j & 1;
-        ok = ptx::mbar_wait(bar(V_FULL + vs), vph, abort_flag) &&
-             ptx::mbar_wait(bar(P_FULL + pbuf), (j >> 1) & 1, abort_flag);
+        const int buf = j & 1;
+        ok = ptx::mbar_wait(bar(P_FULL + buf), (j >> 1) & 1, abort_flag);
         if (!ok) break;
         ptx::tc_fence_after();
         // V is [kv token][d]: MN-major B operand; 64-wide d blocks are KV_TILE_BYTES/2 apart; 16 tokens = 2048 bytes
-        const uint64_t vd = vd0 + (uint64_t)((vs * KV_TILE_BYTES) >> 4);
-        const uint32_t p_tmem = tmem + pbuf * NKV;
+        const uint64_t vd = vd0 + (uint64_t)((buf * KV_TILE_BYTES) >> 4);
+        const uint32_t p_tmem = tmem + buf * NKV;
 #pragma unroll
         for (int k = 0; k < NKV / 16; ++k) {
           const uint64_t bd = vd + (uint64_t)((k * 16 * 128) >> 4);
-          if (P_TMEM)  // A = P from tensor memory: 16 bf16 per K step = 8 packed columns
-            ptx::mma_bf16_ts(tmem + 2 * NKV, p_tmem + k * 8, bd, IDESC_PV, (j > 0 || k > 0) ? 1u : 0u);
-          else
-            ptx::mma_bf16_ss(tmem + 2 * NKV, pd0 + (uint64_t)((k * 32) >> 4), bd, IDESC_PV, (j > 0 || k > 0) ? 1u : 0u);
+          // A = P from tensor memory: 16 bf16 per K step = 8 packed columns
+          ptx::mma_bf16_ts(tmem + 2 * NKV, p_tmem + k * 8, bd, IDESC_PV, (j > 0 || k > 0) ? 1u : 0u);
         }
-        ptx::mma_commit(bar(V_EMPTY + vs));
-        ptx::mma_commit(bar(P_EMPTY));
-        if (++vs == VST) { vs = 0; vph ^= 1; }
-        if (!qk_done) ok = issue_qk(j + 1);
+        ptx::mma_commit(bar(PV_DONE + buf));
       }
     }
     __syncwarp();
@@ -364,16 +346,14 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
     bool ok = ptx::mbar_wait(bar(META), 0, abort_flag);
     const int n_steps = ok ? misc->n_steps : 0;
     float m_used = -INFINITY, l = 0.f;
-    uint8_t* prow = smem + OFF_P + m * 128;
 
-    int vs = 0, vph = 0;
     for (int j = 0; j < n_steps && ok; ++j) {
       const int buf = j & 1;
-      ok = ptx::mbar_wait(bar(V_FULL + vs), vph, abort_flag);   // bias / kvbase of the step visible
+      // bias / kvbase of the step visible; the MMA thread relies on this wait for the V tile as well
+      ok = ptx::mbar_wait(bar(V_FULL + buf), (j >> 1) & 1, abort_flag);
       if (!ok) break;
-      const float bias = misc->bias[vs][t];
-      const int kv0 = misc->kvbase[vs];
-      if (++vs == VST) { vs = 0; vph ^= 1; }
+      const float bias = misc->bias[buf][t];
+      const int kv0 = misc->kvbase[buf];
       ok = ptx::mbar_wait(bar(S_FULL + buf), (j >> 1) & 1, abort_flag);
       if (!ok) break;
       ptx::tc_fence_after();
@@ -385,10 +365,6 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
         DASH_TMEM_LD32(hi, lane_addr + buf * NKV + 32);
       }
       ptx::tmem_wait_ld();
-      if (!P_TMEM) {
-        ptx::tc_fence_before();
-        ptx::mbar_arrive(bar(S_EMPTY + buf));
-      }
 
       // logit (log2 domain) = s*c1 + b2; c1 > 0, so the row maximum can be taken on the raw scores
       const bool selected = bias > -INFINITY;
@@ -436,14 +412,12 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
         for (int c = 0; c < 32; ++c) packed[c] = 0u;
       }
 
-      // O is stable (and the shared-memory P buffer free) once the previous step's PV has completed
+      // O is stable once the previous step's PV has completed
       const bool fix = j > 0 && __any_sync(0xffffffffu, moved);
-      if (!P_TMEM || fix) {
-        ok = ptx::mbar_wait(bar(P_EMPTY), (j & 1) ^ 1, abort_flag);
+      if (fix) {
+        ok = ptx::mbar_wait(bar(PV_DONE + (buf ^ 1)), ((j - 1) >> 1) & 1, abort_flag);
         if (!ok) break;
         ptx::tc_fence_after();
-      }
-      if (fix) {
         // rescale this row of the accumulator: O *= 2^(m_old - m_new)
 #pragma unroll 1
         for (int q = 0; q < HD / 32; ++q) {
@@ -454,27 +428,16 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
           for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * corr);
           DASH_TMEM_ST32(lane_addr + 2 * NKV + q * 32, o);
         }
-        if (!P_TMEM) ptx::tmem_wait_st();
       }
-      if (P_TMEM) {
-        // P row -> the first 32 columns of this step's S buffer (two bf16 per column)
-        DASH_TMEM_ST32(lane_addr + buf * NKV, packed);
-        ptx::tmem_wait_st();
-      } else {
-        // P row -> shared memory, K-major with the 128-byte swizzle (16-byte chunk q of row m sits at q ^ (m & 7))
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-          uint4 v = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
-          *reinterpret_cast<uint4*>(prow + ((q ^ (m & 7)) << 4)) = v;
-        }
-        ptx::fence_proxy_async_smem();
-      }
+      // P row -> the first 32 columns of this step's S buffer (two bf16 per column)
+      DASH_TMEM_ST32(lane_addr + buf * NKV, packed);
+      ptx::tmem_wait_st();
       ptx::tc_fence_before();
       ptx::mbar_arrive(bar(P_FULL + (j & 1)));
     }
 
     // epilogue: O / l -> global (row m is 128 contiguous bf16 of token i_row, head r*g_q + hh)
-    if (ok && n_steps > 0) ok = ptx::mbar_wait(bar(P_EMPTY), (n_steps - 1) & 1, abort_flag);
+    if (ok && n_steps > 0) ok = ptx::mbar_wait(bar(PV_DONE + ((n_steps - 1) & 1)), ((n_steps - 1) >> 1) & 1, abort_flag);
     if (ok && n_steps > 0) {
       ptx::tc_fence_after();
       const float inv = l > 0.f ? 1.f / l : 0.f;
