@@ -174,7 +174,10 @@ int dash_attn_fwd_decode(const dash_params* p, const void* Q, const void* Kcache
                          const float* Kbar, const int32_t* kv_len, void* O, void* workspace,
                          size_t workspace_bytes, void* stream);
 
-/* Zeroes the status word (enqueued on stream).  Call once after allocating a workspace. */
+/* Zeroes the status word (enqueued on stream).  Call once after allocating a workspace, and again after an
+ * error: the word is sticky (the first error wins), and while it is non-zero the tensor-core kernels launched
+ * on that workspace retire without computing, so that one wait that ran out costs one wait limit, not one per
+ * thread block; their outputs are then undefined. */
 int dash_attn_reset_status(void* workspace, void* stream);
 
 /* Synchronises `stream` and returns the workspace's status word (DASH_OK or a device-side error). */

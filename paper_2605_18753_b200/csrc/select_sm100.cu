@@ -133,6 +133,10 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   // barriers and tensor memory are set up; from here on the kernel reads the planes the previous kernel wrote
   chain_wait();
   chain_release();
+  // an error already in the status word (a wait that ran out in an earlier block or kernel) makes every role
+  // leave at its first wait, so the rest of the grid retires in microseconds instead of a wait limit per block
+  if (a.sb && *reinterpret_cast<volatile int*>(&a.sb->status) != 0) *abort_flag = 1;
+  __syncthreads();
 
   if (warp == 4) {
     // ---------------- producer: Q tile, then the three planes of every 64-chunk block of summaries
