@@ -2,19 +2,22 @@
 //
 // Tile: one (batch, KV head) and TQ = 128/g_q consecutive query tokens; the 128 rows of the MMA tile are
 // (token, head-of-group) pairs, token-major.  A tile never straddles a chunk, so its rows share the own
-// chunk; it walks the UNION of its rows' routed chunks in ascending order, 64 KV tokens per step, own
-// chunk last.  A row that did not route a chunk gets bias -inf for that step (probability exactly 0), so
-// every row still attends to its own selection only.
+// chunk; it takes the own chunk first (its tiles can be fetched before the mask has been read), then walks
+// the UNION of its rows' routed chunks in ascending order, 64 KV tokens per step.  A row that did not route
+// a chunk gets bias -inf for that step (probability exactly 0), so every row still attends to its own
+// selection only.
 //
-// Warp roles (192 threads, two blocks per SM so one block's softmax overlaps the other's MMAs):
+// Warp roles (224 threads, two blocks per SM so one block's softmax overlaps the other's MMAs):
 //   warps 0-3  softmax: S (TMEM) -> registers, logit = S/sqrt(d) + bias, causal mask inside the own chunk,
-//              online softmax with a lazily moved row maximum, P (bf16) -> shared memory, rescale of the O
-//              accumulator in TMEM when the maximum moved, final O / l -> global.
-//   warp 4     producer: OR of the tile's mask words = union list; per step the TMA loads of the K and V
-//              tiles (128-byte swizzle, no multicast) and the per-token bias of the step (each lane walks
-//              its token's compact bias list with a cursor).
-//   warp 5     MMA issuer: S = Q K^T (M128 N64 K128) into one of two TMEM buffers, O += P V (M128 N128 K64),
-//              tcgen05.commit to the mbarriers that release the stages; owns the TMEM allocation.
+//              online softmax with a lazily moved row maximum, P (bf16) -> TMEM over the S columns, rescale of
+//              the O accumulator in TMEM when the maximum moved, final O / l -> global.
+//   warp 4     K producer: TMA loads of Q and of the K tiles (128-byte swizzle, no multicast); OR of the tile's
+//              mask words = union list.
+//   warp 6     V producer: walks the same union list; TMA loads of the V tiles and the per-token bias of each
+//              step (each lane walks its tokens' compact bias lists with register-buffered cursors).
+//   warp 5     MMA issuer: S_{j+1} = Q K_{j+1}^T (M128 N64 K128) into one of two TMEM buffers, then O += P_j V_j
+//              (M128 N128 K64, P from TMEM); one tcgen05.commit per product, to the mbarrier that the softmax
+//              warps and the producer of the stage both listen to; owns the TMEM allocation.
 // Every wait is bounded; a wait that runs out raises DASH_ERR_TIMEOUT in the status word and every role
 // leaves its loop, frees TMEM and returns.
 #include <cuda.h>
@@ -139,6 +142,29 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
       ptx::tma_load_4d(sbase + OFF_Q, &tmQ, bar(Q_FULL), 0, r * g_q, i0, b);
       ptx::tma_load_4d(sbase + OFF_Q + Q_BYTES / 2, &tmQ, bar(Q_FULL), 64, r * g_q, i0, b);
     }
+    // The own chunk goes first: its tiles need nothing from the mask, so they are in flight (and the first
+    // S = Q K^T can run) while the union of the routed chunks is still being formed.  Stages 0/1 are free.
+    for (int sub = 0; sub < own_steps; ++sub) {
+      const int kv0 = c_own * dm.B + sub * NKV;
+      if (do_k) {
+        if (lane == 0) {
+          const uint32_t dst = sbase + OFF_K + sub * KV_TILE_BYTES;
+          ptx::mbar_arrive_expect_tx(bar(K_FULL + sub), KV_TILE_BYTES);
+          ptx::tma_load_4d(dst, &tmK, bar(K_FULL + sub), 0, r, kv0, b);
+          ptx::tma_load_4d(dst + KV_TILE_BYTES / 2, &tmK, bar(K_FULL + sub), 64, r, kv0, b);
+        }
+      } else {
+        for (int t = lane; t < TQ; t += 32) misc->bias[sub][t] = 0.f;
+        if (lane == 0) misc->kvbase[sub] = kv0;
+        __syncwarp();
+        if (lane == 0) {
+          const uint32_t dst = sbase + OFF_V + sub * KV_TILE_BYTES;
+          ptx::mbar_arrive_expect_tx(bar(V_FULL + sub), KV_TILE_BYTES);
+          ptx::tma_load_4d(dst, &tmV, bar(V_FULL + sub), 0, r, kv0, b);
+          ptx::tma_load_4d(dst + KV_TILE_BYTES / 2, &tmV, bar(V_FULL + sub), 64, r, kv0, b);
+        }
+      }
+    }
     // union of the tile's mask words (lane t owns tokens t, t+32)
     const int n_words = (c_own >> 5) + 1;
     const long long row0 = ((long long)b * dm.h_kv + r) * dm.seq_q;
@@ -237,14 +263,15 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
       }
       return true;
     };
-    int j = 0;
+    int j = own_steps;                 // the own chunk's steps are already under way
     bool ok = true;
     Blk cur, nxt;
     bool has = pop(nxt);
     while (has && ok) {
       cur = nxt;
       has = pop(nxt);
-      const int nsub = (cur.c == c_own) ? own_steps : sub_per_blk;
+      if (cur.c == c_own) break;       // last of the walk, done first
+      const int nsub = sub_per_blk;
       for (int sub = 0; sub < nsub && ok; ++sub, ++j) {
         const int kv0 = cur.c * dm.B + sub * NKV;
         const int st = j & 1, prev_ph = ((j >> 1) - 1) & 1;   // stage, and the phase of step j-2 on the completion barriers
@@ -288,9 +315,7 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
     // Per step: S_{j+1} = Q K_{j+1}^T (needs only its K tile), then O += P_j V_j.  V_FULL is not tested here: the
     // softmax threads wait for it (the step's bias arrives with it) before they arrive on P_FULL.
     if (lane == 0) {
-      bool ok = ptx::mbar_wait(bar(META), 0, abort_flag);
-      const int n_steps = ok ? misc->n_steps : 0;
-      ok = ok && ptx::mbar_wait(bar(Q_FULL), 0, abort_flag);
+      bool ok = ptx::mbar_wait(bar(Q_FULL), 0, abort_flag);
       constexpr uint32_t IDESC_QK = ptx::idesc_bf16_f32(128, NKV, false, false);
       constexpr uint32_t IDESC_PV = ptx::idesc_bf16_f32(128, HD, false, true);
       // Descriptors differ only in the 14-bit start-address field (16-byte units, no carry into the next
@@ -315,7 +340,9 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
         ptx::mma_commit(bar(S_FULL + buf));
         return true;
       };
-      if (ok && n_steps > 0) ok = issue_qk(0);
+      if (ok) ok = issue_qk(0);          // the own chunk: there is always a step 0, whatever the union holds
+      ok = ok && ptx::mbar_wait(bar(META), 0, abort_flag);
+      const int n_steps = ok ? misc->n_steps : 0;
       for (int j = 0; j < n_steps && ok; ++j) {
         if (j + 1 < n_steps) ok = issue_qk(j + 1);
         if (!ok) break;
@@ -343,11 +370,17 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
     const int i_row = i0 + t;
     const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
     const float c1 = dm.sm_scale * 1.4426950408889634f;
-    bool ok = ptx::mbar_wait(bar(META), 0, abort_flag);
-    const int n_steps = ok ? misc->n_steps : 0;
+    bool ok = true;
+    int n_steps = 0x7fffffff;                // known from step 1 on; step 0 (the own chunk) always exists
     float m_used = -INFINITY, l = 0.f;
 
-    for (int j = 0; j < n_steps && ok; ++j) {
+    for (int j = 0; ok; ++j) {
+      if (j == 1) {
+        ok = ptx::mbar_wait(bar(META), 0, abort_flag);
+        if (!ok) break;
+        n_steps = misc->n_steps;
+      }
+      if (j >= n_steps) break;
       const int buf = j & 1;
       // bias / kvbase of the step visible; the MMA thread relies on this wait for the V tile as well
       ok = ptx::mbar_wait(bar(V_FULL + buf), (j >> 1) & 1, abort_flag);
