@@ -83,8 +83,10 @@ typedef struct dash_params {
 } dash_params;
 
 /* Bytes of workspace that select / fwd_prefill / fwd_decode / attend_* need for these parameters
- * (0 if the parameters are invalid).  The workspace must be 256-byte aligned.  Its first 256 bytes
- * hold the status word; the rest is scratch whose contents mean nothing between calls. */
+ * (0 if the parameters are invalid).  The workspace must be 256-byte aligned.  It starts with the
+ * status word followed by arrival counters that the library keeps at zero between calls (16,640 bytes
+ * in all, cleared by dash_attn_reset_status, which must therefore run once before the first use);
+ * the rest is scratch whose contents mean nothing between calls. */
 size_t dash_attn_workspace_bytes(const dash_params* p);
 
 /* Entries the blk_idx / blk_bias lists need, and where a row's region starts (see top of file).

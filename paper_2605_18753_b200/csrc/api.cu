@@ -81,7 +81,7 @@ static int make_dims(const dash_params* p, Dims* dm) {
 static WorkspaceLayout layout(const Dims& dm) {
   WorkspaceLayout w;
   size_t off = 0;
-  w.status = off; off += 256;
+  w.status = off; off += STATUS_REGION_BYTES;   // status word + arrival counters
   w.kbar = off; off += align256((size_t)dm.batch * dm.h_kv * (size_t)max(dm.T_s, 1) * dm.d * sizeof(float));
   w.mask = off; off += align256((size_t)dm.batch * dm.h_kv * (size_t)dm.seq_q * dm.W * sizeof(uint32_t));
   w.count = off; off += align256((size_t)dm.batch * dm.h_kv * (size_t)dm.seq_q * sizeof(int));
@@ -275,7 +275,7 @@ int dash_attn_fwd_decode(const dash_params* p, const void* Q, const void* Kcache
 
 int dash_attn_reset_status(void* workspace, void* stream) {
   if (!workspace) return DASH_ERR_WORKSPACE;
-  return cuda_status(cudaMemsetAsync(workspace, 0, 256, (cudaStream_t)stream));
+  return cuda_status(cudaMemsetAsync(workspace, 0, STATUS_REGION_BYTES, (cudaStream_t)stream));
 }
 
 int dash_attn_last_status(const void* workspace, void* stream) {

@@ -41,6 +41,13 @@ struct StatusBlock {
   int pad[61];
 };
 static_assert(sizeof(StatusBlock) == 256, "status block is the first 256 bytes of the workspace");
+// Behind the status block the workspace holds arrival counters, one per (batch, KV head), for kernels whose last
+// thread block of a group finishes the group's work (split-KV decode: the last split merges).  They are zero
+// between launches: the block that sees the last arrival clears its counter, and resetting the status word
+// clears them all.  Groups beyond the capacity fall back to a separate merge kernel.
+constexpr int ARRIVAL_COUNTERS = 4096;
+constexpr size_t STATUS_REGION_BYTES = 256 + ARRIVAL_COUNTERS * sizeof(int);
+__host__ __device__ inline int* arrival_counters(StatusBlock* sb) { return reinterpret_cast<int*>(sb + 1); }
 
 __device__ inline void report_error(StatusBlock* sb, int status, int detail) {
   if (!sb) return;
@@ -178,9 +185,10 @@ cudaError_t launch_attend_decode_ex(const Dims& dm, const void* Q, const void* K
                                     const int* count, const int* blk_idx, const float* blk_bias, void* O,
                                     float* partials, StatusBlock* sb, cudaStream_t st);
 int decode_sm100_min_splits(const Dims& dm);
+// O non-null: the last split of every (batch, KV head) merges the partials itself (needs sb's arrival counters)
 cudaError_t launch_decode_sm100(const Dims& dm, int n_split, const void* Q, const void* K, const void* V,
                                 const int* kv_len, const int* count, const int* blk_idx, const float* blk_bias,
-                                float* partials, StatusBlock* sb, cudaStream_t st);
+                                float* partials, void* O, StatusBlock* sb, cudaStream_t st);
 bool prefill_sm100_supported(const Dims& dm);
 cudaError_t launch_attend_prefill_sm100(const Dims& dm, const void* Q, const void* K, const void* V,
                                         const uint32_t* mask, const float* blk_bias, void* O, StatusBlock* sb,

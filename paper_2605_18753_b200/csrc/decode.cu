@@ -244,8 +244,11 @@ cudaError_t launch_attend_decode_ex(const Dims& dm, const void* Q, const void* K
   if (decode_use_sm100(dm)) {
     // bf16, head_dim 128, chunks of 64 or 128: TMA-fed tensor-core split kernel, then the common merge
     const int ns = decode_num_splits(dm);
-    cudaError_t e = launch_decode_sm100(dm, ns, Q, K, V, kv_len, count, blk_idx, blk_bias, partials, sb, st);
-    if (e != cudaSuccess) return e;
+    // with a workspace (status block + arrival counters) the last split of each group merges in the same kernel
+    const bool fused = sb != nullptr && dm.batch * dm.h_kv <= ARRIVAL_COUNTERS;
+    cudaError_t e = launch_decode_sm100(dm, ns, Q, K, V, kv_len, count, blk_idx, blk_bias, partials, fused ? O : nullptr,
+                                        sb, st);
+    if (e != cudaSuccess || fused) return e;
     return launch_merge<__nv_bfloat16, 128>(dm, ns, partials, O, st);
   }
   return launch_attend_decode(dm, Q, K, V, kv_len, count, blk_idx, blk_bias, O, partials, st);

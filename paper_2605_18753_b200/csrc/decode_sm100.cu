@@ -46,6 +46,7 @@ struct MiscD {
   int nvalid[NST][2];
   float red[2][4][NH];
   float lred[4][NH];
+  int is_last;               // this block saw the last arrival of its (batch, KV head)
   int idx_s[MAX_RANGE];      // first KV token of each owned sub-block
   float bias_s[MAX_RANGE];
   int nval_s[MAX_RANGE];
@@ -62,6 +63,7 @@ struct DecodeArgs {
   const float* blk_bias;
   const __nv_bfloat16* Q;
   float* partials;
+  __nv_bfloat16* O;      // non-null: fused merge by the last split of each (batch, KV head)
   StatusBlock* sb;
 };
 
@@ -374,6 +376,7 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         pp[1] = misc->lred[0][h] + misc->lred[1][h] + misc->lred[2][h] + misc->lred[3][h];
       }
     }
+    __threadfence();        // the partial is visible device-wide before this block counts itself as arrived
     ptx::tc_fence_before();
   }
 
@@ -381,6 +384,42 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   if (warp == 5) {
     ptx::tc_fence_after();
     ptx::tmem_dealloc(tmem, TMEM_COLS);
+  }
+  if (a.O != nullptr) {
+    // ---------------- the last split of this (batch, KV head) to arrive merges all of them, in split order
+    int* counter = arrival_counters(a.sb) + grp;
+    if (tid == 0) {
+      const bool last = atomicAdd(counter, 1) == n_split - 1;
+      if (last) *counter = 0;          // every split has arrived: the counter is ready for the next launch
+      misc->is_last = last ? 1 : 0;
+    }
+    __syncthreads();
+    if (misc->is_last) {
+      __threadfence();
+      constexpr int VPL = HD / 32;
+      for (int h = warp; h < G; h += DEC_THREADS / 32) {
+        const long long bh = (long long)b * dm.h_q + (long long)r * G + h;
+        const float* p = a.partials + bh * n_split * (HD + 2);
+        float M = -INFINITY;
+        for (int s = 0; s < n_split; ++s) M = fmaxf(M, __ldcg(p + s * (HD + 2)));
+        float Lsum = 0.f, acc[VPL];
+#pragma unroll
+        for (int v = 0; v < VPL; ++v) acc[v] = 0.f;
+        for (int s = 0; s < n_split; ++s) {
+          const float ms = __ldcg(p + s * (HD + 2));
+          if (ms == -INFINITY) continue;
+          const float w = __expf(ms - M);
+          Lsum += w * __ldcg(p + s * (HD + 2) + 1);
+          const float2* po = reinterpret_cast<const float2*>(p + s * (HD + 2) + 2 + lane * VPL);   // 8-byte aligned
+          const float2 oa = __ldcg(po), ob = __ldcg(po + 1);
+          acc[0] += w * oa.x; acc[1] += w * oa.y; acc[2] += w * ob.x; acc[3] += w * ob.y;
+        }
+        const float inv = Lsum > 0.f ? 1.f / Lsum : 0.f;
+        __nv_bfloat16* op = a.O + (long long)b * dm.os[0] + (long long)(r * G + h) * dm.os[2] + lane * VPL;
+#pragma unroll
+        for (int v = 0; v < VPL; ++v) op[v] = __float2bfloat16_rn(acc[v] * inv);
+      }
+    }
   }
   if (tid == 0 && misc->abort_flag) report_error(a.sb, DASH_ERR_TIMEOUT, 301);
 }
@@ -425,8 +464,9 @@ int decode_sm100_min_splits(const Dims& dm) {
 
 cudaError_t launch_decode_sm100(const Dims& dm, int n_split, const void* Q, const void* K, const void* V,
                                 const int* kv_len, const int* count, const int* blk_idx, const float* blk_bias,
-                                float* partials, StatusBlock* sb, cudaStream_t st) {
+                                float* partials, void* O, StatusBlock* sb, cudaStream_t st) {
   DecodeArgs a;
+  a.O = (__nv_bfloat16*)O;
   a.dm = dm; a.n_split = n_split; a.kv_len = kv_len; a.count = count; a.blk_idx = blk_idx; a.blk_bias = blk_bias;
   a.Q = (const __nv_bfloat16*)Q; a.partials = partials; a.sb = sb;
   CUtensorMap tk, tv;
