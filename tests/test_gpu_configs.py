@@ -1,6 +1,7 @@
 """Full-size parity on the long-context, decode and alpha-sweep workloads, in the launch configuration the
 benchmark uses.  The oracle cannot evaluate these sizes whole, so it computes a seeded sample of rows one by
-one (first/last rows of chunks, rows in the tail, random rows) for a sample of KV heads; the mask of every
+one (first/last rows of chunks, rows in the tail, random rows: about 4000 (row, KV head) pairs per 64K setting,
+1000 per sweep setting, 16 of the 128 decode groups) for a sample of KV heads; the mask of every
 sampled row must equal the oracle's except inside the 1e-4 borderline band; every row whose mask equals the
 oracle's (at these lengths most rows have SOME chunk within 1e-4 of the threshold, so rows are not dropped for
 merely containing one) must agree in its outputs within the bf16 tolerance.  Achieved block sparsity is printed per setting."""
@@ -71,7 +72,7 @@ def _prefill_sampled(w, rows, kv_heads, batches=(0,)):
 @pytest.mark.parametrize("name", ["prefill_64k_s75", "prefill_64k_s90"])
 def test_prefill_64k(name):
     w = synth.workload(name)
-    s = _prefill_sampled(w, _sample_rows(w.seq, w.block, 40, 1), kv_heads=[0, 6])
+    s = _prefill_sampled(w, _sample_rows(w.seq, w.block, 2048, 1), kv_heads=[0, 6])
     assert 0.5 < s < 0.99
 
 
@@ -79,7 +80,7 @@ def test_prefill_64k(name):
 @pytest.mark.parametrize("alpha", [1.25, 1.5, 2.0])
 def test_alpha_sweep_32k(alpha, block):
     w = synth.workload("sweep_32k", alpha=alpha, block=block)
-    _prefill_sampled(w, _sample_rows(w.seq, w.block, 24, 2), kv_heads=[3], batches=(1,))
+    _prefill_sampled(w, _sample_rows(w.seq, w.block, 1024, 2), kv_heads=[3], batches=(1,))
 
 
 def test_decode_128k():
@@ -104,7 +105,8 @@ def test_decode_128k():
     count = rt["count"].cpu().numpy()
     got, want = [], []
     sup, vis = [], []
-    for bb, r in [(0, 0), (1, 3), (2, 7), (15, 5)]:
+    for bb, r in [(0, 0), (1, 3), (2, 7), (15, 5), (3, 1), (4, 2), (5, 4), (6, 6), (7, 0), (8, 3), (9, 7), (10, 5),
+                  (11, 1), (12, 2), (13, 4), (14, 6)]:
         L = lens[bb]
         ref = orc.forward_decode(H.to_np64(q[bb:bb + 1, r * g_q:(r + 1) * g_q]), H.to_np64(Kc[bb:bb + 1, :L, r:r + 1]),
                                  H.to_np64(Vc[bb:bb + 1, :L, r:r + 1]), [L], B=w.block, alpha=w.alpha, gamma=w.gamma,
@@ -123,7 +125,7 @@ def test_decode_128k():
         assert int(count[bb, r, 0]) == ro.support.size
         got.append(o[bb, r * g_q:(r + 1) * g_q].float().cpu().double().numpy())
         want.append(ref["O"][0])
-    assert len(got) >= 2
+    assert len(got) >= 10
     mx, mean = H.check_outputs(np.stack(got), np.stack(want), q.dtype, "decode_128k")
     print(f"\n[decode_128k] groups compared {len(got)} sampled sparsity {orc.block_sparsity(sup, vis):.3f} "
           f"max-abs {mx:.2e} mean-abs {mean:.2e}")

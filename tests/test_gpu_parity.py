@@ -239,14 +239,15 @@ def _fwd_prefill_case(w, rows, kv_heads=None, min_clean=0.9):
     return H.check_outputs(_gather_O(O, keys, w.h_q // w.h_kv), want, Q.dtype, f"fwd_prefill {w.name}")
 
 
-def test_fwd_prefill_8k_config_sampled_rows():
-    """The 8K prefill workload at full size, in the configuration the benchmark times; the oracle computes a
-    seeded sample of rows (first/last rows of chunks, rows after planted chunks, two whole tiles)."""
-    w = synth.workload("prefill_8k")
-    rng = np.random.default_rng(0)
-    rows = set(rng.integers(0, w.seq, 96).tolist()) | {0, 63, 64, 65, 127, 128, w.seq - 1, w.seq - 64, w.seq - 65}
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_fwd_prefill_8k_config_sampled_rows(seed):
+    """The 8K prefill workload at full size, in the configuration the benchmark times (seed 0) and on two more
+    seeds; the oracle computes a seeded sample of rows (first/last rows of chunks, random rows, two whole tiles)."""
+    w = synth.workload("prefill_8k", seed=seed)
+    rng = np.random.default_rng(seed)
+    rows = set(rng.integers(0, w.seq, 1024).tolist()) | {0, 63, 64, 65, 127, 128, w.seq - 1, w.seq - 64, w.seq - 65}
     rows |= set(range(4096, 4096 + 32)) | set(range(8000, 8032))
-    for sigma in (10.0, 1e8):
+    for sigma in ((10.0, 1e8) if seed == 0 else (10.0,)):
         _fwd_prefill_case(w.with_(sigma=sigma), sorted(rows), kv_heads=[0, 5])
 
 
