@@ -275,25 +275,49 @@ def main():
     value = f_total / (ms * 1e-3) / 1e12
     executed, n_steps_total = executed_flops_from_mask(rt["mask"], w)
 
-    # end to end: pinned host inputs -> device, forward, output -> pinned host, all inside the timed region
+    # end to end: pinned host inputs -> device, forward, output -> pinned host, all inside the timed region.
+    # Every step copies its own inputs in and its own output out; as a serving loop would, the copies of
+    # neighbouring steps overlap the compute (two buffer sets; one stream each for H2D, compute and D2H).
     hQ, hK, hV = (t.cpu().pin_memory() for t in (Q, K, V))
     hO = torch.empty_like(hQ).pin_memory()
-    dQ, dK, dV, dO = (torch.empty_like(t) for t in (Q, K, V, O))
-    pe = B.params_for_prefill(dQ, dK, dV, dO, block=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma)
+    sets = []
+    for _ in range(2):
+        dQ, dK, dV, dO = (torch.empty_like(t) for t in (Q, K, V, O))
+        sets.append({"Q": dQ, "K": dK, "V": dV, "O": dO,
+                     "p": B.params_for_prefill(dQ, dK, dV, dO, block=w.block, alpha=w.alpha, gamma=w.gamma,
+                                               sigma=w.sigma),
+                     "in_ready": torch.cuda.Event(), "cmp_done": torch.cuda.Event(), "out_done": torch.cuda.Event()})
+    s_in, s_cmp, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
 
-    def e2e_step():
-        dQ.copy_(hQ, non_blocking=True); dK.copy_(hK, non_blocking=True); dV.copy_(hV, non_blocking=True)
-        B.dash_attn_fwd_prefill(pe, dQ, dK, dV, dO, ws)
-        hO.copy_(dO, non_blocking=True)
+    def e2e_step(i):
+        st = sets[i & 1]
+        with torch.cuda.stream(s_in):
+            if i >= 2:
+                s_in.wait_event(st["cmp_done"])           # the forward of step i-2 has read this input set
+            st["Q"].copy_(hQ, non_blocking=True); st["K"].copy_(hK, non_blocking=True); st["V"].copy_(hV, non_blocking=True)
+            st["in_ready"].record(s_in)
+        with torch.cuda.stream(s_cmp):
+            s_cmp.wait_event(st["in_ready"])
+            if i >= 2:
+                s_cmp.wait_event(st["out_done"])          # the output of step i-2 has left this output buffer
+            B.dash_attn_fwd_prefill(st["p"], st["Q"], st["K"], st["V"], st["O"], ws)
+            st["cmp_done"].record(s_cmp)
+        with torch.cuda.stream(s_out):
+            s_out.wait_event(st["cmp_done"])
+            hO.copy_(st["O"], non_blocking=True)
+            st["out_done"].record(s_out)
 
-    for _ in range(3):
-        e2e_step()
+    for i in range(4):
+        e2e_step(i)
+    torch.cuda.synchronize()
     barrier()
     a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    a.record()
-    for _ in range(args.steps):
-        e2e_step()
-    b_.record()
+    a.record(s_in)
+    s_cmp.wait_event(a); s_out.wait_event(a)
+    for i in range(args.steps):
+        e2e_step(i + 4)
+    b_.record(s_out)                                      # behind the last step's D2H, which is behind everything else
+    torch.cuda.synchronize()
     barrier()
     e2e_ms, _ = combine_timing(a.elapsed_time(b_) / args.steps, 0.0, device=dev)
     h2d = sum(t.numel() * t.element_size() for t in (hQ, hK, hV))
