@@ -15,6 +15,8 @@
 // 32 chunks.  Waits are bounded as in the Stage 2 kernel.
 #include <cuda.h>
 
+#include <type_traits>
+
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 
@@ -243,13 +245,19 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     // on the left.  The start is the root
     // of the same equation with every candidate taken as active (closed form for alpha = 2 and 1.5), clamped to
     // max - 1 <= tau* < max, which saves the slow first halvings of a start at max - 1.
-    const int max_it = e_int ? MAX_NEWTON : MAX_NEWTON_GENERIC;
+    // The body below runs with the exponent as a compile-time constant for alpha = 1.5 (integer power 2, the
+    // paper's setting): the per-candidate loops then hold no tests of it.  Other exponents take the same code
+    // with the run-time value.
+    auto solve = [&](auto ei_tag) {
+    constexpr int EI_STATIC = decltype(ei_tag)::value;
+    const int ei = EI_STATIC >= 0 ? EI_STATIC : e_int;
+    const int max_it = ei ? MAX_NEWTON : MAX_NEWTON_GENERIC;
     auto start_tau = [&](float mx, float s1, float s2) -> float {   // s1, s2: sums of (x - mx), (x - mx)^2
       const float n = (float)n_cand;
       float t = -1.f;
-      if (e_int == 1) {
+      if (ei == 1) {
         t = (s1 - 1.f) / n;
-      } else if (e_int == 2) {
+      } else if (ei == 2) {
         const float mean = s1 / n, ss = s2 - s1 * mean;
         if (ss < 1.f) t = mean - sqrtf((1.f - ss) / n);
       }
@@ -258,7 +266,7 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     auto newton_step = [&](float f, float g, bool& done) {
       if (done) return;
       if (fabsf(f - 1.f) <= NEWTON_F_TOL || !(g > 0.f)) { done = true; return; }
-      const float nt = tau + newton_delta(f, g, e_int, e);
+      const float nt = tau + newton_delta(f, g, ei, e);
       if (nt == tau) done = true; else tau = nt;
     };
     float xr[4][32];                               // the whole row, when it has at most 128 candidates
@@ -278,32 +286,62 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           for (int c = 0; c < 32; ++c) xr[k][c] = -INFINITY;
         }
       }
-      float mx = -INFINITY;
+      // several independent chains per reduction: one chain of 128 dependent operations would cost its latency 128 times
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
       for (int k = 0; k < 4; ++k)
 #pragma unroll
-        for (int c = 0; c < 32; ++c) mx = fmaxf(mx, xr[k][c]);
-      float s1 = 0.f, s2 = 0.f;
+        for (int c = 0; c < 32; ++c) mx4[c & 3] = fmaxf(mx4[c & 3], xr[k][c]);
+      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+      float2 s1v[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)}, s2v[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+      const float2 nmx = make_float2(-mx, -mx);
 #pragma unroll
       for (int k = 0; k < 4; ++k)
 #pragma unroll
-        for (int c = 0; c < 32; ++c) {
-          const float y = xr[k][c] > -INFINITY ? xr[k][c] - mx : 0.f;
-          s1 += y;
-          s2 = fmaf(y, y, s2);
+        for (int c = 0; c < 32; c += 2) {
+          float2 y = __fadd2_rn(make_float2(xr[k][c], xr[k][c + 1]), nmx);     // two candidates per instruction
+          y.x = xr[k][c] > -INFINITY ? y.x : 0.f;
+          y.y = xr[k][c + 1] > -INFINITY ? y.y : 0.f;
+          s1v[(c >> 1) & 1] = __fadd2_rn(s1v[(c >> 1) & 1], y);
+          s2v[(c >> 1) & 1] = __ffma2_rn(y, y, s2v[(c >> 1) & 1]);
         }
+      const float s1 = (s1v[0].x + s1v[0].y) + (s1v[1].x + s1v[1].y);
+      const float s2 = (s2v[0].x + s2v[0].y) + (s2v[1].x + s2v[1].y);
       tau = start_tau(mx, s1, s2);
       bool done = false;
       for (int it = 0; it < max_it; ++it) {
         float f[4] = {0.f, 0.f, 0.f, 0.f}, g[4] = {0.f, 0.f, 0.f, 0.f};
+        if constexpr (EI_STATIC == 2) {
+          // alpha = 1.5: F += m^2, G += m, two candidates per packed instruction, four chains of pairs
+          float2 fv[4], gv[4];
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          if (k < n_chunks) {
+          for (int q = 0; q < 4; ++q) fv[q] = gv[q] = make_float2(0.f, 0.f);
+          const float2 ntau = make_float2(-tau, -tau);
 #pragma unroll
-            for (int c = 0; c < 32; ++c) {
-              const float mm = fmaxf(xr[k][c] - tau, 0.f);
-              f[c & 3] += pow_e(mm, e_int, e);
-              g[c & 3] += pow_em1(mm, e_int, e);
+          for (int k = 0; k < 4; ++k) {
+            if (k < n_chunks) {
+#pragma unroll
+              for (int c = 0; c < 32; c += 2) {
+                float2 mm = __fadd2_rn(make_float2(xr[k][c], xr[k][c + 1]), ntau);
+                mm.x = fmaxf(mm.x, 0.f);
+                mm.y = fmaxf(mm.y, 0.f);
+                fv[(c >> 1) & 3] = __ffma2_rn(mm, mm, fv[(c >> 1) & 3]);
+                gv[(c >> 1) & 3] = __fadd2_rn(gv[(c >> 1) & 3], mm);
+              }
+            }
+          }
+#pragma unroll
+          for (int q = 0; q < 4; ++q) { f[q] = fv[q].x + fv[q].y; g[q] = gv[q].x + gv[q].y; }
+        } else {
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            if (k < n_chunks) {
+#pragma unroll
+              for (int c = 0; c < 32; ++c) {
+                const float mm = fmaxf(xr[k][c] - tau, 0.f);
+                f[c & 3] += pow_e(mm, ei, e);
+                g[c & 3] += pow_em1(mm, ei, e);
+              }
             }
           }
         }
@@ -351,8 +389,8 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           for (int c = 0; c < 32; ++c) {
             float mm = fmaxf(fmaf(__uint_as_float(v[c]), xs, -tau), 0.f);
             mm = c < lim ? mm : 0.f;
-            f[c & 3] += pow_e(mm, e_int, e);
-            g[c & 3] += pow_em1(mm, e_int, e);
+            f[c & 3] += pow_e(mm, ei, e);
+            g[c & 3] += pow_em1(mm, ei, e);
           }
         }
         ok = exchange((f[0] + f[1]) + (f[2] + f[3]), (g[0] + g[1]) + (g[2] + g[3]));
@@ -409,7 +447,7 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           for (int kk = 0; kk < 4; ++kk)
             if (kk == k) {
 #pragma unroll
-              for (int c = 0; c < 32; ++c) pe[c] = pow_e(fmaxf(xr[kk][c] - tau, 0.f), e_int, e);
+              for (int c = 0; c < 32; ++c) pe[c] = pow_e(fmaxf(xr[kk][c] - tau, 0.f), ei, e);
             }
         } else {
           uint32_t v[32];
@@ -419,14 +457,14 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 #pragma unroll
           for (int c = 0; c < 32; ++c) {
             const float mm = fmaxf(fmaf(__uint_as_float(v[c]), xs, -tau), 0.f);
-            pe[c] = c < lim ? pow_e(mm, e_int, e) : 0.f;
+            pe[c] = c < lim ? pow_e(mm, ei, e) : 0.f;
           }
         }
         group_sums(pe);
         uint32_t bits = 0;
-        uint32_t lwv[32];
+        uint32_t lwv[OWN];
 #pragma unroll
-        for (int c = 0; c < 32; ++c) lwv[c] = 0x7f800000u;        // +inf: not routed
+        for (int c = 0; c < OWN; ++c) lwv[c] = 0x7f800000u;       // +inf: not routed
 #pragma unroll
         for (int q = 0; q < OWN; ++q) {
           if (pe[q] > 0.f) {
@@ -438,7 +476,7 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         }
 #pragma unroll
         for (int o = 1; o < G; o <<= 1) bits |= __shfl_xor_sync(0xffffffffu, bits, o);
-        DASH_TMEM_ST32(lane_addr + k * 32, lwv);                 // slot q of this lane = chunk own0 + q of step k
+        ptx::tmem_st_n<OWN>(lane_addr + k * 32, lwv);            // slot q of this lane = chunk own0 + q of step k
         if (row_valid && hh == 0) {
           const int wj = cr * (CLUSTER_COLS / 32) + k;         // mask word of this step
           mrow[wj] = bits | (((c_own >> 5) == wj) ? (1u << (c_own & 31)) : 0u);
@@ -463,8 +501,8 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       }
       const float mu = nsel_all > 0 ? slog_all / (float)nsel_all : 0.f;
       for (int k = 0; k < n_chunks && ok; ++k) {
-        uint32_t lwv[32];
-        DASH_TMEM_LD32(lwv, lane_addr + k * 32);
+        uint32_t lwv[OWN];
+        ptx::tmem_ld_n<OWN>(lwv, lane_addr + k * 32);
         ptx::tmem_wait_ld();
         uint32_t bits = 0;
 #pragma unroll
@@ -486,6 +524,8 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         base += __popc(bits);
       }
     }
+    };
+    if (e_int == 2) solve(std::integral_constant<int, 2>{}); else solve(std::integral_constant<int, -1>{});
     ptx::tc_fence_before();
   }
 
