@@ -46,6 +46,7 @@ class Workload:
     shift: float = 2.0
     n_planted: int = 8
     seed: int = 0
+    q_corr: float = 0.0  # AR(1) coefficient of the query noise along the token axis (0 = independent queries)
 
     def as_dict(self):
         return asdict(self)
@@ -124,6 +125,31 @@ def _keys_values(w: Workload, n_tokens: int, u, planted, device):
     return K, V
 
 
+def _ar1_along_tokens(x: torch.Tensor, c: float) -> torch.Tensor:
+    """x[i] <- c x[i-1] + sqrt(1 - c^2) x[i] along dim 0 (x[0] kept): unit variance, lag-1 correlation c.
+
+    Evaluated segment by segment as a scaled cumulative sum in float64 (c^-L stays below 1e6 inside a segment)."""
+    if c <= 0.0:
+        return x
+    n = x.shape[0]
+    L = max(1, min(n, int(13.8 / -math.log(c))))
+    s = math.sqrt(1.0 - c * c)
+    out = torch.empty_like(x)
+    prev = None
+    for a in range(0, n, L):
+        seg = x[a:a + L].to(torch.float64) * s
+        if prev is None:
+            seg[0] = x[0].to(torch.float64)
+        t = torch.arange(seg.shape[0], device=x.device, dtype=torch.float64)
+        up = (c ** t).view(-1, *([1] * (x.dim() - 1)))
+        acc = torch.cumsum(seg / up, dim=0) * up
+        if prev is not None:
+            acc = acc + up * c * prev
+        prev = acc[-1]
+        out[a:a + L] = acc.to(x.dtype)
+    return out
+
+
 def make_prefill_inputs(w: Workload, device="cpu"):
     """Returns dict(Q [b,n,h_q,d], K [b,n,h_kv,d], V, planted [b,h_kv,n_planted])."""
     assert w.kind == "prefill"
@@ -142,6 +168,7 @@ def make_prefill_inputs(w: Workload, device="cpu"):
     gq = _gen(w.seed, 4, device)
     for bb in range(b):
         q32 = torch.randn(n, h_q, d, generator=gq, device=device, dtype=torch.float32)
+        q32 = _ar1_along_tokens(q32, w.q_corr)
         q32 += (w.rho * math.sqrt(d)) * u[bb].repeat_interleave(g_q, dim=0)[None, :, :]
         Q[bb] = q32.to(dt)
         del q32
