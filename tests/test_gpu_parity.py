@@ -196,6 +196,8 @@ def test_fwd_prefill_tiny_fp32(name, sigmas):
     dict(seq=600, h_q=4, h_kv=2, head_dim=64, block=32, alpha=1.25, gamma=2.0),
     dict(seq=1500, h_q=32, h_kv=2, head_dim=128, block=64, seed=1),
     dict(seq=1111, h_q=2, h_kv=2, head_dim=128, block=64, seed=2),
+    dict(seq=1300, h_q=16, h_kv=2, head_dim=128, block=64, seed=3),          # g_q = 8 on the tensor-core paths
+    dict(seq=900, h_q=4, h_kv=2, head_dim=128, block=128, seed=4),           # g_q = 2, chunks of 128
 ])
 def test_fwd_prefill_small(kw):
     w = _wl(**kw)
@@ -299,6 +301,8 @@ def _decode_case(w, kv_len, use_lists_from_oracle=False):
     (dict(kind="decode", batch=2, seq=1024, h_q=4, h_kv=4, head_dim=64, block=32, alpha=2.0), [1024, 65]),
     (dict(kind="decode", batch=2, seq=4096, h_q=16, h_kv=1, head_dim=128, block=128, alpha=1.25, gamma=2.0), [4095, 129]),
     (dict(kind="decode", batch=1, seq=3000, h_q=2, h_kv=2, head_dim=128, block=64, dtype="f32"), [2999]),
+    (dict(kind="decode", batch=2, seq=5000, h_q=16, h_kv=2, head_dim=128, block=64), [5000, 4097]),     # g_q = 8
+    (dict(kind="decode", batch=2, seq=3000, h_q=4, h_kv=2, head_dim=128, block=128, alpha=2.0), [3000, 2050]),   # g_q = 2
 ])
 def test_decode_matches_oracle(kw, kv_len):
     w = _wl(**kw)
