@@ -127,12 +127,12 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   const uint32_t tmem = misc->tmem_base;
 
   // barriers and tensor memory are set up; everything below reads what the routing kernels wrote
+  int L = a.kv_len ? a.kv_len[b] : dm.seq_kv;   // the caller's input, not a product of the chain: read it before the wait
   chain_wait();
   chain_release();
   // an error already in the status word makes every role leave at its first wait (see the prefill kernel)
   if (a.sb && *reinterpret_cast<volatile int*>(&a.sb->status) != 0) *abort_flag = 1;
   __syncthreads();
-  int L = a.kv_len ? a.kv_len[b] : dm.seq_kv;
   L = max(1, min(L, dm.seq_kv));
   const int c_own = (L - 1) / dm.B;
   const long long grp = (long long)b * dm.h_kv + r;

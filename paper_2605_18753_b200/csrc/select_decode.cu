@@ -56,9 +56,9 @@ decode_scores_kernel(Dims dm, const T* __restrict__ Q, const float* __restrict__
   constexpr int VPL = D / 32;   // floats per lane of one summary row
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int r = blockIdx.y, b = blockIdx.z;
+  int L = kv_len ? kv_len[b] : dm.seq_kv;     // the caller's input, not a product of the chain: read it before the wait
   chain_wait();
   chain_release();
-  int L = kv_len ? kv_len[b] : dm.seq_kv;
   L = max(1, min(L, dm.seq_kv));
   const int n_cand = min((L - 1) / dm.B, dm.T_s);
   const int c_begin = blockIdx.x * SC_ROWS_PER_BLOCK;
@@ -82,10 +82,10 @@ decode_scores_kernel(Dims dm, const T* __restrict__ Q, const float* __restrict__
     for (int u = 0; u < RB; ++u) {
       const int c = min(c0 + u, c_end - 1);
       if constexpr (VPL == 4) {
-        const float4 f = *reinterpret_cast<const float4*>(kb + (long long)c * D);
+        const float4 f = __ldcs(reinterpret_cast<const float4*>(kb + (long long)c * D));   // read once: streaming
         kv[u][0] = f.x; kv[u][1] = f.y; kv[u][2] = f.z; kv[u][3] = f.w;
       } else {
-        const float2 f = *reinterpret_cast<const float2*>(kb + (long long)c * D);
+        const float2 f = __ldcs(reinterpret_cast<const float2*>(kb + (long long)c * D));
         kv[u][0] = f.x; kv[u][1] = f.y;
       }
     }
@@ -122,9 +122,9 @@ decode_route_kernel(Dims dm, const float* __restrict__ xs, const int* __restrict
   static_assert(NW == 32, "one lane per warp segment in the Newton phase");
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int r = blockIdx.x, b = blockIdx.y;
+  int L = kv_len ? kv_len[b] : dm.seq_kv;     // the caller's input, not a product of the chain: read it before the wait
   chain_wait();
   chain_release();
-  int L = kv_len ? kv_len[b] : dm.seq_kv;
   L = max(1, min(L, dm.seq_kv));
   const int c_own = (L - 1) / dm.B;
   const int n_cand = min(c_own, dm.T_s);
@@ -170,7 +170,7 @@ decode_route_kernel(Dims dm, const float* __restrict__ xs, const int* __restrict
   const int e_int = dm.e_int;
   const float e = dm.e;
   {
-    constexpr int NWH = G <= 8 ? NW / G : 1;      // warps per team (named barriers 1..8); one warp per head beyond
+    constexpr int NWH = G < 8 ? 8 / G : 1;        // warps per team: eight Newton warps in all (named barriers 1..4)
     constexpr int TEAM = NWH * 32;
     const int g = min(warp / NWH, G - 1), sw = warp % NWH;
     const bool in_team = warp < G * NWH;
