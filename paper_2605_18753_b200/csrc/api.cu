@@ -164,7 +164,7 @@ int dash_attn_block_summaries(const dash_params* p, const void* K, const float* 
   if (num_blocks < 0) num_blocks = dm.T_s - first_block;
   if (first_block + num_blocks > dm.T_s) return DASH_ERR_INVALID_ARG;
   if ((rc = check_device()) != DASH_OK) return rc;
-  return cuda_status(launch_summaries(dm, K, qbar, qbar_chunk_stride, kv_len, first_block, num_blocks, Kbar,
+  return cuda_status(launch_summaries(dm, K, qbar, qbar_chunk_stride, kv_len, first_block, num_blocks, Kbar, nullptr,
                                       (cudaStream_t)stream));
 }
 
@@ -235,15 +235,21 @@ int dash_attn_fwd_prefill(const dash_params* p, const void* Q, const void* K, co
   cudaStream_t st = (cudaStream_t)stream;
   StatusBlock* sb = at<StatusBlock>(workspace, wl.status);
   const float* kb = Kbar;
+  bool planes_ready = false;
   if (!kb) {
     float* kbw = at<float>(workspace, wl.kbar);
-    if ((rc = cuda_status(launch_summaries(dm, K, qbar, qbar_chunk_stride, nullptr, 0, dm.T_s, kbw, st))) != DASH_OK) return rc;
+    // the tensor-core routing kernel reads Kbar as three bf16 planes: the summary kernel writes them directly
+    void* planes = select_sm100_token_limit(dm) > 0 ? at<void>(workspace, wl.planes) : nullptr;
+    if ((rc = cuda_status(launch_summaries(dm, K, qbar, qbar_chunk_stride, nullptr, 0, dm.T_s, kbw, planes, st))) != DASH_OK)
+      return rc;
     kb = kbw;
+    planes_ready = planes != nullptr && dm.T_s > 0;
   }
   uint32_t* mask = mask_out ? mask_out : at<uint32_t>(workspace, wl.mask);
   float* bias = at<float>(workspace, wl.blk_bias);
   if ((rc = cuda_status(launch_select(dm, Q, kb, nullptr, mask, at<int>(workspace, wl.count), nullptr, bias, nullptr,
-                                      at<void>(workspace, wl.planes), at<float>(workspace, wl.xscratch), sb, st))) != DASH_OK)
+                                      at<void>(workspace, wl.planes), at<float>(workspace, wl.xscratch), sb, st,
+                                      planes_ready))) != DASH_OK)
     return rc;
   return run_attend_prefill(dm, Q, K, V, mask, bias, O, sb, st);
 }

@@ -158,12 +158,16 @@ int validate_params(const dash_params* p, Dims* dm);
 int validate_device();
 
 // Launchers (one per translation unit).  All return a cudaError_t from the launch.
+// planes non-null: also writes the three bf16 planes (hi + mid + lo = fp32 value) the tensor-core routing kernel
+// reads, [3][batch * h_kv * T_s][d], so that no separate split pass is needed
 cudaError_t launch_summaries(const Dims& dm, const void* K, const float* qbar, long long qbar_chunk_stride,
-                             const int* kv_len, int first_block, int num_blocks, float* Kbar, cudaStream_t st);
+                             const int* kv_len, int first_block, int num_blocks, float* Kbar, void* planes,
+                             cudaStream_t st);
 size_t select_smem_bytes(const Dims& dm, int* tq_out);
+// planes_ready: `scratch` already holds the bf16 planes of Kbar (written by launch_summaries)
 cudaError_t launch_select(const Dims& dm, const void* Q, const float* Kbar, const int* kv_len, uint32_t* mask,
                           int* count, int* blk_idx, float* blk_bias, float* tau, void* scratch, float* xscratch,
-                          StatusBlock* sb, cudaStream_t st);
+                          StatusBlock* sb, cudaStream_t st, bool planes_ready = false);
 size_t select_decode_scratch_bytes(const Dims& dm);
 bool select_decode_supported(const Dims& dm);
 cudaError_t launch_select_decode(const Dims& dm, const void* Q, const float* Kbar, const int* kv_len, uint32_t* mask,
@@ -173,7 +177,7 @@ int select_sm100_token_limit(const Dims& dm);
 size_t select_sm100_scratch_bytes(const Dims& dm);
 cudaError_t launch_select_sm100(const Dims& dm, int token_limit, const void* Q, const float* Kbar, void* planes,
                                 uint32_t* mask, int* count, int* blk_idx, float* blk_bias, float* tau,
-                                StatusBlock* sb, cudaStream_t st);
+                                StatusBlock* sb, cudaStream_t st, bool planes_ready = false);
 cudaError_t launch_attend_prefill_generic(const Dims& dm, const void* Q, const void* K, const void* V,
                                           const uint32_t* mask, const float* blk_bias, void* O, cudaStream_t st);
 int decode_num_splits(const Dims& dm);

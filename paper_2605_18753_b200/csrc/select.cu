@@ -283,7 +283,7 @@ static cudaError_t launch_rows(const Dims& dm, const SelectPlan& pl, int token_b
 
 cudaError_t launch_select(const Dims& dm, const void* Q, const float* Kbar, const int* kv_len, uint32_t* mask,
                           int* count, int* blk_idx, float* blk_bias, float* tau, void* scratch, float* xscratch,
-                          StatusBlock* sb, cudaStream_t st) {
+                          StatusBlock* sb, cudaStream_t st, bool planes_ready) {
   // decode: streaming score kernel + per-(batch, KV head) routing kernel
   if (dm.decode && xscratch && select_decode_supported(dm))
     return launch_select_decode(dm, Q, Kbar, kv_len, mask, count, blk_idx, blk_bias, tau, xscratch, st);
@@ -292,7 +292,8 @@ cudaError_t launch_select(const Dims& dm, const void* Q, const float* Kbar, cons
   int token_base = 0;
   const int tc_tokens = scratch ? select_sm100_token_limit(dm) : 0;
   if (tc_tokens > 0) {
-    cudaError_t e = launch_select_sm100(dm, tc_tokens, Q, Kbar, scratch, mask, count, blk_idx, blk_bias, tau, sb, st);
+    cudaError_t e = launch_select_sm100(dm, tc_tokens, Q, Kbar, scratch, mask, count, blk_idx, blk_bias, tau, sb, st,
+                                        planes_ready);
     if (e != cudaSuccess || tc_tokens >= dm.seq_q) return e;
     token_base = tc_tokens;
   }

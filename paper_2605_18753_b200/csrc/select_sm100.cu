@@ -624,13 +624,16 @@ static cudaError_t launch_band_g(const Dims& dm, const CUtensorMap& tq, const CU
 
 cudaError_t launch_select_sm100(const Dims& dm, int token_limit, const void* Q, const float* Kbar, void* planes,
                                 uint32_t* mask, int* count, int* blk_idx, float* blk_bias, float* tau,
-                                StatusBlock* sb, cudaStream_t st) {
+                                StatusBlock* sb, cudaStream_t st, bool planes_ready) {
   const long long plane_rows = (long long)dm.batch * dm.h_kv * dm.T_s;
   const long long n = plane_rows * dm.d;
-  cudaError_t e = launch_chained(kbar_split_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, st, Kbar,
-                                 (__nv_bfloat16*)planes, n);
-  count_launch();
-  if (e != cudaSuccess) return e;
+  cudaError_t e = cudaSuccess;
+  if (!planes_ready) {       // the summaries came from the caller: split them here
+    e = launch_chained(kbar_split_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, st, Kbar,
+                       (__nv_bfloat16*)planes, n);
+    count_launch();
+    if (e != cudaSuccess) return e;
+  }
 
   SelectTcArgs a;
   a.dm = dm;

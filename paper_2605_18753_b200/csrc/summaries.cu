@@ -15,7 +15,8 @@ constexpr int SUM_UNROLL = 8;
 template <typename T, int D>
 __global__ void __launch_bounds__(SUM_WARPS * 32)
 summaries_kernel(Dims dm, const T* __restrict__ K, const float* __restrict__ qbar, long long qbar_chunk_stride,
-                 const int* __restrict__ kv_len, int first_block, int num_blocks, float* __restrict__ Kbar) {
+                 const int* __restrict__ kv_len, int first_block, int num_blocks, float* __restrict__ Kbar,
+                 __nv_bfloat16* __restrict__ planes, long long plane_elems) {
   constexpr int VPL = D / 32;  // elements per lane: 2 (d=64) or 4 (d=128)
   const int lane = threadIdx.x & 31;
   const long long warp = (long long)blockIdx.x * SUM_WARPS + (threadIdx.x >> 5);
@@ -97,21 +98,38 @@ summaries_kernel(Dims dm, const T* __restrict__ K, const float* __restrict__ qba
 #pragma unroll
     for (int v = 0; v < VPL; ++v) acc[v] *= inv;
   }
-  float* op = Kbar + (((long long)b * dm.h_kv + r) * dm.T_s + c) * D + lane * VPL;
+  const long long at = (((long long)b * dm.h_kv + r) * dm.T_s + c) * D + lane * VPL;
+  float* op = Kbar + at;
 #pragma unroll
   for (int v = 0; v < VPL; ++v) op[v] = acc[v];
+  if (planes) {
+    // x = hi + mid + lo exactly (three bf16 roundings of the successive remainders)
+#pragma unroll
+    for (int v = 0; v < VPL; ++v) {
+      const float x = acc[v];
+      const __nv_bfloat16 hi = __float2bfloat16_rn(x);
+      const float r1 = x - __bfloat162float(hi);
+      const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+      const float r2 = r1 - __bfloat162float(mid);
+      planes[at + v] = hi;
+      planes[plane_elems + at + v] = mid;
+      planes[2 * plane_elems + at + v] = __float2bfloat16_rn(r2);
+    }
+  }
 }
 
 cudaError_t launch_summaries(const Dims& dm, const void* K, const float* qbar, long long qbar_chunk_stride,
-                             const int* kv_len, int first_block, int num_blocks, float* Kbar, cudaStream_t st) {
+                             const int* kv_len, int first_block, int num_blocks, float* Kbar, void* planes,
+                             cudaStream_t st) {
   if (num_blocks <= 0) return cudaSuccess;
+  const long long plane_elems = (long long)dm.batch * dm.h_kv * dm.T_s * dm.d;
   const long long total = (long long)dm.batch * dm.h_kv * num_blocks;
   const unsigned grid = (unsigned)((total + SUM_WARPS - 1) / SUM_WARPS);
   const dim3 block(SUM_WARPS * 32);
   cudaError_t le = cudaSuccess;
 #define DASH_LAUNCH_SUM(T, D)                                                                               \
   le = launch_chained(summaries_kernel<T, D>, dim3(grid), block, 0, st, dm, (const T*)K, qbar,              \
-                      qbar_chunk_stride, kv_len, first_block, num_blocks, Kbar)
+                      qbar_chunk_stride, kv_len, first_block, num_blocks, Kbar, (__nv_bfloat16*)planes, plane_elems)
   if (dm.B % SUM_UNROLL != 0) return cudaErrorInvalidValue;
   if (dm.dtype == DASH_BF16) {
     if (dm.d == 128) DASH_LAUNCH_SUM(__nv_bfloat16, 128); else DASH_LAUNCH_SUM(__nv_bfloat16, 64);
