@@ -440,26 +440,8 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       }
     };
     if (ok) {
-      for (int k = 0; k < n_chunks; ++k) {
-        float pe[32];
-        if (in_regs) {
-#pragma unroll
-          for (int kk = 0; kk < 4; ++kk)
-            if (kk == k) {
-#pragma unroll
-              for (int c = 0; c < 32; ++c) pe[c] = pow_e(fmaxf(xr[kk][c] - tau, 0.f), ei, e);
-            }
-        } else {
-          uint32_t v[32];
-          DASH_TMEM_LD32(v, lane_addr + k * 32);
-          ptx::tmem_wait_ld();
-          const int lim = n_loc - k * 32;
-#pragma unroll
-          for (int c = 0; c < 32; ++c) {
-            const float mm = fmaxf(fmaf(__uint_as_float(v[c]), xs, -tau), 0.f);
-            pe[c] = c < lim ? pow_e(mm, ei, e) : 0.f;
-          }
-        }
+      // one 32-chunk step: pe holds this lane's [x - tau]_+^e on entry and is consumed
+      auto chunk_step = [&](int k, float (&pe)[32]) {
         group_sums(pe);
         uint32_t bits = 0;
         uint32_t lwv[OWN];
@@ -482,6 +464,31 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           mrow[wj] = bits | (((c_own >> 5) == wj) ? (1u << (c_own & 31)) : 0u);
         }
         nsel += __popc(bits);
+      };
+      if (in_regs) {
+        // the register-resident row is spent after this sweep: raise it to the power in place, no second copy
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          if (k < n_chunks) {
+#pragma unroll
+            for (int c = 0; c < 32; ++c) xr[k][c] = pow_e(fmaxf(xr[k][c] - tau, 0.f), ei, e);
+            chunk_step(k, xr[k]);
+          }
+        }
+      } else {
+        for (int k = 0; k < n_chunks; ++k) {
+          float pe[32];
+          uint32_t v[32];
+          DASH_TMEM_LD32(v, lane_addr + k * 32);
+          ptx::tmem_wait_ld();
+          const int lim = n_loc - k * 32;
+#pragma unroll
+          for (int c = 0; c < 32; ++c) {
+            const float mm = fmaxf(fmaf(__uint_as_float(v[c]), xs, -tau), 0.f);
+            pe[c] = c < lim ? pow_e(mm, ei, e) : 0.f;
+          }
+          chunk_step(k, pe);
+        }
       }
       ptx::tmem_wait_st();
 #pragma unroll
