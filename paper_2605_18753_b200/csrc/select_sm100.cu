@@ -349,49 +349,84 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         if (__all_sync(0xffffffffu, done)) break;
       }
     } else if (ok && n_cand > 0) {
-      // longer rows stream from tensor memory every pass (and, in a cluster, meet the other blocks' partial sums)
-      float mx = -INFINITY;
-      for (int k = 0; k < n_chunks; ++k) {
-        uint32_t v[32];
-        DASH_TMEM_LD32(v, lane_addr + k * 32);
-        ptx::tmem_wait_ld();
+      // longer rows stream from tensor memory every pass (and, in a cluster, meet the other blocks' partial sums).
+      // The 32-column loads are software-pipelined over two register buffers: with one block per SM a solver
+      // warp has its scheduler to itself, so an exposed load latency per chunk would be pure idle time.
+      auto stream = [&](auto&& body) {
+        uint32_t va[32], vb[32];
+        DASH_TMEM_LD32(va, lane_addr);
+        for (int k = 0; k < n_chunks; k += 2) {
+          DASH_TMEM_WAIT_LD32(va);
+          if (k + 1 < n_chunks) DASH_TMEM_LD32(vb, lane_addr + (k + 1) * 32);
+          body(va, k);
+          if (k + 1 < n_chunks) {
+            DASH_TMEM_WAIT_LD32(vb);
+            if (k + 2 < n_chunks) DASH_TMEM_LD32(va, lane_addr + (k + 2) * 32);
+            body(vb, k + 1);
+          }
+        }
+      };
+      // columns past the row's last candidate (only in the last chunk) hold scores of later chunks: -inf them
+      auto cut_tail = [&](uint32_t (&v)[32], int k) {
         const int lim = n_loc - k * 32;
+        if (lim < 32) {
 #pragma unroll
-        for (int c = 0; c < 32; ++c) mx = fmaxf(mx, c < lim ? __uint_as_float(v[c]) : -INFINITY);
-      }
-      mx *= xs;
+          for (int c = 0; c < 32; ++c) v[c] = c < lim ? v[c] : 0xff800000u;
+        }
+      };
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+      stream([&](uint32_t (&v)[32], int k) {
+        cut_tail(v, k);
+#pragma unroll
+        for (int c = 0; c < 32; ++c) mx4[c & 3] = fmaxf(mx4[c & 3], __uint_as_float(v[c]));
+      });
+      float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * xs;
       ok = exchange(mx, 0.f);
       for (int pr = 0; pr < CS; ++pr) mx = fmaxf(mx, xa[pr]);
-      float s1 = 0.f, s2 = 0.f;
-      for (int k = 0; k < n_chunks; ++k) {
-        uint32_t v[32];
-        DASH_TMEM_LD32(v, lane_addr + k * 32);
-        ptx::tmem_wait_ld();
+      float s1v[4] = {0.f, 0.f, 0.f, 0.f}, s2v[4] = {0.f, 0.f, 0.f, 0.f};
+      stream([&](uint32_t (&v)[32], int k) {
         const int lim = n_loc - k * 32;
 #pragma unroll
         for (int c = 0; c < 32; ++c) {
           const float y = c < lim ? fmaf(__uint_as_float(v[c]), xs, -mx) : 0.f;
-          s1 += y;
-          s2 = fmaf(y, y, s2);
+          s1v[c & 3] += y;
+          s2v[c & 3] = fmaf(y, y, s2v[c & 3]);
         }
-      }
-      ok = ok && exchange(s1, s2);
+      });
+      ok = ok && exchange((s1v[0] + s1v[1]) + (s1v[2] + s1v[3]), (s2v[0] + s2v[1]) + (s2v[2] + s2v[3]));
       tau = start_tau(mx, xsum_a(), xsum_b());
       bool done = false;
       for (int it = 0; it < max_it && ok; ++it) {
         float f[4] = {0.f, 0.f, 0.f, 0.f}, g[4] = {0.f, 0.f, 0.f, 0.f};
-        for (int k = 0; k < n_chunks; ++k) {
-          uint32_t v[32];
-          DASH_TMEM_LD32(v, lane_addr + k * 32);
-          ptx::tmem_wait_ld();
-          const int lim = n_loc - k * 32;
+        if constexpr (EI_STATIC == 2) {
+          // alpha = 1.5: two candidates per packed instruction (scale and shift, F += m^2, G += m)
+          float2 fv[4], gv[4];
 #pragma unroll
-          for (int c = 0; c < 32; ++c) {
-            float mm = fmaxf(fmaf(__uint_as_float(v[c]), xs, -tau), 0.f);
-            mm = c < lim ? mm : 0.f;
-            f[c & 3] += pow_e(mm, ei, e);
-            g[c & 3] += pow_em1(mm, ei, e);
-          }
+          for (int q = 0; q < 4; ++q) fv[q] = gv[q] = make_float2(0.f, 0.f);
+          const float2 xs2 = make_float2(xs, xs), ntau = make_float2(-tau, -tau);
+          stream([&](uint32_t (&v)[32], int k) {
+            cut_tail(v, k);               // -inf * xs - tau = -inf: contributes nothing
+#pragma unroll
+            for (int c = 0; c < 32; c += 2) {
+              float2 mm = __ffma2_rn(make_float2(__uint_as_float(v[c]), __uint_as_float(v[c + 1])), xs2, ntau);
+              mm.x = fmaxf(mm.x, 0.f);
+              mm.y = fmaxf(mm.y, 0.f);
+              fv[(c >> 1) & 3] = __ffma2_rn(mm, mm, fv[(c >> 1) & 3]);
+              gv[(c >> 1) & 3] = __fadd2_rn(gv[(c >> 1) & 3], mm);
+            }
+          });
+#pragma unroll
+          for (int q = 0; q < 4; ++q) { f[q] = fv[q].x + fv[q].y; g[q] = gv[q].x + gv[q].y; }
+        } else {
+          stream([&](uint32_t (&v)[32], int k) {
+            cut_tail(v, k);               // -inf * xs - tau = -inf: contributes nothing
+#pragma unroll
+            for (int c = 0; c < 32; ++c) {
+              const float mm = fmaxf(fmaf(__uint_as_float(v[c]), xs, -tau), 0.f);
+              f[c & 3] += pow_e(mm, ei, e);
+              g[c & 3] += pow_em1(mm, ei, e);
+            }
+          });
         }
         ok = exchange((f[0] + f[1]) + (f[2] + f[3]), (g[0] + g[1]) + (g[2] + g[3]));
         if (!ok) break;
