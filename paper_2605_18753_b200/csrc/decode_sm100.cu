@@ -9,7 +9,8 @@
 // One softmax thread per key row (= TMEM lane of S^T); the per-head running maximum is shared through a
 // small shared-memory reduction, the accumulator O^T is only 16 TMEM columns, so rescaling it is cheap.
 // The routed list (plus the row's own, possibly partial, chunk) is cut into n_split contiguous ranges of
-// 64-token sub-blocks, one thread block each; partial (m, l, O) go to the merge kernel in split order.
+// 64-token sub-blocks, one thread block each; the block that sees the last arrival of its (batch, KV head)
+// merges the partial (m, l, O) of all splits in split order (or, without a workspace, a separate merge kernel does).
 // Every wait is bounded (DASH_ERR_TIMEOUT in the status word).
 #include <cuda.h>
 
@@ -372,7 +373,7 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       float* pp = a.partials + pbase + (long long)h * n_split * (HD + 2);
       pp[2 + tid] = (n_steps > 0) ? __uint_as_float(o[h]) : 0.f;   // thread tid holds O^T[d = tid][h]
       if (tid == h) {
-        pp[0] = (n_steps > 0) ? m[h] * 0.6931471805599453f : -INFINITY;   // the merge kernel works in natural-log units
+        pp[0] = (n_steps > 0) ? m[h] * 0.6931471805599453f : -INFINITY;   // the merge works in natural-log units
         pp[1] = misc->lred[0][h] + misc->lred[1][h] + misc->lred[2][h] + misc->lred[3][h];
       }
     }

@@ -7,8 +7,8 @@
 //                         chunk logits x = gamma(alpha-1) <q, kbar_c>/sqrt(d) of the g_q heads to a small
 //                         fp32 scratch (b * h_q * T_s floats, stays in L2);
 //   decode_route_kernel   one thread block of 32 warps per (batch, KV head) loads its g_q logit rows into shared
-//                         memory, finds tau per head (Newton from max - 1: monotone from below; a team of
-//                         32 / g_q warps per head), then forms the group weights, mask words, log w, mu and
+//                         memory, finds tau per head (Newton from max - 1: monotone from below; eight
+//                         warps in all, a team of 8 / g_q per head), then forms the group weights, mask words, log w, mu and
 //                         the compact (chunk, bias) list.
 #include <type_traits>
 

@@ -8,8 +8,9 @@
 // must match a float64 evaluation except within 1e-4 of the threshold.
 //
 // Each of the 128 solver threads owns one row = one TMEM lane, so the threshold search needs no
-// cross-thread reduction: a pass streams the row out of tensor memory 32 columns at a time.  tau is found
-// by Newton's method from max(x) - 1 (f convex and decreasing: monotone from below, finite for alpha = 2).
+// cross-thread reduction: rows of up to 128 candidates are held in registers over all passes, longer ones
+// stream out of tensor memory 32 columns at a time (loads software-pipelined over two register buffers).
+// tau is found by Newton's method (f convex and decreasing: monotone from below, finite for alpha = 2).
 // The GQA group's heads sit in adjacent lanes; the group weights, the 32-chunk mask words, log w, mu and the
 // compact bias lists are formed through a small shared-memory exchange tile, one warp-synchronous step per
 // 32 chunks.  Waits are bounded as in the Stage 2 kernel.
