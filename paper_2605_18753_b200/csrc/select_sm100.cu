@@ -1,7 +1,7 @@
 // Stage 1 on tensor cores for sm_100a (Eq. 2, Eq. 4, Algorithm 2, Proposition 1), bf16 queries, head_dim 128.
 //
 // Tile = the 128 (token, head-of-group) rows of TQ = 128/g_q consecutive tokens of one (batch, KV head);
-// they share their candidate chunks.  The whole score tile X[128 rows][n_cand <= 512 chunks] is produced by
+// they share their candidate chunks.  The whole score tile X[128 rows][<= 512 chunks per block] is produced by
 // tcgen05.mma into tensor memory and never leaves the SM (Algorithm 2 writes it to HBM).  The fp32
 // summaries are split beforehand into three bf16 planes (hi + mid + lo = the fp32 value exactly), so that
 // Q (exact in bf16) times the three planes, accumulated in fp32, carries fp32-class accuracy: the support
@@ -11,9 +11,11 @@
 // cross-thread reduction: rows of up to 128 candidates are held in registers over all passes, longer ones
 // stream out of tensor memory 32 columns at a time (loads software-pipelined over two register buffers).
 // tau is found by Newton's method (f convex and decreasing: monotone from below, finite for alpha = 2).
-// The GQA group's heads sit in adjacent lanes; the group weights, the 32-chunk mask words, log w, mu and the
-// compact bias lists are formed through a small shared-memory exchange tile, one warp-synchronous step per
-// 32 chunks.  Waits are bounded as in the Stage 2 kernel.
+// The GQA group's heads sit in adjacent lanes; the group weights come from a halving shuffle exchange, one
+// warp-synchronous step per 32 chunks; log w is parked in tensor memory until mu is known, then the compact
+// bias lists are written.  Rows longer than one block's tensor memory are split over a thread-block cluster
+// whose blocks all-reduce the per-row sums through distributed shared memory.  Waits are bounded as in the
+// Stage 2 kernel.
 #include <cuda.h>
 
 #include <type_traits>
