@@ -326,3 +326,50 @@ def test_decode_equals_last_prefill_row_on_gpu():
     wsd = B.alloc_workspace(pd)
     B.dash_attn_fwd_decode(pd, q1, K, V, kbar, None, o1, wsd)
     assert (o1.float() - O[:, -1].float()).abs().max().item() <= 2e-2
+
+
+# ------------------------------------------------------------------ strided tensors
+
+@pytest.mark.parametrize("layout", ["packed_qkv", "head_major"])
+def test_fwd_prefill_and_decode_on_strided_views(layout):
+    """Q, K, V, O as views of larger buffers (one packed [b, n, h_q + 2 h_kv, d] projection output; a head-major
+    [b, h, n, d] buffer): only the element strides in the parameter block change, the results must not."""
+    w = _wl(seq=1200, h_q=8, h_kv=2, head_dim=128, block=64, seed=5)
+    inp = synth.make_prefill_inputs(w, DEV)
+    Q, K, V = inp["Q"], inp["K"], inp["V"]
+    O = torch.empty_like(Q)
+    p = B.params_for_prefill(Q, K, V, O, block=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma)
+    ws = B.alloc_workspace(p)
+    B.dash_attn_fwd_prefill(p, Q, K, V, O, ws)
+    assert B.dash_attn_last_status(ws) == 0
+
+    b, n, h_q, h_kv, d = w.batch, w.seq, w.h_q, w.h_kv, w.head_dim
+    if layout == "packed_qkv":
+        buf = torch.full((b, n, h_q + 2 * h_kv, d), float("nan"), dtype=Q.dtype, device=DEV)
+        buf[:, :, :h_q] = Q
+        buf[:, :, h_q:h_q + h_kv] = K
+        buf[:, :, h_q + h_kv:] = V
+        Qs, Ks, Vs = buf[:, :, :h_q], buf[:, :, h_q:h_q + h_kv], buf[:, :, h_q + h_kv:]
+        Os = torch.full((b, n, h_q + 3, d), float("nan"), dtype=Q.dtype, device=DEV)[:, :, 3:]
+    else:
+        Qs = Q.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)       # storage [b, h, n, d], viewed [b, n, h, d]
+        Ks = K.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+        Vs = V.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+        Os = torch.empty(b, h_q, n, d, dtype=Q.dtype, device=DEV).permute(0, 2, 1, 3)
+    assert not Qs.is_contiguous() and Qs.stride(-1) == 1
+    ps = B.params_for_prefill(Qs, Ks, Vs, Os, block=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma)
+    ws2 = B.alloc_workspace(ps)
+    B.dash_attn_fwd_prefill(ps, Qs, Ks, Vs, Os, ws2)
+    assert B.dash_attn_last_status(ws2) == 0
+    assert torch.equal(Os, O)
+
+    # decode on the same views: the last token against the strided cache
+    q1 = Qs[:, -1]
+    o1 = torch.empty(b, h_q, d, dtype=Q.dtype, device=DEV)
+    pd = B.params_for_decode(q1, Ks, Vs, o1, block=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma)
+    kbar = B.alloc_kbar(pd)
+    B.dash_attn_block_summaries(pd, Ks, kbar)
+    wsd = B.alloc_workspace(pd)
+    B.dash_attn_fwd_decode(pd, q1, Ks, Vs, kbar, None, o1, wsd)
+    assert B.dash_attn_last_status(wsd) == 0
+    assert (o1.float() - O[:, -1].float()).abs().max().item() <= 2e-2
