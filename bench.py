@@ -177,6 +177,105 @@ def run_reference(args, w):
     print(json.dumps(line), flush=True)
 
 
+def run_paper_protocol(args):
+    """SECONDARY measurement, not the contract line: the paper's own Stage-2 speed protocol (random chunk masks
+    at a fixed sparsity, GQA 16:1 with 32 query / 2 KV heads, d = 128, chunks of 64; prefill batch 1, decode
+    batch 24) next to dense SDPA on the same tensors.  Random masks share nothing between neighbouring
+    queries, the worst case for a kernel that walks the union of a tile's chunks: the inflation is printed."""
+    from paper_2605_18753_b200 import binding as B
+    B.lib()
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
+    h_q, h_kv, d, blk = 32, 2, 128, 64
+    g_q = h_q // h_kv
+
+    def timed(fn, iters=5, warm=2):
+        for _ in range(warm):
+            fn()
+        ts = []
+        for k in range(iters):
+            flush.fill_(k)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); fn(); b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        return float(np.mean(ts))
+
+    def pack_bits(bits):                       # bool [..., W * 32] -> int32 words, chunk c = bit c & 31 of word c >> 5
+        v = bits.view(*bits.shape[:-1], -1, 32).to(torch.int64)
+        w = (v << torch.arange(32, device=bits.device, dtype=torch.int64)).sum(-1)
+        return torch.where(w >= 2 ** 31, w - 2 ** 32, w).to(torch.int32)
+
+    rows = []
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(0)
+    for n in (16384, 32768, 65536):
+        Q = torch.randn(1, n, h_q, d, generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+        K = torch.randn(1, n, h_kv, d, generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+        V = torch.randn(1, n, h_kv, d, generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+        O = torch.empty_like(Q)
+        p = B.params_for_prefill(Q, K, V, O, block=blk, alpha=1.5, gamma=1.0, sigma=1e8)
+        ws = B.alloc_workspace(p, dev)
+        T_a = n // blk
+        W = (T_a + 31) // 32
+        bias = torch.zeros(max(B.dash_attn_list_capacity(p), 1), dtype=torch.float32, device=dev)   # prior off
+        q, k, v = (t.transpose(1, 2) for t in (Q, K, V))
+        t_dense = timed(lambda: torch.nn.functional.scaled_dot_product_attention(q, k, v, is_causal=True, enable_gqa=True))
+        own = torch.arange(n, device=dev) // blk
+        cidx = torch.arange(W * 32, device=dev)
+        for sparsity in (0.75, 0.875, 0.9375):
+            mask = torch.empty(1, h_kv, n, W, dtype=torch.int32, device=dev)
+            count = torch.empty(1, h_kv, n, dtype=torch.int32, device=dev)
+            for r in range(h_kv):
+                for i0 in range(0, n, 8192):           # bounded temporaries
+                    i1 = min(n, i0 + 8192)
+                    u = torch.rand(i1 - i0, W * 32, generator=gen, device=dev)
+                    routed = (u < (1.0 - sparsity)) & (cidx[None, :] < own[i0:i1, None])
+                    count[0, r, i0:i1] = routed.sum(-1).to(torch.int32)
+                    mask[0, r, i0:i1] = pack_bits(routed | (cidx[None, :] == own[i0:i1, None]))
+            w_like = argparse.Namespace(h_q=h_q, h_kv=h_kv, block=blk)
+            t = timed(lambda: B.dash_attn_attend_prefill(p, Q, K, V, mask, bias, O, ws))
+            assert B.dash_attn_last_status(ws) == 0
+            f_sel = selected_flops_from_count(count, blk, d, g_q)
+            f_exec, _ = executed_flops_from_mask(mask, w_like)
+            rows.append({"mode": "prefill", "n": n, "sparsity": sparsity, "attend_ms": t, "sdpa_dense_ms": t_dense,
+                         "speedup_vs_dense": t_dense / t, "selected_tflops": f_sel / (t * 1e-3) / 1e12,
+                         "union_inflation": f_exec / f_sel})
+        del Q, K, V, O, ws, bias
+
+    # decode: batch 24, one query per sequence, random routed lists
+    bs = 24
+    for n in (16384, 32768, 65536):
+        q1 = torch.randn(bs, h_q, d, generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+        Kc = torch.randn(bs, n, h_kv, d, generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+        Vc = torch.randn(bs, n, h_kv, d, generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+        o1 = torch.empty_like(q1)
+        pd = B.params_for_decode(q1, Kc, Vc, o1, block=blk, alpha=1.5, gamma=1.0, sigma=1e8)
+        wsd = B.alloc_workspace(pd, dev)
+        T_s = (n - 1) // blk
+        lens = torch.full((bs,), n, dtype=torch.int32, device=dev)
+        kd, vd, qd = Kc.transpose(1, 2), Vc.transpose(1, 2), q1[:, :, None, :]
+        t_dense = timed(lambda: torch.nn.functional.scaled_dot_product_attention(qd, kd, vd, enable_gqa=True))
+        for sparsity in (0.75, 0.875, 0.9375):
+            kk = max(1, int(round((1.0 - sparsity) * T_s)))
+            u = torch.rand(bs * h_kv, T_s, generator=gen, device=dev)
+            idx = torch.sort(torch.topk(u, kk, dim=-1).indices, dim=-1).values.to(torch.int32)
+            blk_idx = torch.zeros(bs * h_kv, max(n // blk, 1), dtype=torch.int32, device=dev)
+            blk_idx[:, :kk] = idx
+            cnt = torch.full((bs, h_kv, 1), kk, dtype=torch.int32, device=dev)
+            bias = torch.zeros_like(blk_idx, dtype=torch.float32)
+            t = timed(lambda: B.dash_attn_attend_decode(pd, q1, Kc, Vc, lens, cnt, blk_idx, bias, o1, wsd))
+            assert B.dash_attn_last_status(wsd) == 0
+            byts = bs * h_kv * (kk + 1) * blk * d * 2 * 2
+            rows.append({"mode": "decode", "n": n, "batch": bs, "sparsity": sparsity, "attend_ms": t,
+                         "sdpa_dense_ms": t_dense, "speedup_vs_dense": t_dense / t,
+                         "hbm_gbs_on_bytes_touched": byts / (t * 1e-3) / 1e9})
+        del q1, Kc, Vc, o1, wsd
+    print(json.dumps({"metric": "paper_protocol_stage2 (secondary)", "heads": "32/2", "head_dim": d, "block": blk,
+                      "data": "random tensors, random chunk masks", "rows": rows}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -186,7 +285,12 @@ def main():
     ap.add_argument("--workload", default="prefill_8k")
     ap.add_argument("--no-extras", action="store_true", help="skip the SDPA / decode / long-context side measurements")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--paper-protocol", action="store_true",
+                    help="secondary: the paper's Stage-2 speed protocol (random masks, 32/2 heads) instead of the contract line")
     args = ap.parse_args()
+    if args.paper_protocol:
+        run_paper_protocol(args)
+        return
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
     from paper_2605_18753_b200 import synth
