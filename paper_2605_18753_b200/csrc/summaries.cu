@@ -45,14 +45,19 @@ summaries_kernel(Dims dm, const T* __restrict__ K, const float* __restrict__ qba
   };
 
   if (qbar == nullptr) {
-    for (int t0 = 0; t0 < dm.B; t0 += SUM_UNROLL) {
-      float kv[SUM_UNROLL][VPL];
+    // plain mean: 16 rows in flight per warp (a small prefill has fewer warps than the SMs can hold, so the depth
+    // of each warp's load queue is what covers the DRAM latency)
+    constexpr int MU = 2 * SUM_UNROLL;
+    for (int t0 = 0; t0 < dm.B; t0 += MU) {
+      float kv[MU][VPL];
 #pragma unroll
-      for (int u = 0; u < SUM_UNROLL; ++u) loadv(kp + (long long)(t0 + u) * dm.ks[1], kv[u]);
+      for (int u = 0; u < MU; ++u) loadv(kp + (long long)min(t0 + u, dm.B - 1) * dm.ks[1], kv[u]);
 #pragma unroll
-      for (int u = 0; u < SUM_UNROLL; ++u)
+      for (int u = 0; u < MU; ++u)
+        if (t0 + u < dm.B) {
 #pragma unroll
-        for (int v = 0; v < VPL; ++v) acc[v] += kv[u][v];
+          for (int v = 0; v < VPL; ++v) acc[v] += kv[u][v];
+        }
     }
     const float inv = 1.f / (float)dm.B;
 #pragma unroll
