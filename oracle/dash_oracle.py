@@ -37,6 +37,16 @@ design notes):
   chunks; D_i is the incomplete tail chunk (empty when B divides n), bias 0.
   Parity unpinned by the paper beyond brute force on tiny inputs.
 * Decode: ``kv_len`` counts the new token; the query sits at ``kv_len - 1``.
+* Local window (``local_blocks = L``; appendix "Long-context adaptation", training
+  settings: the sliding window is the diagonal block and the last block).  Read
+  as: the L chunks just before the diagonal chunk belong to D_i together with
+  the causal part of the diagonal chunk: attended in full with bias 0, counted
+  in |D_i|, and not scored, so the routed candidates are the chunks before
+  c_i - L.  L = 0 is Algorithms 2-3 as printed; L = 1 with B = 64 gives
+  |D_i| = 64 + (i mod 64) + 1 tokens (the appendix counts "64-127", i.e.
+  without the query's own position).  The other possible reading (the previous
+  chunk forced into the support but still scored) is not built; parity between
+  the two is unpinned by the paper.  Causal mode only.
 """
 from __future__ import annotations
 
@@ -219,6 +229,7 @@ class RowRouting:
     support: np.ndarray = field(default_factory=lambda: np.zeros(0, dtype=np.int64))  # routed chunk ids, ascending
     bias: np.ndarray = field(default_factory=lambda: np.zeros(0))         # [len(support)] d of Prop. 1
     log_w: np.ndarray = field(default_factory=lambda: np.zeros(0))        # [len(support)]
+    local: np.ndarray = field(default_factory=lambda: np.zeros(0, dtype=np.int64))  # window chunks before the diagonal one
 
 
 def route_row(q_g: np.ndarray, Kbar_r: np.ndarray, n_cand: int, alpha: float,
@@ -327,18 +338,27 @@ def attend_row_definition_form(q_g: np.ndarray, K_r: np.ndarray, V_r: np.ndarray
 # Whole rows / whole problems.
 # --------------------------------------------------------------------------
 
-def _row_geometry(i: int, length: int, B: int, causal: bool):
-    """(number of candidate chunks, diagonal token range) of query position i."""
+def _row_geometry(i: int, length: int, B: int, causal: bool, local_blocks: int = 0):
+    """(number of candidate chunks, token range of D_i) of query position i.
+
+    With a local window of L chunks, D_i starts L chunks before the diagonal
+    chunk (or at token 0) and the candidates are the chunks before that.
+    """
     T_s = length // B
+    if local_blocks < 0:
+        raise ValueError("local_blocks must be >= 0")
     if causal:
-        c_i = i // B
-        return min(c_i, T_s), c_i * B, i + 1
+        c_lo = max(i // B - local_blocks, 0)
+        return min(c_lo, T_s), c_lo * B, i + 1
+    if local_blocks:
+        raise ValueError("the local window is defined for the causal mode only")
     return T_s, T_s * B, length
 
 
 def forward_row(Q_b: np.ndarray, K_b: np.ndarray, V_b: np.ndarray, Kbar_b: np.ndarray,
                 i: int, r: int, *, B: int, alpha: float, gamma: float, sigma: float,
-                causal: bool = True, length: int | None = None, q_row: np.ndarray | None = None):
+                causal: bool = True, length: int | None = None, q_row: np.ndarray | None = None,
+                local_blocks: int = 0):
     """One query row i of KV head r of one sequence.
 
     Q_b [n, h_q, d] (or pass ``q_row`` [h_q, d] for decode), K_b, V_b
@@ -349,8 +369,10 @@ def forward_row(Q_b: np.ndarray, K_b: np.ndarray, V_b: np.ndarray, Kbar_b: np.nd
     g_q = qh.shape[0] // h_kv
     q_g = np.asarray(qh[r * g_q:(r + 1) * g_q], dtype=np.float64)
     length = K_b.shape[0] if length is None else int(length)
-    n_cand, dlo, dhi = _row_geometry(i, length, B, causal)
+    n_cand, dlo, dhi = _row_geometry(i, length, B, causal, local_blocks)
     rt = route_row(q_g, Kbar_b[:, r, :], n_cand, alpha, gamma, sigma)
+    if causal:
+        rt.local = np.arange(dlo // B, i // B, dtype=np.int64)
     o = attend_row(q_g, K_b[:length, r, :], V_b[:length, r, :], B, rt.support, rt.bias, dlo, dhi)
     return rt, o
 
@@ -368,7 +390,7 @@ def pack_mask_words(support: np.ndarray, diag_chunk: int | None, n_words: int) -
 
 def forward_prefill(Q: np.ndarray, K: np.ndarray, V: np.ndarray, *, B: int, alpha: float,
                     gamma: float = 1.0, sigma: float = 10.0, causal: bool = True,
-                    qbar: np.ndarray | None = None, rows=None, kv_heads=None):
+                    qbar: np.ndarray | None = None, rows=None, kv_heads=None, local_blocks: int = 0):
     """Prefill over [b, n, h, d] tensors.  ``rows``/``kv_heads`` restrict the work to a sample.
 
     Returns a dict: Kbar [b, T_s, h_kv, d]; O [b, n, h_q, d] (NaN where not
@@ -389,7 +411,7 @@ def forward_prefill(Q: np.ndarray, K: np.ndarray, V: np.ndarray, *, B: int, alph
         for r in kv_heads:
             for i in rows:
                 rt, o = forward_row(Q[bb], K[bb], V[bb], Kbar[bb], i, r, B=B, alpha=alpha,
-                                    gamma=gamma, sigma=sigma, causal=causal)
+                                    gamma=gamma, sigma=sigma, causal=causal, local_blocks=local_blocks)
                 routing[(bb, r, i)] = rt
                 O[bb, i, r * g_q:(r + 1) * g_q, :] = o
     return {"Kbar": Kbar, "O": O, "routing": routing}
@@ -397,7 +419,7 @@ def forward_prefill(Q: np.ndarray, K: np.ndarray, V: np.ndarray, *, B: int, alph
 
 def forward_decode(Q: np.ndarray, Kc: np.ndarray, Vc: np.ndarray, kv_len, *, B: int, alpha: float,
                    gamma: float = 1.0, sigma: float = 10.0, qbar: np.ndarray | None = None,
-                   Kbar: np.ndarray | None = None, batches=None, kv_heads=None):
+                   Kbar: np.ndarray | None = None, batches=None, kv_heads=None, local_blocks: int = 0):
     """Decode: Q [b, h_q, d] (one new token per sequence), caches [b, cap, h_kv, d], kv_len [b].
 
     The query of sequence bb sits at position kv_len[bb] - 1 (the new token is
@@ -430,7 +452,7 @@ def forward_decode(Q: np.ndarray, Kc: np.ndarray, Vc: np.ndarray, kv_len, *, B: 
                 Kbar_r = Kb[:, r:r + 1, :]
             q_row = Q[bb, r * g_q:(r + 1) * g_q, :]
             rt, o = forward_row(None, K_b, V_b, Kbar_r, L - 1, 0, B=B, alpha=alpha, gamma=gamma,
-                                sigma=sigma, causal=True, length=L, q_row=q_row)
+                                sigma=sigma, causal=True, length=L, q_row=q_row, local_blocks=local_blocks)
             routing[(bb, r)] = rt
             O[bb, r * g_q:(r + 1) * g_q, :] = o
     return {"O": O, "routing": routing}

@@ -216,3 +216,96 @@ def test_mask_packing_and_statistics():
     assert list(w) == [0x80000001, 0x00000001, (1 << 6) | (1 << 31)]
     assert orc.block_sparsity([0, 1, 2], [0, 3, 8]) == pytest.approx(1 - 6 / 14)
     assert orc.selected_flops([2], [5], 64, 128, 4) == 4 * 128 * 4 * (128 + 5)
+
+
+# ------------------------------------------------------------------ local window (diagonal + previous chunks)
+
+def test_local_window_zero_is_the_printed_algorithms():
+    Q, K, V = _case(80, n=120)
+    a = orc.forward_prefill(Q, K, V, B=16, alpha=1.5, gamma=3.0, sigma=2.0)
+    b = orc.forward_prefill(Q, K, V, B=16, alpha=1.5, gamma=3.0, sigma=2.0, local_blocks=0)
+    assert np.array_equal(a["O"], b["O"])
+    assert all(rt.local.size == 0 for rt in b["routing"].values())
+
+
+@pytest.mark.parametrize("L", [1, 2, 3])
+def test_local_window_against_dense_masked_attention(L):
+    """Token-level brute force: the window chunks and the causal part of the diagonal chunk get bias 0, the
+    routed chunks (all before the window) their bias, everything else -inf; softmax written out here."""
+    Q, K, V = _case(81, n=150)
+    B, d = 16, 8
+    res = orc.forward_prefill(Q, K, V, B=B, alpha=1.5, gamma=3.0, sigma=2.0, local_blocks=L)
+    routed_any = False
+    for r in range(2):
+        for i in range(150):
+            rt = res["routing"][(0, r, i)]
+            c_i = i // B
+            lo = max(c_i - L, 0)
+            assert rt.n_cand == lo and list(rt.local) == list(range(lo, c_i))
+            assert all(c < lo for c in rt.support)
+            routed_any |= rt.support.size > 0
+            M = np.full(150, -np.inf)
+            for c, dc in zip(rt.support, rt.bias):
+                M[c * B:(c + 1) * B] = dc
+            M[lo * B:i + 1] = 0.0
+            for h in (2 * r, 2 * r + 1):
+                z = K[0, :, r] @ Q[0, i, h] / math.sqrt(d) + M
+                p = np.exp(z - z.max())
+                p /= p.sum()
+                assert np.allclose(res["O"][0, i, h], p @ V[0, :, r], atol=1e-12)
+    assert routed_any
+
+
+def test_local_window_covering_everything_is_dense_causal_attention():
+    """A window at least as long as the sequence leaves nothing to route: the result is plain causal softmax
+    attention whatever alpha, gamma and sigma are."""
+    Q, K, V = _case(82, n=96, scale=1.0)
+    res = orc.forward_prefill(Q, K, V, B=16, alpha=1.25, gamma=5.0, sigma=0.5, local_blocks=6)
+    for h in range(4):
+        ref = torch.nn.functional.scaled_dot_product_attention(
+            torch.from_numpy(Q[0, :, h])[None], torch.from_numpy(K[0, :, h // 2])[None],
+            torch.from_numpy(V[0, :, h // 2])[None], is_causal=True)[0].numpy()
+        assert np.allclose(res["O"][0, :, h], ref, atol=1e-12)
+    assert all(rt.n_cand == 0 for rt in res["routing"].values())
+
+
+@pytest.mark.parametrize("sigma", [1.0, 10.0, 1e8])
+def test_local_window_bias_form_equals_definition_form(sigma):
+    """Proposition 1 with |D_i| = window tokens + causal diagonal tokens (Eq. 9-10 count tokens)."""
+    Q, K, V = _case(83)
+    B = 16
+    Kbar = orc.block_summaries(K[0], B)
+    for L in (1, 2):
+        for i in (15, 16, 40, 63, 100, 199):
+            for r in (0, 1):
+                rt, o = orc.forward_row(Q[0], K[0], V[0], Kbar, i, r, B=B, alpha=1.5, gamma=3.0, sigma=sigma,
+                                        local_blocks=L)
+                lo = max(i // B - L, 0)
+                o2 = orc.attend_row_definition_form(Q[0, i, 2 * r:2 * r + 2], K[0, :, r], V[0, :, r], B,
+                                                    rt.support, rt.w[rt.support] if rt.n_cand else np.zeros(0),
+                                                    sigma, lo * B, i + 1)
+                assert np.allclose(o, o2, rtol=1e-11, atol=1e-12)
+
+
+def test_local_window_size_matches_the_training_setting():
+    """B = 64, one window chunk: D_i holds 64 + (i mod 64) + 1 tokens once a previous chunk exists (the
+    appendix's "64-127 tokens" counts the positions before the query)."""
+    for i in (64, 100, 127, 128, 1000):
+        n_cand, dlo, dhi = orc._row_geometry(i, 4096, 64, True, 1)
+        assert dhi - dlo - 1 == 64 + i % 64 and 64 <= dhi - dlo - 1 <= 127
+        assert n_cand == i // 64 - 1
+
+
+def test_local_window_decode_equals_last_prefill_row():
+    Q, K, V = _case(84, n=150)
+    pre = orc.forward_prefill(Q, K, V, B=16, alpha=1.5, gamma=3.0, sigma=5.0, rows=[99, 149], local_blocks=2)
+    for L in (100, 150):
+        dec = orc.forward_decode(Q[:, L - 1], K, V, [L], B=16, alpha=1.5, gamma=3.0, sigma=5.0, local_blocks=2)
+        assert np.allclose(dec["O"][0], pre["O"][0, L - 1], atol=1e-13)
+        assert np.array_equal(dec["routing"][(0, 1)].local, pre["routing"][(0, 1, L - 1)].local)
+
+
+def test_local_window_is_causal_only():
+    Q, K, V = _case(85, n=64)
+    with pytest.raises(ValueError):
+        orc.forward_prefill(Q, K, V, B=16, alpha=1.5, causal=False, local_blocks=1)
