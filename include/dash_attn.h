@@ -26,6 +26,11 @@
  *     summaries; T_a = ceil(seq_kv / block) chunks exist; W = ceil(T_a / 32) mask words per row.
  *   - Query head h uses KV head h / (h_q / h_kv) (Section 3.2).
  *   - Only causal = 1 (the paper's setting) is implemented; causal = 0 returns DASH_ERR_UNSUPPORTED.
+ *   - Local window (p->local_blocks = L > 0): the chunks c_own-L .. c_own-1 of a row are not candidates of
+ *     the entmax routing; they are attended like the own chunk (all their tokens, bias 0) and do not enter
+ *     the mean of log w.  In the routing outputs they appear as ordinary list entries with bias exactly 0
+ *     behind the routed ones (they have the largest chunk indices), their mask bits are set and count
+ *     includes them, so Stage 2 needs no other description of the window.
  *
  * Routing outputs (Stage 1 -> Stage 2)
  *   mask     uint32 [batch, h_kv, seq_q, W]: bit (c & 31) of word (c >> 5) is set iff chunk c is
@@ -77,7 +82,10 @@ typedef struct dash_params {
   float alpha;          /* > 1; 1.25, 1.5 and 2 have integer exponents and take the fast path */
   float gamma;          /* Stage-1 temperature multiplying the chunk logit (Eq. 4) */
   float sigma;          /* prior strength of Eq. 8, > 0 */
-  int32_t reserved;     /* 0 */
+  int32_t local_blocks; /* L >= 0 window chunks before the own chunk that every row attends in full with
+                           bias 0 and that are not scored (appendix "Long-context adaptation": the sliding
+                           window of the trained models is the own chunk plus the previous one, L = 1);
+                           0 = Algorithms 2-3 as printed */
   const int32_t* q_to_kv; /* host, h_q entries, or NULL for h / (h_q/h_kv); only that map is accepted */
   int64_t q_stride[3], k_stride[3], v_stride[3], o_stride[3]; /* elements: batch, token, head */
 } dash_params;

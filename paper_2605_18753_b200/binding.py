@@ -41,7 +41,7 @@ class DashParams(ctypes.Structure):
         ("struct_size", c_uint32), ("batch", c_int32), ("seq_q", c_int32), ("seq_kv", c_int32),
         ("h_q", c_int32), ("h_kv", c_int32), ("head_dim", c_int32), ("block", c_int32),
         ("dtype", c_int32), ("causal", c_int32), ("alpha", c_float), ("gamma", c_float), ("sigma", c_float),
-        ("reserved", c_int32), ("q_to_kv", POINTER(c_int32)),
+        ("local_blocks", c_int32), ("q_to_kv", POINTER(c_int32)),
         ("q_stride", c_int64 * 3), ("k_stride", c_int64 * 3), ("v_stride", c_int64 * 3), ("o_stride", c_int64 * 3),
     ]
 
@@ -130,7 +130,7 @@ def _strides3(t: torch.Tensor, decode_q: bool = False):
 
 
 def make_params(*, batch, seq_q, seq_kv, h_q, h_kv, head_dim, block, dtype, alpha, gamma=1.0, sigma=10.0,
-                causal=1, q_stride=None, k_stride=None, v_stride=None, o_stride=None) -> DashParams:
+                causal=1, local_blocks=0, q_stride=None, k_stride=None, v_stride=None, o_stride=None) -> DashParams:
     """Fills a dash_params; strides default to contiguous [b, n, h, d] (decode Q/O: [b, h, d])."""
     p = DashParams()
     p.struct_size = ctypes.sizeof(DashParams)
@@ -139,7 +139,7 @@ def make_params(*, batch, seq_q, seq_kv, h_q, h_kv, head_dim, block, dtype, alph
     p.dtype = dtype if isinstance(dtype, int) else _dtype_code(dtype)
     p.causal = causal
     p.alpha, p.gamma, p.sigma = alpha, gamma, sigma
-    p.reserved = 0
+    p.local_blocks = local_blocks
     p.q_to_kv = None
     dq = (seq_q * h_q * head_dim, h_q * head_dim, head_dim) if seq_q == seq_kv else (h_q * head_dim, 0, head_dim)
     dk = (seq_kv * h_kv * head_dim, h_kv * head_dim, head_dim)
@@ -149,17 +149,18 @@ def make_params(*, batch, seq_q, seq_kv, h_q, h_kv, head_dim, block, dtype, alph
     return p
 
 
-def params_for_prefill(Q, K, V, O, *, block, alpha, gamma=1.0, sigma=10.0) -> DashParams:
+def params_for_prefill(Q, K, V, O, *, block, alpha, gamma=1.0, sigma=10.0, local_blocks=0) -> DashParams:
     b, n, h_q, d = Q.shape
     return make_params(batch=b, seq_q=n, seq_kv=K.shape[1], h_q=h_q, h_kv=K.shape[2], head_dim=d, block=block,
-                       dtype=Q.dtype, alpha=alpha, gamma=gamma, sigma=sigma, q_stride=_strides3(Q),
+                       dtype=Q.dtype, alpha=alpha, gamma=gamma, sigma=sigma, local_blocks=local_blocks, q_stride=_strides3(Q),
                        k_stride=_strides3(K), v_stride=_strides3(V), o_stride=_strides3(O))
 
 
-def params_for_decode(Q, Kc, Vc, O, *, block, alpha, gamma=1.0, sigma=10.0) -> DashParams:
+def params_for_decode(Q, Kc, Vc, O, *, block, alpha, gamma=1.0, sigma=10.0, local_blocks=0) -> DashParams:
     b, h_q, d = Q.shape
     return make_params(batch=b, seq_q=1, seq_kv=Kc.shape[1], h_q=h_q, h_kv=Kc.shape[2], head_dim=d, block=block,
-                       dtype=Q.dtype, alpha=alpha, gamma=gamma, sigma=sigma, q_stride=_strides3(Q, True),
+                       dtype=Q.dtype, alpha=alpha, gamma=gamma, sigma=sigma, local_blocks=local_blocks,
+                       q_stride=_strides3(Q, True),
                        k_stride=_strides3(Kc), v_stride=_strides3(Vc), o_stride=_strides3(O, True))
 
 

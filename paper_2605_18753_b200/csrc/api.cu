@@ -36,7 +36,7 @@ static int make_dims(const dash_params* p, Dims* dm) {
   if (p->dtype != DASH_F32 && p->dtype != DASH_BF16) return DASH_ERR_INVALID_ARG;
   if (!(p->alpha > 1.f) || !(p->gamma > 0.f) || !(p->sigma > 0.f)) return DASH_ERR_INVALID_ARG;
   if (!std::isfinite(p->alpha) || !std::isfinite(p->gamma) || !std::isfinite(p->sigma)) return DASH_ERR_INVALID_ARG;
-  if (p->reserved != 0) return DASH_ERR_INVALID_ARG;
+  if (p->local_blocks < 0 || p->local_blocks > (1 << 24)) return DASH_ERR_INVALID_ARG;
   if (p->seq_q != p->seq_kv && p->seq_q != 1) return DASH_ERR_INVALID_ARG;
   const int g_q = p->h_q / p->h_kv;
   if (p->q_to_kv) {
@@ -55,6 +55,7 @@ static int make_dims(const dash_params* p, Dims* dm) {
   dm->batch = p->batch; dm->seq_q = p->seq_q; dm->seq_kv = p->seq_kv;
   dm->h_q = p->h_q; dm->h_kv = p->h_kv; dm->d = p->head_dim; dm->B = p->block; dm->g_q = g_q;
   dm->dtype = p->dtype;
+  dm->local_blocks = p->local_blocks;
   dm->T_s = p->seq_kv / p->block;
   dm->T_a = (p->seq_kv + p->block - 1) / p->block;
   dm->W = (dm->T_a + 31) / 32;

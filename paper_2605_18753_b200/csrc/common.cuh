@@ -17,6 +17,7 @@ struct Dims {
   int T_a;      // all chunks: ceil(seq_kv / B)
   int W;        // mask words per row: ceil(T_a / 32)
   int decode;   // 1: one query row per sequence at kv_len[b]-1
+  int local_blocks;  // window chunks before the own chunk: attended with bias 0, not scored
   int e_int;    // 1/(alpha-1) when it is 1, 2 or 4 (alpha = 2, 1.5, 1.25); 0 otherwise
   float e;      // 1/(alpha-1)
   float x_scale;   // gamma (alpha-1) / sqrt(d): chunk logit scale (Algorithm 2, step 1)

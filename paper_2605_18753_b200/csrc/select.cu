@@ -11,6 +11,8 @@
 //   3. Group weights w_c = mean_h [x_hc - tau_h]_+^e, support bit = (max_h (x_hc - tau_h) > 0), 32 chunks
 //      per ballot = one mask word (Algorithm 2 steps 7-13); log w in a scaled form; mu = mean log w;
 //      bias = (log w - mu)/sigma compacted into the row's list (steps 15-19), the own chunk's bit is set.
+// With a local window of L chunks the last L chunks before the own one are not scored: their bits are set and
+// they close the row's list with bias 0 (they take no part in tau, w or mu).
 #include "common.cuh"
 
 namespace dash {
@@ -79,18 +81,18 @@ select_kernel(Dims dm, int TQ, int xs_stride, int token_base, const T* __restric
   chain_wait();
   chain_release();
 
-  int i0, c_own, n_cand;
+  int i0, c_own;
   if (dm.decode) {
     int L = kv_len ? kv_len[b] : dm.seq_kv;
     L = max(1, min(L, dm.seq_kv));
     i0 = 0;
     c_own = (L - 1) / dm.B;
-    n_cand = min(c_own, dm.T_s);
   } else {
     i0 = token_base + tile * TQ;
     c_own = i0 / dm.B;
-    n_cand = min(c_own, dm.T_s);
   }
+  const int n_vis = min(c_own, dm.T_s);                 // chunks before the own one: routed candidates, then the window
+  const int n_cand = max(n_vis - dm.local_blocks, 0);   // scored by entmax
 
   // ---- stage the query rows in fp32 (row = token * g_q + head-in-group)
   for (int idx = tid; idx < R_PAD * (D / 4); idx += SEL_THREADS) {
@@ -220,6 +222,9 @@ select_kernel(Dims dm, int TQ, int xs_stride, int token_base, const T* __restric
       }
       uint32_t word = __ballot_sync(0xffffffffu, sel);
       nsel += __popc(word);
+      const bool local = c >= n_cand && c < n_vis;
+      if (local) x0[c] = -INFINITY;  // -inf marks a window chunk: listed with bias 0
+      word |= __ballot_sync(0xffffffffu, local);
       if ((c_own >> 5) == j) word |= 1u << (c_own & 31);
       if (lane == (j & 31)) myword = word;
       if ((j & 31) == 31 || j == dm.W - 1) {
@@ -227,21 +232,21 @@ select_kernel(Dims dm, int TQ, int xs_stride, int token_base, const T* __restric
       }
     }
     slog = warp_sum(slog);
-    if (lane == 0) count[row_id] = nsel;
+    if (lane == 0) count[row_id] = nsel + (n_vis - n_cand);
 
     // pass 2: bias = (log w - mu) / sigma, compacted in ascending chunk order
-    if (nsel > 0) {
-      const float mu = slog / (float)nsel;
+    if (nsel + (n_vis - n_cand) > 0) {
+      const float mu = nsel > 0 ? slog / (float)nsel : 0.f;
       const long long loff = ((long long)b * dm.h_kv + r) * dm.list_rows + list_row_offset(dm, i);
       int base = 0;
-      for (int j = 0; j * 32 < n_cand; ++j) {
+      for (int j = 0; j * 32 < n_vis; ++j) {
         const int c = j * 32 + lane;
-        const float lw = (c < n_cand) ? x0[c] : INFINITY;
+        const float lw = (c < n_vis) ? x0[c] : INFINITY;
         const bool sel = lw < INFINITY;
         const uint32_t word = __ballot_sync(0xffffffffu, sel);
         if (sel) {
           const long long pos = loff + base + __popc(word & ((1u << lane) - 1u));
-          blk_bias[pos] = (lw - mu) * dm.inv_sigma;
+          blk_bias[pos] = lw == -INFINITY ? 0.f : (lw - mu) * dm.inv_sigma;
           if (blk_idx) blk_idx[pos] = c;
         }
         base += __popc(word);

@@ -10,6 +10,8 @@
 //                         memory, finds tau per head (Newton from max - 1: monotone from below; eight
 //                         warps in all, a team of 8 / g_q per head), then forms the group weights, mask words, log w, mu and
 //                         the compact (chunk, bias) list.
+// With a local window of L chunks the last L chunks before the own one are not scored; the routing kernel sets
+// their bits and appends them to the list with bias 0.
 #include <type_traits>
 
 #include "common.cuh"
@@ -60,7 +62,7 @@ decode_scores_kernel(Dims dm, const T* __restrict__ Q, const float* __restrict__
   chain_wait();
   chain_release();
   L = max(1, min(L, dm.seq_kv));
-  const int n_cand = min((L - 1) / dm.B, dm.T_s);
+  const int n_cand = max(min((L - 1) / dm.B, dm.T_s) - dm.local_blocks, 0);   // window chunks are not scored
   const int c_begin = blockIdx.x * SC_ROWS_PER_BLOCK;
   const int c_end = min(n_cand, c_begin + SC_ROWS_PER_BLOCK);
   if (c_begin >= c_end) return;
@@ -127,8 +129,9 @@ decode_route_kernel(Dims dm, const float* __restrict__ xs, const int* __restrict
   chain_release();
   L = max(1, min(L, dm.seq_kv));
   const int c_own = (L - 1) / dm.B;
-  const int n_cand = min(c_own, dm.T_s);
-  const int stride = route_stride(n_cand);
+  const int n_vis = min(c_own, dm.T_s);                 // chunks before the own one: candidates, then the window
+  const int n_cand = max(n_vis - dm.local_blocks, 0);   // scored by entmax
+  const int stride = route_stride(n_vis);
   float* X = sm;                                 // [G][stride] all logits of the group
   float* taus = X + (size_t)G * stride;          // [G] (32 floats reserved)
   float2* part = reinterpret_cast<float2*>(taus + 32);   // [RT_THREADS] per-lane (F, G) partials + [G] control words;
@@ -288,9 +291,13 @@ decode_route_kernel(Dims dm, const float* __restrict__ xs, const int* __restrict
         lw = e * logf(mstar) + logf(s) - log_gq;
       }
     }
-    const uint32_t word = __ballot_sync(0xffffffffu, sel);
     const float ls = warp_sum(sel ? lw : 0.f);
-    if (c < n_cand) X[c] = lw;                      // +inf marks "not routed"
+    if (c >= n_cand && c < n_vis) {                 // window chunk: listed with bias 0, outside mu
+      sel = true;
+      lw = -INFINITY;
+    }
+    const uint32_t word = __ballot_sync(0xffffffffu, sel);
+    if (c < n_vis) X[c] = lw;                       // +inf marks "not routed", -inf a window chunk
     if (lane == 0) {
       mrow[j] = word | (((c_own >> 5) == j) ? (1u << (c_own & 31)) : 0u);
       wsum[j] = ls;
@@ -323,18 +330,19 @@ decode_route_kernel(Dims dm, const float* __restrict__ xs, const int* __restrict
     }
   }
   __syncthreads();
-  const int nsel = wcnt[dm.W];
-  if (nsel > 0) {
-    const float mu = wsum[0] / (float)nsel;
+  const int nlist = wcnt[dm.W];                  // routed + window chunks
+  const int nsel = nlist - (n_vis - n_cand);     // routed only: the denominator of mu
+  if (nlist > 0) {
+    const float mu = nsel > 0 ? wsum[0] / (float)nsel : 0.f;
     const long long loff = grp * dm.list_rows;
-    for (int j = warp; j * 32 < n_cand; j += RT_THREADS / 32) {
+    for (int j = warp; j * 32 < n_vis; j += RT_THREADS / 32) {
       const int c = j * 32 + lane;
-      const float lw = (c < n_cand) ? X[c] : INFINITY;
+      const float lw = (c < n_vis) ? X[c] : INFINITY;
       const bool sel = lw < INFINITY;
       const uint32_t word = __ballot_sync(0xffffffffu, sel);
       if (sel) {
         const long long pos = loff + wcnt[j] + __popc(word & ((1u << lane) - 1u));
-        blk_bias[pos] = (lw - mu) * dm.inv_sigma;
+        blk_bias[pos] = lw == -INFINITY ? 0.f : (lw - mu) * dm.inv_sigma;
         if (blk_idx) blk_idx[pos] = c;
       }
     }

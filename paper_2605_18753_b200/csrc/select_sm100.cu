@@ -106,7 +106,8 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   constexpr int g_q = G;
   const int i0 = tile * TQ;
   const int c_own = i0 / dm.B;
-  const int n_cand = min(c_own, dm.T_s);                       // candidates of the tile's rows
+  // candidates of the tile's rows; with a local window its chunks are not scored (window_rows_kernel lists them)
+  const int n_cand = min(max(c_own - dm.local_blocks, 0), dm.T_s);   // (c_own <= T_s in a prefill)
   const int c_lo = cr * CLUSTER_COLS;                          // first candidate this block holds
   const int n_loc = CS > 1 ? max(0, min(CLUSTER_COLS, n_cand - c_lo)) : n_cand;
   const int n_blk = (n_loc + SC - 1) / SC;
@@ -667,6 +668,34 @@ static cudaError_t launch_band_g(const Dims& dm, const CUtensorMap& tq, const CU
   }
 }
 
+// Local window: the chunks [c_own - L, c_own) of every row are attended with bias 0 without being scored.  The
+// routing kernel above leaves them out; this one (launched behind it only when L > 0) sets their mask bits,
+// appends them to the row's list behind the routed chunks and adds them to the count.  One thread per row.
+__global__ void __launch_bounds__(256)
+window_rows_kernel(Dims dm, int token_limit, uint32_t* __restrict__ mask, int* __restrict__ count,
+                   int* __restrict__ blk_idx, float* __restrict__ blk_bias) {
+  chain_wait();
+  chain_release();
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long long total = (long long)dm.batch * dm.h_kv * token_limit;
+  if (idx >= total) return;
+  const int i = (int)(idx % token_limit);
+  const long long grp = idx / token_limit;
+  const int n_vis = min(i / dm.B, dm.T_s);
+  const int n_cand = max(n_vis - dm.local_blocks, 0);
+  if (n_vis == n_cand) return;
+  const long long row_id = grp * dm.seq_q + i;
+  uint32_t* mrow = mask + row_id * dm.W;
+  const int routed = count[row_id];
+  const long long loff = grp * dm.list_rows + list_row_offset(dm, i) + routed;
+  for (int c = n_cand; c < n_vis; ++c) {
+    mrow[c >> 5] |= 1u << (c & 31);
+    blk_bias[loff + (c - n_cand)] = 0.f;
+    if (blk_idx) blk_idx[loff + (c - n_cand)] = c;
+  }
+  count[row_id] = routed + (n_vis - n_cand);
+}
+
 cudaError_t launch_select_sm100(const Dims& dm, int token_limit, const void* Q, const float* Kbar, void* planes,
                                 uint32_t* mask, int* count, int* blk_idx, float* blk_bias, float* tau,
                                 StatusBlock* sb, cudaStream_t st, bool planes_ready) {
@@ -727,6 +756,12 @@ cudaError_t launch_select_sm100(const Dims& dm, int token_limit, const void* Q, 
     a.tmem_cols = cols;
     if (cols <= 256) e = launch_band_g<1, 1>(dm, tq, tkb, a, (long long)a.n_tiles * groups, st);
     else e = launch_band_g<2, 1>(dm, tq, tkb, a, (long long)a.n_tiles * groups, st);
+  }
+  if (e == cudaSuccess && dm.local_blocks > 0) {
+    const long long rows = (long long)groups * token_limit;
+    e = launch_chained(window_rows_kernel, dim3((unsigned)((rows + 255) / 256)), dim3(256), 0, st, dm, token_limit,
+                       mask, count, blk_idx, blk_bias);
+    count_launch();
   }
   return e;
 }

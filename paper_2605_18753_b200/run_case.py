@@ -3,7 +3,7 @@
     python -m paper_2605_18753_b200.run_case prefill_8k --iters 5
     python -m paper_2605_18753_b200.run_case decode_128k --batch 4 --iters 3      # 2 GiB of KV cache instead of 8
 
-A quick way to see the path work on a given shape (overrides: --batch, --seq, --block, --alpha), and a small,
+A quick way to see the path work on a given shape (overrides: --batch, --seq, --block, --alpha, --local-blocks), and a small,
 self-terminating command to put under a profiler.  Inputs are the seeded synthetic tensors of `synth`."""
 from __future__ import annotations
 
@@ -23,6 +23,7 @@ def main() -> None:
     ap.add_argument("--seq", type=int)
     ap.add_argument("--block", type=int)
     ap.add_argument("--alpha", type=float)
+    ap.add_argument("--local-blocks", type=int, default=0, help="window chunks before the own chunk (0 = none)")
     args = ap.parse_args()
     over = {k: getattr(args, k) for k in ("batch", "seq", "block", "alpha") if getattr(args, k) is not None}
     w = synth.workload(args.workload, **over)
@@ -33,14 +34,16 @@ def main() -> None:
         inp = synth.make_prefill_inputs(w, dev)
         Q, K, V = inp["Q"], inp["K"], inp["V"]
         O = torch.empty_like(Q)
-        p = B.params_for_prefill(Q, K, V, O, block=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma)
+        p = B.params_for_prefill(Q, K, V, O, block=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma,
+                                 local_blocks=args.local_blocks)
         ws = B.alloc_workspace(p)
         step = lambda: B.dash_attn_fwd_prefill(p, Q, K, V, O, ws)
     else:
         di = synth.make_decode_inputs(w, dev)
         q, Kc, Vc, kl = di["Q"], di["K"], di["V"], di["kv_len"]
         O = torch.empty_like(q)
-        p = B.params_for_decode(q, Kc, Vc, O, block=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma)
+        p = B.params_for_decode(q, Kc, Vc, O, block=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma,
+                                local_blocks=args.local_blocks)
         kbar = B.alloc_kbar(p)
         B.dash_attn_block_summaries(p, Kc, kbar, kv_len=kl)
         ws = B.alloc_workspace(p)

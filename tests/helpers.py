@@ -18,7 +18,8 @@ def tol_for(dtype: torch.dtype):
     return (2e-2, 2e-3) if dtype == torch.bfloat16 else (1e-4, 1e-5)
 
 
-def oracle_prefill_rows(Q, K, V, *, B, alpha, gamma, sigma, rows, kv_heads=None, batches=None, qbar=None):
+def oracle_prefill_rows(Q, K, V, *, B, alpha, gamma, sigma, rows, kv_heads=None, batches=None, qbar=None,
+                        local_blocks=0):
     """Oracle routing + outputs for the given rows.  Returns dict[(b, r, i)] -> (RowRouting, O [g_q, d])."""
     Qn, Kn, Vn = to_np64(Q), to_np64(K), to_np64(V)
     b, n, h_q, d = Qn.shape
@@ -29,7 +30,7 @@ def oracle_prefill_rows(Q, K, V, *, B, alpha, gamma, sigma, rows, kv_heads=None,
         for r in (range(h_kv) if kv_heads is None else kv_heads):
             for i in rows:
                 out[(bb, r, int(i))] = orc.forward_row(Qn[bb], Kn[bb], Vn[bb], Kbar, int(i), r, B=B, alpha=alpha,
-                                                       gamma=gamma, sigma=sigma)
+                                                       gamma=gamma, sigma=sigma, local_blocks=local_blocks)
     return out
 
 
@@ -69,6 +70,16 @@ def compare_routing(rt: orc.RowRouting, own_chunk, mask_words: np.ndarray, count
     if own_chunk is not None:
         assert own_chunk in got, "own chunk's bit must be set"
         got.discard(own_chunk)
+    # window chunks (local_blocks > 0): bits set, listed behind the routed chunks with bias exactly 0, counted
+    local = [int(c) for c in rt.local]
+    assert set(local) <= got, "every window chunk's bit must be set"
+    got -= set(local)
+    assert count >= len(local), "count includes the window chunks"
+    count -= len(local)
+    if local:
+        assert (np.asarray(bias_list[count:count + len(local)]) == 0.0).all(), "window chunks carry bias 0"
+        if idx_list is not None:
+            assert list(idx_list[count:count + len(local)]) == local, "window chunks close the list in order"
     want = set(int(c) for c in rt.support)
     border = set(int(c) for c in np.nonzero(np.abs(rt.margin) <= BORDERLINE)[0]) if rt.n_cand else set()
     diff = got ^ want

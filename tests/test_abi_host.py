@@ -67,13 +67,21 @@ def test_workspace_and_list_geometry(lib):
 @pytest.mark.parametrize("kw,code", [
     (dict(h_q=30), -1), (dict(alpha=1.0), -1), (dict(sigma=0.0), -1), (dict(gamma=-1.0), -1),
     (dict(seq_q=100), -1), (dict(head_dim=96), -2), (dict(block=48), -2), (dict(causal=0), -2),
-    (dict(h_q=24, h_kv=8), -2), (dict(dtype=7), -1), (dict(batch=0), -1),
+    (dict(h_q=24, h_kv=8), -2), (dict(dtype=7), -1), (dict(batch=0), -1), (dict(local_blocks=-1), -1),
 ])
 def test_invalid_parameters_are_rejected_on_the_host(lib, kw, code):
     p = _p(**kw)
     assert B.dash_attn_workspace_bytes(p) == 0
     rc = lib.dash_attn_block_summaries(ctypes.byref(p), 16, None, 0, None, 0, -1, 16, None)
     assert rc == code
+
+
+def test_local_window_changes_no_size(lib):
+    """The window chunks are list entries like the routed ones: same workspace, same list geometry."""
+    a, b = _p(), _p(local_blocks=1)
+    assert B.dash_attn_workspace_bytes(a) == B.dash_attn_workspace_bytes(b) > 0
+    assert B.dash_attn_list_capacity(a) == B.dash_attn_list_capacity(b)
+    assert B.dash_attn_list_offset(a, 0, 3, 130) == B.dash_attn_list_offset(b, 0, 3, 130)
 
 
 def test_null_and_misaligned_pointers_and_short_workspace(lib):

@@ -67,10 +67,11 @@ def test_block_summaries_incremental_and_kv_len():
 
 # ------------------------------------------------------------------ Stage 1
 
-def _run_select(w, inp, with_idx=True):
+def _run_select(w, inp, with_idx=True, local_blocks=0):
     Q, K, V = inp["Q"], inp["K"], inp["V"]
     O = torch.empty_like(Q)
-    p = B.params_for_prefill(Q, K, V, O, block=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma)
+    p = B.params_for_prefill(Q, K, V, O, block=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma,
+                             local_blocks=local_blocks)
     kbar = B.alloc_kbar(p)
     B.dash_attn_block_summaries(p, K, kbar)
     ws = B.alloc_workspace(p)
@@ -84,9 +85,9 @@ def _run_select(w, inp, with_idx=True):
     return p, kbar, ws, rt
 
 
-def _check_select(w, inp, p, rt, rows, kv_heads=None):
+def _check_select(w, inp, p, rt, rows, kv_heads=None, local_blocks=0):
     ora = H.oracle_prefill_rows(inp["Q"], inp["K"], inp["V"], B=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma,
-                                rows=rows, kv_heads=kv_heads)
+                                rows=rows, kv_heads=kv_heads, local_blocks=local_blocks)
     mask = rt["mask"].cpu().numpy().view(np.uint32)
     count = rt["count"].cpu().numpy()
     idx = rt["blk_idx"].cpu().numpy()
@@ -205,11 +206,12 @@ def test_fwd_prefill_small(kw):
     _fwd_prefill_case(w, rows)
 
 
-def _fwd_prefill_case(w, rows, kv_heads=None, min_clean=0.9):
+def _fwd_prefill_case(w, rows, kv_heads=None, min_clean=0.9, local_blocks=0):
     inp = synth.make_prefill_inputs(w, DEV)
     Q, K, V = inp["Q"], inp["K"], inp["V"]
     O = torch.full_like(Q, float("nan"))
-    p = B.params_for_prefill(Q, K, V, O, block=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma)
+    p = B.params_for_prefill(Q, K, V, O, block=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma,
+                             local_blocks=local_blocks)
     ws = B.alloc_workspace(p)
     T_a = (w.seq + w.block - 1) // w.block
     mask = torch.empty(w.batch, w.h_kv, w.seq, (T_a + 31) // 32, dtype=torch.int32, device=DEV)
@@ -217,12 +219,12 @@ def _fwd_prefill_case(w, rows, kv_heads=None, min_clean=0.9):
     assert B.dash_attn_last_status(ws) == 0
     assert torch.isfinite(O.float()).all()
     ora = H.oracle_prefill_rows(Q, K, V, B=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma, rows=rows,
-                                kv_heads=kv_heads)
+                                kv_heads=kv_heads, local_blocks=local_blocks)
     mk = mask.cpu().numpy().view(np.uint32)
     keys = []
     n_excluded = 0
     for (b, r, i), (ro, o) in ora.items():
-        want = orc.pack_mask_words(ro.support, i // w.block, mk.shape[-1])
+        want = orc.pack_mask_words(np.concatenate([ro.support, ro.local]), i // w.block, mk.shape[-1])
         if np.array_equal(mk[b, r, i], want):
             # rows holding a member or non-member inside the borderline band are compared on the mask only:
             # at finite sigma their bias (log of a near-zero weight) is ill-conditioned by construction
@@ -232,7 +234,7 @@ def _fwd_prefill_case(w, rows, kv_heads=None, min_clean=0.9):
                 keys.append((b, r, i))
         else:
             got = {c for c in range(T_a) if (int(mk[b, r, i, c >> 5]) >> (c & 31)) & 1}
-            diff = got ^ (set(int(c) for c in ro.support) | {i // w.block})
+            diff = got ^ (set(int(c) for c in ro.support) | set(int(c) for c in ro.local) | {i // w.block})
             border = set(int(c) for c in np.nonzero(np.abs(ro.margin) <= H.BORDERLINE)[0])
             assert diff <= border, (b, r, i, sorted(diff))
             n_excluded += 1
@@ -255,17 +257,18 @@ def test_fwd_prefill_8k_config_sampled_rows(seed):
 
 # ------------------------------------------------------------------ decode
 
-def _decode_case(w, kv_len, use_lists_from_oracle=False):
+def _decode_case(w, kv_len, use_lists_from_oracle=False, local_blocks=0):
     inp = synth.make_decode_inputs(w, DEV, kv_len=kv_len)
     Q, Kc, Vc, lens = inp["Q"], inp["K"], inp["V"], inp["kv_len"]
     O = torch.full_like(Q, float("nan"))
-    p = B.params_for_decode(Q, Kc, Vc, O, block=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma)
+    p = B.params_for_decode(Q, Kc, Vc, O, block=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma,
+                            local_blocks=local_blocks)
     kbar = B.alloc_kbar(p)
     kbar.fill_(float("nan"))
     B.dash_attn_block_summaries(p, Kc, kbar, kv_len=lens)
     ws = B.alloc_workspace(p)
     ora = orc.forward_decode(H.to_np64(Q), H.to_np64(Kc), H.to_np64(Vc), lens.cpu().numpy(), B=w.block, alpha=w.alpha,
-                             gamma=w.gamma, sigma=w.sigma)
+                             gamma=w.gamma, sigma=w.sigma, local_blocks=local_blocks)
     if use_lists_from_oracle:
         mask, count, idx, bias = H.routing_to_abi({(b, r, 0): rt for (b, r), rt in ora["routing"].items()}, p,
                                                   B.dash_attn_list_offset)
@@ -373,3 +376,71 @@ def test_fwd_prefill_and_decode_on_strided_views(layout):
     B.dash_attn_fwd_decode(pd, q1, Ks, Vs, kbar, None, o1, wsd)
     assert B.dash_attn_last_status(wsd) == 0
     assert (o1.float() - O[:, -1].float()).abs().max().item() <= 2e-2
+
+
+# ------------------------------------------------------------------ local window (own chunk + previous chunks)
+
+@pytest.mark.parametrize("kw,L", [
+    (dict(), 1), (dict(), 3), (dict(alpha=2.0, seq=300), 2), (dict(dtype="f32", seq=300, gamma=3.0), 1),
+    (dict(h_q=8, h_kv=2, head_dim=128, block=32, seq=1000), 1),
+    (dict(h_q=16, h_kv=1, head_dim=128, block=64, seq=1500, batch=2), 2),
+    (dict(h_q=8, h_kv=1, head_dim=128, block=16, seq=9000), 1),      # clusters of two blocks
+    (dict(h_q=32, h_kv=2, head_dim=128, block=32, seq=700), 40),     # window longer than the sequence: nothing routed
+    (dict(h_q=4, h_kv=2, head_dim=128, block=64, seq=2100), 31), (dict(h_q=4, h_kv=2, head_dim=128, block=64, seq=2100), 33),
+])
+def test_select_with_local_window(kw, L):
+    w = _wl(**kw)
+    inp = synth.make_prefill_inputs(w, DEV)
+    p, kbar, ws, rt = _run_select(w, inp, local_blocks=L)
+    step = 7 if w.seq < 12000 else 41
+    rows = sorted(set(list(range(0, w.seq, step)) + [w.seq - 1] + list(range(min(w.seq, (L + 2) * w.block)))))
+    ora, clean, nb, nd = _check_select(w, inp, p, rt, rows, local_blocks=L)
+    assert nd <= nb
+    assert all(v[0].local.size == min(L, i // w.block) for (b, r, i), v in ora.items())
+
+
+@pytest.mark.parametrize("kw,L", [
+    (dict(seq=640, h_q=8, h_kv=2, head_dim=128, block=64, seed=3), 1),
+    (dict(seq=900, h_q=4, h_kv=2, head_dim=128, block=128, seed=4), 2),
+    (dict(seq=500, dtype="f32", gamma=3.0), 1),
+    (dict(seq=1300, h_q=32, h_kv=2, head_dim=128, block=64, seed=5), 1),
+])
+def test_fwd_prefill_with_local_window(kw, L):
+    w = _wl(**kw)
+    rows = sorted(set(list(range(0, w.seq, 5)) + [w.seq - 1, w.seq - 2] + list(range(min(w.seq, 3 * w.block)))))
+    _fwd_prefill_case(w, rows, local_blocks=L)
+
+
+def test_fwd_prefill_8k_config_with_the_training_window():
+    """The 8K workload with the window of the paper's trained models (own chunk + previous chunk)."""
+    w = synth.workload("prefill_8k")
+    rng = np.random.default_rng(7)
+    rows = set(rng.integers(0, w.seq, 512).tolist()) | {0, 63, 64, 65, 127, 128, 129, w.seq - 1, w.seq - 64, w.seq - 65}
+    _fwd_prefill_case(w, sorted(rows), kv_heads=[1, 6], local_blocks=1)
+
+
+def test_window_covering_the_sequence_is_dense_causal_attention():
+    """Nothing is left to route when the window reaches back to token 0: the forward pass must equal dense causal
+    softmax attention (torch SDPA in fp32 on the same bf16 tensors), whatever alpha and sigma are."""
+    w = _wl(seq=1000, h_q=8, h_kv=2, head_dim=128, block=64, alpha=1.25, sigma=0.5)
+    inp = synth.make_prefill_inputs(w, DEV)
+    Q, K, V = inp["Q"], inp["K"], inp["V"]
+    O = torch.full_like(Q, float("nan"))
+    p = B.params_for_prefill(Q, K, V, O, block=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma, local_blocks=16)
+    ws = B.alloc_workspace(p)
+    B.dash_attn_fwd_prefill(p, Q, K, V, O, ws)
+    assert B.dash_attn_last_status(ws) == 0
+    q, k, v = (t.float().transpose(1, 2) for t in (Q, K, V))
+    ref = torch.nn.functional.scaled_dot_product_attention(q, k, v, is_causal=True, enable_gqa=True).transpose(1, 2)
+    H.check_outputs(O.float().cpu().double().numpy(), ref.cpu().double().numpy(), Q.dtype, "window = everything")
+
+
+@pytest.mark.parametrize("kw,kv_len,L", [
+    (dict(kind="decode", batch=3, seq=2000, h_q=8, h_kv=2, head_dim=128, block=64), [2000, 1, 777], 1),
+    (dict(kind="decode", batch=2, seq=5000, h_q=32, h_kv=8, head_dim=128, block=64), [5000, 4097], 2),
+    (dict(kind="decode", batch=2, seq=600, h_q=4, h_kv=2, head_dim=64, block=16, dtype="f32"), [600, 33], 3),
+    (dict(kind="decode", batch=2, seq=1500, h_q=8, h_kv=2, head_dim=128, block=64), [1500, 130], 50),
+])
+def test_decode_with_local_window(kw, kv_len, L):
+    w = _wl(**kw)
+    _decode_case(w, kv_len, local_blocks=L)
