@@ -25,7 +25,12 @@
  *   - 0-based positions.  Chunk of token j is j / block.  T_s = seq_kv / block complete chunks have
  *     summaries; T_a = ceil(seq_kv / block) chunks exist; W = ceil(T_a / 32) mask words per row.
  *   - Query head h uses KV head h / (h_q / h_kv) (Section 3.2).
- *   - Only causal = 1 (the paper's setting) is implemented; causal = 0 returns DASH_ERR_UNSUPPORTED.
+ *   - causal = 1 is the paper's setting and the one the tensor-core kernels serve.  causal = 0 (prefill only;
+ *     the paper does not define it) is read as: every complete chunk is a candidate of every row; the
+ *     incomplete tail chunk (index T_s, present when seq_kv is not a multiple of block) takes the own chunk's
+ *     part -- attended whole by every row with bias 0 -- and there is no causal mask.  It runs on the CUDA-core
+ *     kernels; the list region of row i then starts at (b*h_kv + r) * seq_q * T_s + i * T_s.  A decode shape
+ *     with causal = 0 returns DASH_ERR_UNSUPPORTED, causal = 0 with local_blocks > 0 DASH_ERR_INVALID_ARG.
  *   - Local window (p->local_blocks = L > 0): the chunks c_own-L .. c_own-1 of a row are not candidates of
  *     the entmax routing; they are attended like the own chunk (all their tokens, bias 0) and do not enter
  *     the mean of log w.  In the routing outputs they appear as ordinary list entries with bias exactly 0
@@ -57,7 +62,7 @@ extern "C" {
 typedef enum {
   DASH_OK = 0,
   DASH_ERR_INVALID_ARG = -1, /* null pointer, non-positive size, bad stride/alignment, struct_size mismatch */
-  DASH_ERR_UNSUPPORTED = -2, /* valid request outside what is built (head_dim, block, non-causal, ...) */
+  DASH_ERR_UNSUPPORTED = -2, /* valid request outside what is built (head_dim, block, non-causal decode, ...) */
   DASH_ERR_WORKSPACE = -3,   /* workspace null, misaligned or smaller than dash_attn_workspace_bytes() */
   DASH_ERR_CAPACITY = -4,    /* device side: a list or queue overran its region */
   DASH_ERR_CUDA = -5,        /* a CUDA runtime / driver call failed */
@@ -78,7 +83,7 @@ typedef struct dash_params {
   int32_t head_dim;     /* 64 or 128 */
   int32_t block;        /* chunk size B: 16, 32, 64 or 128 */
   int32_t dtype;        /* dash_dtype of Q, K, V, O */
-  int32_t causal;       /* 1 */
+  int32_t causal;       /* 1 (the paper's setting) or 0 (see Conventions) */
   float alpha;          /* > 1; 1.25, 1.5 and 2 have integer exponents and take the fast path */
   float gamma;          /* Stage-1 temperature multiplying the chunk logit (Eq. 4) */
   float sigma;          /* prior strength of Eq. 8, > 0 */

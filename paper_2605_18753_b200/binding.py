@@ -149,10 +149,11 @@ def make_params(*, batch, seq_q, seq_kv, h_q, h_kv, head_dim, block, dtype, alph
     return p
 
 
-def params_for_prefill(Q, K, V, O, *, block, alpha, gamma=1.0, sigma=10.0, local_blocks=0) -> DashParams:
+def params_for_prefill(Q, K, V, O, *, block, alpha, gamma=1.0, sigma=10.0, local_blocks=0, causal=1) -> DashParams:
     b, n, h_q, d = Q.shape
     return make_params(batch=b, seq_q=n, seq_kv=K.shape[1], h_q=h_q, h_kv=K.shape[2], head_dim=d, block=block,
-                       dtype=Q.dtype, alpha=alpha, gamma=gamma, sigma=sigma, local_blocks=local_blocks, q_stride=_strides3(Q),
+                       dtype=Q.dtype, alpha=alpha, gamma=gamma, sigma=sigma, local_blocks=local_blocks, causal=causal,
+                       q_stride=_strides3(Q),
                        k_stride=_strides3(K), v_stride=_strides3(V), o_stride=_strides3(O))
 
 

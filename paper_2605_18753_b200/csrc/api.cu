@@ -46,7 +46,9 @@ static int make_dims(const dash_params* p, Dims* dm) {
   if (p->head_dim != 64 && p->head_dim != 128) return DASH_ERR_UNSUPPORTED;
   if (p->block != 16 && p->block != 32 && p->block != 64 && p->block != 128) return DASH_ERR_UNSUPPORTED;
   if (g_q != 1 && g_q != 2 && g_q != 4 && g_q != 8 && g_q != 16) return DASH_ERR_UNSUPPORTED;
-  if (p->causal != 1) return DASH_ERR_UNSUPPORTED;
+  if (p->causal != 0 && p->causal != 1) return DASH_ERR_INVALID_ARG;
+  if (p->causal == 0 && p->local_blocks != 0) return DASH_ERR_INVALID_ARG;   // the window is a causal notion
+  if (p->causal == 0 && p->seq_q == 1 && p->seq_kv != 1) return DASH_ERR_UNSUPPORTED;   // decode is causal by nature
   if (!check_strides((const long long*)p->q_stride, p->dtype) || !check_strides((const long long*)p->k_stride, p->dtype) ||
       !check_strides((const long long*)p->v_stride, p->dtype) || !check_strides((const long long*)p->o_stride, p->dtype))
     return DASH_ERR_INVALID_ARG;
@@ -56,6 +58,7 @@ static int make_dims(const dash_params* p, Dims* dm) {
   dm->h_q = p->h_q; dm->h_kv = p->h_kv; dm->d = p->head_dim; dm->B = p->block; dm->g_q = g_q;
   dm->dtype = p->dtype;
   dm->local_blocks = p->local_blocks;
+  dm->causal = p->causal;
   dm->T_s = p->seq_kv / p->block;
   dm->T_a = (p->seq_kv + p->block - 1) / p->block;
   dm->W = (dm->T_a + 31) / 32;
@@ -70,6 +73,8 @@ static int make_dims(const dash_params* p, Dims* dm) {
   }
   if (dm->decode) {
     dm->list_rows = dm->T_s;
+  } else if (!dm->causal) {
+    dm->list_rows = (long long)p->seq_q * dm->T_s;
   } else {
     const long long n = p->seq_q;
     const long long c = n / p->block;

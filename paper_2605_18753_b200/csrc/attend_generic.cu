@@ -29,7 +29,7 @@ attend_prefill_generic_kernel(Dims dm, const T* __restrict__ Q, const T* __restr
   const int i = dm.seq_q - 1 - (int)((gw / dm.h_q) % dm.seq_q);  // long rows first
   const int b = (int)(gw / ((long long)dm.h_q * dm.seq_q));
   const int r = h / dm.g_q;
-  const int c_own = i / dm.B;
+  const int c_own = dm.causal ? i / dm.B : dm.T_s;   // non-causal: the incomplete tail chunk, seen whole by every row
 
   const T* qp = Q + (long long)b * dm.qs[0] + (long long)i * dm.qs[1] + (long long)h * dm.qs[2];
   for (int k = lane; k < D; k += 32) qs[warp][k] = to_f32<T>(qp[k]) * dm.sm_scale;
@@ -54,7 +54,7 @@ attend_prefill_generic_kernel(Dims dm, const T* __restrict__ Q, const T* __restr
       if (c > c_own) continue;  // a mask that marks a future chunk is ignored (causal)
       const float bias = (c == c_own) ? 0.f : brow[cursor];
       if (c != c_own) ++cursor;
-      const int t_end = (c == c_own) ? (i + 1) : min((c + 1) * dm.B, dm.seq_kv);
+      const int t_end = (c == c_own && dm.causal) ? (i + 1) : min((c + 1) * dm.B, dm.seq_kv);
       for (int t0 = c * dm.B; t0 < t_end; t0 += 32) {
         const int t = t0 + lane;
         float s = -INFINITY;

@@ -17,6 +17,7 @@ struct Dims {
   int T_a;      // all chunks: ceil(seq_kv / B)
   int W;        // mask words per row: ceil(T_a / 32)
   int decode;   // 1: one query row per sequence at kv_len[b]-1
+  int causal;        // 1: the paper's setting; 0: every row sees every complete chunk (prefill only)
   int local_blocks;  // window chunks before the own chunk: attended with bias 0, not scored
   int e_int;    // 1/(alpha-1) when it is 1, 2 or 4 (alpha = 2, 1.5, 1.25); 0 otherwise
   float e;      // 1/(alpha-1)
@@ -30,6 +31,7 @@ struct Dims {
 // Start of row i's list region inside its (batch, KV head) slab.
 __host__ __device__ inline long long list_row_offset(const Dims& dm, int i) {
   if (dm.decode) return 0;
+  if (!dm.causal) return (long long)i * dm.T_s;
   long long c = i / dm.B;
   return (long long)dm.B * c * (c - 1) / 2 + (long long)(i % dm.B) * c;
 }

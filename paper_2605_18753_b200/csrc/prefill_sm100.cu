@@ -543,7 +543,7 @@ bool make_map(CUtensorMap* out, const void* base, long long tokens, int heads, i
 }  // namespace
 
 bool prefill_sm100_supported(const Dims& dm) {
-  if (dm.decode || dm.dtype != DASH_BF16 || dm.d != HD) return false;
+  if (dm.decode || !dm.causal || dm.dtype != DASH_BF16 || dm.d != HD) return false;
   if (dm.B != 64 && dm.B != 128) return false;
   const int tq = 128 / dm.g_q;
   if (dm.g_q < 2 || tq > MAX_TQ || tq > dm.B) return false;

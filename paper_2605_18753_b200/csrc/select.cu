@@ -36,7 +36,7 @@ static bool plan_select(const Dims& dm, SelectPlan* pl) {
   if (!dm.decode) {
     while (tq * 2 * dm.g_q <= 32 && tq * 2 <= dm.B) tq *= 2;
   }
-  const int max_cand = dm.decode ? dm.T_s : min(dm.T_s, (dm.seq_q - 1) / dm.B);
+  const int max_cand = (dm.decode || !dm.causal) ? dm.T_s : min(dm.T_s, (dm.seq_q - 1) / dm.B);
   const int xs = ((max_cand + SEL_CT - 1) / SEL_CT) * SEL_CT + 4;
   for (;; tq /= 2) {
     const int rows = tq * dm.g_q;
@@ -89,8 +89,11 @@ select_kernel(Dims dm, int TQ, int xs_stride, int token_base, const T* __restric
     c_own = (L - 1) / dm.B;
   } else {
     i0 = token_base + tile * TQ;
-    c_own = i0 / dm.B;
+    // non-causal: every complete chunk is a candidate of every row; the incomplete tail chunk (index T_s, if
+    // the length is not a multiple of the chunk size) plays the own chunk's part: attended with bias 0
+    c_own = dm.causal ? i0 / dm.B : dm.T_s;
   }
+  const bool has_own = c_own < dm.T_a;
   const int n_vis = min(c_own, dm.T_s);                 // chunks before the own one: routed candidates, then the window
   const int n_cand = max(n_vis - dm.local_blocks, 0);   // scored by entmax
 
@@ -225,7 +228,7 @@ select_kernel(Dims dm, int TQ, int xs_stride, int token_base, const T* __restric
       const bool local = c >= n_cand && c < n_vis;
       if (local) x0[c] = -INFINITY;  // -inf marks a window chunk: listed with bias 0
       word |= __ballot_sync(0xffffffffu, local);
-      if ((c_own >> 5) == j) word |= 1u << (c_own & 31);
+      if (has_own && (c_own >> 5) == j) word |= 1u << (c_own & 31);
       if (lane == (j & 31)) myword = word;
       if ((j & 31) == 31 || j == dm.W - 1) {
         if (lane <= (j & 31)) mrow[(j & ~31) + lane] = myword;

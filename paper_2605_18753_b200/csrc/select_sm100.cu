@@ -615,7 +615,7 @@ bool encode4(CUtensorMap* out, const void* base, const cuuint64_t* dims, const c
 // Tokens [0, select_sm100_token_limit) can be routed by the tensor-core kernel (0: not applicable).  A block
 // holds 512 candidates per row in tensor memory; clusters of 2 or 4 blocks extend that to 1024 / 2048.
 int select_sm100_token_limit(const Dims& dm) {
-  if (dm.decode || dm.dtype != DASH_BF16 || dm.d != HD || dm.T_s < 1) return 0;
+  if (dm.decode || !dm.causal || dm.dtype != DASH_BF16 || dm.d != HD || dm.T_s < 1) return 0;
   const int tq = 128 / dm.g_q;
   if (dm.g_q < 2 || tq > dm.B) return 0;
   if (get_encode() == nullptr) return 0;

@@ -19,7 +19,7 @@ def tol_for(dtype: torch.dtype):
 
 
 def oracle_prefill_rows(Q, K, V, *, B, alpha, gamma, sigma, rows, kv_heads=None, batches=None, qbar=None,
-                        local_blocks=0):
+                        local_blocks=0, causal=True):
     """Oracle routing + outputs for the given rows.  Returns dict[(b, r, i)] -> (RowRouting, O [g_q, d])."""
     Qn, Kn, Vn = to_np64(Q), to_np64(K), to_np64(V)
     b, n, h_q, d = Qn.shape
@@ -30,7 +30,8 @@ def oracle_prefill_rows(Q, K, V, *, B, alpha, gamma, sigma, rows, kv_heads=None,
         for r in (range(h_kv) if kv_heads is None else kv_heads):
             for i in rows:
                 out[(bb, r, int(i))] = orc.forward_row(Qn[bb], Kn[bb], Vn[bb], Kbar, int(i), r, B=B, alpha=alpha,
-                                                       gamma=gamma, sigma=sigma, local_blocks=local_blocks)
+                                                       gamma=gamma, sigma=sigma, local_blocks=local_blocks,
+                                                       causal=causal)
     return out
 
 

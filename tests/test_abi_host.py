@@ -66,7 +66,8 @@ def test_workspace_and_list_geometry(lib):
 
 @pytest.mark.parametrize("kw,code", [
     (dict(h_q=30), -1), (dict(alpha=1.0), -1), (dict(sigma=0.0), -1), (dict(gamma=-1.0), -1),
-    (dict(seq_q=100), -1), (dict(head_dim=96), -2), (dict(block=48), -2), (dict(causal=0), -2),
+    (dict(seq_q=100), -1), (dict(head_dim=96), -2), (dict(block=48), -2), (dict(causal=2), -1), (dict(causal=0, local_blocks=1), -1),
+    (dict(causal=0, seq_q=1), -2),
     (dict(h_q=24, h_kv=8), -2), (dict(dtype=7), -1), (dict(batch=0), -1), (dict(local_blocks=-1), -1),
 ])
 def test_invalid_parameters_are_rejected_on_the_host(lib, kw, code):
@@ -82,6 +83,14 @@ def test_local_window_changes_no_size(lib):
     assert B.dash_attn_workspace_bytes(a) == B.dash_attn_workspace_bytes(b) > 0
     assert B.dash_attn_list_capacity(a) == B.dash_attn_list_capacity(b)
     assert B.dash_attn_list_offset(a, 0, 3, 130) == B.dash_attn_list_offset(b, 0, 3, 130)
+
+
+def test_non_causal_list_geometry(lib):
+    """Without the causal mask every row has all T_s complete chunks as candidates: fixed-size list regions."""
+    p = _p(seq_q=200, seq_kv=200, causal=0)
+    assert B.dash_attn_list_capacity(p) == 8 * 200 * 3
+    assert B.dash_attn_list_offset(p, 0, 2, 7) == 2 * 600 + 21
+    assert B.dash_attn_workspace_bytes(p) > 0
 
 
 def test_null_and_misaligned_pointers_and_short_workspace(lib):

@@ -444,3 +444,47 @@ def test_window_covering_the_sequence_is_dense_causal_attention():
 def test_decode_with_local_window(kw, kv_len, L):
     w = _wl(**kw)
     _decode_case(w, kv_len, local_blocks=L)
+
+
+# ------------------------------------------------------------------ non-causal reading (CUDA-core kernels)
+
+@pytest.mark.parametrize("kw", [
+    dict(seq=200), dict(seq=192), dict(seq=333, dtype="f32", gamma=3.0), dict(seq=15),
+    dict(seq=700, h_q=8, h_kv=2, head_dim=128, block=64, alpha=2.0),
+    dict(seq=640, h_q=16, h_kv=2, head_dim=128, block=32, alpha=1.25, gamma=2.0, batch=2),
+])
+def test_non_causal_prefill_matches_oracle(kw):
+    """causal = 0: all complete chunks are candidates of every row, the incomplete tail chunk is attended whole
+    with bias 0, no causal mask.  Routing lists and outputs against the oracle's non-causal reading."""
+    w = _wl(**kw)
+    inp = synth.make_prefill_inputs(w, DEV)
+    Q, K, V = inp["Q"], inp["K"], inp["V"]
+    O = torch.full_like(Q, float("nan"))
+    p = B.params_for_prefill(Q, K, V, O, block=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma, causal=0)
+    T_s, T_a = w.seq // w.block, (w.seq + w.block - 1) // w.block
+    own = T_s if T_a > T_s else None
+    kbar = B.alloc_kbar(p)
+    B.dash_attn_block_summaries(p, K, kbar)
+    ws = B.alloc_workspace(p)
+    rt = B.alloc_routing(p, with_tau=True)
+    B.dash_attn_select(p, Q, kbar, rt["mask"], rt["count"], rt["blk_idx"], rt["blk_bias"], ws, tau=rt["tau"])
+    assert B.dash_attn_last_status(ws) == 0
+    rows = sorted(set(list(range(0, w.seq, 3)) + [w.seq - 1]))
+    ora = H.oracle_prefill_rows(Q, K, V, B=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma, rows=rows, causal=False)
+    mask = rt["mask"].cpu().numpy().view(np.uint32)
+    count, idx, bias = rt["count"].cpu().numpy(), rt["blk_idx"].cpu().numpy(), rt["blk_bias"].cpu().numpy()
+    clean = {}
+    for (b, r, i), (ro, o) in ora.items():
+        assert ro.n_cand == T_s
+        off = B.dash_attn_list_offset(p, b, r, i)
+        assert off == (b * w.h_kv + r) * w.seq * T_s + i * T_s
+        nb, nd, ok = H.compare_routing(ro, own, mask[b, r, i], int(count[b, r, i]), bias[off:], idx[off:], w.sigma,
+                                       1.0 / (w.alpha - 1.0))
+        clean[(b, r, i)] = ok and not (ro.n_cand and (np.abs(ro.margin) <= H.BORDERLINE).any())
+    B.dash_attn_fwd_prefill(p, Q, K, V, O, ws)
+    assert B.dash_attn_last_status(ws) == 0
+    keys = [k for k, ok in clean.items() if ok]
+    assert len(keys) >= 0.9 * len(ora)
+    if T_s == 0:
+        assert all(v[0].support.size == 0 for v in ora.values())
+    H.check_outputs(_gather_O(O, keys, w.h_q // w.h_kv), np.stack([ora[k][1] for k in keys]), Q.dtype, "non-causal")
