@@ -145,13 +145,25 @@ decode_route_kernel(Dims dm, const float* __restrict__ xs, const int* __restrict
   // ---- logits -> shared memory, row maxima
   float mx[G];
 #pragma unroll
-  for (int g = 0; g < G; ++g) {
-    mx[g] = -INFINITY;
-    for (int c = tid; c < n_cand; c += RT_THREADS) {
-      const float x = xg[(long long)g * dm.T_s + c];
-      X[(size_t)g * stride + c] = x;
-      mx[g] = fmaxf(mx[g], x);
-    }
+  for (int g = 0; g < G; ++g) mx[g] = -INFINITY;
+  // all of a thread's loads of one sweep are issued before the first is used (one L2 round trip per sweep)
+  for (int c0 = 0; c0 < n_cand; c0 += 2 * RT_THREADS) {
+    float v[G][2];
+#pragma unroll
+    for (int g = 0; g < G; ++g)
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        const int c = c0 + u * RT_THREADS + tid;
+        v[g][u] = c < n_cand ? __ldcg(xg + (long long)g * dm.T_s + c) : -INFINITY;
+      }
+#pragma unroll
+    for (int g = 0; g < G; ++g)
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        const int c = c0 + u * RT_THREADS + tid;
+        if (c < n_cand) X[(size_t)g * stride + c] = v[g][u];
+        mx[g] = fmaxf(mx[g], v[g][u]);
+      }
   }
   // maxima through the integer warp reduction (one instruction instead of five shuffles): floats map to
   // signed integers of the same order by flipping the magnitude bits of the negative ones

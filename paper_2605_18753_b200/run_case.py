@@ -24,15 +24,21 @@ def main() -> None:
     ap.add_argument("--block", type=int)
     ap.add_argument("--alpha", type=float)
     ap.add_argument("--local-blocks", type=int, default=0, help="window chunks before the own chunk (0 = none)")
+    ap.add_argument("--kv-layout", choices=("token_major", "head_major"), default="token_major",
+                    help="memory order of K and V: [b, n, h_kv, d] (default) or [b, h_kv, n, d] behind the same strided view")
     args = ap.parse_args()
     over = {k: getattr(args, k) for k in ("batch", "seq", "block", "alpha") if getattr(args, k) is not None}
     w = synth.workload(args.workload, **over)
     dev = "cuda"
+
+    def relayout(t):
+        # same logical [b, n, h, d] tensor; head-major memory makes a chunk's rows of one head contiguous
+        return t.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3) if args.kv_layout == "head_major" else t
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)     # larger than L2
 
     if w.kind == "prefill":
         inp = synth.make_prefill_inputs(w, dev)
-        Q, K, V = inp["Q"], inp["K"], inp["V"]
+        Q, K, V = inp["Q"], relayout(inp["K"]), relayout(inp["V"])
         O = torch.empty_like(Q)
         p = B.params_for_prefill(Q, K, V, O, block=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma,
                                  local_blocks=args.local_blocks)
@@ -40,7 +46,8 @@ def main() -> None:
         step = lambda: B.dash_attn_fwd_prefill(p, Q, K, V, O, ws)
     else:
         di = synth.make_decode_inputs(w, dev)
-        q, Kc, Vc, kl = di["Q"], di["K"], di["V"], di["kv_len"]
+        q, Kc, Vc, kl = di["Q"], relayout(di["K"]), relayout(di["V"]), di["kv_len"]
+        del di
         O = torch.empty_like(q)
         p = B.params_for_decode(q, Kc, Vc, O, block=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma,
                                 local_blocks=args.local_blocks)
