@@ -1,6 +1,7 @@
 // Shared declarations of the DashAttention CUDA library (internal; the public ABI is include/dash_attn.h).
 #pragma once
 
+#include <atomic>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -137,6 +138,20 @@ __device__ __forceinline__ float newton_delta(float F, float G, int e_int, float
 #ifdef __CUDACC__
 __device__ __forceinline__ void chain_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void chain_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// cudaFuncSetAttribute applies to the current device only, and a process may drive several GPUs: one bit per
+// device remembers where a kernel's dynamic shared-memory limit has already been raised.
+template <typename Kern>
+inline cudaError_t allow_dynamic_smem(Kern kern, size_t bytes, std::atomic<unsigned long long>& done) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const bool tracked = dev >= 0 && dev < 64;
+  if (tracked && ((done.load(std::memory_order_relaxed) >> dev) & 1ull)) return cudaSuccess;
+  e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+  if (e == cudaSuccess && tracked) done.fetch_or(1ull << dev, std::memory_order_relaxed);
+  return e;
+}
 
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_chained(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,

@@ -16,6 +16,7 @@
 
 #include "common.cuh"
 #include "sm100_ptx.cuh"
+#include "tensor_map.cuh"
 
 namespace dash {
 
@@ -425,31 +426,12 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   if (tid == 0 && misc->abort_flag) report_error(a.sb, DASH_ERR_TIMEOUT, 301);
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-EncodeTiledFn get_encode() {
-  static EncodeTiledFn fn = nullptr;
-  if (!fn) {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(p);
-  }
-  return fn;
-}
 bool make_kv_map(CUtensorMap* out, const void* base, const Dims& dm, const long long* s) {
-  EncodeTiledFn enc = get_encode();
-  if (!enc) return false;
   cuuint64_t dims[4] = {(cuuint64_t)HD, (cuuint64_t)dm.h_kv, (cuuint64_t)dm.seq_kv, (cuuint64_t)dm.batch};
   auto st = [](long long e) { return (cuuint64_t)((e > 0 ? e : 8) * 2); };
   cuuint64_t strides[3] = {st(s[2]), st(s[1]), st(s[0])};
   cuuint32_t box[4] = {64u, 1u, (cuuint32_t)SUB, 1u};
-  cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
-  return enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
-             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return encode_bf16_sw128_4d(out, base, dims, strides, box);
 }
 
 }  // namespace
@@ -458,7 +440,7 @@ bool make_kv_map(CUtensorMap* out, const void* base, const Dims& dm, const long 
 int decode_sm100_min_splits(const Dims& dm) {
   if (!dm.decode || dm.dtype != DASH_BF16 || dm.d != HD) return 0;
   if (dm.B != 64 && dm.B != 128) return 0;
-  if (dm.qs[2] % 8 != 0 || get_encode() == nullptr) return 0;
+  if (dm.qs[2] % 8 != 0 || tensor_map_encoder() == nullptr) return 0;
   const int max_items = (dm.T_s + 1) * (dm.B / SUB);
   return (max_items + MAX_RANGE - 1) / MAX_RANGE;
 }
@@ -476,13 +458,9 @@ cudaError_t launch_decode_sm100(const Dims& dm, int n_split, const void* Q, cons
   cudaError_t le = cudaSuccess;
 #define DASH_DEC_TC(G)                                                                                          \
   {                                                                                                             \
-    static bool configured = false;                                                                             \
-    if (!configured) {                                                                                          \
-      cudaError_t e = cudaFuncSetAttribute(decode_sm100_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
-                                           DEC_SMEM);                                                           \
-      if (e != cudaSuccess) return e;                                                                           \
-      configured = true;                                                                                        \
-    }                                                                                                           \
+    static std::atomic<unsigned long long> configured{0};                                                       \
+    cudaError_t e = allow_dynamic_smem(decode_sm100_kernel<G>, DEC_SMEM, configured);                           \
+    if (e != cudaSuccess) return e;                                                                             \
     le = launch_chained(decode_sm100_kernel<G>, grid, dim3(DEC_THREADS), DEC_SMEM, st, tk, tv, a);              \
   }
   switch (dm.g_q) {

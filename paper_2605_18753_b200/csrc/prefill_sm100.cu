@@ -24,6 +24,7 @@
 
 #include "common.cuh"
 #include "sm100_ptx.cuh"
+#include "tensor_map.cuh"
 
 namespace dash {
 
@@ -508,36 +509,15 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
 
 // ---------------------------------------------------------------- host side
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn get_encode() {
-  static EncodeTiledFn fn = nullptr;
-  if (!fn) {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(p);
-  }
-  return fn;
-}
-
 // [batch, tokens, heads, 128] bf16 tensor with element strides s[3]; box = 64 x box_heads x box_tokens x 1.
 bool make_map(CUtensorMap* out, const void* base, long long tokens, int heads, int batch, const long long* s,
               int box_heads, int box_tokens) {
-  EncodeTiledFn enc = get_encode();
-  if (!enc) return false;
   cuuint64_t dims[4] = {(cuuint64_t)HD, (cuuint64_t)heads, (cuuint64_t)tokens, (cuuint64_t)batch};
   // a size-1 dimension may come with stride 0; any positive multiple of 16 bytes is accepted there
   auto st = [](long long e) { return (cuuint64_t)((e > 0 ? e : 8) * 2); };
   cuuint64_t strides[3] = {st(s[2]), st(s[1]), st(s[0])};
   cuuint32_t box[4] = {64u, (cuuint32_t)box_heads, (cuuint32_t)box_tokens, 1u};
-  cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
-  return enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
-             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return encode_bf16_sw128_4d(out, base, dims, strides, box);
 }
 
 }  // namespace
@@ -548,7 +528,7 @@ bool prefill_sm100_supported(const Dims& dm) {
   const int tq = 128 / dm.g_q;
   if (dm.g_q < 2 || tq > MAX_TQ || tq > dm.B) return false;
   if (dm.os[2] % 8 != 0 || dm.os[1] % 8 != 0) return false;
-  return get_encode() != nullptr;
+  return tensor_map_encoder() != nullptr;
 }
 
 cudaError_t launch_attend_prefill_sm100(const Dims& dm, const void* Q, const void* K, const void* V,
@@ -566,12 +546,8 @@ cudaError_t launch_attend_prefill_sm100(const Dims& dm, const void* Q, const voi
   if (!make_map(&tq, Q, dm.seq_q, dm.h_q, dm.batch, dm.qs, dm.g_q, a.TQ)) return cudaErrorInvalidValue;
   if (!make_map(&tk, K, dm.seq_kv, dm.h_kv, dm.batch, dm.ks, 1, NKV)) return cudaErrorInvalidValue;
   if (!make_map(&tv, V, dm.seq_kv, dm.h_kv, dm.batch, dm.vs, 1, NKV)) return cudaErrorInvalidValue;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(attend_prefill_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PF_SMEM);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  static std::atomic<unsigned long long> configured{0};
+  if (cudaError_t e = allow_dynamic_smem(attend_prefill_sm100_kernel, PF_SMEM, configured); e != cudaSuccess) return e;
   const long long blocks = (long long)a.n_tiles * dm.batch * dm.h_kv;
   cudaError_t le = launch_chained(attend_prefill_sm100_kernel, dim3((unsigned)blocks), dim3(PF_THREADS), PF_SMEM, st, tq,
                                   tk, tv, a);

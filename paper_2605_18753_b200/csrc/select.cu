@@ -263,12 +263,8 @@ static cudaError_t launch_one(const Dims& dm, const SelectPlan& pl, int token_ba
                               const int* kv_len, uint32_t* mask, int* count, int* blk_idx, float* blk_bias,
                               float* tau, cudaStream_t st) {
   auto kern = select_kernel<T, D, RPT, CPT>;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SEL_SMEM_BUDGET);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  static std::atomic<unsigned long long> configured{0};
+  if (cudaError_t e = allow_dynamic_smem(kern, SEL_SMEM_BUDGET, configured); e != cudaSuccess) return e;
   const int tiles = dm.decode ? 1 : (dm.seq_q - token_base + pl.TQ - 1) / pl.TQ;
   dim3 grid(tiles, dm.h_kv, dm.batch);
   cudaError_t le = launch_chained(kern, grid, dim3(SEL_THREADS), pl.smem, st, dm, pl.TQ, pl.xs_stride, token_base,

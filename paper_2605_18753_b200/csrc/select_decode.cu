@@ -407,13 +407,9 @@ cudaError_t launch_select_decode(const Dims& dm, const void* Q, const float* Kba
   cudaError_t re = cudaSuccess;
 #define DASH_RT(G)                                                                                                  \
   {                                                                                                                 \
-    static bool configured = false;                                                                                 \
-    if (!configured) {                                                                                              \
-      cudaError_t e = cudaFuncSetAttribute(decode_route_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize,     \
-                                           200 * 1024);                                                             \
-      if (e != cudaSuccess) return e;                                                                               \
-      configured = true;                                                                                            \
-    }                                                                                                               \
+    static std::atomic<unsigned long long> configured{0};                                                           \
+    cudaError_t e = allow_dynamic_smem(decode_route_kernel<G>, 200 * 1024, configured);                             \
+    if (e != cudaSuccess) return e;                                                                                 \
     re = launch_chained(decode_route_kernel<G>, dim3(dm.h_kv, dm.batch), dim3(RT_THREADS), smem, st, dm,           \
                         (const float*)scratch, kv_len, mask, count, blk_idx, blk_bias, tau);                       \
   }

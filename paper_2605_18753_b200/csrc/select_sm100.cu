@@ -22,6 +22,7 @@
 
 #include "common.cuh"
 #include "sm100_ptx.cuh"
+#include "tensor_map.cuh"
 
 namespace dash {
 
@@ -584,32 +585,6 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   if (CS > 1) ptx::cluster_sync_all();     // nobody leaves while a peer may still write into its shared memory
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn get_encode() {
-  static EncodeTiledFn fn = nullptr;
-  if (!fn) {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(p);
-  }
-  return fn;
-}
-
-bool encode4(CUtensorMap* out, const void* base, const cuuint64_t* dims, const cuuint64_t* strides_bytes,
-             const cuuint32_t* box) {
-  EncodeTiledFn enc = get_encode();
-  if (!enc) return false;
-  cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
-  return enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides_bytes, box, estr,
-             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 }  // namespace
 
 // Tokens [0, select_sm100_token_limit) can be routed by the tensor-core kernel (0: not applicable).  A block
@@ -618,7 +593,7 @@ int select_sm100_token_limit(const Dims& dm) {
   if (dm.decode || !dm.causal || dm.dtype != DASH_BF16 || dm.d != HD || dm.T_s < 1) return 0;
   const int tq = 128 / dm.g_q;
   if (dm.g_q < 2 || tq > dm.B) return 0;
-  if (get_encode() == nullptr) return 0;
+  if (tensor_map_encoder() == nullptr) return 0;
   const long long lim = (long long)(4 * CLUSTER_COLS + 1) * dm.B;   // own chunk index <= 2048
   return (int)(lim < dm.seq_q ? lim : dm.seq_q);
 }
@@ -631,12 +606,8 @@ template <int NST, int G, int CS>
 static cudaError_t launch_band(const CUtensorMap& tq, const CUtensorMap& tkb, const SelectTcArgs& a, long long clusters,
                                cudaStream_t st) {
   auto kern = select_sm100_kernel<NST, G, CS>;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemPlan<NST>::TOTAL);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  static std::atomic<unsigned long long> configured{0};
+  if (cudaError_t e = allow_dynamic_smem(kern, SmemPlan<NST>::TOTAL, configured); e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(clusters * CS));
   cfg.blockDim = dim3(SEL_TC_THREADS);
@@ -721,13 +692,13 @@ cudaError_t launch_select_sm100(const Dims& dm, int token_limit, const void* Q, 
     auto sb2 = [](long long el) { return (cuuint64_t)((el > 0 ? el : 8) * 2); };
     cuuint64_t strides[3] = {sb2(dm.qs[2]), sb2(dm.qs[1]), sb2(dm.qs[0])};
     cuuint32_t box[4] = {64u, (cuuint32_t)dm.g_q, (cuuint32_t)a.TQ, 1u};
-    if (!encode4(&tq, Q, dims, strides, box)) return cudaErrorInvalidValue;
+    if (!encode_bf16_sw128_4d(&tq, Q, dims, strides, box)) return cudaErrorInvalidValue;
   }
   {
     cuuint64_t dims[4] = {(cuuint64_t)HD, (cuuint64_t)(3 * plane_rows), 1, 1};
     cuuint64_t strides[3] = {(cuuint64_t)HD * 2, (cuuint64_t)(3 * plane_rows) * HD * 2, (cuuint64_t)(3 * plane_rows) * HD * 2};
     cuuint32_t box[4] = {64u, (cuuint32_t)SC, 1u, 1u};
-    if (!encode4(&tkb, planes, dims, strides, box)) return cudaErrorInvalidValue;
+    if (!encode_bf16_sw128_4d(&tkb, planes, dims, strides, box)) return cudaErrorInvalidValue;
   }
   // Bands of tiles by candidate count: <= 512 one block per tile, <= 1024 clusters of 2, <= 2048 clusters of 4.
   // Tiles are TQ tokens; a tile's candidate count is its own chunk index i0 / B.
