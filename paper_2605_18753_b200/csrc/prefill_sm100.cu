@@ -62,6 +62,13 @@ constexpr uint32_t PF_SMEM = OFF_MISC + sizeof(Misc);
 static_assert(PF_SMEM <= 115712, "two blocks per SM need <= 113 KiB each");
 
 
+// max of three in one instruction
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
 struct PrefillArgs {
   Dims dm;
   int TQ;            // tokens per tile
@@ -411,13 +418,17 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
           for (int c = 0; c < NKV; ++c)
             if (c >= n_vis) sreg[c] = 0xff800000u;   // -inf
         }
+        // three-input maxima: 32 instructions for the 64 scores, in eight independent chains, then a tree
+        float ch[8];
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {   // eight independent chains, then a tree
-          float a = __uint_as_float(sreg[c]);
+        for (int c = 0; c < 8; ++c) ch[c] = __uint_as_float(sreg[c]);
 #pragma unroll
-          for (int k = 8; k < NKV; k += 8) a = fmaxf(a, __uint_as_float(sreg[c + k]));
-          mr = fmaxf(mr, a);
-        }
+        for (int k = 8; k + 16 <= NKV; k += 16)
+#pragma unroll
+          for (int c = 0; c < 8; ++c) ch[c] = max3(ch[c], __uint_as_float(sreg[c + k]), __uint_as_float(sreg[c + k + 8]));
+#pragma unroll
+        for (int c = 0; c < 8; ++c) ch[c] = fmaxf(ch[c], __uint_as_float(sreg[c + NKV - 8]));
+        mr = fmaxf(max3(ch[0], ch[1], ch[2]), fmaxf(max3(ch[3], ch[4], ch[5]), fmaxf(ch[6], ch[7])));
       }
       const float mloc = fmaf(mr, c1, b2);           // -inf when not selected
       float corr = 1.f;
@@ -431,16 +442,19 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
       uint32_t packed[32];
       if (selected) {
         const float off = b2 - m_used;
-        float lsum[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        // scale-and-shift and the row sum on packed pairs (one instruction per two scores)
+        const float2 c1v = make_float2(c1, c1), offv = make_float2(off, off);
+        float2 lsum[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
 #pragma unroll
         for (int c = 0; c < NKV; c += 2) {
-          const float p0 = exp2f(fmaf(__uint_as_float(sreg[c]), c1, off));
-          const float p1 = exp2f(fmaf(__uint_as_float(sreg[c + 1]), c1, off));
-          lsum[(c >> 1) & 7] += p0 + p1;
-          __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
+          const float2 t = __ffma2_rn(make_float2(__uint_as_float(sreg[c]), __uint_as_float(sreg[c + 1])), c1v, offv);
+          const float2 pp = make_float2(exp2f(t.x), exp2f(t.y));
+          lsum[(c >> 1) & 3] = __fadd2_rn(lsum[(c >> 1) & 3], pp);
+          __nv_bfloat162 h = __floats2bfloat162_rn(pp.x, pp.y);
           packed[c >> 1] = *reinterpret_cast<uint32_t*>(&h);
         }
-        l += ((lsum[0] + lsum[1]) + (lsum[2] + lsum[3])) + ((lsum[4] + lsum[5]) + (lsum[6] + lsum[7]));
+        const float2 ls = __fadd2_rn(__fadd2_rn(lsum[0], lsum[1]), __fadd2_rn(lsum[2], lsum[3]));
+        l += ls.x + ls.y;
       } else {
 #pragma unroll
         for (int c = 0; c < 32; ++c) packed[c] = 0u;
