@@ -238,7 +238,7 @@ def _fwd_prefill_case(w, rows, kv_heads=None, min_clean=0.9, local_blocks=0):
             border = set(int(c) for c in np.nonzero(np.abs(ro.margin) <= H.BORDERLINE)[0])
             assert diff <= border, (b, r, i, sorted(diff))
             n_excluded += 1
-    assert len(keys) >= min_clean * len(ora), (len(keys), len(ora), n_excluded)
+    assert len(keys) >= min_clean * len(ora), f"too few clean rows: {len(keys)} of {len(ora)} ({n_excluded} excluded)"
     want = np.stack([ora[k][1] for k in keys])
     return H.check_outputs(_gather_O(O, keys, w.h_q // w.h_kv), want, Q.dtype, f"fwd_prefill {w.name}")
 
@@ -295,7 +295,7 @@ def _decode_case(w, kv_len, use_lists_from_oracle=False, local_blocks=0):
     got = O.float().cpu().double().numpy()
     g_q = w.h_q // w.h_kv
     sel = np.repeat(clean, g_q, axis=1)
-    assert sel.any() and (sel.mean() >= 0.8 or sel.size < 64)
+    assert sel.any() and (sel.mean() >= 0.8 or sel.size < 64), "too few clean groups"
     H.check_outputs(got[sel], ora["O"][sel], Q.dtype, "fwd_decode")
 
 
