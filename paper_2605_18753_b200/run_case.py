@@ -24,6 +24,7 @@ def main() -> None:
     ap.add_argument("--block", type=int)
     ap.add_argument("--alpha", type=float)
     ap.add_argument("--local-blocks", type=int, default=0, help="window chunks before the own chunk (0 = none)")
+    ap.add_argument("--graph", action="store_true", help="record the forward pass into a CUDA graph and time its replays")
     ap.add_argument("--kv-layout", choices=("token_major", "head_major"), default="token_major",
                     help="memory order of K and V: [b, n, h_kv, d] (default) or [b, h_kv, n, d] behind the same strided view")
     args = ap.parse_args()
@@ -55,6 +56,14 @@ def main() -> None:
         B.dash_attn_block_summaries(p, Kc, kbar, kv_len=kl)
         ws = B.alloc_workspace(p)
         step = lambda: B.dash_attn_fwd_decode(p, q, Kc, Vc, kbar, kl, O, ws)
+
+    if args.graph:
+        step()                                   # first use outside the capture
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            step()
+        step = graph.replay
 
     times = []
     for it in range(args.iters + 1):
