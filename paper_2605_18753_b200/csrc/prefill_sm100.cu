@@ -34,16 +34,9 @@ constexpr int NKV = 64;           // KV tokens per step
 constexpr int KST = 2, VST = 2;   // ring depths: stage = step parity, like the S/P buffers, so that the two
                                   // MMA completion barriers of a step also release its K and V stages
 constexpr int PF_THREADS = 224;   // 4 softmax warps, K producer, MMA issuer, V/bias producer
-constexpr int HD = 128;           // head_dim
 constexpr uint32_t TMEM_COLS = 256;  // S0 [0,64), S1 [64,128), O [128,256)
 constexpr float RESCALE_LOG2 = 8.f;  // the running maximum is moved only when it grew by more than this
 
-constexpr uint32_t Q_BYTES = 128 * HD * 2;           // 32 KiB: two 128x64 K-major regions
-constexpr uint32_t KV_TILE_BYTES = NKV * HD * 2;     // 16 KiB: two 64x64 regions
-constexpr uint32_t OFF_Q = 0;
-constexpr uint32_t OFF_K = OFF_Q + Q_BYTES;
-constexpr uint32_t OFF_V = OFF_K + KST * KV_TILE_BYTES;
-constexpr uint32_t OFF_MISC = OFF_V + VST * KV_TILE_BYTES;
 constexpr int MAX_TQ = 64;
 // S_FULL[j&1]: QK of step j complete (S readable; K stage j&1 reusable).  PV_DONE[j&1]: PV of step j complete (O stable;
 // S/P buffer and V stage j&1 reusable).  Every tcgen05.commit and every barrier test costs the issuing thread as
@@ -58,8 +51,19 @@ struct Misc {
   int kvbase[VST];
   float bias[VST][MAX_TQ];
 };
-constexpr uint32_t PF_SMEM = OFF_MISC + sizeof(Misc);
-static_assert(PF_SMEM <= 115712, "two blocks per SM need <= 113 KiB each");
+// Shared-memory layout for head_dim HD (64 or 128): tiles are K-major regions of 64 elements (128 bytes, the
+// swizzle span) per row, one region per 64 of head_dim.
+template <int HD>
+struct PfLayout {
+  static constexpr uint32_t Q_BYTES = 128 * HD * 2;           // HD = 128: 32 KiB, two 128x64 regions
+  static constexpr uint32_t KV_TILE_BYTES = NKV * HD * 2;     // HD = 128: 16 KiB, two 64x64 regions
+  static constexpr uint32_t OFF_Q = 0;
+  static constexpr uint32_t OFF_K = OFF_Q + Q_BYTES;
+  static constexpr uint32_t OFF_V = OFF_K + KST * KV_TILE_BYTES;
+  static constexpr uint32_t OFF_MISC = OFF_V + VST * KV_TILE_BYTES;
+  static constexpr uint32_t SMEM = OFF_MISC + sizeof(Misc);
+  static_assert(SMEM <= 115712, "two blocks per SM need <= 113 KiB each");
+};
 
 
 // max of three in one instruction
@@ -79,9 +83,13 @@ struct PrefillArgs {
   StatusBlock* sb;
 };
 
+template <int HD>
 __global__ void __launch_bounds__(PF_THREADS, 2)
 attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                             const __grid_constant__ CUtensorMap tmV, PrefillArgs a) {
+  using LY = PfLayout<HD>;
+  constexpr uint32_t Q_BYTES = LY::Q_BYTES, KV_TILE_BYTES = LY::KV_TILE_BYTES, OFF_Q = LY::OFF_Q, OFF_K = LY::OFF_K,
+                     OFF_V = LY::OFF_V, OFF_MISC = LY::OFF_MISC;
   extern __shared__ __align__(1024) uint8_t smem[];
   Misc* misc = reinterpret_cast<Misc*>(smem + OFF_MISC);
   const Dims& dm = a.dm;
@@ -148,7 +156,7 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
       ptx::prefetch_tensormap(&tmV);
       ptx::mbar_arrive_expect_tx(bar(Q_FULL), Q_BYTES);
       ptx::tma_load_4d(sbase + OFF_Q, &tmQ, bar(Q_FULL), 0, r * g_q, i0, b);
-      ptx::tma_load_4d(sbase + OFF_Q + Q_BYTES / 2, &tmQ, bar(Q_FULL), 64, r * g_q, i0, b);
+      if constexpr (HD == 128) ptx::tma_load_4d(sbase + OFF_Q + Q_BYTES / 2, &tmQ, bar(Q_FULL), 64, r * g_q, i0, b);
     }
     // The own chunk goes first: its tiles need nothing from the mask, so they are in flight (and the first
     // S = Q K^T can run) while the union of the routed chunks is still being formed.  Stages 0/1 are free.
@@ -159,7 +167,7 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
           const uint32_t dst = sbase + OFF_K + sub * KV_TILE_BYTES;
           ptx::mbar_arrive_expect_tx(bar(K_FULL + sub), KV_TILE_BYTES);
           ptx::tma_load_4d(dst, &tmK, bar(K_FULL + sub), 0, r, kv0, b);
-          ptx::tma_load_4d(dst + KV_TILE_BYTES / 2, &tmK, bar(K_FULL + sub), 64, r, kv0, b);
+          if constexpr (HD == 128) ptx::tma_load_4d(dst + KV_TILE_BYTES / 2, &tmK, bar(K_FULL + sub), 64, r, kv0, b);
         }
       } else {
         for (int t = lane; t < TQ; t += 32) misc->bias[sub][t] = 0.f;
@@ -169,7 +177,7 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
           const uint32_t dst = sbase + OFF_V + sub * KV_TILE_BYTES;
           ptx::mbar_arrive_expect_tx(bar(V_FULL + sub), KV_TILE_BYTES);
           ptx::tma_load_4d(dst, &tmV, bar(V_FULL + sub), 0, r, kv0, b);
-          ptx::tma_load_4d(dst + KV_TILE_BYTES / 2, &tmV, bar(V_FULL + sub), 64, r, kv0, b);
+          if constexpr (HD == 128) ptx::tma_load_4d(dst + KV_TILE_BYTES / 2, &tmV, bar(V_FULL + sub), 64, r, kv0, b);
         }
       }
     }
@@ -290,7 +298,7 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
             const uint32_t dst = sbase + OFF_K + st * KV_TILE_BYTES;
             ptx::mbar_arrive_expect_tx(bar(K_FULL + st), KV_TILE_BYTES);
             ptx::tma_load_4d(dst, &tmK, bar(K_FULL + st), 0, r, kv0, b);
-            ptx::tma_load_4d(dst + KV_TILE_BYTES / 2, &tmK, bar(K_FULL + st), 64, r, kv0, b);
+            if constexpr (HD == 128) ptx::tma_load_4d(dst + KV_TILE_BYTES / 2, &tmK, bar(K_FULL + st), 64, r, kv0, b);
           }
           continue;
         }
@@ -307,7 +315,7 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
           const uint32_t dst = sbase + OFF_V + vs * KV_TILE_BYTES;
           ptx::mbar_arrive_expect_tx(bar(V_FULL + vs), KV_TILE_BYTES);
           ptx::tma_load_4d(dst, &tmV, bar(V_FULL + vs), 0, r, kv0, b);
-          ptx::tma_load_4d(dst + KV_TILE_BYTES / 2, &tmV, bar(V_FULL + vs), 64, r, kv0, b);
+          if constexpr (HD == 128) ptx::tma_load_4d(dst + KV_TILE_BYTES / 2, &tmV, bar(V_FULL + vs), 64, r, kv0, b);
         }
       }
     }
@@ -524,9 +532,9 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
 // ---------------------------------------------------------------- host side
 
 // [batch, tokens, heads, 128] bf16 tensor with element strides s[3]; box = 64 x box_heads x box_tokens x 1.
-bool make_map(CUtensorMap* out, const void* base, long long tokens, int heads, int batch, const long long* s,
+bool make_map(CUtensorMap* out, const void* base, int hd, long long tokens, int heads, int batch, const long long* s,
               int box_heads, int box_tokens) {
-  cuuint64_t dims[4] = {(cuuint64_t)HD, (cuuint64_t)heads, (cuuint64_t)tokens, (cuuint64_t)batch};
+  cuuint64_t dims[4] = {(cuuint64_t)hd, (cuuint64_t)heads, (cuuint64_t)tokens, (cuuint64_t)batch};
   // a size-1 dimension may come with stride 0; any positive multiple of 16 bytes is accepted there
   auto st = [](long long e) { return (cuuint64_t)((e > 0 ? e : 8) * 2); };
   cuuint64_t strides[3] = {st(s[2]), st(s[1]), st(s[0])};
@@ -537,7 +545,7 @@ bool make_map(CUtensorMap* out, const void* base, long long tokens, int heads, i
 }  // namespace
 
 bool prefill_sm100_supported(const Dims& dm) {
-  if (dm.decode || !dm.causal || dm.dtype != DASH_BF16 || dm.d != HD) return false;
+  if (dm.decode || !dm.causal || dm.dtype != DASH_BF16 || (dm.d != 64 && dm.d != 128)) return false;
   if (dm.B != 64 && dm.B != 128) return false;
   const int tq = 128 / dm.g_q;
   if (dm.g_q < 2 || tq > MAX_TQ || tq > dm.B) return false;
@@ -557,14 +565,22 @@ cudaError_t launch_attend_prefill_sm100(const Dims& dm, const void* Q, const voi
   a.O = (__nv_bfloat16*)O;
   a.sb = sb;
   CUtensorMap tq, tk, tv;
-  if (!make_map(&tq, Q, dm.seq_q, dm.h_q, dm.batch, dm.qs, dm.g_q, a.TQ)) return cudaErrorInvalidValue;
-  if (!make_map(&tk, K, dm.seq_kv, dm.h_kv, dm.batch, dm.ks, 1, NKV)) return cudaErrorInvalidValue;
-  if (!make_map(&tv, V, dm.seq_kv, dm.h_kv, dm.batch, dm.vs, 1, NKV)) return cudaErrorInvalidValue;
-  static std::atomic<unsigned long long> configured{0};
-  if (cudaError_t e = allow_dynamic_smem(attend_prefill_sm100_kernel, PF_SMEM, configured); e != cudaSuccess) return e;
+  if (!make_map(&tq, Q, dm.d, dm.seq_q, dm.h_q, dm.batch, dm.qs, dm.g_q, a.TQ)) return cudaErrorInvalidValue;
+  if (!make_map(&tk, K, dm.d, dm.seq_kv, dm.h_kv, dm.batch, dm.ks, 1, NKV)) return cudaErrorInvalidValue;
+  if (!make_map(&tv, V, dm.d, dm.seq_kv, dm.h_kv, dm.batch, dm.vs, 1, NKV)) return cudaErrorInvalidValue;
   const long long blocks = (long long)a.n_tiles * dm.batch * dm.h_kv;
-  cudaError_t le = launch_chained(attend_prefill_sm100_kernel, dim3((unsigned)blocks), dim3(PF_THREADS), PF_SMEM, st, tq,
-                                  tk, tv, a);
+  cudaError_t le = cudaSuccess;
+  if (dm.d == 128) {
+    static std::atomic<unsigned long long> configured{0};
+    if (cudaError_t e = allow_dynamic_smem(attend_prefill_sm100_kernel<128>, PfLayout<128>::SMEM, configured); e != cudaSuccess) return e;
+    le = launch_chained(attend_prefill_sm100_kernel<128>, dim3((unsigned)blocks), dim3(PF_THREADS), PfLayout<128>::SMEM,
+                        st, tq, tk, tv, a);
+  } else {
+    static std::atomic<unsigned long long> configured{0};
+    if (cudaError_t e = allow_dynamic_smem(attend_prefill_sm100_kernel<64>, PfLayout<64>::SMEM, configured); e != cudaSuccess) return e;
+    le = launch_chained(attend_prefill_sm100_kernel<64>, dim3((unsigned)blocks), dim3(PF_THREADS), PfLayout<64>::SMEM, st,
+                        tq, tk, tv, a);
+  }
   count_launch();
   return le;
 }

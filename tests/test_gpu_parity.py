@@ -199,6 +199,8 @@ def test_fwd_prefill_tiny_fp32(name, sigmas):
     dict(seq=1111, h_q=2, h_kv=2, head_dim=128, block=64, seed=2),
     dict(seq=1300, h_q=16, h_kv=2, head_dim=128, block=64, seed=3),          # g_q = 8 on the tensor-core paths
     dict(seq=900, h_q=4, h_kv=2, head_dim=128, block=128, seed=4),           # g_q = 2, chunks of 128
+    dict(seq=1500, h_q=8, h_kv=2, head_dim=64, block=64, seed=6),            # head_dim 64 on the tensor-core kernels
+    dict(seq=1100, h_q=16, h_kv=1, head_dim=64, block=128, seed=7, alpha=2.0),
 ])
 def test_fwd_prefill_small(kw):
     w = _wl(**kw)
