@@ -29,10 +29,10 @@ namespace dash {
 namespace {
 
 constexpr int SC = 64;               // candidate chunks per MMA block / staged summary tile
-constexpr int HD = 128;
+constexpr int HD_MAX = 128;          // the shared-memory layout is the one of head_dim 128; head_dim 64 fills half of each tile
 constexpr int SEL_TC_THREADS = 192;
-constexpr uint32_t Q_BYTES = 128 * HD * 2;            // 32 KiB
-constexpr uint32_t PLANE_BYTES = SC * HD * 2;         // 16 KiB per plane per stage
+constexpr uint32_t Q_BYTES = 128 * HD_MAX * 2;        // 32 KiB
+constexpr uint32_t PLANE_BYTES = SC * HD_MAX * 2;     // 16 KiB per plane per stage
 constexpr uint32_t STAGE_BYTES = 3 * PLANE_BYTES;     // hi, mid, lo
 constexpr int XCH_STRIDE = 33;
 constexpr uint32_t XCH_BYTES = 128 * XCH_STRIDE * 4;
@@ -82,7 +82,7 @@ __global__ void kbar_split_kernel(const float* __restrict__ kbar, __nv_bfloat16*
   planes[2 * n + i] = __float2bfloat16_rn(r2);
 }
 
-template <int NST, int G, int CS>
+template <int NST, int G, int CS, int HD>
 __global__ void __launch_bounds__(SEL_TC_THREADS, NST == 1 ? 2 : 1)
 select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKB, SelectTcArgs a) {
   using SP = SmemPlan<NST>;
@@ -150,21 +150,21 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     if (lane == 0 && n_loc > 0) {
       ptx::prefetch_tensormap(&tmQ);
       ptx::prefetch_tensormap(&tmKB);
-      ptx::mbar_arrive_expect_tx(bar(Q_FULL), Q_BYTES);
+      ptx::mbar_arrive_expect_tx(bar(Q_FULL), 128 * HD * 2);
       ptx::tma_load_4d(sbase + SP::OFF_Q, &tmQ, bar(Q_FULL), 0, r * g_q, i0, b);
-      ptx::tma_load_4d(sbase + SP::OFF_Q + Q_BYTES / 2, &tmQ, bar(Q_FULL), 64, r * g_q, i0, b);
+      if constexpr (HD == 128) ptx::tma_load_4d(sbase + SP::OFF_Q + Q_BYTES / 2, &tmQ, bar(Q_FULL), 64, r * g_q, i0, b);
       const long long row0 = ((long long)b * dm.h_kv + r) * dm.T_s + c_lo;
       bool ok = true;
       for (int cb = 0; cb < n_blk && ok; ++cb) {
         const int s = cb % NST;
         ok = ptx::mbar_wait(bar(KB_EMPTY + s), ((cb / NST) & 1) ^ 1, abort_flag);
         if (!ok) break;
-        ptx::mbar_arrive_expect_tx(bar(KB_FULL + s), STAGE_BYTES);
+        ptx::mbar_arrive_expect_tx(bar(KB_FULL + s), 3 * SC * HD * 2);
         for (int pl = 0; pl < 3; ++pl) {
           const uint32_t dst = sbase + SP::OFF_KB + s * STAGE_BYTES + pl * PLANE_BYTES;
           const int row = (int)(pl * a.plane_rows + row0 + (long long)cb * SC);
           ptx::tma_load_4d(dst, &tmKB, bar(KB_FULL + s), 0, row, 0, 0);
-          ptx::tma_load_4d(dst + PLANE_BYTES / 2, &tmKB, bar(KB_FULL + s), 64, row, 0, 0);
+          if constexpr (HD == 128) ptx::tma_load_4d(dst + PLANE_BYTES / 2, &tmKB, bar(KB_FULL + s), 64, row, 0, 0);
         }
       }
       if (!ok) {
@@ -590,7 +590,7 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 // Tokens [0, select_sm100_token_limit) can be routed by the tensor-core kernel (0: not applicable).  A block
 // holds 512 candidates per row in tensor memory; clusters of 2 or 4 blocks extend that to 1024 / 2048.
 int select_sm100_token_limit(const Dims& dm) {
-  if (dm.decode || !dm.causal || dm.dtype != DASH_BF16 || dm.d != HD || dm.T_s < 1) return 0;
+  if (dm.decode || !dm.causal || dm.dtype != DASH_BF16 || (dm.d != 64 && dm.d != 128) || dm.T_s < 1) return 0;
   const int tq = 128 / dm.g_q;
   if (dm.g_q < 2 || tq > dm.B) return 0;
   if (tensor_map_encoder() == nullptr) return 0;
@@ -602,10 +602,10 @@ size_t select_sm100_scratch_bytes(const Dims& dm) {
   return (size_t)3 * dm.batch * dm.h_kv * (size_t)(dm.T_s > 0 ? dm.T_s : 1) * dm.d * sizeof(__nv_bfloat16);
 }
 
-template <int NST, int G, int CS>
+template <int NST, int G, int CS, int HD>
 static cudaError_t launch_band(const CUtensorMap& tq, const CUtensorMap& tkb, const SelectTcArgs& a, long long clusters,
                                cudaStream_t st) {
-  auto kern = select_sm100_kernel<NST, G, CS>;
+  auto kern = select_sm100_kernel<NST, G, CS, HD>;
   static std::atomic<unsigned long long> configured{0};
   if (cudaError_t e = allow_dynamic_smem(kern, SmemPlan<NST>::TOTAL, configured); e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
@@ -630,11 +630,20 @@ static cudaError_t launch_band(const CUtensorMap& tq, const CUtensorMap& tkb, co
 template <int NST, int CS>
 static cudaError_t launch_band_g(const Dims& dm, const CUtensorMap& tq, const CUtensorMap& tkb, const SelectTcArgs& a,
                                  long long clusters, cudaStream_t st) {
+  if (dm.d == 64) {
+    switch (dm.g_q) {
+      case 2: return launch_band<NST, 2, CS, 64>(tq, tkb, a, clusters, st);
+      case 4: return launch_band<NST, 4, CS, 64>(tq, tkb, a, clusters, st);
+      case 8: return launch_band<NST, 8, CS, 64>(tq, tkb, a, clusters, st);
+      case 16: return launch_band<NST, 16, CS, 64>(tq, tkb, a, clusters, st);
+      default: return cudaErrorInvalidValue;
+    }
+  }
   switch (dm.g_q) {
-    case 2: return launch_band<NST, 2, CS>(tq, tkb, a, clusters, st);
-    case 4: return launch_band<NST, 4, CS>(tq, tkb, a, clusters, st);
-    case 8: return launch_band<NST, 8, CS>(tq, tkb, a, clusters, st);
-    case 16: return launch_band<NST, 16, CS>(tq, tkb, a, clusters, st);
+    case 2: return launch_band<NST, 2, CS, 128>(tq, tkb, a, clusters, st);
+    case 4: return launch_band<NST, 4, CS, 128>(tq, tkb, a, clusters, st);
+    case 8: return launch_band<NST, 8, CS, 128>(tq, tkb, a, clusters, st);
+    case 16: return launch_band<NST, 16, CS, 128>(tq, tkb, a, clusters, st);
     default: return cudaErrorInvalidValue;
   }
 }
@@ -688,15 +697,16 @@ cudaError_t launch_select_sm100(const Dims& dm, int token_limit, const void* Q, 
 
   CUtensorMap tq, tkb;
   {
-    cuuint64_t dims[4] = {(cuuint64_t)HD, (cuuint64_t)dm.h_q, (cuuint64_t)dm.seq_q, (cuuint64_t)dm.batch};
+    cuuint64_t dims[4] = {(cuuint64_t)dm.d, (cuuint64_t)dm.h_q, (cuuint64_t)dm.seq_q, (cuuint64_t)dm.batch};
     auto sb2 = [](long long el) { return (cuuint64_t)((el > 0 ? el : 8) * 2); };
     cuuint64_t strides[3] = {sb2(dm.qs[2]), sb2(dm.qs[1]), sb2(dm.qs[0])};
     cuuint32_t box[4] = {64u, (cuuint32_t)dm.g_q, (cuuint32_t)a.TQ, 1u};
     if (!encode_bf16_sw128_4d(&tq, Q, dims, strides, box)) return cudaErrorInvalidValue;
   }
   {
-    cuuint64_t dims[4] = {(cuuint64_t)HD, (cuuint64_t)(3 * plane_rows), 1, 1};
-    cuuint64_t strides[3] = {(cuuint64_t)HD * 2, (cuuint64_t)(3 * plane_rows) * HD * 2, (cuuint64_t)(3 * plane_rows) * HD * 2};
+    const cuuint64_t hd = (cuuint64_t)dm.d;
+    cuuint64_t dims[4] = {hd, (cuuint64_t)(3 * plane_rows), 1, 1};
+    cuuint64_t strides[3] = {hd * 2, (cuuint64_t)(3 * plane_rows) * hd * 2, (cuuint64_t)(3 * plane_rows) * hd * 2};
     cuuint32_t box[4] = {64u, (cuuint32_t)SC, 1u, 1u};
     if (!encode_bf16_sw128_4d(&tkb, planes, dims, strides, box)) return cudaErrorInvalidValue;
   }

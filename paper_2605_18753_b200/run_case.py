@@ -3,7 +3,7 @@
     python -m paper_2605_18753_b200.run_case prefill_8k --iters 5
     python -m paper_2605_18753_b200.run_case decode_128k --batch 4 --iters 3      # 2 GiB of KV cache instead of 8
 
-A quick way to see the path work on a given shape (overrides: --batch, --seq, --block, --alpha, --local-blocks), and a small,
+A quick way to see the path work on a given shape (overrides: --batch, --seq, --block, --alpha, --head-dim, --local-blocks), and a small,
 self-terminating command to put under a profiler.  Inputs are the seeded synthetic tensors of `synth`."""
 from __future__ import annotations
 
@@ -23,12 +23,13 @@ def main() -> None:
     ap.add_argument("--seq", type=int)
     ap.add_argument("--block", type=int)
     ap.add_argument("--alpha", type=float)
+    ap.add_argument("--head-dim", type=int, dest="head_dim")
     ap.add_argument("--local-blocks", type=int, default=0, help="window chunks before the own chunk (0 = none)")
     ap.add_argument("--graph", action="store_true", help="record the forward pass into a CUDA graph and time its replays")
     ap.add_argument("--kv-layout", choices=("token_major", "head_major"), default="token_major",
                     help="memory order of K and V: [b, n, h_kv, d] (default) or [b, h_kv, n, d] behind the same strided view")
     args = ap.parse_args()
-    over = {k: getattr(args, k) for k in ("batch", "seq", "block", "alpha") if getattr(args, k) is not None}
+    over = {k: getattr(args, k) for k in ("batch", "seq", "block", "alpha", "head_dim") if getattr(args, k) is not None}
     w = synth.workload(args.workload, **over)
     dev = "cuda"
 
