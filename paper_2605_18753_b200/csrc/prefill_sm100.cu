@@ -43,17 +43,20 @@ constexpr int MAX_TQ = 64;
 // much as an MMA, so each product signals exactly one barrier and the producers listen to the same ones.
 enum Bar { Q_FULL = 0, META, S_FULL = 2, PV_DONE = 4, P_FULL = 6, V_FULL = 8, K_FULL = 10, N_BARS = 12 };
 static_assert(KST == 2 && VST == 2, "stage = step parity");
-struct Misc {
+// CPS = chunks per 64-token step: 1 for chunks of 64 or 128 tokens, 2 / 4 for chunks of 32 / 16 (a step then
+// packs that many chunks of the union list, each with its own per-token bias).
+template <int CPS>
+struct MiscT {
   unsigned long long bar[N_BARS];
   uint32_t tmem_base;
   int n_steps;
   int abort_flag;
-  int kvbase[VST];
-  float bias[VST][MAX_TQ];
+  int kvbase[VST][CPS];
+  float bias[VST][CPS][MAX_TQ];
 };
 // Shared-memory layout for head_dim HD (64 or 128): tiles are K-major regions of 64 elements (128 bytes, the
 // swizzle span) per row, one region per 64 of head_dim.
-template <int HD>
+template <int HD, int CPS>
 struct PfLayout {
   static constexpr uint32_t Q_BYTES = 128 * HD * 2;           // HD = 128: 32 KiB, two 128x64 regions
   static constexpr uint32_t KV_TILE_BYTES = NKV * HD * 2;     // HD = 128: 16 KiB, two 64x64 regions
@@ -61,7 +64,7 @@ struct PfLayout {
   static constexpr uint32_t OFF_K = OFF_Q + Q_BYTES;
   static constexpr uint32_t OFF_V = OFF_K + KST * KV_TILE_BYTES;
   static constexpr uint32_t OFF_MISC = OFF_V + VST * KV_TILE_BYTES;
-  static constexpr uint32_t SMEM = OFF_MISC + sizeof(Misc);
+  static constexpr uint32_t SMEM = OFF_MISC + sizeof(MiscT<CPS>);
   static_assert(SMEM <= 115712, "two blocks per SM need <= 113 KiB each");
 };
 
@@ -83,11 +86,12 @@ struct PrefillArgs {
   StatusBlock* sb;
 };
 
-template <int HD>
+template <int HD, int CPS>
 __global__ void __launch_bounds__(PF_THREADS, 2)
 attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                             const __grid_constant__ CUtensorMap tmV, PrefillArgs a) {
-  using LY = PfLayout<HD>;
+  using LY = PfLayout<HD, CPS>;
+  using Misc = MiscT<CPS>;
   constexpr uint32_t Q_BYTES = LY::Q_BYTES, KV_TILE_BYTES = LY::KV_TILE_BYTES, OFF_Q = LY::OFF_Q, OFF_K = LY::OFF_K,
                      OFF_V = LY::OFF_V, OFF_MISC = LY::OFF_MISC;
   extern __shared__ __align__(1024) uint8_t smem[];
@@ -160,8 +164,37 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
     }
     // The own chunk goes first: its tiles need nothing from the mask, so they are in flight (and the first
     // S = Q K^T can run) while the union of the routed chunks is still being formed.  Stages 0/1 are free.
+    // A step's K or V tile for chunks smaller than the step: CPS boxes of NKV / CPS tokens, one per packed chunk.
+    [[maybe_unused]] auto load_packed = [&](const CUtensorMap* tm, uint32_t dst, uint32_t barrier, const int* kvs) {
+      ptx::mbar_arrive_expect_tx(barrier, KV_TILE_BYTES);
+#pragma unroll
+      for (int s = 0; s < CPS; ++s) {
+        const uint32_t d = dst + s * (NKV / CPS) * 128;
+        ptx::tma_load_4d(d, tm, barrier, 0, r, kvs[s], b);
+        if constexpr (HD == 128) ptx::tma_load_4d(d + KV_TILE_BYTES / 2, tm, barrier, 64, r, kvs[s], b);
+      }
+    };
     for (int sub = 0; sub < own_steps; ++sub) {
       const int kv0 = c_own * dm.B + sub * NKV;
+      if constexpr (CPS > 1) {
+        // the own chunk fills the first slot of step 0; the other slots repeat it with bias -inf (probability 0)
+        int kvs[CPS];
+#pragma unroll
+        for (int s = 0; s < CPS; ++s) kvs[s] = kv0;
+        if (do_k) {
+          if (lane == 0) load_packed(&tmK, sbase + OFF_K, bar(K_FULL), kvs);
+        } else {
+          for (int t = lane; t < TQ; t += 32) {
+            misc->bias[0][0][t] = 0.f;
+#pragma unroll
+            for (int s = 1; s < CPS; ++s) misc->bias[0][s][t] = -INFINITY;
+          }
+          if (lane < CPS) misc->kvbase[0][lane] = kv0;
+          __syncwarp();
+          if (lane == 0) load_packed(&tmV, sbase + OFF_V, bar(V_FULL), kvs);
+        }
+        continue;
+      }
       if (do_k) {
         if (lane == 0) {
           const uint32_t dst = sbase + OFF_K + sub * KV_TILE_BYTES;
@@ -170,8 +203,8 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
           if constexpr (HD == 128) ptx::tma_load_4d(dst + KV_TILE_BYTES / 2, &tmK, bar(K_FULL + sub), 64, r, kv0, b);
         }
       } else {
-        for (int t = lane; t < TQ; t += 32) misc->bias[sub][t] = 0.f;
-        if (lane == 0) misc->kvbase[sub] = kv0;
+        for (int t = lane; t < TQ; t += 32) misc->bias[sub][0][t] = 0.f;
+        if (lane == 0) misc->kvbase[sub][0] = kv0;
         __syncwarp();
         if (lane == 0) {
           const uint32_t dst = sbase + OFF_V + sub * KV_TILE_BYTES;
@@ -195,7 +228,7 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
       total += __popc(u);
     }
     // the own chunk is always in the union (its bit is set in every row); it contributes own_steps steps
-    const int n_steps = (total - 1) * sub_per_blk + own_steps;
+    const int n_steps = CPS > 1 ? (total - 1 + CPS - 1) / CPS + own_steps : (total - 1) * sub_per_blk + own_steps;
     if (lane == 0 && do_k) {
       misc->n_steps = n_steps;
       ptx::mbar_arrive(bar(META));
@@ -283,6 +316,49 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
     bool ok = true;
     Blk cur, nxt;
     bool has = pop(nxt);
+    if constexpr (CPS > 1) {
+      // chunks of 32 / 16 tokens: a step packs the next CPS chunks of the union; a short last step repeats its
+      // last chunk with bias -inf
+      while (has && ok) {
+        Blk grp[CPS];
+        int m = 0;
+        while (m < CPS && has) {
+          cur = nxt;
+          has = pop(nxt);
+          if (cur.c == c_own) { has = false; break; }      // last of the walk, done first
+          grp[m++] = cur;
+        }
+        if (m == 0) break;
+#pragma unroll
+        for (int s = 1; s < CPS; ++s)
+          if (s >= m) { grp[s].c = grp[m - 1].c; grp[s].bv[0] = grp[s].bv[1] = -INFINITY; }
+        int kvs[CPS];
+#pragma unroll
+        for (int s = 0; s < CPS; ++s) kvs[s] = grp[s].c * dm.B;
+        const int st = j & 1, prev_ph = ((j >> 1) - 1) & 1;
+        if (do_k) {
+          if (j >= 2) ok = ptx::mbar_wait(bar(S_FULL + st), prev_ph, abort_flag);
+          if (!ok) break;
+          if (lane == 0) load_packed(&tmK, sbase + OFF_K + st * KV_TILE_BYTES, bar(K_FULL + st), kvs);
+        } else {
+          if (j >= 2) ok = ptx::mbar_wait(bar(PV_DONE + st), prev_ph, abort_flag);
+          if (!ok) break;
+#pragma unroll
+          for (int s = 0; s < CPS; ++s)
+            for (int q = 0; q < 2; ++q) {
+              const int t = lane + 32 * q;
+              if (t < TQ) misc->bias[st][s][t] = grp[s].bv[q];
+            }
+#pragma unroll
+          for (int s = 0; s < CPS; ++s)
+            if (lane == s) misc->kvbase[st][s] = kvs[s];
+          __syncwarp();
+          if (lane == 0) load_packed(&tmV, sbase + OFF_V + st * KV_TILE_BYTES, bar(V_FULL + st), kvs);
+        }
+        ++j;
+      }
+      has = false;
+    }
     while (has && ok) {
       cur = nxt;
       has = pop(nxt);
@@ -307,9 +383,9 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
         if (!ok) break;
         for (int q = 0; q < 2; ++q) {
           const int t = lane + 32 * q;
-          if (t < TQ) misc->bias[vs][t] = cur.bv[q];
+          if (t < TQ) misc->bias[vs][0][t] = cur.bv[q];
         }
-        if (lane == 0) misc->kvbase[vs] = kv0;
+        if (lane == 0) misc->kvbase[vs][0] = kv0;
         __syncwarp();
         if (lane == 0) {
           const uint32_t dst = sbase + OFF_V + vs * KV_TILE_BYTES;
@@ -401,8 +477,10 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
       // bias / kvbase of the step visible; the MMA thread relies on this wait for the V tile as well
       ok = ptx::mbar_wait(bar(V_FULL + buf), (j >> 1) & 1, abort_flag);
       if (!ok) break;
-      const float bias = misc->bias[buf][t];
-      const int kv0 = misc->kvbase[buf];
+      float b2s[CPS];                                // per packed chunk: bias in the log2 domain (-inf: not routed)
+#pragma unroll
+      for (int s = 0; s < CPS; ++s) b2s[s] = misc->bias[buf][s][t] * 1.4426950408889634f;
+      const int kv0 = misc->kvbase[buf][0];
       ok = ptx::mbar_wait(bar(S_FULL + buf), (j >> 1) & 1, abort_flag);
       if (!ok) break;
       ptx::tc_fence_after();
@@ -416,11 +494,38 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
       ptx::tmem_wait_ld();
 
       // logit (log2 domain) = s*c1 + b2; c1 > 0, so the row maximum can be taken on the raw scores
-      const bool selected = bias > -INFINITY;
-      const float b2 = bias * 1.4426950408889634f;
       const int n_vis = i_row - kv0 + 1;             // causal: KV token kv0 + c visible iff c < n_vis
+      bool selected;
+      float mloc;
+      if constexpr (CPS > 1) {
+        // packed chunks: each slot of W columns has its own bias; only the own chunk (slot 0 of step 0) can be cut
+        // by the causal mask (routed chunks lie wholly before the row)
+        constexpr int W = NKV / CPS;
+        mloc = -INFINITY;
+#pragma unroll
+        for (int s = 0; s < CPS; ++s) {
+          if (b2s[s] > -INFINITY) {
+            if (s == 0 && n_vis < W) {
+#pragma unroll
+              for (int c = 0; c < W; ++c)
+                if (c >= n_vis) sreg[c] = 0xff800000u;   // -inf
+            }
+            float ch[4];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) ch[c] = __uint_as_float(sreg[s * W + c]);
+#pragma unroll
+            for (int k = 4; k < W; k += 4)
+#pragma unroll
+              for (int c = 0; c < 4; ++c) ch[c] = fmaxf(ch[c], __uint_as_float(sreg[s * W + c + k]));
+            mloc = fmaxf(mloc, fmaf(fmaxf(fmaxf(ch[0], ch[1]), fmaxf(ch[2], ch[3])), c1, b2s[s]));
+          }
+        }
+        selected = mloc > -INFINITY;
+      }
+      const float b2 = b2s[0];
       float mr = -INFINITY;
-      if (selected) {
+      if constexpr (CPS == 1) selected = b2 > -INFINITY;
+      if (CPS == 1 && selected) {
         if (n_vis < NKV) {                           // only inside the own chunk
 #pragma unroll
           for (int c = 0; c < NKV; ++c)
@@ -438,7 +543,7 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
         for (int c = 0; c < 8; ++c) ch[c] = fmaxf(ch[c], __uint_as_float(sreg[c + NKV - 8]));
         mr = fmaxf(max3(ch[0], ch[1], ch[2]), fmaxf(max3(ch[3], ch[4], ch[5]), fmaxf(ch[6], ch[7])));
       }
-      const float mloc = fmaf(mr, c1, b2);           // -inf when not selected
+      if constexpr (CPS == 1) mloc = fmaf(mr, c1, b2);           // -inf when not selected
       float corr = 1.f;
       bool moved = false;
       if (mloc > m_used + RESCALE_LOG2 || (m_used == -INFINITY && mloc > -INFINITY)) {
@@ -449,12 +554,16 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
       l *= corr;
       uint32_t packed[32];
       if (selected) {
-        const float off = b2 - m_used;
-        // scale-and-shift and the row sum on packed pairs (one instruction per two scores)
-        const float2 c1v = make_float2(c1, c1), offv = make_float2(off, off);
+        // scale-and-shift and the row sum on packed pairs (one instruction per two scores); a slot that is not
+        // routed has offset -inf, so its probabilities come out as exactly 0
+        const float2 c1v = make_float2(c1, c1);
+        float2 offs[CPS];
+#pragma unroll
+        for (int s = 0; s < CPS; ++s) offs[s] = make_float2(b2s[s] - m_used, b2s[s] - m_used);
         float2 lsum[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
 #pragma unroll
         for (int c = 0; c < NKV; c += 2) {
+          const float2 offv = offs[c / (NKV / CPS)];
           const float2 t = __ffma2_rn(make_float2(__uint_as_float(sreg[c]), __uint_as_float(sreg[c + 1])), c1v, offv);
           const float2 pp = make_float2(exp2f(t.x), exp2f(t.y));
           lsum[(c >> 1) & 3] = __fadd2_rn(lsum[(c >> 1) & 3], pp);
@@ -546,7 +655,7 @@ bool make_map(CUtensorMap* out, const void* base, int hd, long long tokens, int 
 
 bool prefill_sm100_supported(const Dims& dm) {
   if (dm.decode || !dm.causal || dm.dtype != DASH_BF16 || (dm.d != 64 && dm.d != 128)) return false;
-  if (dm.B != 64 && dm.B != 128) return false;
+  if (dm.B != 16 && dm.B != 32 && dm.B != 64 && dm.B != 128) return false;
   const int tq = 128 / dm.g_q;
   if (dm.g_q < 2 || tq > MAX_TQ || tq > dm.B) return false;
   if (dm.os[2] % 8 != 0 || dm.os[1] % 8 != 0) return false;
@@ -565,22 +674,29 @@ cudaError_t launch_attend_prefill_sm100(const Dims& dm, const void* Q, const voi
   a.O = (__nv_bfloat16*)O;
   a.sb = sb;
   CUtensorMap tq, tk, tv;
+  const int box_kv = dm.B < NKV ? dm.B : NKV;      // chunks below 64 tokens are fetched one box per chunk
   if (!make_map(&tq, Q, dm.d, dm.seq_q, dm.h_q, dm.batch, dm.qs, dm.g_q, a.TQ)) return cudaErrorInvalidValue;
-  if (!make_map(&tk, K, dm.d, dm.seq_kv, dm.h_kv, dm.batch, dm.ks, 1, NKV)) return cudaErrorInvalidValue;
-  if (!make_map(&tv, V, dm.d, dm.seq_kv, dm.h_kv, dm.batch, dm.vs, 1, NKV)) return cudaErrorInvalidValue;
+  if (!make_map(&tk, K, dm.d, dm.seq_kv, dm.h_kv, dm.batch, dm.ks, 1, box_kv)) return cudaErrorInvalidValue;
+  if (!make_map(&tv, V, dm.d, dm.seq_kv, dm.h_kv, dm.batch, dm.vs, 1, box_kv)) return cudaErrorInvalidValue;
   const long long blocks = (long long)a.n_tiles * dm.batch * dm.h_kv;
   cudaError_t le = cudaSuccess;
-  if (dm.d == 128) {
-    static std::atomic<unsigned long long> configured{0};
-    if (cudaError_t e = allow_dynamic_smem(attend_prefill_sm100_kernel<128>, PfLayout<128>::SMEM, configured); e != cudaSuccess) return e;
-    le = launch_chained(attend_prefill_sm100_kernel<128>, dim3((unsigned)blocks), dim3(PF_THREADS), PfLayout<128>::SMEM,
-                        st, tq, tk, tv, a);
-  } else {
-    static std::atomic<unsigned long long> configured{0};
-    if (cudaError_t e = allow_dynamic_smem(attend_prefill_sm100_kernel<64>, PfLayout<64>::SMEM, configured); e != cudaSuccess) return e;
-    le = launch_chained(attend_prefill_sm100_kernel<64>, dim3((unsigned)blocks), dim3(PF_THREADS), PfLayout<64>::SMEM, st,
-                        tq, tk, tv, a);
+#define DASH_PF(HDV, CPSV)                                                                                          \
+  {                                                                                                                 \
+    static std::atomic<unsigned long long> configured{0};                                                           \
+    if (cudaError_t e = allow_dynamic_smem(attend_prefill_sm100_kernel<HDV, CPSV>, PfLayout<HDV, CPSV>::SMEM,       \
+                                           configured);                                                             \
+        e != cudaSuccess)                                                                                           \
+      return e;                                                                                                     \
+    le = launch_chained(attend_prefill_sm100_kernel<HDV, CPSV>, dim3((unsigned)blocks), dim3(PF_THREADS),           \
+                        PfLayout<HDV, CPSV>::SMEM, st, tq, tk, tv, a);                                              \
   }
+  const int cps = NKV / box_kv;
+  if (dm.d == 128) {
+    if (cps == 1) DASH_PF(128, 1) else if (cps == 2) DASH_PF(128, 2) else DASH_PF(128, 4)
+  } else {
+    if (cps == 1) DASH_PF(64, 1) else if (cps == 2) DASH_PF(64, 2) else DASH_PF(64, 4)
+  }
+#undef DASH_PF
   count_launch();
   return le;
 }
