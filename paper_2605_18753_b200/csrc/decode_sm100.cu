@@ -40,20 +40,27 @@ constexpr uint32_t OFF_MISC = OFF_PT + PT_BYTES;
 constexpr uint32_t TMEM_COLS = 64;      // S^T buffers at columns 0 and 16, O^T at 32
 enum BarD { Q_READY = 0, S_FULL = 1, P_FULL = 3, P_EMPTY = 5, RED_BAR = 6, LRED_BAR = 8, K_FULL = 9, K_EMPTY = 9 + NST,
             V_FULL = 9 + 2 * NST, V_EMPTY = 9 + 3 * NST, N_BARS = 9 + 4 * NST };
-struct MiscD {
+// CPS = routed chunks per 64-token sub-block: 1 for chunks of 64 / 128 tokens, 2 / 4 for chunks of 32 / 16 (a
+// sub-block then gathers that many chunks of the list, each fetched by its own TMA box and carrying its own bias).
+template <int CPS>
+struct MiscT {
+  static constexpr int RANGE = MAX_RANGE / CPS;   // sub-blocks one thread block can own
   unsigned long long bar[N_BARS];
   uint32_t tmem_base;
   int abort_flag;
-  float bias2[NST][2];
+  float bias2[NST][2][CPS];
   int nvalid[NST][2];
   float red[2][4][NH];
   float lred[4][NH];
   int is_last;               // this block saw the last arrival of its (batch, KV head)
-  int idx_s[MAX_RANGE];      // first KV token of each owned sub-block
-  float bias_s[MAX_RANGE];
-  int nval_s[MAX_RANGE];
+  int idx_s[RANGE][CPS];     // first KV token of each chunk slot of each owned sub-block
+  float bias_s[RANGE][CPS];
+  int nval_s[RANGE];         // valid rows of the sub-block
 };
-constexpr uint32_t DEC_SMEM = OFF_MISC + sizeof(MiscD);
+constexpr size_t MISC_BYTES = sizeof(MiscT<1>) > sizeof(MiscT<2>)
+                                  ? (sizeof(MiscT<1>) > sizeof(MiscT<4>) ? sizeof(MiscT<1>) : sizeof(MiscT<4>))
+                                  : (sizeof(MiscT<2>) > sizeof(MiscT<4>) ? sizeof(MiscT<2>) : sizeof(MiscT<4>));
+constexpr uint32_t DEC_SMEM = OFF_MISC + (uint32_t)MISC_BYTES;   // one size for every instantiation
 static_assert(DEC_SMEM <= 232448, "shared memory budget");
 
 struct DecodeArgs {
@@ -83,9 +90,11 @@ __device__ __forceinline__ void tmem_st16(uint32_t addr, const uint32_t* r) {
                : "memory");
 }
 
-template <int G>
+template <int G, int CPS>
 __global__ void __launch_bounds__(DEC_THREADS, 1)
 decode_sm100_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, DecodeArgs a) {
+  using MiscD = MiscT<CPS>;
+  constexpr int W = SUB / CPS;          // rows of one chunk slot inside a sub-block
   extern __shared__ __align__(1024) uint8_t smem[];
   MiscD* misc = reinterpret_cast<MiscD*>(smem + OFF_MISC);
   const Dims& dm = a.dm;
@@ -138,8 +147,9 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   L = max(1, min(L, dm.seq_kv));
   const int c_own = (L - 1) / dm.B;
   const long long grp = (long long)b * dm.h_kv + r;
-  const int spb = dm.B / SUB;                                   // sub-blocks per routed chunk
-  const int n_routed_sub = a.count[grp] * spb;
+  const int spb = CPS > 1 ? 1 : dm.B / SUB;                     // sub-blocks per routed chunk (chunks >= 64 tokens)
+  const int n_routed = a.count[grp];
+  const int n_routed_sub = CPS > 1 ? (n_routed + CPS - 1) / CPS : n_routed * spb;
   const int own_tokens = L - c_own * dm.B;                       // 1 .. B
   const int n_items = n_routed_sub + (own_tokens + SUB - 1) / SUB;
   const int per = (n_items + n_split - 1) / n_split;
@@ -154,6 +164,28 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     // owned sub-blocks -> (first token, bias, valid rows), staged once so the walk has no dependent global reads
     for (int k = lane; k < n_own; k += 32) {
       const int it = lo + k;
+      if constexpr (CPS > 1) {
+        if (it < n_routed_sub) {
+          // CPS consecutive list entries; a short last group repeats its last chunk in rows that are marked invalid
+          const int e0 = it * CPS, m = min(CPS, n_routed - e0);
+#pragma unroll
+          for (int s = 0; s < CPS; ++s) {
+            const int e = e0 + min(s, m - 1);
+            misc->idx_s[k][s] = a.blk_idx[loff + e] * dm.B;
+            misc->bias_s[k][s] = a.blk_bias[loff + e];
+          }
+          misc->nval_s[k] = m * dm.B;
+        } else {
+          // the own chunk (shorter than a sub-block): the rows behind it are fetched but marked invalid
+#pragma unroll
+          for (int s = 0; s < CPS; ++s) {
+            misc->idx_s[k][s] = c_own * dm.B + s * W;
+            misc->bias_s[k][s] = 0.f;
+          }
+          misc->nval_s[k] = L - c_own * dm.B;
+        }
+        continue;
+      }
       int tok0, nv;
       float bs;
       if (it < n_routed_sub) {
@@ -167,7 +199,7 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         bs = 0.f;
         nv = min(SUB, L - tok0);
       }
-      misc->idx_s[k] = tok0; misc->bias_s[k] = bs; misc->nval_s[k] = nv;
+      misc->idx_s[k][0] = tok0; misc->bias_s[k][0] = bs; misc->nval_s[k] = nv;
     }
     __syncwarp();
     if (lane == 0) {
@@ -177,27 +209,34 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       int s = 0, ph = 1;
       for (int j = 0; j < n_steps && ok; ++j) {
         const int k0 = 2 * j, k1 = (2 * j + 1 < n_own) ? 2 * j + 1 : 2 * j;   // an odd tail repeats its last sub-block
-        const int t0 = misc->idx_s[k0], t1 = misc->idx_s[k1];
+        // one 128-row tile: sub-blocks k0 and k1, each CPS boxes of W rows, for both halves of head_dim
+        auto load_tile = [&](const CUtensorMap* tm, uint32_t dst, uint32_t barrier) {
+          ptx::mbar_arrive_expect_tx(barrier, TILE_BYTES);
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            const int k = h ? k1 : k0;
+#pragma unroll
+            for (int q = 0; q < CPS; ++q) {
+              const int tok = misc->idx_s[k][q];
+              const uint32_t d = dst + (h * SUB + q * W) * 128;
+              ptx::tma_load_4d(d, tm, barrier, 0, r, tok, b);
+              ptx::tma_load_4d(d + TILE_BYTES / 2, tm, barrier, 64, r, tok, b);
+            }
+          }
+        };
         ok = ptx::mbar_wait(bar(K_EMPTY + s), ph, abort_flag);
         if (!ok) break;
-        uint32_t dst = sbase + OFF_K + s * TILE_BYTES;
-        ptx::mbar_arrive_expect_tx(bar(K_FULL + s), TILE_BYTES);
-        ptx::tma_load_4d(dst, &tmK, bar(K_FULL + s), 0, r, t0, b);
-        ptx::tma_load_4d(dst + SUB * 128, &tmK, bar(K_FULL + s), 0, r, t1, b);
-        ptx::tma_load_4d(dst + TILE_BYTES / 2, &tmK, bar(K_FULL + s), 64, r, t0, b);
-        ptx::tma_load_4d(dst + TILE_BYTES / 2 + SUB * 128, &tmK, bar(K_FULL + s), 64, r, t1, b);
+        load_tile(&tmK, sbase + OFF_K + s * TILE_BYTES, bar(K_FULL + s));
         ok = ptx::mbar_wait(bar(V_EMPTY + s), ph, abort_flag);
         if (!ok) break;
-        misc->bias2[s][0] = misc->bias_s[k0];
-        misc->bias2[s][1] = misc->bias_s[k1];
+#pragma unroll
+        for (int q = 0; q < CPS; ++q) {
+          misc->bias2[s][0][q] = misc->bias_s[k0][q];
+          misc->bias2[s][1][q] = misc->bias_s[k1][q];
+        }
         misc->nvalid[s][0] = misc->nval_s[k0];
         misc->nvalid[s][1] = (k1 != k0) ? misc->nval_s[k1] : 0;
-        dst = sbase + OFF_V + s * TILE_BYTES;
-        ptx::mbar_arrive_expect_tx(bar(V_FULL + s), TILE_BYTES);
-        ptx::tma_load_4d(dst, &tmV, bar(V_FULL + s), 0, r, t0, b);
-        ptx::tma_load_4d(dst + SUB * 128, &tmV, bar(V_FULL + s), 0, r, t1, b);
-        ptx::tma_load_4d(dst + TILE_BYTES / 2, &tmV, bar(V_FULL + s), 64, r, t0, b);
-        ptx::tma_load_4d(dst + TILE_BYTES / 2 + SUB * 128, &tmV, bar(V_FULL + s), 64, r, t1, b);
+        load_tile(&tmV, sbase + OFF_V + s * TILE_BYTES, bar(V_FULL + s));
         if (++s == NST) { s = 0; ph ^= 1; }
       }
       if (!ok) {
@@ -279,7 +318,7 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     for (int j = 0; j < n_steps && ok; ++j) {
       ok = ptx::mbar_wait(bar(V_FULL + vs), vph, abort_flag);     // step metadata visible, V tile landed
       if (!ok) break;
-      const float b2 = misc->bias2[vs][half] * 1.4426950408889634f;
+      const float b2 = misc->bias2[vs][half][CPS > 1 ? row / W : 0] * 1.4426950408889634f;
       const int nval = misc->nvalid[vs][half];
       const bool valid = row < nval;
       ok = ptx::mbar_wait(bar(S_FULL + (j & 1)), (j >> 1) & 1, abort_flag);
@@ -430,7 +469,7 @@ bool make_kv_map(CUtensorMap* out, const void* base, const Dims& dm, const long 
   cuuint64_t dims[4] = {(cuuint64_t)HD, (cuuint64_t)dm.h_kv, (cuuint64_t)dm.seq_kv, (cuuint64_t)dm.batch};
   auto st = [](long long e) { return (cuuint64_t)((e > 0 ? e : 8) * 2); };
   cuuint64_t strides[3] = {st(s[2]), st(s[1]), st(s[0])};
-  cuuint32_t box[4] = {64u, 1u, (cuuint32_t)SUB, 1u};
+  cuuint32_t box[4] = {64u, 1u, (cuuint32_t)(dm.B < SUB ? dm.B : SUB), 1u};   // chunks below 64 tokens: one box per chunk
   return encode_bf16_sw128_4d(out, base, dims, strides, box);
 }
 
@@ -439,8 +478,13 @@ bool make_kv_map(CUtensorMap* out, const void* base, const Dims& dm, const long 
 // Splits needed so that no thread block owns more than MAX_RANGE sub-blocks (0: shape not served here).
 int decode_sm100_min_splits(const Dims& dm) {
   if (!dm.decode || dm.dtype != DASH_BF16 || dm.d != HD) return 0;
-  if (dm.B != 64 && dm.B != 128) return 0;
+  if (dm.B != 16 && dm.B != 32 && dm.B != 64 && dm.B != 128) return 0;
   if (dm.qs[2] % 8 != 0 || tensor_map_encoder() == nullptr) return 0;
+  if (dm.B < SUB) {
+    const int cps = SUB / dm.B, range = MAX_RANGE / cps;
+    const int max_items = (dm.T_s + cps - 1) / cps + 1;
+    return (max_items + range - 1) / range;
+  }
   const int max_items = (dm.T_s + 1) * (dm.B / SUB);
   return (max_items + MAX_RANGE - 1) / MAX_RANGE;
 }
@@ -456,21 +500,24 @@ cudaError_t launch_decode_sm100(const Dims& dm, int n_split, const void* Q, cons
   if (!make_kv_map(&tk, K, dm, dm.ks) || !make_kv_map(&tv, V, dm, dm.vs)) return cudaErrorInvalidValue;
   dim3 grid(n_split, dm.h_kv, dm.batch);
   cudaError_t le = cudaSuccess;
-#define DASH_DEC_TC(G)                                                                                          \
+#define DASH_DEC_TC(G, C)                                                                                       \
   {                                                                                                             \
     static std::atomic<unsigned long long> configured{0};                                                       \
-    cudaError_t e = allow_dynamic_smem(decode_sm100_kernel<G>, DEC_SMEM, configured);                           \
+    cudaError_t e = allow_dynamic_smem(decode_sm100_kernel<G, C>, DEC_SMEM, configured);                        \
     if (e != cudaSuccess) return e;                                                                             \
-    le = launch_chained(decode_sm100_kernel<G>, grid, dim3(DEC_THREADS), DEC_SMEM, st, tk, tv, a);              \
+    le = launch_chained(decode_sm100_kernel<G, C>, grid, dim3(DEC_THREADS), DEC_SMEM, st, tk, tv, a);           \
   }
-  switch (dm.g_q) {
-    case 1: DASH_DEC_TC(1); break;
-    case 2: DASH_DEC_TC(2); break;
-    case 4: DASH_DEC_TC(4); break;
-    case 8: DASH_DEC_TC(8); break;
-    case 16: DASH_DEC_TC(16); break;
-    default: return cudaErrorInvalidValue;
+#define DASH_DEC_G(C)                                  \
+  switch (dm.g_q) {                                    \
+    case 1: DASH_DEC_TC(1, C); break;                  \
+    case 2: DASH_DEC_TC(2, C); break;                  \
+    case 4: DASH_DEC_TC(4, C); break;                  \
+    case 8: DASH_DEC_TC(8, C); break;                  \
+    case 16: DASH_DEC_TC(16, C); break;                \
+    default: return cudaErrorInvalidValue;             \
   }
+  if (dm.B >= SUB) { DASH_DEC_G(1) } else if (dm.B == 32) { DASH_DEC_G(2) } else { DASH_DEC_G(4) }
+#undef DASH_DEC_G
 #undef DASH_DEC_TC
   count_launch();
   return le;

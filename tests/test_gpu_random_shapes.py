@@ -49,14 +49,15 @@ def test_random_shapes_any_path(seed):
 
 @pytest.mark.parametrize("seed", [21])
 def test_random_shapes_tensor_core_paths(seed):
-    """bf16, head_dim 128, chunks of 64 / 128, g_q >= 2: the shapes the TMA / tcgen05 kernels serve."""
+    """bf16, g_q >= 2, every chunk size and both head dims: mostly shapes the TMA / tcgen05 kernels serve."""
     rng = np.random.default_rng(seed)
     done = 0
     for _ in range(120):
         g_q = int(rng.choice([2, 4, 8, 16])); h_kv = int(rng.choice([1, 2]))
         seq = int(rng.integers(1, 9000))
         batch = int(rng.choice([1, 2]))
-        kw = dict(seq=seq, h_q=g_q * h_kv, h_kv=h_kv, head_dim=128, block=int(rng.choice([64, 128])), dtype="bf16",
+        kw = dict(seq=seq, h_q=g_q * h_kv, h_kv=h_kv, head_dim=int(rng.choice([128, 128, 64])),
+                  block=int(rng.choice([16, 32, 64, 128])), dtype="bf16",
                   alpha=float(rng.choice([1.25, 1.5, 1.5, 2.0, 1.6])), gamma=float(rng.choice([1.0, 2.0])), batch=batch,
                   seed=int(rng.integers(0, 1000)), sigma=float(rng.choice([1.0, 10.0, 1e8])),
                   n_planted=int(rng.choice([2, 5, 9])))
