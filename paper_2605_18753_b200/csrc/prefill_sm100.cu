@@ -1,7 +1,8 @@
 // Stage 2, prefill, tensor-core path for sm_100a (Eq. 7 in the form of Proposition 1; Algorithm 3).
 //
-// Tile: one (batch, KV head) and TQ = 128/g_q consecutive query tokens; the 128 rows of the MMA tile are
-// (token, head-of-group) pairs, token-major.  A tile never straddles a chunk, so its rows share the own
+// Tile: one (batch, KV head) and TQ = min(128/g_q, chunk size) consecutive query tokens; the rows of the MMA tile
+// are (token, head-of-group) pairs, token-major (with chunks shorter than 128/g_q tokens the tile holds fewer than
+// 128 live rows; the rest are zero queries whose results are dropped).  A tile never straddles a chunk, so its rows share the own
 // chunk; it takes the own chunk first (its tiles can be fetched before the mask has been read), then walks
 // the UNION of its rows' routed chunks in ascending order, 64 KV tokens per step.  A row that did not route
 // a chunk gets bias -inf for that step (probability exactly 0), so every row still attends to its own
@@ -86,7 +87,9 @@ struct PrefillArgs {
   StatusBlock* sb;
 };
 
-template <int HD, int CPS>
+// SHORT: the tile has fewer than 128 live rows (chunks shorter than 128 / g_q tokens); full tiles compile without
+// any of the padding-row handling.
+template <int HD, int CPS, bool SHORT>
 __global__ void __launch_bounds__(PF_THREADS, 2)
 attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                             const __grid_constant__ CUtensorMap tmV, PrefillArgs a) {
@@ -141,6 +144,15 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem = misc->tmem_base;
+  // Rows of the Q tile beyond the tile's TQ * g_q live rows (chunks shorter than 128 / g_q tokens) are never written by
+  // the TMA box: they are zeroed once, so that their scores are finite; their probabilities are forced to 0 below.
+  if constexpr (SHORT) {
+    const int first = TQ * g_q * 8;                 // 16-byte pieces before the first dead row (a row is 128 bytes)
+    for (int regn = 0; regn < HD / 64; ++regn)
+      for (int k = first + tid; k < 128 * 8; k += PF_THREADS)
+        *reinterpret_cast<uint4*>(smem + OFF_Q + regn * (Q_BYTES / (HD / 64)) + k * 16) = make_uint4(0u, 0u, 0u, 0u);
+    ptx::fence_proxy_async_smem();
+  }
   // barriers and tensor memory are set up; from here on the kernel reads what the routing kernels wrote
   chain_wait();
   chain_release();
@@ -154,11 +166,12 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
     // Two warps walk the same union list: warp 4 feeds the K ring (and loads Q), warp 6 feeds the V ring and
     // the per-token bias of each step.  Split like this, a full V ring never holds back the next K tile.
     const bool do_k = (warp == 4), do_v = (warp == 6);
+    const int TR = SHORT ? 128 / g_q : TQ;   // token slots of the 128 tile rows; slots TQ .. TR-1 are padding (bias -inf)
     if (lane == 0 && do_k) {
       ptx::prefetch_tensormap(&tmQ);
       ptx::prefetch_tensormap(&tmK);
       ptx::prefetch_tensormap(&tmV);
-      ptx::mbar_arrive_expect_tx(bar(Q_FULL), Q_BYTES);
+      ptx::mbar_arrive_expect_tx(bar(Q_FULL), SHORT ? (uint32_t)(TQ * g_q * HD * 2) : Q_BYTES);   // the box holds the live rows
       ptx::tma_load_4d(sbase + OFF_Q, &tmQ, bar(Q_FULL), 0, r * g_q, i0, b);
       if constexpr (HD == 128) ptx::tma_load_4d(sbase + OFF_Q + Q_BYTES / 2, &tmQ, bar(Q_FULL), 64, r * g_q, i0, b);
     }
@@ -184,8 +197,8 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
         if (do_k) {
           if (lane == 0) load_packed(&tmK, sbase + OFF_K, bar(K_FULL), kvs);
         } else {
-          for (int t = lane; t < TQ; t += 32) {
-            misc->bias[0][0][t] = 0.f;
+          for (int t = lane; t < TR; t += 32) {
+            misc->bias[0][0][t] = t < TQ ? 0.f : -INFINITY;     // token slots beyond TQ: padding rows of a short tile
 #pragma unroll
             for (int s = 1; s < CPS; ++s) misc->bias[0][s][t] = -INFINITY;
           }
@@ -203,7 +216,7 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
           if constexpr (HD == 128) ptx::tma_load_4d(dst + KV_TILE_BYTES / 2, &tmK, bar(K_FULL + sub), 64, r, kv0, b);
         }
       } else {
-        for (int t = lane; t < TQ; t += 32) misc->bias[sub][0][t] = 0.f;
+        for (int t = lane; t < TR; t += 32) misc->bias[sub][0][t] = t < TQ ? 0.f : -INFINITY;   // beyond TQ: padding rows
         if (lane == 0) misc->kvbase[sub][0] = kv0;
         __syncwarp();
         if (lane == 0) {
@@ -347,7 +360,7 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
           for (int s = 0; s < CPS; ++s)
             for (int q = 0; q < 2; ++q) {
               const int t = lane + 32 * q;
-              if (t < TQ) misc->bias[st][s][t] = grp[s].bv[q];
+              if (t < TR) misc->bias[st][s][t] = t < TQ ? grp[s].bv[q] : -INFINITY;
             }
 #pragma unroll
           for (int s = 0; s < CPS; ++s)
@@ -383,7 +396,7 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
         if (!ok) break;
         for (int q = 0; q < 2; ++q) {
           const int t = lane + 32 * q;
-          if (t < TQ) misc->bias[vs][0][t] = cur.bv[q];
+          if (t < TR) misc->bias[vs][0][t] = t < TQ ? cur.bv[q] : -INFINITY;
         }
         if (lane == 0) misc->kvbase[vs][0] = kv0;
         __syncwarp();
@@ -460,6 +473,7 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
     const int m = tid;                       // tile row = TMEM lane
     const int t = m / g_q, hh = m % g_q;     // token in tile, head in group
     const int i_row = i0 + t;
+    const bool row_live = t < TQ;            // false for the padding rows of a tile shorter than 128 rows
     const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
     const float c1 = dm.sm_scale * 1.4426950408889634f;
     bool ok = true;
@@ -479,7 +493,7 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
       if (!ok) break;
       float b2s[CPS];                                // per packed chunk: bias in the log2 domain (-inf: not routed)
 #pragma unroll
-      for (int s = 0; s < CPS; ++s) b2s[s] = misc->bias[buf][s][t] * 1.4426950408889634f;
+      for (int s = 0; s < CPS; ++s) b2s[s] = misc->bias[buf][s][t] * 1.4426950408889634f;   // -inf on padding rows
       const int kv0 = misc->kvbase[buf][0];
       ok = ptx::mbar_wait(bar(S_FULL + buf), (j >> 1) & 1, abort_flag);
       if (!ok) break;
@@ -612,7 +626,7 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
         uint32_t o[32];
         DASH_TMEM_LD32(o, lane_addr + 2 * NKV + q * 32);
         ptx::tmem_wait_ld();
-        if (i_row < dm.seq_q) {
+        if (i_row < dm.seq_q && (!SHORT || row_live)) {
 #pragma unroll
           for (int c = 0; c < 32; c += 8) {
             uint4 v;
@@ -656,8 +670,7 @@ bool make_map(CUtensorMap* out, const void* base, int hd, long long tokens, int 
 bool prefill_sm100_supported(const Dims& dm) {
   if (dm.decode || !dm.causal || dm.dtype != DASH_BF16 || (dm.d != 64 && dm.d != 128)) return false;
   if (dm.B != 16 && dm.B != 32 && dm.B != 64 && dm.B != 128) return false;
-  const int tq = 128 / dm.g_q;
-  if (dm.g_q < 2 || tq > MAX_TQ || tq > dm.B) return false;
+  if (dm.g_q < 2 || 128 / dm.g_q > MAX_TQ) return false;
   if (dm.os[2] % 8 != 0 || dm.os[1] % 8 != 0) return false;
   return tensor_map_encoder() != nullptr;
 }
@@ -667,7 +680,7 @@ cudaError_t launch_attend_prefill_sm100(const Dims& dm, const void* Q, const voi
                                         cudaStream_t st) {
   PrefillArgs a;
   a.dm = dm;
-  a.TQ = 128 / dm.g_q;
+  a.TQ = 128 / dm.g_q < dm.B ? 128 / dm.g_q : dm.B;     // a tile stays inside one chunk
   a.n_tiles = (dm.seq_q + a.TQ - 1) / a.TQ;
   a.mask = mask;
   a.blk_bias = blk_bias;
@@ -680,22 +693,24 @@ cudaError_t launch_attend_prefill_sm100(const Dims& dm, const void* Q, const voi
   if (!make_map(&tv, V, dm.d, dm.seq_kv, dm.h_kv, dm.batch, dm.vs, 1, box_kv)) return cudaErrorInvalidValue;
   const long long blocks = (long long)a.n_tiles * dm.batch * dm.h_kv;
   cudaError_t le = cudaSuccess;
-#define DASH_PF(HDV, CPSV)                                                                                          \
+#define DASH_PF(HDV, CPSV, SHORTV)                                                                                  \
   {                                                                                                                 \
     static std::atomic<unsigned long long> configured{0};                                                           \
-    if (cudaError_t e = allow_dynamic_smem(attend_prefill_sm100_kernel<HDV, CPSV>, PfLayout<HDV, CPSV>::SMEM,       \
-                                           configured);                                                             \
+    if (cudaError_t e = allow_dynamic_smem(attend_prefill_sm100_kernel<HDV, CPSV, SHORTV>,                          \
+                                           PfLayout<HDV, CPSV>::SMEM, configured);                                  \
         e != cudaSuccess)                                                                                           \
       return e;                                                                                                     \
-    le = launch_chained(attend_prefill_sm100_kernel<HDV, CPSV>, dim3((unsigned)blocks), dim3(PF_THREADS),           \
+    le = launch_chained(attend_prefill_sm100_kernel<HDV, CPSV, SHORTV>, dim3((unsigned)blocks), dim3(PF_THREADS),   \
                         PfLayout<HDV, CPSV>::SMEM, st, tq, tk, tv, a);                                              \
   }
+#define DASH_PF_HD(HDV)                                                                    \
+  if (cps == 1) DASH_PF(HDV, 1, false)                                                     \
+  else if (cps == 2) { if (short_tile) DASH_PF(HDV, 2, true) else DASH_PF(HDV, 2, false) } \
+  else { if (short_tile) DASH_PF(HDV, 4, true) else DASH_PF(HDV, 4, false) }
   const int cps = NKV / box_kv;
-  if (dm.d == 128) {
-    if (cps == 1) DASH_PF(128, 1) else if (cps == 2) DASH_PF(128, 2) else DASH_PF(128, 4)
-  } else {
-    if (cps == 1) DASH_PF(64, 1) else if (cps == 2) DASH_PF(64, 2) else DASH_PF(64, 4)
-  }
+  const bool short_tile = a.TQ * dm.g_q < 128;      // only with chunks below 64 tokens
+  if (dm.d == 128) { DASH_PF_HD(128) } else { DASH_PF_HD(64) }
+#undef DASH_PF_HD
 #undef DASH_PF
   count_launch();
   return le;

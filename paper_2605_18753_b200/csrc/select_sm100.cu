@@ -82,7 +82,9 @@ __global__ void kbar_split_kernel(const float* __restrict__ kbar, __nv_bfloat16*
   planes[2 * n + i] = __float2bfloat16_rn(r2);
 }
 
-template <int NST, int G, int CS, int HD>
+// SHORT: the tile has fewer than 128 live rows (chunks shorter than 128 / g_q tokens); full tiles compile without
+// any of the padding-row handling.
+template <int NST, int G, int CS, int HD, bool SHORT>
 __global__ void __launch_bounds__(SEL_TC_THREADS, NST == 1 ? 2 : 1)
 select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKB, SelectTcArgs a) {
   using SP = SmemPlan<NST>;
@@ -133,6 +135,15 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     ptx::tmem_relinquish();
     ptx::tc_fence_before();
   }
+  // Rows of the Q tile beyond its TQ * g_q live rows (chunks shorter than 128 / g_q tokens) are never written by the
+  // TMA box: zero queries give zero logits, and nothing those rows compute is stored.
+  if constexpr (SHORT) {
+    const int first = TQ * g_q * 8;                 // 16-byte pieces before the first dead row (a row is 128 bytes)
+    for (int regn = 0; regn < HD / 64; ++regn)
+      for (int k = first + tid; k < 128 * 8; k += SEL_TC_THREADS)
+        *reinterpret_cast<uint4*>(smem + SP::OFF_Q + regn * (Q_BYTES / 2) + k * 16) = make_uint4(0u, 0u, 0u, 0u);
+    ptx::fence_proxy_async_smem();
+  }
   __syncthreads();
   if (CS > 1) ptx::cluster_sync_all();     // every block's barriers exist before anybody arrives on them remotely
   ptx::tc_fence_after();
@@ -150,7 +161,7 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     if (lane == 0 && n_loc > 0) {
       ptx::prefetch_tensormap(&tmQ);
       ptx::prefetch_tensormap(&tmKB);
-      ptx::mbar_arrive_expect_tx(bar(Q_FULL), 128 * HD * 2);
+      ptx::mbar_arrive_expect_tx(bar(Q_FULL), SHORT ? (uint32_t)(TQ * g_q * HD * 2) : 128 * HD * 2);   // the box holds the live rows
       ptx::tma_load_4d(sbase + SP::OFF_Q, &tmQ, bar(Q_FULL), 0, r * g_q, i0, b);
       if constexpr (HD == 128) ptx::tma_load_4d(sbase + SP::OFF_Q + Q_BYTES / 2, &tmQ, bar(Q_FULL), 64, r * g_q, i0, b);
       const long long row0 = ((long long)b * dm.h_kv + r) * dm.T_s + c_lo;
@@ -204,7 +215,7 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const int m = tid;
     const int t = m / g_q, hh = m % g_q;
     const int i = i0 + t;
-    const bool row_valid = i < dm.seq_q;
+    const bool row_valid = SHORT ? (i < dm.seq_q && t < TQ) : i < dm.seq_q;   // (a short tile ends with zero-query rows)
     const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
     const int e_int = dm.e_int;
     const float e = dm.e, xs = dm.x_scale;
@@ -591,8 +602,7 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 // holds 512 candidates per row in tensor memory; clusters of 2 or 4 blocks extend that to 1024 / 2048.
 int select_sm100_token_limit(const Dims& dm) {
   if (dm.decode || !dm.causal || dm.dtype != DASH_BF16 || (dm.d != 64 && dm.d != 128) || dm.T_s < 1) return 0;
-  const int tq = 128 / dm.g_q;
-  if (dm.g_q < 2 || tq > dm.B) return 0;
+  if (dm.g_q < 2) return 0;
   if (tensor_map_encoder() == nullptr) return 0;
   const long long lim = (long long)(4 * CLUSTER_COLS + 1) * dm.B;   // own chunk index <= 2048
   return (int)(lim < dm.seq_q ? lim : dm.seq_q);
@@ -602,10 +612,10 @@ size_t select_sm100_scratch_bytes(const Dims& dm) {
   return (size_t)3 * dm.batch * dm.h_kv * (size_t)(dm.T_s > 0 ? dm.T_s : 1) * dm.d * sizeof(__nv_bfloat16);
 }
 
-template <int NST, int G, int CS, int HD>
+template <int NST, int G, int CS, int HD, bool SHORT = false>
 static cudaError_t launch_band(const CUtensorMap& tq, const CUtensorMap& tkb, const SelectTcArgs& a, long long clusters,
                                cudaStream_t st) {
-  auto kern = select_sm100_kernel<NST, G, CS, HD>;
+  auto kern = select_sm100_kernel<NST, G, CS, HD, SHORT>;
   static std::atomic<unsigned long long> configured{0};
   if (cudaError_t e = allow_dynamic_smem(kern, SmemPlan<NST>::TOTAL, configured); e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
@@ -630,6 +640,16 @@ static cudaError_t launch_band(const CUtensorMap& tq, const CUtensorMap& tkb, co
 template <int NST, int CS>
 static cudaError_t launch_band_g(const Dims& dm, const CUtensorMap& tq, const CUtensorMap& tkb, const SelectTcArgs& a,
                                  long long clusters, cudaStream_t st) {
+  if (a.TQ * dm.g_q < 128) {      // short tiles: only g_q = 2 (chunks of 16 or 32) and g_q = 4 (chunks of 16)
+    if (dm.d == 64) {
+      if (dm.g_q == 2) return launch_band<NST, 2, CS, 64, true>(tq, tkb, a, clusters, st);
+      if (dm.g_q == 4) return launch_band<NST, 4, CS, 64, true>(tq, tkb, a, clusters, st);
+    } else {
+      if (dm.g_q == 2) return launch_band<NST, 2, CS, 128, true>(tq, tkb, a, clusters, st);
+      if (dm.g_q == 4) return launch_band<NST, 4, CS, 128, true>(tq, tkb, a, clusters, st);
+    }
+    return cudaErrorInvalidValue;
+  }
   if (dm.d == 64) {
     switch (dm.g_q) {
       case 2: return launch_band<NST, 2, CS, 64>(tq, tkb, a, clusters, st);
@@ -691,7 +711,7 @@ cudaError_t launch_select_sm100(const Dims& dm, int token_limit, const void* Q, 
 
   SelectTcArgs a;
   a.dm = dm;
-  a.TQ = 128 / dm.g_q;
+  a.TQ = 128 / dm.g_q < dm.B ? 128 / dm.g_q : dm.B;     // a tile stays inside one chunk
   a.plane_rows = plane_rows;
   a.mask = mask; a.count = count; a.blk_idx = blk_idx; a.blk_bias = blk_bias; a.tau = tau; a.sb = sb;
 

@@ -204,7 +204,9 @@ def test_fwd_prefill_tiny_fp32(name, sigmas):
     dict(seq=1300, h_q=8, h_kv=2, head_dim=128, block=32, seed=8),           # two chunks of 32 per 64-token step
     dict(seq=1000, h_q=16, h_kv=2, head_dim=128, block=16, seed=9),          # four chunks of 16 per step (g_q = 8)
     dict(seq=777, h_q=16, h_kv=1, head_dim=64, block=16, seed=10, alpha=1.25, gamma=2.0),
-    dict(seq=2100, h_q=4, h_kv=2, head_dim=128, block=32, seed=11, n_planted=6),   # g_q = 2: 64-token tiles, chunks of 32: not served
+    dict(seq=2100, h_q=4, h_kv=2, head_dim=128, block=32, seed=11, n_planted=6),   # g_q = 2, chunks of 32: tiles of 32 tokens, 64 live rows
+    dict(seq=1500, h_q=8, h_kv=2, head_dim=128, block=16, seed=12),                # g_q = 4, chunks of 16: tiles of 16 tokens
+    dict(seq=900, h_q=2, h_kv=1, head_dim=64, block=16, seed=13, alpha=2.0),        # g_q = 2, chunks of 16: 32 live rows
 ])
 def test_fwd_prefill_small(kw):
     w = _wl(**kw)
