@@ -117,6 +117,8 @@ def _check_select(w, inp, p, rt, rows, kv_heads=None, local_blocks=0):
     dict(h_q=8, h_kv=1, head_dim=128, block=16, seq=9000),      # rows beyond 512 candidates: clusters of two blocks
     dict(h_q=16, h_kv=1, head_dim=128, block=16, seq=17000, n_planted=6),   # beyond 1024: clusters of four
     dict(h_q=4, h_kv=2, head_dim=128, block=64, seq=2100, alpha=2.0), dict(h_q=32, h_kv=2, head_dim=128, block=32, seq=700),
+    dict(h_q=4, h_kv=1, head_dim=128, block=16, seq=9000),      # tiles of 16 tokens (64 live rows) in clusters of two blocks
+    dict(h_q=4, h_kv=2, head_dim=64, block=32, seq=3000, alpha=1.25),   # g_q = 2: tiles of 32 tokens, head_dim 64
 ])
 def test_select_matches_oracle(kw):
     w = _wl(**kw)
