@@ -25,9 +25,9 @@
  *   - 0-based positions.  Chunk of token j is j / block.  T_s = seq_kv / block complete chunks have
  *     summaries; T_a = ceil(seq_kv / block) chunks exist; W = ceil(T_a / 32) mask words per row.
  *   - Query head h uses KV head h / (h_q / h_kv) (Section 3.2).
- *   - Which kernels run: bf16 tensors with g_q = h_q / h_kv >= 2 take the TMA / tcgen05 kernels (prefill: head_dim
- *     64 or 128, every chunk size; decode: head_dim 128, every chunk size); fp32 tensors, g_q = 1, head_dim 64 in
- *     decode and the non-causal mode take CUDA-core kernels that compute the same thing (the correctness path).
+ *   - Which kernels run: bf16 tensors take the TMA / tcgen05 kernels (head_dim 64 or 128, every chunk size; prefill
+ *     needs g_q = h_q / h_kv >= 2, decode takes every group size); fp32 tensors, g_q = 1 in prefill and the
+ *     non-causal mode take CUDA-core kernels that compute the same thing (the correctness path).
  *     The choice is made from the parameters alone, never from the data, and is the same on every call.
  *   - causal = 1 is the paper's setting and the one the tensor-core kernels serve.  causal = 0 (prefill only;
  *     the paper does not define it) is read as: every complete chunk is a candidate of every row; the

@@ -265,7 +265,8 @@ cudaError_t launch_attend_decode_ex(const Dims& dm, const void* Q, const void* K
     cudaError_t e = launch_decode_sm100(dm, ns, Q, K, V, kv_len, count, blk_idx, blk_bias, partials, fused ? O : nullptr,
                                         sb, st);
     if (e != cudaSuccess || fused) return e;
-    return launch_merge<__nv_bfloat16, 128>(dm, ns, partials, O, st);
+    return dm.d == 128 ? launch_merge<__nv_bfloat16, 128>(dm, ns, partials, O, st)
+                       : launch_merge<__nv_bfloat16, 64>(dm, ns, partials, O, st);
   }
   return launch_attend_decode(dm, Q, K, V, kv_len, count, blk_idx, blk_bias, O, partials, st);
 }

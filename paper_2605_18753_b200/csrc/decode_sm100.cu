@@ -22,15 +22,15 @@ namespace dash {
 
 namespace {
 
-constexpr int HD = 128;
+constexpr int HD_MAX = 128;             // the shared-memory layout is the one of head_dim 128 (head_dim 64 fills half a tile)
 constexpr int SUB = 64;                 // KV tokens per sub-block (one TMA box pair)
 constexpr int STEP = 128;               // KV tokens per step = MMA M
 constexpr int NST = 3;                  // K/V ring depth
 constexpr int NH = 16;                  // heads padded to the MMA N
 constexpr int DEC_THREADS = 192;
 constexpr int MAX_RANGE = 512;          // sub-blocks one thread block can own
-constexpr uint32_t TILE_BYTES = STEP * HD * 2;   // 32 KiB: two regions (d halves) of 128 rows x 128 B
-constexpr uint32_t QT_BYTES = NH * HD * 2;       // 4 KiB: two regions of 16 rows x 128 B
+constexpr uint32_t TILE_BYTES = STEP * HD_MAX * 2;   // 32 KiB: two regions (d halves) of 128 rows x 128 B
+constexpr uint32_t QT_BYTES = NH * HD_MAX * 2;       // 4 KiB: two regions of 16 rows x 128 B
 constexpr uint32_t PT_BYTES = NH * STEP * 2;     // 4 KiB: two regions (key halves) of 16 rows x 128 B
 constexpr uint32_t OFF_K = 0;
 constexpr uint32_t OFF_V = OFF_K + NST * TILE_BYTES;
@@ -90,7 +90,12 @@ __device__ __forceinline__ void tmem_st16(uint32_t addr, const uint32_t* r) {
                : "memory");
 }
 
-template <int G, int CPS>
+// head_dim 64 (HD = 64): K and V tiles are one 128-byte region per row.  S^T = K Q^T has four K steps.  The
+// accumulator O^T would have only 64 rows, which is not an M = 128 shape, so the two 64-key sub-blocks of a step are
+// stacked along M instead: A = [V_a^T ; V_b^T] (two MN blocks of 64, 8 KiB apart), K = 64 keys, B = [P_a^T | P_b^T]
+// (N = 32): rows 0-63 / columns 0-15 hold V_a^T P_a^T and rows 64-127 / columns 16-31 hold V_b^T P_b^T (the other two
+// quadrants are not used); the two are added when the partial is written.
+template <int G, int CPS, int HD>
 __global__ void __launch_bounds__(DEC_THREADS, 1)
 decode_sm100_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, DecodeArgs a) {
   using MiscD = MiscT<CPS>;
@@ -211,7 +216,7 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         const int k0 = 2 * j, k1 = (2 * j + 1 < n_own) ? 2 * j + 1 : 2 * j;   // an odd tail repeats its last sub-block
         // one 128-row tile: sub-blocks k0 and k1, each CPS boxes of W rows, for both halves of head_dim
         auto load_tile = [&](const CUtensorMap* tm, uint32_t dst, uint32_t barrier) {
-          ptx::mbar_arrive_expect_tx(barrier, TILE_BYTES);
+          ptx::mbar_arrive_expect_tx(barrier, STEP * HD * 2);
 #pragma unroll
           for (int h = 0; h < 2; ++h) {
             const int k = h ? k1 : k0;
@@ -220,7 +225,7 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
               const int tok = misc->idx_s[k][q];
               const uint32_t d = dst + (h * SUB + q * W) * 128;
               ptx::tma_load_4d(d, tm, barrier, 0, r, tok, b);
-              ptx::tma_load_4d(d + TILE_BYTES / 2, tm, barrier, 64, r, tok, b);
+              if constexpr (HD == 128) ptx::tma_load_4d(d + TILE_BYTES / 2, tm, barrier, 64, r, tok, b);
             }
           }
         };
@@ -250,10 +255,12 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     // ---------------- MMA issuer
     if (lane == 0 && n_steps > 0) {
       constexpr uint32_t IDESC_S = ptx::idesc_bf16_f32(128, NH, false, false);
-      constexpr uint32_t IDESC_O = ptx::idesc_bf16_f32(128, NH, true, false);
+      constexpr uint32_t IDESC_O = ptx::idesc_bf16_f32(128, HD == 128 ? NH : 2 * NH, true, false);
       const uint64_t kd0 = ptx::smem_desc_sw128(sbase + OFF_K, 16, 1024);
       const uint64_t qd0 = ptx::smem_desc_sw128(sbase + OFF_QT, 16, 1024);
-      const uint64_t vd0 = ptx::smem_desc_sw128(sbase + OFF_V, TILE_BYTES / 2, 1024);   // MN-major A: d halves 16 KiB apart
+      // MN-major A: the two MN blocks of 64 are the d halves, 16 KiB apart (head_dim 128), or the two 64-key
+      // sub-blocks of the step, 8 KiB apart (head_dim 64)
+      const uint64_t vd0 = ptx::smem_desc_sw128(sbase + OFF_V, HD == 128 ? TILE_BYTES / 2 : SUB * 128, 1024);
       const uint64_t pd0 = ptx::smem_desc_sw128(sbase + OFF_PT, 16, 1024);
       bool ok = ptx::mbar_wait(bar(Q_READY), 0, abort_flag);
       int ks = 0, kph = 0;
@@ -282,9 +289,11 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         ptx::tc_fence_after();
         const uint64_t vd = vd0 + (uint64_t)((vs * TILE_BYTES) >> 4);
 #pragma unroll
-        for (int k = 0; k < STEP / 16; ++k) {
+        for (int k = 0; k < (HD == 128 ? STEP : SUB) / 16; ++k) {
           const uint64_t ad = vd + (uint64_t)((k * 16 * 128) >> 4);                                   // 16 key rows = 2048 B
-          const uint64_t bd = pd0 + (uint64_t)(((k >> 2) * (PT_BYTES / 2) + (k & 3) * 32) >> 4);
+          // head_dim 128: P^T is two K-major regions (key halves) of 16 rows; head_dim 64: the same bytes read as one
+          // region of 32 rows (sub-block a's heads, then sub-block b's), 64 keys long
+          const uint64_t bd = pd0 + (uint64_t)(((HD == 128 ? (k >> 2) * (PT_BYTES / 2) : 0) + (k & 3) * 32) >> 4);
           ptx::mma_bf16_ss(tmem + 2 * NH, ad, bd, IDESC_O, (j > 0 || k > 0) ? 1u : 0u);
         }
         ptx::mma_commit(bar(V_EMPTY + vs));
@@ -301,7 +310,8 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     for (int ch = tid; ch < NH * 16; ch += 128) {
       const int h = ch >> 4, c16 = ch & 15;            // 16-byte chunk c16 of head h: d = c16*8 .. +7
       uint4 v = make_uint4(0u, 0u, 0u, 0u);
-      if (h < G) v = *reinterpret_cast<const uint4*>(a.Q + (long long)b * dm.qs[0] + (long long)(r * G + h) * dm.qs[2] + c16 * 8);
+      if (h < G && c16 * 8 < HD)
+        v = *reinterpret_cast<const uint4*>(a.Q + (long long)b * dm.qs[0] + (long long)(r * G + h) * dm.qs[2] + c16 * 8);
       const uint32_t off = (c16 >> 3) * (QT_BYTES / 2) + h * 128 + (((c16 & 7) ^ (h & 7)) << 4);
       *reinterpret_cast<uint4*>(smem + OFF_QT + off) = v;
       *reinterpret_cast<uint4*>(smem + OFF_PT + off) = make_uint4(0u, 0u, 0u, 0u);
@@ -361,12 +371,14 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       if (!ok) break;
       ptx::tc_fence_after();
       if (j > 0 && changed) {
+        // head_dim 64: this lane's live accumulator columns are h (sub-block a, lanes 0-63) or NH + h (lanes 64-127)
+        const uint32_t o_addr = lane_addr + 2 * NH + ((HD == 64 && half) ? NH : 0);
         uint32_t o[16];
-        tmem_ld16(o, lane_addr + 2 * NH);
+        tmem_ld16(o, o_addr);
         ptx::tmem_wait_ld();
 #pragma unroll
         for (int h = 0; h < G; ++h) o[h] = __float_as_uint(__uint_as_float(o[h]) * corr[h]);
-        tmem_st16(lane_addr + 2 * NH, o);
+        tmem_st16(o_addr, o);
         ptx::tmem_wait_st();
       }
       // P^T[head h][key tid]: K-major rows of 64 keys, 128-byte swizzle
@@ -404,14 +416,29 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
 #pragma unroll
     for (int h = 0; h < 16; ++h) o[h] = 0u;
     if (ok && n_steps > 0) {
-      tmem_ld16(o, lane_addr + 2 * NH);
+      tmem_ld16(o, lane_addr + 2 * NH + ((HD == 64 && (tid >> 6)) ? NH : 0));
       ptx::tmem_wait_ld();
+    }
+    if constexpr (HD == 64) {
+      // O^T[d][h] = (sub-block a's part in lane d) + (sub-block b's part in lane 64 + d): the upper lanes hand theirs
+      // over through the P^T tile, which no product reads any more
+      float* comb = reinterpret_cast<float*>(smem + OFF_PT);       // [64][16]
+      if (tid >= 64) {
+#pragma unroll
+        for (int h = 0; h < G; ++h) comb[(tid - 64) * NH + h] = __uint_as_float(o[h]);
+      }
+      ptx::mbar_arrive(bar(LRED_BAR));
+      ok = ptx::mbar_wait(bar(LRED_BAR), 1, abort_flag) && ok;
+      if (tid < 64) {
+#pragma unroll
+        for (int h = 0; h < G; ++h) o[h] = __float_as_uint(__uint_as_float(o[h]) + comb[tid * NH + h]);
+      }
     }
     const long long pbase = (((long long)b * dm.h_q + (long long)r * G) * n_split + split) * (HD + 2);
 #pragma unroll
     for (int h = 0; h < G; ++h) {
       float* pp = a.partials + pbase + (long long)h * n_split * (HD + 2);
-      pp[2 + tid] = (n_steps > 0) ? __uint_as_float(o[h]) : 0.f;   // thread tid holds O^T[d = tid][h]
+      if (tid < HD) pp[2 + tid] = (n_steps > 0) ? __uint_as_float(o[h]) : 0.f;   // thread tid holds O^T[d = tid][h]
       if (tid == h) {
         pp[0] = (n_steps > 0) ? m[h] * 0.6931471805599453f : -INFINITY;   // the merge works in natural-log units
         pp[1] = misc->lred[0][h] + misc->lred[1][h] + misc->lred[2][h] + misc->lred[3][h];
@@ -452,8 +479,12 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
           const float w = __expf(ms - M);
           Lsum += w * __ldcg(p + s * (HD + 2) + 1);
           const float2* po = reinterpret_cast<const float2*>(p + s * (HD + 2) + 2 + lane * VPL);   // 8-byte aligned
-          const float2 oa = __ldcg(po), ob = __ldcg(po + 1);
-          acc[0] += w * oa.x; acc[1] += w * oa.y; acc[2] += w * ob.x; acc[3] += w * ob.y;
+          const float2 oa = __ldcg(po);
+          acc[0] += w * oa.x; acc[1] += w * oa.y;
+          if constexpr (VPL == 4) {
+            const float2 ob = __ldcg(po + 1);
+            acc[2] += w * ob.x; acc[3] += w * ob.y;
+          }
         }
         const float inv = Lsum > 0.f ? 1.f / Lsum : 0.f;
         __nv_bfloat16* op = a.O + (long long)b * dm.os[0] + (long long)(r * G + h) * dm.os[2] + lane * VPL;
@@ -466,7 +497,7 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
 }
 
 bool make_kv_map(CUtensorMap* out, const void* base, const Dims& dm, const long long* s) {
-  cuuint64_t dims[4] = {(cuuint64_t)HD, (cuuint64_t)dm.h_kv, (cuuint64_t)dm.seq_kv, (cuuint64_t)dm.batch};
+  cuuint64_t dims[4] = {(cuuint64_t)dm.d, (cuuint64_t)dm.h_kv, (cuuint64_t)dm.seq_kv, (cuuint64_t)dm.batch};
   auto st = [](long long e) { return (cuuint64_t)((e > 0 ? e : 8) * 2); };
   cuuint64_t strides[3] = {st(s[2]), st(s[1]), st(s[0])};
   cuuint32_t box[4] = {64u, 1u, (cuuint32_t)(dm.B < SUB ? dm.B : SUB), 1u};   // chunks below 64 tokens: one box per chunk
@@ -477,7 +508,7 @@ bool make_kv_map(CUtensorMap* out, const void* base, const Dims& dm, const long 
 
 // Splits needed so that no thread block owns more than MAX_RANGE sub-blocks (0: shape not served here).
 int decode_sm100_min_splits(const Dims& dm) {
-  if (!dm.decode || dm.dtype != DASH_BF16 || dm.d != HD) return 0;
+  if (!dm.decode || dm.dtype != DASH_BF16 || (dm.d != 64 && dm.d != 128)) return 0;
   if (dm.B != 16 && dm.B != 32 && dm.B != 64 && dm.B != 128) return 0;
   if (dm.qs[2] % 8 != 0 || tensor_map_encoder() == nullptr) return 0;
   if (dm.B < SUB) {
@@ -500,13 +531,15 @@ cudaError_t launch_decode_sm100(const Dims& dm, int n_split, const void* Q, cons
   if (!make_kv_map(&tk, K, dm, dm.ks) || !make_kv_map(&tv, V, dm, dm.vs)) return cudaErrorInvalidValue;
   dim3 grid(n_split, dm.h_kv, dm.batch);
   cudaError_t le = cudaSuccess;
-#define DASH_DEC_TC(G, C)                                                                                       \
+#define DASH_DEC_HD(G, C, H)                                                                                    \
   {                                                                                                             \
     static std::atomic<unsigned long long> configured{0};                                                       \
-    cudaError_t e = allow_dynamic_smem(decode_sm100_kernel<G, C>, DEC_SMEM, configured);                        \
+    cudaError_t e = allow_dynamic_smem(decode_sm100_kernel<G, C, H>, DEC_SMEM, configured);                     \
     if (e != cudaSuccess) return e;                                                                             \
-    le = launch_chained(decode_sm100_kernel<G, C>, grid, dim3(DEC_THREADS), DEC_SMEM, st, tk, tv, a);           \
+    le = launch_chained(decode_sm100_kernel<G, C, H>, grid, dim3(DEC_THREADS), DEC_SMEM, st, tk, tv, a);        \
   }
+#define DASH_DEC_TC(G, C) \
+  if (dm.d == 128) DASH_DEC_HD(G, C, 128) else DASH_DEC_HD(G, C, 64)
 #define DASH_DEC_G(C)                                  \
   switch (dm.g_q) {                                    \
     case 1: DASH_DEC_TC(1, C); break;                  \
@@ -519,6 +552,7 @@ cudaError_t launch_decode_sm100(const Dims& dm, int n_split, const void* Q, cons
   if (dm.B >= SUB) { DASH_DEC_G(1) } else if (dm.B == 32) { DASH_DEC_G(2) } else { DASH_DEC_G(4) }
 #undef DASH_DEC_G
 #undef DASH_DEC_TC
+#undef DASH_DEC_HD
   count_launch();
   return le;
 }

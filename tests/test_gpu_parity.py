@@ -319,6 +319,9 @@ def _decode_case(w, kv_len, use_lists_from_oracle=False, local_blocks=0):
     (dict(kind="decode", batch=3, seq=2500, h_q=8, h_kv=2, head_dim=128, block=32), [2500, 33, 1999]),   # two chunks per sub-block
     (dict(kind="decode", batch=2, seq=1800, h_q=16, h_kv=2, head_dim=128, block=16, alpha=1.25, gamma=2.0), [1800, 1001]),
     (dict(kind="decode", batch=2, seq=9000, h_q=4, h_kv=1, head_dim=128, block=16), [9000, 8191]),      # long lists, four per sub-block
+    (dict(kind="decode", batch=3, seq=4000, h_q=16, h_kv=2, head_dim=64, block=64), [4000, 1, 2049]),   # head_dim 64: stacked sub-blocks
+    (dict(kind="decode", batch=2, seq=3000, h_q=8, h_kv=2, head_dim=64, block=128, alpha=2.0), [2999, 130]),
+    (dict(kind="decode", batch=2, seq=2500, h_q=2, h_kv=1, head_dim=64, block=32), [2500, 1777]),
 ])
 def test_decode_matches_oracle(kw, kv_len):
     w = _wl(**kw)
