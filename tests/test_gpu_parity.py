@@ -167,6 +167,9 @@ def _gather_O(O, keys, g_q):
     dict(), dict(dtype="f32"), dict(h_q=8, h_kv=2, head_dim=128, block=64, seq=1000, sigma=1.0),
     dict(h_q=4, h_kv=4, head_dim=128, block=32, seq=333, alpha=2.0), dict(seq=17), dict(seq=5),
     dict(h_q=16, h_kv=1, head_dim=128, block=128, seq=700, alpha=1.25, gamma=2.0),
+    dict(h_q=8, h_kv=2, head_dim=128, block=32, seq=900, gamma=2.0),     # packed chunks (two per step), every row compared
+    dict(h_q=8, h_kv=1, head_dim=64, block=16, seq=500, gamma=2.0),      # four per step, head_dim 64
+    dict(h_q=4, h_kv=2, head_dim=128, block=16, seq=400, gamma=2.0),     # short tiles (32 live rows)
 ])
 def test_attend_prefill_with_oracle_lists(kw):
     """Stage 2 alone, fed the oracle's own routing: no exclusions, every row must match."""
