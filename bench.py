@@ -99,15 +99,17 @@ def selected_flops_from_count(count: torch.Tensor, B: int, d: int, g_q: int) -> 
 
 
 def executed_flops_from_mask(mask: torch.Tensor, w) -> tuple:
-    """FLOPs the Stage-2 tensor-core kernel executes: it walks, per tile of 128/g_q tokens, the UNION of the
-    rows' routed chunks in 64-token steps, each step costing 4*128*128*64 FLOPs whatever the rows select."""
+    """FLOPs the Stage-2 tensor-core kernel executes: it walks, per tile of min(128/g_q, chunk) tokens, the UNION of
+    the rows' routed chunks in 64-token steps (chunks of 128 tokens take two steps, chunks of 32 / 16 are packed two /
+    four to a step), each step costing 4*128*128*64 FLOPs whatever the rows select."""
     b, h_kv, n, W = mask.shape
     g_q = w.h_q // w.h_kv
-    tq = max(1, 128 // g_q)
-    if n % tq != 0 or tq > w.block:
+    tq = min(max(1, 128 // g_q), w.block)
+    if n % tq != 0:
         return float("nan"), 0
     steps = 0
     sub = max(1, w.block // 64)
+    cps = max(1, 64 // w.block)
     for bb in range(b):                                    # one sequence at a time bounds the temporary
         m = mask[bb].view(h_kv, n // tq, tq, W)
         u = m[:, :, 0, :].clone()
@@ -118,7 +120,8 @@ def executed_flops_from_mask(mask: torch.Tensor, w) -> tuple:
             bits += ((u >> k) & 1).sum(dim=-1)
         own_first = (torch.arange(n // tq, device=mask.device) * tq) % w.block   # offset of the tile in its own chunk
         own_steps = own_first // 64 + 1
-        steps += int(((bits - 1) * sub + own_steps[None, :]).sum().item())
+        routed_steps = (bits - 1) * sub if cps == 1 else (bits - 1 + cps - 1) // cps
+        steps += int((routed_steps + own_steps[None, :]).sum().item())
     return float(steps) * 4.0 * 128 * 128 * 64, steps
 
 

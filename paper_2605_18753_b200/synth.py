@@ -66,6 +66,12 @@ WORKLOADS = {
     # C2: prefill 8K, ~75 % block sparsity
     "prefill_8k": Workload("prefill_8k", "prefill", 1, 8192, 32, 8, 128, 64, 1.5, "bf16", "planted",
                            rho=0.72, shift=2.0),
+    # the 8K prefill with the finer chunks of the paper's chunk-size study (its sparsities there: 75.7 % at 32,
+    # 77.0 % at 16); same tensors' recipe, shift re-calibrated for chunks of 16
+    "prefill_8k_b32": Workload("prefill_8k_b32", "prefill", 1, 8192, 32, 8, 128, 32, 1.5, "bf16", "planted",
+                               rho=0.72, shift=1.78),
+    "prefill_8k_b16": Workload("prefill_8k_b16", "prefill", 1, 8192, 32, 8, 128, 16, 1.5, "bf16", "planted",
+                               rho=0.72, shift=1.77),
     # C3: prefill 64K at ~75 % and ~90 %
     "prefill_64k_s75": Workload("prefill_64k_s75", "prefill", 1, 65536, 32, 8, 128, 64, 1.5, "bf16", "planted",
                                 rho=0.72, shift=1.56),
