@@ -277,7 +277,7 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
     };
 #pragma unroll
     for (int q = 0; q < 2; ++q) {
-      if (do_v) {
+      if (do_v && CPS == 1) {
         load_group(q, 0, bq[q]);
         load_group(q, 4, bn[q]);
       } else {
@@ -328,26 +328,53 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
     int j = own_steps;                 // the own chunk's steps are already under way
     bool ok = true;
     Blk cur, nxt;
-    bool has = pop(nxt);
+    bool has = false;
+    if constexpr (CPS == 1) has = pop(nxt);
     if constexpr (CPS > 1) {
-      // chunks of 32 / 16 tokens: a step packs the next CPS chunks of the union; a short last step repeats its
-      // last chunk with bias -inf
-      while (has && ok) {
-        Blk grp[CPS];
+      // Chunks of 32 / 16 tokens: a step packs the next CPS chunks of the union; a short last step repeats its
+      // last chunk with bias -inf.  A row's bias for a chunk is read straight from its list: the entry number is the
+      // count of the row's routed bits below the chunk (previous words' totals kept in `seen`), so the loads of a
+      // whole step are issued together, before the wait for the stage, and nothing walks the lists entry by entry.
+      int seen[2] = {0, 0};
+      auto routed_bits = [&](uint32_t word) -> uint32_t {    // a row's routed chunks in word w: the own chunk and later ones cleared
+        return w == n_words - 1 ? word & own_word_keep & ~(1u << (c_own & 31)) : word;
+      };
+      bool walking = true;
+      while (walking && ok) {
+        int cs[CPS];
+        float bvs[CPS][2];
         int m = 0;
-        while (m < CPS && has) {
-          cur = nxt;
-          has = pop(nxt);
-          if (cur.c == c_own) { has = false; break; }      // last of the walk, done first
-          grp[m++] = cur;
+        while (m < CPS) {
+          while (u == 0u && walking) {
+            seen[0] += __popc(routed_bits(rw[0]));
+            seen[1] += __popc(routed_bits(rw[1]));
+            if (++w >= n_words) { walking = false; break; }
+            rw[0] = rw_n[0]; rw[1] = rw_n[1];
+            u = union_of(w, rw);
+            if (w + 1 < n_words) load_rows(w + 1, rw_n);
+          }
+          if (!walking) break;
+          const int bit = __ffs(u) - 1;
+          u &= u - 1;
+          const int c = w * 32 + bit;
+          if (c == c_own) { walking = false; break; }        // last of the walk, done first
+          cs[m] = c;
+#pragma unroll
+          for (int q = 0; q < 2; ++q) {
+            const uint32_t rb = routed_bits(rw[q]);
+            const bool member = do_v && ((rb >> bit) & 1u);
+            const int e = seen[q] + __popc(rb & ((1u << bit) - 1u));
+            bvs[m][q] = member ? __ldg(a.blk_bias + loff[q] + e) : -INFINITY;
+          }
+          ++m;
         }
         if (m == 0) break;
 #pragma unroll
         for (int s = 1; s < CPS; ++s)
-          if (s >= m) { grp[s].c = grp[m - 1].c; grp[s].bv[0] = grp[s].bv[1] = -INFINITY; }
+          if (s >= m) { cs[s] = cs[m - 1]; bvs[s][0] = bvs[s][1] = -INFINITY; }
         int kvs[CPS];
 #pragma unroll
-        for (int s = 0; s < CPS; ++s) kvs[s] = grp[s].c * dm.B;
+        for (int s = 0; s < CPS; ++s) kvs[s] = cs[s] * dm.B;
         const int st = j & 1, prev_ph = ((j >> 1) - 1) & 1;
         if (do_k) {
           if (j >= 2) ok = ptx::mbar_wait(bar(S_FULL + st), prev_ph, abort_flag);
@@ -360,7 +387,7 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
           for (int s = 0; s < CPS; ++s)
             for (int q = 0; q < 2; ++q) {
               const int t = lane + 32 * q;
-              if (t < TR) misc->bias[st][s][t] = t < TQ ? grp[s].bv[q] : -INFINITY;
+              if (t < TR) misc->bias[st][s][t] = t < TQ ? bvs[s][q] : -INFINITY;
             }
 #pragma unroll
           for (int s = 0; s < CPS; ++s)
@@ -370,7 +397,6 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
         }
         ++j;
       }
-      has = false;
     }
     while (has && ok) {
       cur = nxt;
