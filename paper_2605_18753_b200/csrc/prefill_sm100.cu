@@ -15,7 +15,8 @@
 //   warp 4     K producer: TMA loads of Q and of the K tiles (128-byte swizzle, no multicast); OR of the tile's
 //              mask words = union list.
 //   warp 6     V producer: walks the same union list; TMA loads of the V tiles and the per-token bias of each
-//              step (each lane walks its tokens' compact bias lists with register-buffered cursors).
+//              step (a row's list entry for a chunk = its routed bits below the chunk + the totals of the earlier mask
+//              words: read by direct index, a whole step's loads issued together before the wait for the stage).
 //   warp 5     MMA issuer: S_{j+1} = Q K_{j+1}^T (M128 N64 K128) into one of two TMEM buffers, then O += P_j V_j
 //              (M128 N128 K64, P from TMEM); one tcgen05.commit per product, to the mbarrier that the softmax
 //              warps and the producer of the stage both listen to; owns the TMEM allocation.
@@ -246,8 +247,7 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
       misc->n_steps = n_steps;
       ptx::mbar_arrive(bar(META));
     }
-    // per-lane cursors into the compact bias lists of this lane's tokens (lane t owns tokens t and t+32)
-    int cursor[2] = {0, 0};
+    // start of the compact bias lists of this lane's tokens (lane t owns tokens t and t+32)
     long long loff[2];
     for (int q = 0; q < 2; ++q) {
       const int t = lane + 32 * q;
@@ -265,76 +265,20 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
       if (w == n_words - 1) u = (u & own_word_keep) | (1u << (c_own & 31));
       return u;
     };
-    // Bias list entries are consumed in order, so every lane keeps the next 4..8 entries of each of its
-    // rows in registers (two groups of four; the second group is loading while the first is consumed).
-    // A dependent global read per step would otherwise put a DRAM latency on every step of the walk.
-    float bq[2][4], bn[2][4];
-    int taken[2] = {0, 0};                 // entries of the current group already handed out
-    const int row_cap = c_own;             // list entries a row can hold (= its candidate count)
-    auto load_group = [&](int q, int first, float* dst) {
-#pragma unroll
-      for (int k = 0; k < 4; ++k) dst[k] = (first + k < row_cap) ? __ldg(a.blk_bias + loff[q] + first + k) : 0.f;
-    };
-#pragma unroll
-    for (int q = 0; q < 2; ++q) {
-      if (do_v && CPS == 1) {
-        load_group(q, 0, bq[q]);
-        load_group(q, 4, bn[q]);
-      } else {
-#pragma unroll
-        for (int k = 0; k < 4; ++k) bq[q][k] = bn[q][k] = 0.f;
-      }
-    }
-    auto take = [&](int q) -> float {
-      const int k = taken[q];
-      const float v = k == 0 ? bq[q][0] : k == 1 ? bq[q][1] : k == 2 ? bq[q][2] : bq[q][3];
-      ++cursor[q];
-      if (++taken[q] == 4) {
-        taken[q] = 0;
-#pragma unroll
-        for (int kk = 0; kk < 4; ++kk) bq[q][kk] = bn[q][kk];
-        load_group(q, cursor[q] + 4, bn[q]);
-      }
-      return v;
-    };
-    // The walk is a generator of (chunk, per-token bias) pairs; mask words are read one word ahead.
-    struct Blk { int c; float bv[2]; };
+    // The walk pops the chunks of the union in ascending order; mask words are read one word ahead.
     int w = 0;
     uint32_t rw[2], rw_n[2] = {0u, 0u};
     load_rows(0, rw);
     uint32_t u = union_of(0, rw);
     if (n_words > 1) load_rows(1, rw_n);
-    auto pop = [&](Blk& out) -> bool {
-      while (u == 0u) {
-        if (++w >= n_words) return false;
-        rw[0] = rw_n[0]; rw[1] = rw_n[1];
-        u = union_of(w, rw);
-        if (w + 1 < n_words) load_rows(w + 1, rw_n);
-      }
-      const int bit = __ffs(u) - 1;
-      u &= u - 1;
-      out.c = w * 32 + bit;
-#pragma unroll
-      for (int q = 0; q < 2; ++q) {
-        out.bv[q] = -INFINITY;
-        if (out.c == c_own) {
-          out.bv[q] = 0.f;
-        } else if (do_v && ((rw[q] >> bit) & 1u)) {
-          out.bv[q] = take(q);
-        }
-      }
-      return true;
-    };
     int j = own_steps;                 // the own chunk's steps are already under way
     bool ok = true;
-    Blk cur, nxt;
-    bool has = false;
-    if constexpr (CPS == 1) has = pop(nxt);
-    if constexpr (CPS > 1) {
-      // Chunks of 32 / 16 tokens: a step packs the next CPS chunks of the union; a short last step repeats its
-      // last chunk with bias -inf.  A row's bias for a chunk is read straight from its list: the entry number is the
-      // count of the row's routed bits below the chunk (previous words' totals kept in `seen`), so the loads of a
-      // whole step are issued together, before the wait for the stage, and nothing walks the lists entry by entry.
+    {
+      // A step takes the next CPS chunks of the union (CPS > 1: chunks of 32 / 16 tokens packed into the 64-token
+      // step; a short last step repeats its last chunk with bias -inf).  A row's bias for a chunk is read straight
+      // from its list: the entry number is the count of the row's routed bits below the chunk (previous words'
+      // totals kept in `seen`), so the loads of a whole step are issued together, before the wait for the stage,
+      // and nothing walks the lists entry by entry.
       int seen[2] = {0, 0};
       auto routed_bits = [&](uint32_t word) -> uint32_t {    // a row's routed chunks in word w: the own chunk and later ones cleared
         return w == n_words - 1 ? word & own_word_keep & ~(1u << (c_own & 31)) : word;
@@ -372,65 +316,31 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
 #pragma unroll
         for (int s = 1; s < CPS; ++s)
           if (s >= m) { cs[s] = cs[m - 1]; bvs[s][0] = bvs[s][1] = -INFINITY; }
-        int kvs[CPS];
+        // chunks of 128 tokens take two 64-token steps with the same bias
+        for (int sub = 0; sub < (CPS > 1 ? 1 : sub_per_blk) && ok; ++sub, ++j) {
+          int kvs[CPS];
 #pragma unroll
-        for (int s = 0; s < CPS; ++s) kvs[s] = cs[s] * dm.B;
-        const int st = j & 1, prev_ph = ((j >> 1) - 1) & 1;
-        if (do_k) {
-          if (j >= 2) ok = ptx::mbar_wait(bar(S_FULL + st), prev_ph, abort_flag);
-          if (!ok) break;
-          if (lane == 0) load_packed(&tmK, sbase + OFF_K + st * KV_TILE_BYTES, bar(K_FULL + st), kvs);
-        } else {
-          if (j >= 2) ok = ptx::mbar_wait(bar(PV_DONE + st), prev_ph, abort_flag);
-          if (!ok) break;
+          for (int s = 0; s < CPS; ++s) kvs[s] = cs[s] * dm.B + sub * NKV;
+          const int st = j & 1, prev_ph = ((j >> 1) - 1) & 1;   // stage, and the phase of step j-2 on the completion barriers
+          if (do_k) {
+            if (j >= 2) ok = ptx::mbar_wait(bar(S_FULL + st), prev_ph, abort_flag);     // QK of step j-2 has read the stage
+            if (!ok) break;
+            if (lane == 0) load_packed(&tmK, sbase + OFF_K + st * KV_TILE_BYTES, bar(K_FULL + st), kvs);
+          } else {
+            if (j >= 2) ok = ptx::mbar_wait(bar(PV_DONE + st), prev_ph, abort_flag);    // PV of step j-2 has read the stage
+            if (!ok) break;
 #pragma unroll
-          for (int s = 0; s < CPS; ++s)
-            for (int q = 0; q < 2; ++q) {
-              const int t = lane + 32 * q;
-              if (t < TR) misc->bias[st][s][t] = t < TQ ? bvs[s][q] : -INFINITY;
-            }
+            for (int s = 0; s < CPS; ++s)
+              for (int q = 0; q < 2; ++q) {
+                const int t = lane + 32 * q;
+                if (t < TR) misc->bias[st][s][t] = t < TQ ? bvs[s][q] : -INFINITY;
+              }
 #pragma unroll
-          for (int s = 0; s < CPS; ++s)
-            if (lane == s) misc->kvbase[st][s] = kvs[s];
-          __syncwarp();
-          if (lane == 0) load_packed(&tmV, sbase + OFF_V + st * KV_TILE_BYTES, bar(V_FULL + st), kvs);
-        }
-        ++j;
-      }
-    }
-    while (has && ok) {
-      cur = nxt;
-      has = pop(nxt);
-      if (cur.c == c_own) break;       // last of the walk, done first
-      const int nsub = sub_per_blk;
-      for (int sub = 0; sub < nsub && ok; ++sub, ++j) {
-        const int kv0 = cur.c * dm.B + sub * NKV;
-        const int st = j & 1, prev_ph = ((j >> 1) - 1) & 1;   // stage, and the phase of step j-2 on the completion barriers
-        if (do_k) {
-          if (j >= 2) ok = ptx::mbar_wait(bar(S_FULL + st), prev_ph, abort_flag);   // QK of step j-2 has read the stage
-          if (!ok) break;
-          if (lane == 0) {
-            const uint32_t dst = sbase + OFF_K + st * KV_TILE_BYTES;
-            ptx::mbar_arrive_expect_tx(bar(K_FULL + st), KV_TILE_BYTES);
-            ptx::tma_load_4d(dst, &tmK, bar(K_FULL + st), 0, r, kv0, b);
-            if constexpr (HD == 128) ptx::tma_load_4d(dst + KV_TILE_BYTES / 2, &tmK, bar(K_FULL + st), 64, r, kv0, b);
+            for (int s = 0; s < CPS; ++s)
+              if (lane == s) misc->kvbase[st][s] = kvs[s];
+            __syncwarp();
+            if (lane == 0) load_packed(&tmV, sbase + OFF_V + st * KV_TILE_BYTES, bar(V_FULL + st), kvs);
           }
-          continue;
-        }
-        const int vs = st;
-        if (j >= 2) ok = ptx::mbar_wait(bar(PV_DONE + st), prev_ph, abort_flag);     // PV of step j-2 has read the stage
-        if (!ok) break;
-        for (int q = 0; q < 2; ++q) {
-          const int t = lane + 32 * q;
-          if (t < TR) misc->bias[vs][0][t] = t < TQ ? cur.bv[q] : -INFINITY;
-        }
-        if (lane == 0) misc->kvbase[vs][0] = kv0;
-        __syncwarp();
-        if (lane == 0) {
-          const uint32_t dst = sbase + OFF_V + vs * KV_TILE_BYTES;
-          ptx::mbar_arrive_expect_tx(bar(V_FULL + vs), KV_TILE_BYTES);
-          ptx::tma_load_4d(dst, &tmV, bar(V_FULL + vs), 0, r, kv0, b);
-          if constexpr (HD == 128) ptx::tma_load_4d(dst + KV_TILE_BYTES / 2, &tmV, bar(V_FULL + vs), 64, r, kv0, b);
         }
       }
     }
