@@ -441,7 +441,7 @@ def main():
                 "unit": "TFLOP/s", "frac": achieved / peak_tf, "peak_source": f"{peaks['_source']} bf16 burst",
                 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of this kernel on this workload, from the
                 # ncu capture summarised in profiles/attend_prefill_sm100_prefill_8k.md (112.3 MB + 33.6 MB)
-                "traffic": 143.9e6 if w.name == "prefill_8k" else None}
+                "traffic": 142.8e6 if w.name == "prefill_8k" else None}
     extras = {"fwd_ms": ms, "stage_ms": stage_ms, "block_sparsity": sparsity, "selected_tflop": f_sel / 1e12,
               "executed_tflop": executed / 1e12, "union_inflation": executed / f_sel, "tile_steps": n_steps_total,
               "stage2_executed_tflops": executed / (stage_ms["attend"] * 1e-3) / 1e12,
