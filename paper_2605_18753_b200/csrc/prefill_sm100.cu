@@ -232,14 +232,29 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
     const int n_words = (c_own >> 5) + 1;
     const long long row0 = ((long long)b * dm.h_kv + r) * dm.seq_q;
     const uint32_t own_word_keep = (c_own & 31) == 31 ? 0xffffffffu : ((2u << (c_own & 31)) - 1u);
+    // four mask words per sweep: a lane's eight loads are in flight together (one L2 round trip per four words
+    // instead of one per word; the step count below is what the MMA thread waits for before its second product)
     int total = 0;
-    for (int w = 0; w < n_words; ++w) {
-      uint32_t u = 0;
-      for (int t = lane; t < TQ; t += 32)
-        if (i0 + t < dm.seq_q) u |= a.mask[(row0 + i0 + t) * dm.W + w];
-      u = __reduce_or_sync(0xffffffffu, u);
-      if (w == n_words - 1) u = (u & own_word_keep) | (1u << (c_own & 31));  // own chunk: always, and last
-      total += __popc(u);
+    for (int w0 = 0; w0 < n_words; w0 += 4) {
+      uint32_t uu[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+      for (int q = 0; q < 2; ++q) {
+        const int t = lane + 32 * q;
+        if (t < TQ && i0 + t < dm.seq_q) {
+          const uint32_t* mp = a.mask + (row0 + i0 + t) * dm.W + w0;
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            if (w0 + k < n_words) uu[k] |= mp[k];
+        }
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        if (w0 + k < n_words) {
+          uint32_t u = __reduce_or_sync(0xffffffffu, uu[k]);
+          if (w0 + k == n_words - 1) u = (u & own_word_keep) | (1u << (c_own & 31));  // own chunk: always, and last
+          total += __popc(u);
+        }
+      }
     }
     // the own chunk is always in the union (its bit is set in every row); it contributes own_steps steps
     const int n_steps = CPS > 1 ? (total - 1 + CPS - 1) / CPS + own_steps : (total - 1) * sub_per_blk + own_steps;
