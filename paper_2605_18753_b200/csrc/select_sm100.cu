@@ -1,6 +1,7 @@
-// Stage 1 on tensor cores for sm_100a (Eq. 2, Eq. 4, Algorithm 2, Proposition 1), bf16 queries, head_dim 128.
+// Stage 1 on tensor cores for sm_100a (Eq. 2, Eq. 4, Algorithm 2, Proposition 1), bf16 queries, head_dim 128 or 64.
 //
-// Tile = the 128 (token, head-of-group) rows of TQ = 128/g_q consecutive tokens of one (batch, KV head);
+// Tile = the (token, head-of-group) rows of TQ = min(128/g_q, chunk size) consecutive tokens of one (batch, KV head):
+// 128 rows, or fewer live rows followed by zero-query padding when chunks are shorter than 128/g_q tokens;
 // they share their candidate chunks.  The whole score tile X[128 rows][<= 512 chunks per block] is produced by
 // tcgen05.mma into tensor memory and never leaves the SM (Algorithm 2 writes it to HBM).  The fp32
 // summaries are split beforehand into three bf16 planes (hi + mid + lo = the fp32 value exactly), so that
@@ -193,15 +194,16 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         ok = ptx::mbar_wait(bar(KB_FULL + s), (cb / NST) & 1, abort_flag);
         if (!ok) break;
         ptx::tc_fence_after();
-        const uint32_t qa = sbase + SP::OFF_Q;
+        // descriptors differ only in the start-address field (16-byte units, no carry into the next field): built once
+        // per stage, then one add per MMA keeps the issuing thread's instruction stream short
+        const uint64_t qd0 = ptx::smem_desc_sw128(sbase + SP::OFF_Q, 16, 1024);
+        const uint64_t kd0 = ptx::smem_desc_sw128(sbase + SP::OFF_KB + s * STAGE_BYTES, 16, 1024);
 #pragma unroll
         for (int pl = 0; pl < 3; ++pl) {
-          const uint32_t ka = sbase + SP::OFF_KB + s * STAGE_BYTES + pl * PLANE_BYTES;
 #pragma unroll
           for (int k = 0; k < HD / 16; ++k) {
-            const uint32_t koff = (k & 3) * 32;
-            const uint64_t ad = ptx::smem_desc_sw128(qa + (k >> 2) * (Q_BYTES / 2) + koff, 16, 1024);
-            const uint64_t bd = ptx::smem_desc_sw128(ka + (k >> 2) * (PLANE_BYTES / 2) + koff, 16, 1024);
+            const uint64_t ad = qd0 + (uint64_t)(((k >> 2) * (Q_BYTES / 2) + (k & 3) * 32) >> 4);
+            const uint64_t bd = kd0 + (uint64_t)((pl * PLANE_BYTES + (k >> 2) * (PLANE_BYTES / 2) + (k & 3) * 32) >> 4);
             ptx::mma_bf16_ss(tmem + cb * SC, ad, bd, IDESC, (pl > 0 || k > 0) ? 1u : 0u);
           }
         }
