@@ -21,7 +21,11 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 import numpy as np
-import torch
+
+try:                                  # oracle worker processes (spawned) re-import this file and need numpy only
+    import torch
+except Exception:  # pragma: no cover
+    torch = None
 
 METRIC = "dashattention_prefill_fwd_effective_tflops"
 UNIT = "TFLOP/s"
@@ -131,28 +135,79 @@ def sparsity_from_count(count: torch.Tensor, B: int) -> float:
     return float(1.0 - (count.to(torch.float64) + 1).sum().item() / ((vis + 1).sum().item() * count.shape[0] * count.shape[1]))
 
 
-def time_oracle_sample(w, inp, budget_s: float = 15.0):
-    """Times the oracle (as it stands, one thread) on a seeded sample of rows of the workload.
-    Returns (TFLOP/s on selected FLOPs, rows done, seconds)."""
-    from oracle import dash_oracle as orc
+def host_cores() -> int:
+    try:
+        return max(1, len(os.sched_getaffinity(0)))
+    except AttributeError:  # pragma: no cover
+        return max(1, os.cpu_count() or 1)
+
+
+def _oracle_worker(job):
+    """One host core's share of the oracle timing: whole oracle rows (Stage 1 + Stage 2 of one query row and KV
+    head, float64) of random positions of the workload until the budget is spent.  Runs in its own process."""
+    path, wd, seed, budget_s = job
     from threadpoolctl import threadpool_limits
-    Qn = inp["Q"][0].cpu().double().numpy()
-    Kn = inp["K"][0].cpu().double().numpy()
-    Vn = inp["V"][0].cpu().double().numpy()
-    rng = np.random.default_rng(0)
-    g_q = w.h_q // w.h_kv
+    from oracle import dash_oracle as orc
+    Qn, Kn, Vn = (np.load(os.path.join(path, f"{k}.npy"), mmap_mode="r") for k in "QKV")
+    rng = np.random.default_rng(seed)
+    g_q = wd["h_q"] // wd["h_kv"]
     flops, rows = 0.0, 0
     with threadpool_limits(limits=1):
         t0 = time.perf_counter()
-        Kbar = orc.block_summaries(Kn, w.block)
+        Kbar = orc.block_summaries(Kn, wd["block"])
         while time.perf_counter() - t0 < budget_s:
-            i = int(rng.integers(0, w.seq))
-            r = int(rng.integers(0, w.h_kv))
-            rt, _ = orc.forward_row(Qn, Kn, Vn, Kbar, i, r, B=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma)
-            flops += 4.0 * w.head_dim * g_q * (w.block * rt.support.size + (i % w.block) + 1)
+            i = int(rng.integers(0, wd["seq"]))
+            r = int(rng.integers(0, wd["h_kv"]))
+            rt, _ = orc.forward_row(Qn, Kn, Vn, Kbar, i, r, B=wd["block"], alpha=wd["alpha"], gamma=wd["gamma"],
+                                    sigma=wd["sigma"])
+            flops += 4.0 * wd["head_dim"] * g_q * (wd["block"] * rt.support.size + (i % wd["block"]) + 1)
             rows += 1
         dt = time.perf_counter() - t0
-    return flops / dt / 1e12, rows, dt
+    return flops, rows, dt
+
+
+class OraclePool:
+    """The oracle, as it stands, on every host core: one single-threaded process per core, each timing its own
+    random sample of rows of the same tensors (float64 copies of sequence 0, shared through memory-mapped files)."""
+
+    def __init__(self, w, inp):
+        import multiprocessing as mp
+        import tempfile
+        self.w = w
+        self.cores = host_cores()
+        base = "/dev/shm" if os.path.isdir("/dev/shm") and os.access("/dev/shm", os.W_OK) else None
+        self.tmp = tempfile.TemporaryDirectory(prefix="dash_oracle_", dir=base)
+        for k in "QKV":
+            np.save(os.path.join(self.tmp.name, f"{k}.npy"), inp[k][0].detach().cpu().double().numpy())
+        self.pool = mp.get_context("spawn").Pool(self.cores)
+        self.pool.map(_oracle_warm, range(self.cores))             # imports done before anything is timed
+
+    def run(self, budget_s: float, seed0: int = 0):
+        """Returns (TFLOP/s on selected-token FLOPs summed over the cores, rows done, wall seconds)."""
+        wd = self.w.as_dict()
+        t0 = time.perf_counter()
+        res = self.pool.map(_oracle_worker, [(self.tmp.name, wd, seed0 * 1000 + c, budget_s) for c in range(self.cores)])
+        wall = time.perf_counter() - t0
+        return sum(r[0] for r in res) / wall / 1e12, sum(r[1] for r in res), wall
+
+    def close(self):
+        self.pool.close()
+        self.pool.join()
+        self.tmp.cleanup()
+
+
+def _oracle_warm(_):
+    from threadpoolctl import threadpool_limits  # noqa: F401
+    from oracle import dash_oracle  # noqa: F401
+    return 0
+
+
+def config_dict(w, world: int) -> dict:
+    """The workload description both arms print (same keys, same values)."""
+    return {"workload": w.name, "batch_per_gpu": w.batch, "seq": w.seq, "h_q": w.h_q, "h_kv": w.h_kv,
+            "head_dim": w.head_dim, "block": w.block, "alpha": w.alpha, "gamma": w.gamma, "sigma": w.sigma,
+            "rho": w.rho, "shift": w.shift, "l2": "256 MiB buffer written between timed iterations",
+            "parallelism": f"independent batches x{world}"}
 
 
 def run_reference(args, w):
@@ -161,20 +216,24 @@ def run_reference(args, w):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
+    world = int(os.environ.get("WORLD_SIZE", str(args.gpus)))
     inp = synth.make_prefill_inputs(w.with_(batch=1), "cpu")
     per_step = max(2.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
+    pool = OraclePool(w, inp)
     vals, rows = [], 0
     for s in range(args.warmup + args.steps):
-        v, r, dt = time_oracle_sample(w, inp, per_step)
+        v, r, dt = pool.run(per_step, seed0=s)
         if s >= args.warmup:
             vals.append(v); rows += r
+    pool.close()
     value = float(np.mean(vals))
-    sample = f"{rows} random (row, KV head) pairs of {w.name} in {args.steps} steps of {per_step:.0f} s, whole oracle row each"
-    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+    sample = (f"{rows} random (row, KV head) pairs of {w.name} in {args.steps} steps of {per_step:.0f} s on "
+              f"{pool.cores} single-threaded processes, whole oracle row each")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": per_step * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": w.name, **{k: getattr(w, k) for k in ("batch", "seq", "h_q", "h_kv", "head_dim", "block", "alpha", "gamma", "sigma")}},
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+            "config": config_dict(w, world),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": pool.cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line), flush=True)
@@ -279,6 +338,189 @@ def run_paper_protocol(args):
                       "data": "random tensors, random chunk masks", "rows": rows}), flush=True)
 
 
+def self_launch(args) -> int:
+    """`python bench.py --gpus N` with N > 1 and no launcher around it: start the N ranks here (one process per GPU
+    through torch.distributed.run on the loopback address) and return their exit code."""
+    import socket
+    import subprocess
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
+def stats(xs) -> dict:
+    return {"mean": float(np.mean(xs)), "median": float(np.median(xs)), "min": float(np.min(xs))}
+
+
+def load_traffic(workload: str):
+    """DRAM bytes of one Stage-2 launch (dram__bytes_read.sum + dram__bytes_write.sum) from the tracked ncu summary
+    of this workload, or None when there is none."""
+    path = os.path.join(ROOT, "profiles", f"attend_prefill_{workload}.json")
+    if not os.path.exists(path):
+        return None
+    with open(path) as f:
+        d = json.load(f)
+    return float(d["dram_bytes_read"]) + float(d["dram_bytes_write"])
+
+
+def measure_prefill(B, synth, w, dev, peaks, iters: int, warm: int = 3, flush=None, with_sdpa=True, tensors=None,
+                    sdpa_ms=None) -> dict:
+    """One prefill workload: whole forward and the three stages (CUDA events, L2 flushed between iterations), workload
+    statistics from the routing outputs, dense SDPA on the same tensors, and the clocks sampled meanwhile."""
+    sampler = ClockSampler(dev.index or 0)
+    sampler.start()
+    inp = tensors if tensors is not None else synth.make_prefill_inputs(w, dev)
+    Q, K, V = inp["Q"], inp["K"], inp["V"]
+    O = torch.empty_like(Q)
+    p = B.params_for_prefill(Q, K, V, O, block=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma)
+    ws, rt, kbar = B.alloc_workspace(p, dev), B.alloc_routing(p, dev), B.alloc_kbar(p, dev)
+    g_q = w.h_q // w.h_kv
+    for _ in range(warm):
+        flush.fill_(1)
+        B.dash_attn_fwd_prefill(p, Q, K, V, O, ws)
+    torch.cuda.synchronize()
+    fwd, st = [], {"summaries": [], "select": [], "attend": []}
+    for s in range(iters):
+        flush.fill_(s & 0xFF)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(); B.dash_attn_fwd_prefill(p, Q, K, V, O, ws); b.record()
+        torch.cuda.synchronize()
+        fwd.append(a.elapsed_time(b))
+    for s in range(iters):
+        flush.fill_(s & 0xFF)
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+        e[0].record()
+        B.dash_attn_block_summaries(p, K, kbar)
+        e[1].record()
+        B.dash_attn_select(p, Q, kbar, rt["mask"], rt["count"], None, rt["blk_bias"], ws)
+        e[2].record()
+        B.dash_attn_attend_prefill(p, Q, K, V, rt["mask"], rt["blk_bias"], O, ws)
+        e[3].record()
+        torch.cuda.synchronize()
+        for k, name in enumerate(("summaries", "select", "attend")):
+            st[name].append(e[k].elapsed_time(e[k + 1]))
+    assert B.dash_attn_last_status(ws) == 0, "device-side error reported by the library"
+    f_sel = selected_flops_from_count(rt["count"], w.block, w.head_dim, g_q)
+    executed, n_steps = executed_flops_from_mask(rt["mask"], w)
+    att = float(np.median(st["attend"]))
+    out = {"workload": w.name, "batch": w.batch, "seq": w.seq, "block": w.block, "alpha": w.alpha, "shift": w.shift,
+           "fwd_ms": stats(fwd), "stage_ms": {k: stats(v) for k, v in st.items()},
+           "block_sparsity": sparsity_from_count(rt["count"], w.block),
+           "selected_tflop": f_sel / 1e12, "executed_tflop": executed / 1e12, "union_inflation": executed / f_sel,
+           "fwd_selected_tflops": f_sel / (float(np.median(fwd)) * 1e-3) / 1e12,
+           "stage2_selected_tflops": f_sel / (att * 1e-3) / 1e12,
+           "stage2_frac": f_sel / (att * 1e-3) / 1e12 / float(peaks["bf16_tflops"]),
+           "stage2_executed_frac": executed / (att * 1e-3) / 1e12 / float(peaks["bf16_tflops"]),
+           "dense_causal_tflop": 4.0 * w.head_dim * w.h_q * w.batch * w.seq * (w.seq + 1) / 2.0 / 1e12}
+    del ws, rt, kbar
+    if with_sdpa:
+        if sdpa_ms is None:
+            q, k, v = (t.transpose(1, 2) for t in (Q, K, V))
+            sd = lambda: torch.nn.functional.scaled_dot_product_attention(q, k, v, is_causal=True, enable_gqa=True)
+            for _ in range(2):
+                sd()
+            ts = []
+            for s in range(max(3, iters // 2)):
+                flush.fill_(s)
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(); sd(); b.record()
+                torch.cuda.synchronize()
+                ts.append(a.elapsed_time(b))
+            sdpa_ms = float(np.median(ts))
+        out["sdpa_dense_ms"] = sdpa_ms
+        out["speedup_vs_dense_sdpa"] = sdpa_ms / float(np.median(fwd))
+    out["clocks"] = sampler.stop()
+    return out
+
+
+def measure_decode(B, synth, wd, dev, peaks, flush, iters=30) -> dict:
+    """The decode workload: whole step, its two stages, bytes actually touched, dense q-len-1 SDPA."""
+    sampler = ClockSampler(dev.index or 0)
+    sampler.start()
+
+    def timed(fn, iters=iters, warm=3):
+        for _ in range(warm):
+            fn()
+        ts = []
+        for k in range(iters):
+            flush.fill_(k & 0xFF)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); fn(); b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        return stats(ts)
+
+    di = synth.make_decode_inputs(wd, dev)
+    qd, Kc, Vc, lens = di["Q"], di["K"], di["V"], di["kv_len"]
+    od = torch.empty_like(qd)
+    pd = B.params_for_decode(qd, Kc, Vc, od, block=wd.block, alpha=wd.alpha, gamma=wd.gamma, sigma=wd.sigma)
+    kbar = B.alloc_kbar(pd, dev)
+    t_sum = timed(lambda: B.dash_attn_block_summaries(pd, Kc, kbar, kv_len=lens), iters=3, warm=1)
+    wsd = B.alloc_workspace(pd, dev)
+    rt = B.alloc_routing(pd, dev)
+    B.dash_attn_select(pd, qd, kbar, rt["mask"], rt["count"], rt["blk_idx"], rt["blk_bias"], wsd, kv_len=lens)
+    cnt = rt["count"].to(torch.float64)
+    g = wd.batch * wd.h_kv
+    diag = ((lens.to(torch.float64) - 1) % wd.block + 1).sum().item() * wd.h_kv
+    kv_bytes = (cnt.sum().item() * wd.block + diag) * wd.head_dim * 2 * 2
+    kbar_bytes = g * ((wd.seq - 1) // wd.block) * wd.head_dim * 4
+    t_sel = timed(lambda: B.dash_attn_select(pd, qd, kbar, rt["mask"], rt["count"], rt["blk_idx"], rt["blk_bias"], wsd, kv_len=lens))
+    t_att = timed(lambda: B.dash_attn_attend_decode(pd, qd, Kc, Vc, lens, rt["count"], rt["blk_idx"], rt["blk_bias"], od, wsd))
+    t_all = timed(lambda: B.dash_attn_fwd_decode(pd, qd, Kc, Vc, kbar, lens, od, wsd))
+    assert B.dash_attn_last_status(wsd) == 0
+    hbm = float(peaks["hbm_gbs"])
+    out = {"workload": wd.name, "batch": wd.batch, "seq": wd.seq, "fwd_ms": t_all, "select_ms": t_sel, "attend_ms": t_att,
+           "summaries_ms_whole_cache": t_sum,
+           "block_sparsity": float(1.0 - (cnt + 1).sum().item() / (g * ((wd.seq - 1) // wd.block + 1))),
+           "bytes_touched": kv_bytes + kbar_bytes,
+           "hbm_gbs_fwd": (kv_bytes + kbar_bytes) / (t_all["median"] * 1e-3) / 1e9,
+           "hbm_gbs_fwd_best": (kv_bytes + kbar_bytes) / (t_all["min"] * 1e-3) / 1e9,
+           "hbm_gbs_attend_kv_only": kv_bytes / (t_att["median"] * 1e-3) / 1e9,
+           "hbm_frac_fwd": (kv_bytes + kbar_bytes) / (t_all["median"] * 1e-3) / 1e9 / hbm,
+           "hbm_frac_fwd_mean": (kv_bytes + kbar_bytes) / (t_all["mean"] * 1e-3) / 1e9 / hbm,
+           "hbm_peak_gbs": hbm}
+    kd = Kc.transpose(1, 2); vd = Vc.transpose(1, 2); q1 = qd[:, :, None, :]
+    out["sdpa_dense_ms"] = timed(lambda: torch.nn.functional.scaled_dot_product_attention(q1, kd, vd, enable_gqa=True), iters=5)["median"]
+    out["speedup_vs_dense_sdpa"] = out["sdpa_dense_ms"] / t_all["median"]
+    out["clocks"] = sampler.stop()
+    return out
+
+
+def all_config_measurements(B, synth, dev, peaks, flush) -> dict:
+    """Every other configuration of the task beside the headline: the 64K prefill at two sparsities, the
+    (chunk size, alpha) sweep at 32K x batch 2, the 8K prefill with finer chunks, and the decode workload."""
+    out = {}
+
+    def guarded(name, fn):
+        try:
+            out[name] = fn()
+        except Exception as ex:  # a side measurement never breaks the contract line
+            out[name] = {"error": repr(ex)}
+        torch.cuda.empty_cache()
+
+    for name in ("prefill_64k_s75", "prefill_64k_s90"):
+        guarded(name, lambda name=name: measure_prefill(B, synth, synth.workload(name), dev, peaks, iters=6, flush=flush))
+    sdpa = {}
+    for blk in (64, 128):
+        for alpha in (1.25, 1.5, 2.0):
+            w = synth.workload("sweep_32k", block=blk, alpha=alpha)
+            key = f"sweep_32k_b{blk}_a{alpha}"
+
+            def run(w=w):
+                r = measure_prefill(B, synth, w, dev, peaks, iters=4, flush=flush, sdpa_ms=sdpa.get("ms"))
+                sdpa.setdefault("ms", r.get("sdpa_dense_ms"))        # the dense baseline does not depend on B or alpha
+                return r
+            guarded(key, run)
+    for name in ("prefill_8k_b32", "prefill_8k_b16"):
+        guarded(name, lambda name=name: measure_prefill(B, synth, synth.workload(name), dev, peaks, iters=10, flush=flush,
+                                                        with_sdpa=False))
+    guarded("decode_128k", lambda: measure_decode(B, synth, synth.workload("decode_128k"), dev, peaks, flush))
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -286,7 +528,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="prefill_8k")
-    ap.add_argument("--no-extras", action="store_true", help="skip the SDPA / decode / long-context side measurements")
+    ap.add_argument("--no-extras", action="store_true", help="skip the other configurations and the dense-SDPA side numbers")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--paper-protocol", action="store_true",
                     help="secondary: the paper's Stage-2 speed protocol (random masks, 32/2 heads) instead of the contract line")
@@ -294,6 +536,8 @@ def main():
     if args.paper_protocol:
         run_paper_protocol(args)
         return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(self_launch(args))
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
     from paper_2605_18753_b200 import synth
@@ -358,7 +602,7 @@ def main():
     ms_local = float(np.mean(step_ms))
 
     # per-stage timing (same steps, stages called one by one through the C ABI) and workload statistics
-    stage_ms = {"summaries": [], "select": [], "attend": []}
+    stage_all = {"summaries": [], "select": [], "attend": []}
     for s in range(args.steps):
         flush.fill_(s & 0xFF)
         e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
@@ -371,8 +615,8 @@ def main():
         e[3].record()
         torch.cuda.synchronize()
         for k, name in enumerate(("summaries", "select", "attend")):
-            stage_ms[name].append(e[k].elapsed_time(e[k + 1]))
-    stage_ms = {k: float(np.mean(v)) for k, v in stage_ms.items()}
+            stage_all[name].append(e[k].elapsed_time(e[k + 1]))
+    stage_ms = {k: float(np.mean(v)) for k, v in stage_all.items()}
     clocks = sampler.stop()      # sampled from before the warm-up to after the per-stage pass (both under load)
     f_sel = selected_flops_from_count(rt["count"], w.block, w.head_dim, g_q)
     sparsity = sparsity_from_count(rt["count"], w.block)
@@ -429,6 +673,7 @@ def main():
     e2e_ms, _ = combine_timing(a.elapsed_time(b_) / args.steps, 0.0, device=dev)
     h2d = sum(t.numel() * t.element_size() for t in (hQ, hK, hV))
     d2h = hO.numel() * hO.element_size()
+    del sets, hQ, hK, hV, hO
 
     if rank != 0:
         if dist is not None:
@@ -439,10 +684,10 @@ def main():
     achieved = f_sel / (stage_ms["attend"] * 1e-3) / 1e12
     roofline = {"bound": "tensor", "kernel": "attend_prefill (Stage 2)", "achieved": achieved, "peak": peak_tf,
                 "unit": "TFLOP/s", "frac": achieved / peak_tf, "peak_source": f"{peaks['_source']} bf16 burst",
-                # dram__bytes_read.sum + dram__bytes_write.sum of one launch of this kernel on this workload, from the
-                # ncu capture summarised in profiles/attend_prefill_sm100_prefill_8k.md (112.3 MB + 33.6 MB)
-                "traffic": 142.8e6 if w.name == "prefill_8k" else None}
-    extras = {"fwd_ms": ms, "stage_ms": stage_ms, "block_sparsity": sparsity, "selected_tflop": f_sel / 1e12,
+                "traffic": load_traffic(w.name)}
+    extras = {"fwd_ms": ms, "fwd_ms_stats": stats(step_ms), "stage_ms": stage_ms,
+              "stage_ms_stats": {k: stats(v) for k, v in stage_all.items()},
+              "block_sparsity": sparsity, "selected_tflop": f_sel / 1e12,
               "executed_tflop": executed / 1e12, "union_inflation": executed / f_sel, "tile_steps": n_steps_total,
               "stage2_executed_tflops": executed / (stage_ms["attend"] * 1e-3) / 1e12,
               "dense_causal_tflop": f_dense / 1e12, "wall_s_timed_region": t_wall,
@@ -451,23 +696,28 @@ def main():
               "stage2_selected_frac_of_measured_sustained": achieved / float(peaks["bf16_tflops_sustained"]),
               "stage2_executed_frac_of_measured_burst": executed / (stage_ms["attend"] * 1e-3) / 1e12 / peak_tf}
 
-    cpu_val, cpu_rows, cpu_dt = time_oracle_sample(w, {k: v for k, v in inp.items()}, args.cpu_seconds)
-    cpu_baseline = {"value": cpu_val, "unit": UNIT, "cores": 1, "kind": "oracle",
-                    "sample": f"{cpu_rows} random (row, KV head) pairs of {w.name}, whole oracle row each, {cpu_dt:.1f} s"}
+    pool = OraclePool(w, inp)
+    cpu_val, cpu_rows, cpu_dt = pool.run(args.cpu_seconds)
+    pool.close()
+    cpu_baseline = {"value": cpu_val, "unit": UNIT, "cores": pool.cores, "kind": "oracle",
+                    "sample": f"{cpu_rows} random (row, KV head) pairs of {w.name}, whole oracle row each, on {pool.cores} "
+                              f"single-threaded processes for {cpu_dt:.1f} s"}
 
     if not args.no_extras:
         try:
-            extras.update(side_measurements(B, synth, w, Q, K, V, dev, peaks))
+            extras.update(side_measurements(B, synth, w, Q, K, V, dev, peaks, flush))
         except Exception as ex:  # side numbers never break the contract line
             extras["side_error"] = repr(ex)
+        del Q, K, V, O, ws, rt, kbar, inp
+        torch.cuda.empty_cache()
+        extras["configs"] = all_config_measurements(B, synth, dev, peaks, flush)
+        if "decode_128k" in extras["configs"]:
+            extras["decode"] = extras["configs"]["decode_128k"]
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
-            "config": {"workload": w.name, "batch_per_gpu": w.batch, "seq": w.seq, "h_q": w.h_q, "h_kv": w.h_kv,
-                       "head_dim": w.head_dim, "block": w.block, "alpha": w.alpha, "gamma": w.gamma, "sigma": w.sigma,
-                       "rho": w.rho, "shift": w.shift, "l2": "256 MiB buffer written between timed iterations",
-                       "parallelism": f"independent batches x{world}"},
+            "config": config_dict(w, world),
             "clocks": clocks,
             "e2e": {"value": f_total / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
@@ -480,10 +730,10 @@ def main():
         dist.destroy_process_group()
 
 
-def side_measurements(B, synth, w, Q, K, V, dev, peaks) -> dict:
-    """Context numbers beside the contract line: dense SDPA on the same tensors and the decode workload."""
+def side_measurements(B, synth, w, Q, K, V, dev, peaks, flush) -> dict:
+    """Context numbers beside the contract line: dense SDPA on the headline tensors and the same workload with
+    correlated queries."""
     out = {}
-    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
 
     def timed(fn, iters=10, warm=3):
         for _ in range(warm):
@@ -506,56 +756,12 @@ def side_measurements(B, synth, w, Q, K, V, dev, peaks) -> dict:
     # inflation, which caps selected-FLOP efficiency on the headline inputs, mostly disappears.
     try:
         wc = w.with_(q_corr=0.99)
-        ic = synth.make_prefill_inputs(wc, dev)
-        Qc, Kc_, Vc_ = ic["Q"], ic["K"], ic["V"]
-        Oc = torch.empty_like(Qc)
-        pc = B.params_for_prefill(Qc, Kc_, Vc_, Oc, block=wc.block, alpha=wc.alpha, gamma=wc.gamma, sigma=wc.sigma)
-        wsc, rtc, kbc = B.alloc_workspace(pc, dev), B.alloc_routing(pc, dev), B.alloc_kbar(pc, dev)
-        B.dash_attn_block_summaries(pc, Kc_, kbc)
-        B.dash_attn_select(pc, Qc, kbc, rtc["mask"], rtc["count"], None, rtc["blk_bias"], wsc)
-        t_att_c = timed(lambda: B.dash_attn_attend_prefill(pc, Qc, Kc_, Vc_, rtc["mask"], rtc["blk_bias"], Oc, wsc))
-        t_fwd_c = timed(lambda: B.dash_attn_fwd_prefill(pc, Qc, Kc_, Vc_, Oc, wsc))
-        f_sel_c = selected_flops_from_count(rtc["count"], wc.block, wc.head_dim, wc.h_q // wc.h_kv)
-        ex_c, _ = executed_flops_from_mask(rtc["mask"], wc)
-        out["secondary_q_corr_0.99"] = {
-            "workload": wc.name + " with q_corr=0.99", "fwd_ms": t_fwd_c, "attend_ms": t_att_c,
-            "block_sparsity": sparsity_from_count(rtc["count"], wc.block), "union_inflation": ex_c / f_sel_c,
-            "fwd_selected_tflops": f_sel_c / (t_fwd_c * 1e-3) / 1e12,
-            "stage2_selected_tflops": f_sel_c / (t_att_c * 1e-3) / 1e12,
-            "stage2_selected_frac_of_measured_burst": f_sel_c / (t_att_c * 1e-3) / 1e12 / float(peaks["bf16_tflops"])}
-        del ic, Qc, Kc_, Vc_, Oc, wsc, rtc, kbc
+        r = measure_prefill(B, synth, wc, dev, peaks, iters=10, flush=flush, with_sdpa=False)
+        r["workload"] = wc.name + " with q_corr=0.99"
+        r["stage2_selected_frac_of_measured_burst"] = r["stage2_frac"]
+        out["secondary_q_corr_0.99"] = r
     except Exception as ex:
         out["secondary_q_corr_0.99"] = {"error": repr(ex)}
-
-    # decode workload: batch 16, 131072-token cache, ~90 % sparsity
-    wd = synth.workload("decode_128k")
-    di = synth.make_decode_inputs(wd, dev)
-    qd, Kc, Vc, lens = di["Q"], di["K"], di["V"], di["kv_len"]
-    od = torch.empty_like(qd)
-    pd = B.params_for_decode(qd, Kc, Vc, od, block=wd.block, alpha=wd.alpha, gamma=wd.gamma, sigma=wd.sigma)
-    kbar = B.alloc_kbar(pd, dev)
-    out["decode_summaries_ms"] = timed(lambda: B.dash_attn_block_summaries(pd, Kc, kbar, kv_len=lens), iters=3, warm=1)
-    wsd = B.alloc_workspace(pd, dev)
-    rt = B.alloc_routing(pd, dev)
-    B.dash_attn_select(pd, qd, kbar, rt["mask"], rt["count"], rt["blk_idx"], rt["blk_bias"], wsd, kv_len=lens)
-    cnt = rt["count"].to(torch.float64)
-    g = wd.batch * wd.h_kv
-    diag = ((lens.to(torch.float64) - 1) % wd.block + 1).sum().item() * wd.h_kv
-    kv_bytes = (cnt.sum().item() * wd.block + diag) * wd.head_dim * 2 * 2
-    kbar_bytes = g * ((wd.seq - 1) // wd.block) * wd.head_dim * 4
-    t_sel = timed(lambda: B.dash_attn_select(pd, qd, kbar, rt["mask"], rt["count"], rt["blk_idx"], rt["blk_bias"], wsd, kv_len=lens))
-    t_att = timed(lambda: B.dash_attn_attend_decode(pd, qd, Kc, Vc, lens, rt["count"], rt["blk_idx"], rt["blk_bias"], od, wsd))
-    t_all = timed(lambda: B.dash_attn_fwd_decode(pd, qd, Kc, Vc, kbar, lens, od, wsd))
-    hbm = float(peaks["hbm_gbs"])
-    out["decode"] = {"workload": wd.name, "fwd_ms": t_all, "select_ms": t_sel, "attend_ms": t_att,
-                     "block_sparsity": float(1.0 - (cnt + 1).sum().item() / (g * ((wd.seq - 1) // wd.block + 1))),
-                     "bytes_touched": kv_bytes + kbar_bytes,
-                     "hbm_gbs_fwd": (kv_bytes + kbar_bytes) / (t_all * 1e-3) / 1e9,
-                     "hbm_gbs_attend_kv_only": kv_bytes / (t_att * 1e-3) / 1e9,
-                     "hbm_frac_fwd": (kv_bytes + kbar_bytes) / (t_all * 1e-3) / 1e9 / hbm,
-                     "hbm_peak_gbs": hbm}
-    kd = Kc.transpose(1, 2); vd = Vc.transpose(1, 2); q1 = qd[:, :, None, :]
-    out["decode"]["sdpa_dense_ms"] = timed(lambda: torch.nn.functional.scaled_dot_product_attention(q1, kd, vd, enable_gqa=True), iters=5)
     return out
 
 

@@ -15,7 +15,10 @@
  *
  * Conventions
  *   - Every pointer is DEVICE memory unless its comment says "host".  The caller owns every buffer;
- *     the library allocates nothing, keeps no state between calls and launches only on `stream`.
+ *     the library allocates nothing, launches only on `stream` and keeps no state that affects results
+ *     (what it does keep, per process: a launch counter, per-device caches of the SM count, of the
+ *     architecture check and of which kernels had their shared-memory limit raised, and the fixed scratch
+ *     array of dash_attn_attend_decode_static).
  *   - Calls are asynchronous: they return after enqueueing.  Argument errors are detected on the host
  *     before anything is enqueued and are returned synchronously.  Problems only a kernel can see
  *     (a bounded wait that ran out, a capacity overrun) are written to a status word at the start of
@@ -165,8 +168,14 @@ int dash_attn_attend_decode(const dash_params* p, const void* Q, const void* Kca
  * device array that is part of the library image (every GPU that loads the library holds it until exit).
  *
  * Limits and rules:
- *   - batch * h_q * n_split * (head_dim + 2) floats must fit in 4 MiB (n_split = ceil(592 / (batch*h_kv)),
- *     clamped to [1, 32]); larger problems return DASH_ERR_TOO_LARGE and nothing is enqueued.
+ *   - It always runs the CUDA-core split kernel and a separate merge kernel (the kernels that serve fp32 and
+ *     the shapes the tensor-core decode kernel does not take), for every dtype: the result is the one
+ *     dash_attn_attend_decode gives, but for bf16 shapes that call is faster (TMA / tcgen05, merge fused in).
+ *   - The partials need batch * h_q * n_split * (head_dim + 2) floats, where the split count n_split is chosen
+ *     by the library from the problem size and the SM count and is never more than 32 (more than 16 only
+ *     for caches beyond 2^19 tokens).  A problem with
+ *     batch * h_q * 32 * (head_dim + 2) * 4 bytes <= 4 MiB therefore always fits; a larger one may or may not,
+ *     and when it does not the call returns DASH_ERR_TOO_LARGE and nothing is enqueued.
  *   - The call allocates nothing (no cudaMalloc / cudaFree, no allocating library routine).  The first call
  *     on each device looks up the array's device address (a host-side query, no allocation); make that first
  *     call before any stream capture begins.
@@ -204,6 +213,16 @@ int dash_attn_last_status(const void* workspace, void* stream);
 
 /* Number of kernel launches this library has enqueued in this process (for launch accounting). */
 int64_t dash_attn_launch_count(void);
+
+/* Switches for the test-suite; production code never calls this (process-wide, not thread-safe, defaults restored
+ * by (0, 0)).
+ *   wait_limit_cycles  SM clock cycles a bounded device-side wait of the prefill attention kernel may spin before it
+ *                      gives up with DASH_ERR_TIMEOUT; <= 0 restores the default (2e9, about a second).
+ *   skip_own_k_load    1: the tensor-core prefill attention kernel never issues the load of its first K tile, so
+ *                      the waits for it run out -- with a short limit this exercises the time-out path (roles leave
+ *                      their loops, copies in flight land, tensor memory is freed, the status word is set) without
+ *                      hanging or faulting anything. */
+void dash_attn_test_hooks(int64_t wait_limit_cycles, int32_t skip_own_k_load);
 
 const char* dash_attn_strerror(int status);
 

@@ -26,7 +26,7 @@ EXPORTS = [
     "dash_attn_block_summaries", "dash_attn_select", "dash_attn_attend_prefill", "dash_attn_attend_decode",
     "dash_attn_attend_decode_static",
     "dash_attn_fwd_prefill", "dash_attn_fwd_decode", "dash_attn_reset_status", "dash_attn_last_status",
-    "dash_attn_launch_count", "dash_attn_strerror",
+    "dash_attn_launch_count", "dash_attn_strerror", "dash_attn_test_hooks",
 ]
 
 
@@ -85,6 +85,8 @@ def lib() -> ctypes.CDLL:
         L.dash_attn_last_status.argtypes = [c_void_p, c_void_p]
         L.dash_attn_launch_count.restype = c_int64
         L.dash_attn_launch_count.argtypes = []
+        L.dash_attn_test_hooks.restype = None
+        L.dash_attn_test_hooks.argtypes = [c_int64, c_int32]
         L.dash_attn_strerror.restype = c_char_p
         L.dash_attn_strerror.argtypes = [ctypes.c_int]
         _lib = L
@@ -259,6 +261,11 @@ def dash_attn_reset_status(workspace):
 
 def dash_attn_last_status(workspace) -> int:
     return int(lib().dash_attn_last_status(_ptr(workspace), _stream()))
+
+
+def dash_attn_test_hooks(wait_limit_cycles: int = 0, skip_own_k_load: int = 0) -> None:
+    """Test-suite switches (see the header); calling it without arguments restores the defaults."""
+    lib().dash_attn_test_hooks(int(wait_limit_cycles), int(skip_own_k_load))
 
 
 def dash_attn_launch_count() -> int:

@@ -4,12 +4,25 @@
 #include <cmath>
 #include <cstring>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "common.cuh"
 
 namespace dash {
 
+// NVTX range around the launches of one stage (a no-op unless a profiler is attached).
+struct StageRange {
+  explicit StageRange(const char* name) { nvtxRangePushA(name); }
+  ~StageRange() { nvtxRangePop(); }
+};
+
 static std::atomic<long long> g_launches{0};
 void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+
+TestHooks& test_hooks() {
+  static TestHooks hooks;
+  return hooks;
+}
 
 static inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
@@ -104,11 +117,12 @@ static WorkspaceLayout layout(const Dims& dm) {
 static int check_device() {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return DASH_ERR_CUDA;
-  static int cached[64];  // 0 unknown, 1 ok, 2 wrong architecture
-  if (dev >= 0 && dev < 64 && cached[dev]) return cached[dev] == 1 ? DASH_OK : DASH_ERR_ARCH;
+  static std::atomic<int> cached[64];  // per device: 0 unknown, 1 ok, 2 wrong architecture
+  const bool tracked = dev >= 0 && dev < 64;
+  if (const int c = tracked ? cached[dev].load(std::memory_order_relaxed) : 0) return c == 1 ? DASH_OK : DASH_ERR_ARCH;
   int major = 0;
   if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return DASH_ERR_CUDA;
-  if (dev >= 0 && dev < 64) cached[dev] = major == 10 ? 1 : 2;
+  if (tracked) cached[dev].store(major == 10 ? 1 : 2, std::memory_order_relaxed);
   return major == 10 ? DASH_OK : DASH_ERR_ARCH;
 }
 
@@ -127,8 +141,9 @@ template <typename T> static T* at(void* ws, size_t off) { return reinterpret_ca
 static int cuda_status(cudaError_t e) { return e == cudaSuccess ? DASH_OK : DASH_ERR_CUDA; }
 
 static int run_attend_prefill(const Dims& dm, const void* Q, const void* K, const void* V, const uint32_t* mask,
-                              const float* blk_bias, void* O, StatusBlock* sb, cudaStream_t st) {
-  if (prefill_sm100_supported(dm)) return cuda_status(launch_attend_prefill_sm100(dm, Q, K, V, mask, blk_bias, O, sb, st));
+                              const float* blk_bias, void* O, StatusBlock* sb, bool inputs_stable, cudaStream_t st) {
+  if (prefill_sm100_supported(dm))
+    return cuda_status(launch_attend_prefill_sm100(dm, Q, K, V, mask, blk_bias, O, sb, inputs_stable, st));
   return cuda_status(launch_attend_prefill_generic(dm, Q, K, V, mask, blk_bias, O, st));
 }
 
@@ -170,6 +185,7 @@ int dash_attn_block_summaries(const dash_params* p, const void* K, const float* 
   if (num_blocks < 0) num_blocks = dm.T_s - first_block;
   if (first_block + num_blocks > dm.T_s) return DASH_ERR_INVALID_ARG;
   if ((rc = check_device()) != DASH_OK) return rc;
+  StageRange nv("dash_attn: stage 0 summaries");
   return cuda_status(launch_summaries(dm, K, qbar, qbar_chunk_stride, kv_len, first_block, num_blocks, Kbar, nullptr,
                                       (cudaStream_t)stream));
 }
@@ -186,6 +202,7 @@ int dash_attn_select(const dash_params* p, const void* Q, const float* Kbar, con
   WorkspaceLayout wl;
   if ((rc = check_workspace(dm, workspace, workspace_bytes, &wl)) != DASH_OK) return rc;
   if ((rc = check_device()) != DASH_OK) return rc;
+  StageRange nv("dash_attn: stage 1 routing");
   return cuda_status(launch_select(dm, Q, Kbar, kv_len, mask, count, blk_idx, blk_bias, tau,
                                    at<void>(workspace, wl.planes), at<float>(workspace, wl.xscratch), at<StatusBlock>(workspace, wl.status),
                                    (cudaStream_t)stream));
@@ -203,7 +220,10 @@ int dash_attn_attend_prefill(const dash_params* p, const void* Q, const void* K,
   WorkspaceLayout wl;
   if ((rc = check_workspace(dm, workspace, workspace_bytes, &wl)) != DASH_OK) return rc;
   if ((rc = check_device()) != DASH_OK) return rc;
-  return run_attend_prefill(dm, Q, K, V, mask, blk_bias, O, at<StatusBlock>(workspace, wl.status), (cudaStream_t)stream);
+  StageRange nv("dash_attn: stage 2 prefill attention");
+  // the kernel before this one on the stream is unknown here and may have produced Q, K or V
+  return run_attend_prefill(dm, Q, K, V, mask, blk_bias, O, at<StatusBlock>(workspace, wl.status), false,
+                            (cudaStream_t)stream);
 }
 
 int dash_attn_attend_decode(const dash_params* p, const void* Q, const void* Kcache, const void* Vcache,
@@ -219,6 +239,7 @@ int dash_attn_attend_decode(const dash_params* p, const void* Q, const void* Kca
   WorkspaceLayout wl;
   if ((rc = check_workspace(dm, workspace, workspace_bytes, &wl)) != DASH_OK) return rc;
   if ((rc = check_device()) != DASH_OK) return rc;
+  StageRange nv("dash_attn: stage 2 decode attention");
   return cuda_status(launch_attend_decode_ex(dm, Q, Kcache, Vcache, kv_len, count, blk_idx, blk_bias, O,
                                              at<float>(workspace, wl.partials), at<StatusBlock>(workspace, wl.status),
                                              (cudaStream_t)stream));
@@ -246,6 +267,7 @@ int dash_attn_fwd_prefill(const dash_params* p, const void* Q, const void* K, co
     float* kbw = at<float>(workspace, wl.kbar);
     // the tensor-core routing kernel reads Kbar as three bf16 planes: the summary kernel writes them directly
     void* planes = select_sm100_token_limit(dm) > 0 ? at<void>(workspace, wl.planes) : nullptr;
+    StageRange nv("dash_attn: stage 0 summaries");
     if ((rc = cuda_status(launch_summaries(dm, K, qbar, qbar_chunk_stride, nullptr, 0, dm.T_s, kbw, planes, st))) != DASH_OK)
       return rc;
     kb = kbw;
@@ -253,11 +275,16 @@ int dash_attn_fwd_prefill(const dash_params* p, const void* Q, const void* K, co
   }
   uint32_t* mask = mask_out ? mask_out : at<uint32_t>(workspace, wl.mask);
   float* bias = at<float>(workspace, wl.blk_bias);
-  if ((rc = cuda_status(launch_select(dm, Q, kb, nullptr, mask, at<int>(workspace, wl.count), nullptr, bias, nullptr,
-                                      at<void>(workspace, wl.planes), at<float>(workspace, wl.xscratch), sb, st,
-                                      planes_ready))) != DASH_OK)
-    return rc;
-  return run_attend_prefill(dm, Q, K, V, mask, bias, O, sb, st);
+  {
+    StageRange nv("dash_attn: stage 1 routing");
+    if ((rc = cuda_status(launch_select(dm, Q, kb, nullptr, mask, at<int>(workspace, wl.count), nullptr, bias, nullptr,
+                                        at<void>(workspace, wl.planes), at<float>(workspace, wl.xscratch), sb, st,
+                                        planes_ready))) != DASH_OK)
+      return rc;
+  }
+  StageRange nv("dash_attn: stage 2 prefill attention");
+  // the kernel before Stage 2 is this call's own routing kernel, which writes none of Q, K, V
+  return run_attend_prefill(dm, Q, K, V, mask, bias, O, sb, true, st);
 }
 
 int dash_attn_fwd_decode(const dash_params* p, const void* Q, const void* Kcache, const void* Vcache,
@@ -278,9 +305,13 @@ int dash_attn_fwd_decode(const dash_params* p, const void* Q, const void* Kcache
   int* count = at<int>(workspace, wl.count);
   int* idx = at<int>(workspace, wl.blk_idx);
   float* bias = at<float>(workspace, wl.blk_bias);
-  if ((rc = cuda_status(launch_select(dm, Q, Kbar, kv_len, at<uint32_t>(workspace, wl.mask), count, idx, bias, nullptr,
-                                      at<void>(workspace, wl.planes), at<float>(workspace, wl.xscratch), sb, st))) != DASH_OK)
-    return rc;
+  {
+    StageRange nv("dash_attn: stage 1 routing");
+    if ((rc = cuda_status(launch_select(dm, Q, Kbar, kv_len, at<uint32_t>(workspace, wl.mask), count, idx, bias, nullptr,
+                                        at<void>(workspace, wl.planes), at<float>(workspace, wl.xscratch), sb, st))) != DASH_OK)
+      return rc;
+  }
+  StageRange nv("dash_attn: stage 2 decode attention");
   return cuda_status(launch_attend_decode_ex(dm, Q, Kcache, Vcache, kv_len, count, idx, bias, O,
                                              at<float>(workspace, wl.partials), sb, st));
 }
@@ -300,6 +331,12 @@ int dash_attn_last_status(const void* workspace, void* stream) {
 }
 
 int64_t dash_attn_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+void dash_attn_test_hooks(int64_t wait_limit_cycles, int32_t skip_own_k_load) {
+  TestHooks& h = test_hooks();
+  h.wait_limit_cycles = wait_limit_cycles > 0 ? wait_limit_cycles : TestHooks().wait_limit_cycles;
+  h.skip_own_k_load = skip_own_k_load ? 1 : 0;
+}
 
 const char* dash_attn_strerror(int status) {
   switch (status) {

@@ -171,6 +171,12 @@ inline cudaError_t launch_chained(void (*kern)(KArgs...), dim3 grid, dim3 block,
 #endif
 
 void count_launch();
+// Host-side switches for the tests (set through dash_attn_test_hooks; the defaults are what production runs with).
+struct TestHooks {
+  long long wait_limit_cycles = 2000000000LL;   // how long a bounded device-side wait may spin (about 1 s)
+  int skip_own_k_load = 0;                      // 1: the prefill attention kernel never loads its first K tile
+};
+TestHooks& test_hooks();
 // Host-side checks shared by the entry points that live outside api.cu.
 int validate_params(const dash_params* p, Dims* dm);
 int validate_device();
@@ -212,8 +218,9 @@ cudaError_t launch_decode_sm100(const Dims& dm, int n_split, const void* Q, cons
                                 const int* kv_len, const int* count, const int* blk_idx, const float* blk_bias,
                                 float* partials, void* O, StatusBlock* sb, cudaStream_t st);
 bool prefill_sm100_supported(const Dims& dm);
+// inputs_stable: Q, K, V were not written by the kernel launched just before on the stream
 cudaError_t launch_attend_prefill_sm100(const Dims& dm, const void* Q, const void* K, const void* V,
                                         const uint32_t* mask, const float* blk_bias, void* O, StatusBlock* sb,
-                                        cudaStream_t st);
+                                        bool inputs_stable, cudaStream_t st);
 
 }  // namespace dash

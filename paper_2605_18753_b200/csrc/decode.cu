@@ -25,14 +25,21 @@ static bool decode_use_sm100(const Dims& dm) {
 // shared memory), so the time is about ceil(groups * s / SMs) waves of (1/s of a group's work + a fixed cost per
 // block, about 2 % of a long group's work: list staging, first loads, partial write).  At 128 groups on 148 SMs
 // s = 5 leaves a fifth wave a third full, s = 8 fills seven waves almost exactly (measured: 0.155 vs 0.150 ms).
+// SM count of the current device, cached per device (a process may drive several GPUs).
+static int current_sm_count() {
+  static std::atomic<int> cached[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+  const bool tracked = dev >= 0 && dev < 64;
+  int n = tracked ? cached[dev].load(std::memory_order_relaxed) : 0;
+  if (n > 0) return n;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+  if (tracked) cached[dev].store(n, std::memory_order_relaxed);
+  return n;
+}
+
 int decode_num_splits(const Dims& dm) {
-  static int n_sm = 0;
-  if (n_sm == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sm <= 0)
-      n_sm = 148;
-  }
+  const int n_sm = current_sm_count();
   const int groups = dm.batch * dm.h_kv;
   int lo = 1;
   if (decode_use_sm100(dm)) lo = max(lo, decode_sm100_min_splits(dm));   // a block owns at most 512 sub-blocks there

@@ -82,6 +82,9 @@ struct PrefillArgs {
   Dims dm;
   int TQ;            // tokens per tile
   int n_tiles;       // tiles per (batch, KV head)
+  int early_loads;   // 1: Q, K, V are not written by the kernel before this one on the stream (their first loads may precede chain_wait)
+  int inject;        // test hook: 1 = the K producer never loads the own chunk's keys (the waits for them run out)
+  long long wait_limit;   // cycles a bounded wait may spin
   const uint32_t* mask;
   const float* blk_bias;
   __nv_bfloat16* O;
@@ -105,6 +108,8 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
   const uint32_t sbase = ptx::smem_u32(smem);
   auto bar = [&](int i) { return ptx::smem_u32(&misc->bar[i]); };
   volatile int* abort_flag = &misc->abort_flag;
+  const long long wait_limit = a.wait_limit;
+  auto wait_on = [&](uint32_t barrier, uint32_t parity) { return ptx::mbar_wait(barrier, parity, abort_flag, wait_limit); };
 
   const int groups = dm.batch * dm.h_kv;
   const int tile = a.n_tiles - 1 - (int)(blockIdx.x / groups);  // late (long) tiles first
@@ -154,20 +159,19 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
         *reinterpret_cast<uint4*>(smem + OFF_Q + regn * (Q_BYTES / (HD / 64)) + k * 16) = make_uint4(0u, 0u, 0u, 0u);
     ptx::fence_proxy_async_smem();
   }
-  // barriers and tensor memory are set up; from here on the kernel reads what the routing kernels wrote
-  chain_wait();
-  chain_release();
-  // a workspace whose status word already holds an error makes every role leave at its first wait: after one
-  // block's wait has run out, the rest of the grid retires in microseconds instead of a wait limit each
-  if (a.sb && *reinterpret_cast<volatile int*>(&a.sb->status) != 0) *abort_flag = 1;
-  __syncthreads();
-
-  if (warp == 4 || warp == 6) {
-    // =========================== producers ===========================
-    // Two warps walk the same union list: warp 4 feeds the K ring (and loads Q), warp 6 feeds the V ring and
-    // the per-token bias of each step.  Split like this, a full V ring never holds back the next K tile.
-    const bool do_k = (warp == 4), do_v = (warp == 6);
-    const int TR = SHORT ? 128 / g_q : TQ;   // token slots of the 128 tile rows; slots TQ .. TR-1 are padding (bias -inf)
+  // A step's K or V tile for chunks smaller than the step: CPS boxes of NKV / CPS tokens, one per packed chunk.
+  [[maybe_unused]] auto load_packed = [&](const CUtensorMap* tm, uint32_t dst, uint32_t barrier, const int* kvs) {
+    ptx::mbar_arrive_expect_tx(barrier, KV_TILE_BYTES);
+#pragma unroll
+    for (int s = 0; s < CPS; ++s) {
+      const uint32_t d = dst + s * (NKV / CPS) * 128;
+      ptx::tma_load_4d(d, tm, barrier, 0, r, kvs[s], b);
+      if constexpr (HD == 128) ptx::tma_load_4d(d + KV_TILE_BYTES / 2, tm, barrier, 64, r, kvs[s], b);
+    }
+  };
+  // Q and the own chunk's K / V tiles: they need nothing from the routing kernels (and go first anyway).
+  auto own_loads = [&](bool do_k, bool do_v) {
+    const int TR = SHORT ? 128 / g_q : TQ;
     if (lane == 0 && do_k) {
       ptx::prefetch_tensormap(&tmQ);
       ptx::prefetch_tensormap(&tmK);
@@ -178,16 +182,6 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
     }
     // The own chunk goes first: its tiles need nothing from the mask, so they are in flight (and the first
     // S = Q K^T can run) while the union of the routed chunks is still being formed.  Stages 0/1 are free.
-    // A step's K or V tile for chunks smaller than the step: CPS boxes of NKV / CPS tokens, one per packed chunk.
-    [[maybe_unused]] auto load_packed = [&](const CUtensorMap* tm, uint32_t dst, uint32_t barrier, const int* kvs) {
-      ptx::mbar_arrive_expect_tx(barrier, KV_TILE_BYTES);
-#pragma unroll
-      for (int s = 0; s < CPS; ++s) {
-        const uint32_t d = dst + s * (NKV / CPS) * 128;
-        ptx::tma_load_4d(d, tm, barrier, 0, r, kvs[s], b);
-        if constexpr (HD == 128) ptx::tma_load_4d(d + KV_TILE_BYTES / 2, tm, barrier, 64, r, kvs[s], b);
-      }
-    };
     for (int sub = 0; sub < own_steps; ++sub) {
       const int kv0 = c_own * dm.B + sub * NKV;
       if constexpr (CPS > 1) {
@@ -196,7 +190,7 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
 #pragma unroll
         for (int s = 0; s < CPS; ++s) kvs[s] = kv0;
         if (do_k) {
-          if (lane == 0) load_packed(&tmK, sbase + OFF_K, bar(K_FULL), kvs);
+          if (lane == 0 && !a.inject) load_packed(&tmK, sbase + OFF_K, bar(K_FULL), kvs);
         } else {
           for (int t = lane; t < TR; t += 32) {
             misc->bias[0][0][t] = t < TQ ? 0.f : -INFINITY;     // token slots beyond TQ: padding rows of a short tile
@@ -210,7 +204,7 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
         continue;
       }
       if (do_k) {
-        if (lane == 0) {
+        if (lane == 0 && !a.inject) {
           const uint32_t dst = sbase + OFF_K + sub * KV_TILE_BYTES;
           ptx::mbar_arrive_expect_tx(bar(K_FULL + sub), KV_TILE_BYTES);
           ptx::tma_load_4d(dst, &tmK, bar(K_FULL + sub), 0, r, kv0, b);
@@ -228,6 +222,25 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
         }
       }
     }
+  };
+  // Q, K and V are inputs of the whole chain, not outputs of the kernel before this one: when the caller vouches for
+  // that, their first tiles are under way while that kernel still drains
+  if (a.early_loads && (warp == 4 || warp == 6)) own_loads(warp == 4, warp == 6);
+  // barriers and tensor memory are set up; from here on the kernel reads what the routing kernels wrote
+  chain_wait();
+  chain_release();
+  // a workspace whose status word already holds an error makes every role leave at its first wait: after one
+  // block's wait has run out, the rest of the grid retires in microseconds instead of a wait limit each
+  if (a.sb && *reinterpret_cast<volatile int*>(&a.sb->status) != 0) *abort_flag = 1;
+  __syncthreads();
+
+  if (warp == 4 || warp == 6) {
+    // =========================== producers ===========================
+    // Two warps walk the same union list: warp 4 feeds the K ring (and loads Q), warp 6 feeds the V ring and
+    // the per-token bias of each step.  Split like this, a full V ring never holds back the next K tile.
+    const bool do_k = (warp == 4), do_v = (warp == 6);
+    const int TR = SHORT ? 128 / g_q : TQ;   // token slots of the 128 tile rows; slots TQ .. TR-1 are padding (bias -inf)
+    if (!a.early_loads) own_loads(do_k, do_v);
     // union of the tile's mask words (lane t owns tokens t, t+32)
     const int n_words = (c_own >> 5) + 1;
     const long long row0 = ((long long)b * dm.h_kv + r) * dm.seq_q;
@@ -288,6 +301,9 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
     if (n_words > 1) load_rows(1, rw_n);
     int j = own_steps;                 // the own chunk's steps are already under way
     bool ok = true;
+    // last step loaded into each stage (-1: none): what a block that gives up has to let land before it retires
+    int last_j[2] = {-1, -1};
+    for (int sub = 0; sub < (CPS > 1 ? 1 : own_steps); ++sub) last_j[sub] = (do_k && a.inject) ? -1 : sub;
     {
       // A step takes the next CPS chunks of the union (CPS > 1: chunks of 32 / 16 tokens packed into the 64-token
       // step; a short last step repeats its last chunk with bias -inf).  A row's bias for a chunk is read straight
@@ -338,11 +354,12 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
           for (int s = 0; s < CPS; ++s) kvs[s] = cs[s] * dm.B + sub * NKV;
           const int st = j & 1, prev_ph = ((j >> 1) - 1) & 1;   // stage, and the phase of step j-2 on the completion barriers
           if (do_k) {
-            if (j >= 2) ok = ptx::mbar_wait(bar(S_FULL + st), prev_ph, abort_flag);     // QK of step j-2 has read the stage
+            if (j >= 2) ok = wait_on(bar(S_FULL + st), prev_ph);     // QK of step j-2 has read the stage
             if (!ok) break;
             if (lane == 0) load_packed(&tmK, sbase + OFF_K + st * KV_TILE_BYTES, bar(K_FULL + st), kvs);
+            last_j[st] = j;
           } else {
-            if (j >= 2) ok = ptx::mbar_wait(bar(PV_DONE + st), prev_ph, abort_flag);    // PV of step j-2 has read the stage
+            if (j >= 2) ok = wait_on(bar(PV_DONE + st), prev_ph);    // PV of step j-2 has read the stage
             if (!ok) break;
 #pragma unroll
             for (int s = 0; s < CPS; ++s)
@@ -355,23 +372,27 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
               if (lane == s) misc->kvbase[st][s] = kvs[s];
             __syncwarp();
             if (lane == 0) load_packed(&tmV, sbase + OFF_V + st * KV_TILE_BYTES, bar(V_FULL + st), kvs);
+            last_j[st] = j;
           }
         }
       }
     }
     if (!ok && lane == 0) {
       // a wait ran out: let the copies already issued land (bounded) before the block retires
-      for (int s = 0; s < KST && do_k; ++s)
-        for (int k = 0; k < 200000 && !ptx::mbar_try_wait(bar(K_FULL + s), 0) && !ptx::mbar_try_wait(bar(K_FULL + s), 1); ++k) {}
-      for (int s = 0; s < VST && do_v; ++s)
-        for (int k = 0; k < 200000 && !ptx::mbar_try_wait(bar(V_FULL + s), 0) && !ptx::mbar_try_wait(bar(V_FULL + s), 1); ++k) {}
+      for (int s = 0; s < 2; ++s) {
+        if (last_j[s] < 0) continue;
+        const uint32_t full = bar((do_k ? K_FULL : V_FULL) + s), parity = (uint32_t)(last_j[s] >> 1) & 1u;
+        for (int k = 0; k < 200000 && !ptx::mbar_try_wait(full, parity); ++k) {}
+      }
+      if (do_k)
+        for (int k = 0; k < 200000 && !ptx::mbar_try_wait(bar(Q_FULL), 0); ++k) {}
     }
   } else if (warp == 5) {
     // =========================== MMA issuer ===========================
     // Per step: S_{j+1} = Q K_{j+1}^T (needs only its K tile), then O += P_j V_j.  V_FULL is not tested here: the
     // softmax threads wait for it (the step's bias arrives with it) before they arrive on P_FULL.
     if (lane == 0) {
-      bool ok = ptx::mbar_wait(bar(Q_FULL), 0, abort_flag);
+      bool ok = wait_on(bar(Q_FULL), 0);
       constexpr uint32_t IDESC_QK = ptx::idesc_bf16_f32(128, NKV, false, false);
       constexpr uint32_t IDESC_PV = ptx::idesc_bf16_f32(128, HD, false, true);
       // Descriptors differ only in the 14-bit start-address field (16-byte units, no carry into the next
@@ -381,7 +402,7 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
       const uint64_t vd0 = ptx::smem_desc_sw128(sbase + OFF_V, KV_TILE_BYTES / 2, 1024);
       auto issue_qk = [&](int j) -> bool {
         const int buf = j & 1;
-        if (!ptx::mbar_wait(bar(K_FULL + buf), (j >> 1) & 1, abort_flag)) return false;
+        if (!wait_on(bar(K_FULL + buf), (j >> 1) & 1)) return false;
         // the S/P buffer is recycled in MMA issue order (PV of step j-2 precedes this QK)
         ptx::tc_fence_after();
         const uint64_t kd = kd0 + (uint64_t)((buf * KV_TILE_BYTES) >> 4);
@@ -397,13 +418,13 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
         return true;
       };
       if (ok) ok = issue_qk(0);          // the own chunk: there is always a step 0, whatever the union holds
-      ok = ok && ptx::mbar_wait(bar(META), 0, abort_flag);
+      ok = ok && wait_on(bar(META), 0);
       const int n_steps = ok ? misc->n_steps : 0;
       for (int j = 0; j < n_steps && ok; ++j) {
         if (j + 1 < n_steps) ok = issue_qk(j + 1);
         if (!ok) break;
         const int buf = j & 1;
-        ok = ptx::mbar_wait(bar(P_FULL + buf), (j >> 1) & 1, abort_flag);
+        ok = wait_on(bar(P_FULL + buf), (j >> 1) & 1);
         if (!ok) break;
         ptx::tc_fence_after();
         // V is [kv token][d]: MN-major B operand; 64-wide d blocks are KV_TILE_BYTES/2 apart; 16 tokens = 2048 bytes
@@ -433,20 +454,20 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
 
     for (int j = 0; ok; ++j) {
       if (j == 1) {
-        ok = ptx::mbar_wait(bar(META), 0, abort_flag);
+        ok = wait_on(bar(META), 0);
         if (!ok) break;
         n_steps = misc->n_steps;
       }
       if (j >= n_steps) break;
       const int buf = j & 1;
       // bias / kvbase of the step visible; the MMA thread relies on this wait for the V tile as well
-      ok = ptx::mbar_wait(bar(V_FULL + buf), (j >> 1) & 1, abort_flag);
+      ok = wait_on(bar(V_FULL + buf), (j >> 1) & 1);
       if (!ok) break;
       float b2s[CPS];                                // per packed chunk: bias in the log2 domain (-inf: not routed)
 #pragma unroll
       for (int s = 0; s < CPS; ++s) b2s[s] = misc->bias[buf][s][t] * 1.4426950408889634f;   // -inf on padding rows
       const int kv0 = misc->kvbase[buf][0];
-      ok = ptx::mbar_wait(bar(S_FULL + buf), (j >> 1) & 1, abort_flag);
+      ok = wait_on(bar(S_FULL + buf), (j >> 1) & 1);
       if (!ok) break;
       ptx::tc_fence_after();
       uint32_t sreg[64];
@@ -545,7 +566,7 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
       // O is stable once the previous step's PV has completed
       const bool fix = j > 0 && __any_sync(0xffffffffu, moved);
       if (fix) {
-        ok = ptx::mbar_wait(bar(PV_DONE + (buf ^ 1)), ((j - 1) >> 1) & 1, abort_flag);
+        ok = wait_on(bar(PV_DONE + (buf ^ 1)), ((j - 1) >> 1) & 1);
         if (!ok) break;
         ptx::tc_fence_after();
         // rescale this row of the accumulator: O *= 2^(m_old - m_new)
@@ -567,7 +588,7 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
     }
 
     // epilogue: O / l -> global (row m is 128 contiguous bf16 of token i_row, head r*g_q + hh)
-    if (ok && n_steps > 0) ok = ptx::mbar_wait(bar(PV_DONE + ((n_steps - 1) & 1)), ((n_steps - 1) >> 1) & 1, abort_flag);
+    if (ok && n_steps > 0) ok = wait_on(bar(PV_DONE + ((n_steps - 1) & 1)), ((n_steps - 1) >> 1) & 1);
     if (ok && n_steps > 0) {
       ptx::tc_fence_after();
       const float inv = l > 0.f ? 1.f / l : 0.f;
@@ -628,11 +649,14 @@ bool prefill_sm100_supported(const Dims& dm) {
 
 cudaError_t launch_attend_prefill_sm100(const Dims& dm, const void* Q, const void* K, const void* V,
                                         const uint32_t* mask, const float* blk_bias, void* O, StatusBlock* sb,
-                                        cudaStream_t st) {
+                                        bool inputs_stable, cudaStream_t st) {
   PrefillArgs a;
   a.dm = dm;
   a.TQ = 128 / dm.g_q < dm.B ? 128 / dm.g_q : dm.B;     // a tile stays inside one chunk
   a.n_tiles = (dm.seq_q + a.TQ - 1) / a.TQ;
+  a.early_loads = inputs_stable ? 1 : 0;
+  a.inject = test_hooks().skip_own_k_load;
+  a.wait_limit = test_hooks().wait_limit_cycles;
   a.mask = mask;
   a.blk_bias = blk_bias;
   a.O = (__nv_bfloat16*)O;

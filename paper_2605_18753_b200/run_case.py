@@ -25,22 +25,15 @@ def main() -> None:
     ap.add_argument("--alpha", type=float)
     ap.add_argument("--head-dim", type=int, dest="head_dim")
     ap.add_argument("--local-blocks", type=int, default=0, help="window chunks before the own chunk (0 = none)")
-    ap.add_argument("--graph", action="store_true", help="record the forward pass into a CUDA graph and time its replays")
-    ap.add_argument("--kv-layout", choices=("token_major", "head_major"), default="token_major",
-                    help="memory order of K and V: [b, n, h_kv, d] (default) or [b, h_kv, n, d] behind the same strided view")
     args = ap.parse_args()
     over = {k: getattr(args, k) for k in ("batch", "seq", "block", "alpha", "head_dim") if getattr(args, k) is not None}
     w = synth.workload(args.workload, **over)
     dev = "cuda"
-
-    def relayout(t):
-        # same logical [b, n, h, d] tensor; head-major memory makes a chunk's rows of one head contiguous
-        return t.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3) if args.kv_layout == "head_major" else t
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)     # larger than L2
 
     if w.kind == "prefill":
         inp = synth.make_prefill_inputs(w, dev)
-        Q, K, V = inp["Q"], relayout(inp["K"]), relayout(inp["V"])
+        Q, K, V = inp["Q"], inp["K"], inp["V"]
         O = torch.empty_like(Q)
         p = B.params_for_prefill(Q, K, V, O, block=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma,
                                  local_blocks=args.local_blocks)
@@ -48,7 +41,7 @@ def main() -> None:
         step = lambda: B.dash_attn_fwd_prefill(p, Q, K, V, O, ws)
     else:
         di = synth.make_decode_inputs(w, dev)
-        q, Kc, Vc, kl = di["Q"], relayout(di["K"]), relayout(di["V"]), di["kv_len"]
+        q, Kc, Vc, kl = di["Q"], di["K"], di["V"], di["kv_len"]
         del di
         O = torch.empty_like(q)
         p = B.params_for_decode(q, Kc, Vc, O, block=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma,
@@ -57,14 +50,6 @@ def main() -> None:
         B.dash_attn_block_summaries(p, Kc, kbar, kv_len=kl)
         ws = B.alloc_workspace(p)
         step = lambda: B.dash_attn_fwd_decode(p, q, Kc, Vc, kbar, kl, O, ws)
-
-    if args.graph:
-        step()                                   # first use outside the capture
-        torch.cuda.synchronize()
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph):
-            step()
-        step = graph.replay
 
     times = []
     for it in range(args.iters + 1):

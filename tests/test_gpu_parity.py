@@ -219,7 +219,9 @@ def test_fwd_prefill_small(kw):
     _fwd_prefill_case(w, rows)
 
 
-def _fwd_prefill_case(w, rows, kv_heads=None, min_clean=0.9, local_blocks=0):
+def _fwd_prefill_case(w, rows, kv_heads=None, min_clean=0.9, local_blocks=0, qbar_mode="none", give_kbar=False):
+    """qbar_mode: "none" (mean pooling), "head" (one summary query per KV head), "chunk" (one per chunk and KV head);
+    give_kbar: the caller computes the summaries with dash_attn_block_summaries and hands them to the forward."""
     inp = synth.make_prefill_inputs(w, DEV)
     Q, K, V = inp["Q"], inp["K"], inp["V"]
     O = torch.full_like(Q, float("nan"))
@@ -227,12 +229,26 @@ def _fwd_prefill_case(w, rows, kv_heads=None, min_clean=0.9, local_blocks=0):
                              local_blocks=local_blocks)
     ws = B.alloc_workspace(p)
     T_a = (w.seq + w.block - 1) // w.block
+    T_s = w.seq // w.block
     mask = torch.empty(w.batch, w.h_kv, w.seq, (T_a + 31) // 32, dtype=torch.int32, device=DEV)
-    B.dash_attn_fwd_prefill(p, Q, K, V, O, ws, mask_out=mask)
+    qbar, stride = None, 0
+    if qbar_mode == "head":
+        qbar = torch.randn(w.h_kv, w.head_dim, device=DEV, generator=torch.Generator(DEV).manual_seed(w.seed + 50)) * 2
+    elif qbar_mode == "chunk":
+        qbar = torch.randn(max(T_s, 1), w.h_kv, w.head_dim, device=DEV,
+                           generator=torch.Generator(DEV).manual_seed(w.seed + 51)) * 2
+        stride = w.h_kv * w.head_dim
+    if give_kbar:
+        kbar = B.alloc_kbar(p)
+        B.dash_attn_block_summaries(p, K, kbar, qbar, stride)
+        B.dash_attn_fwd_prefill(p, Q, K, V, O, ws, Kbar=kbar, mask_out=mask)
+    else:
+        B.dash_attn_fwd_prefill(p, Q, K, V, O, ws, qbar=qbar, qbar_chunk_stride=stride, mask_out=mask)
     assert B.dash_attn_last_status(ws) == 0
     assert torch.isfinite(O.float()).all()
     ora = H.oracle_prefill_rows(Q, K, V, B=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma, rows=rows,
-                                kv_heads=kv_heads, local_blocks=local_blocks)
+                                kv_heads=kv_heads, local_blocks=local_blocks,
+                                qbar=None if qbar is None else H.to_np64(qbar))
     mk = mask.cpu().numpy().view(np.uint32)
     keys = []
     n_excluded = 0
@@ -254,6 +270,65 @@ def _fwd_prefill_case(w, rows, kv_heads=None, min_clean=0.9, local_blocks=0):
     assert len(keys) >= min_clean * len(ora), f"too few clean rows: {len(keys)} of {len(ora)} ({n_excluded} excluded)"
     want = np.stack([ora[k][1] for k in keys])
     return H.check_outputs(_gather_O(O, keys, w.h_q // w.h_kv), want, Q.dtype, f"fwd_prefill {w.name}")
+
+
+@pytest.mark.parametrize("kw,qbar_mode,give_kbar", [
+    (dict(seq=1024, h_q=8, h_kv=2, head_dim=128, block=64, seed=20), "head", False),    # planes written by Stage 0, weighted
+    (dict(seq=1100, h_q=8, h_kv=2, head_dim=128, block=64, seed=21), "chunk", False),
+    (dict(seq=900, h_q=16, h_kv=2, head_dim=64, block=32, seed=22, alpha=2.0), "chunk", False),
+    (dict(seq=700, dtype="f32", gamma=3.0, seed=23), "head", False),                    # CUDA-core path
+    (dict(seq=1024, h_q=8, h_kv=2, head_dim=128, block=64, seed=24), "none", True),     # caller-supplied summaries
+    (dict(seq=1300, h_q=32, h_kv=2, head_dim=128, block=64, seed=25), "head", True),
+])
+def test_fwd_prefill_with_summary_queries_and_given_summaries(kw, qbar_mode, give_kbar):
+    """The whole forward with a learned summary query (Eq. 3: softmax-weighted pooling, per KV head or per chunk as
+    Algorithm 1's input) and with summaries the caller computed beforehand."""
+    w = _wl(**kw)
+    rows = sorted(set(list(range(0, w.seq, 5)) + [w.seq - 1, w.seq - 2] + list(range(min(w.seq, 2 * w.block)))))
+    _fwd_prefill_case(w, rows, qbar_mode=qbar_mode, give_kbar=give_kbar)
+
+
+def test_select_equal_scores_get_equal_weights():
+    """Duplicated key chunks have identical summaries, hence identical logits: entmax is symmetric, so the copies are
+    routed together (or not at all) and carry the same bias; the rest of the routing still matches the oracle."""
+    w = _wl(seq=1500, h_q=8, h_kv=2, head_dim=128, block=64, seed=30)
+    inp = synth.make_prefill_inputs(w, DEV)
+    K = inp["K"]
+    pairs = [(1, 9), (3, 17), (4, 5)]
+    for a, c in pairs:
+        K[:, c * 64:(c + 1) * 64] = K[:, a * 64:(a + 1) * 64]
+    p, kbar, ws, rt = _run_select(w, inp)
+    assert torch.equal(kbar[:, :, 1], kbar[:, :, 9])
+    rows = sorted(set(list(range(0, w.seq, 3)) + [w.seq - 1]))
+    _check_select(w, inp, p, rt, rows)
+    mask = rt["mask"].cpu().numpy().view(np.uint32)
+    count = rt["count"].cpu().numpy()
+    idx, bias = rt["blk_idx"].cpu().numpy(), rt["blk_bias"].cpu().numpy()
+    n_both = 0
+    for r in range(w.h_kv):
+        for i in range(18 * 64, w.seq, 3):
+            off = B.dash_attn_list_offset(p, 0, r, i)
+            ent = {int(c): float(v) for c, v in zip(idx[off:off + count[0, r, i]], bias[off:off + count[0, r, i]])}
+            for a, c in pairs:
+                assert (a in ent) == (c in ent), (r, i, a, c)
+                assert ((mask[0, r, i, a >> 5] >> (a & 31)) & 1) == ((mask[0, r, i, c >> 5] >> (c & 31)) & 1)
+                if a in ent:
+                    assert ent[a] == ent[c], (r, i, a, c, ent[a], ent[c])
+                    n_both += 1
+    assert n_both > 0
+
+
+def test_select_rows_beyond_2048_candidates():
+    """Chunks of 16 tokens and more than 32784 tokens: the last rows have more than 2048 candidates, beyond what
+    the tensor-core routing kernel keeps on chip; they take the CUDA-core kernel."""
+    w = _wl(seq=33100, h_q=2, h_kv=1, head_dim=64, block=16, seed=31, n_planted=6)
+    inp = synth.make_prefill_inputs(w, DEV)
+    p, kbar, ws, rt = _run_select(w, inp)
+    rows = sorted(set(list(range(32784, w.seq, 9)) + list(range(32700, 32784, 7)) + list(range(0, 32700, 997))
+                      + [w.seq - 1]))
+    ora, clean, nb, nd = _check_select(w, inp, p, rt, rows)
+    assert max(v[0].n_cand for v in ora.values()) > 2048
+    assert nd <= nb
 
 
 @pytest.mark.parametrize("seed", [0, 1, 2])

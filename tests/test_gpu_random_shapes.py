@@ -44,6 +44,8 @@ def test_random_shapes_any_path(seed):
         rows = sorted(set(rng.integers(0, seq, min(seq, 40)).tolist()) | {0, seq - 1})
         lens = [int(rng.integers(1, seq + 1)) for _ in range(batch)]
         done += _run(kind, kw, lens, rows, L)
+    print(f"random shapes (any path) seed {seed}: {done} of 150 draws compared, {150 - done} had too few rows or groups "
+          "free of borderline chunks")
     assert done >= 140
 
 
@@ -51,7 +53,7 @@ def test_random_shapes_any_path(seed):
 def test_random_shapes_tensor_core_paths(seed):
     """bf16, g_q >= 2, every chunk size and both head dims: mostly shapes the TMA / tcgen05 kernels serve."""
     rng = np.random.default_rng(seed)
-    done = 0
+    done, swallowed = 0, []
     for _ in range(120):
         g_q = int(rng.choice([2, 4, 8, 16])); h_kv = int(rng.choice([1, 2]))
         seq = int(rng.integers(1, 9000))
@@ -65,5 +67,10 @@ def test_random_shapes_tensor_core_paths(seed):
         kind = str(rng.choice(["prefill", "prefill", "decode"]))
         rows = sorted(set(rng.integers(0, seq, min(seq, 30)).tolist()) | {0, seq - 1})
         lens = [int(rng.integers(1, seq + 1)) for _ in range(batch)]
-        done += _run(kind, kw, lens, rows, L)
-    assert done >= 110
+        ok = _run(kind, kw, lens, rows, L)
+        done += ok
+        if not ok:
+            swallowed.append((kind, kw, L))
+    print(f"random shapes (tensor-core paths) seed {seed}: {done} of 120 draws compared; not compared: {swallowed}")
+    # a tensor-core-path draw that cannot be compared is a gap in the sweep, not noise: none is accepted
+    assert not swallowed, swallowed

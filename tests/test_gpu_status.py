@@ -62,3 +62,34 @@ def test_status_word_decode_path():
     B.dash_attn_fwd_decode(p, q, Kc, Vc, kbar, kl, o, ws)
     assert B.dash_attn_last_status(ws) == 0
     assert torch.equal(o, good)
+
+
+def test_bounded_wait_really_runs_out_and_the_kernel_returns():
+    """A device-side wait that nothing will ever satisfy: through the test hooks the prefill attention kernel is told
+    not to issue the load of its first K tile and to give up a wait after 2e5 cycles (0.1 ms).  The waits for that tile
+    run out, every role leaves its loop, the copies in flight land, tensor memory is freed and the kernel returns
+    with DASH_ERR_TIMEOUT in the status word -- no hang, no trap, no fault -- and after a reset the same workspace
+    serves a correct forward pass again."""
+    w = synth.workload("prefill_8k", seq=1024)
+    inp = synth.make_prefill_inputs(w, DEV)
+    Q, K, V = inp["Q"], inp["K"], inp["V"]
+    O = torch.empty_like(Q)
+    p = B.params_for_prefill(Q, K, V, O, block=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma)
+    ws = B.alloc_workspace(p)
+    B.dash_attn_fwd_prefill(p, Q, K, V, O, ws)
+    assert B.dash_attn_last_status(ws) == 0
+    good = O.clone()
+    try:
+        B.dash_attn_test_hooks(wait_limit_cycles=200_000, skip_own_k_load=1)
+        O.fill_(float("nan"))
+        t0 = time.time()
+        B.dash_attn_fwd_prefill(p, Q, K, V, O, ws)
+        assert B.dash_attn_last_status(ws) == DASH_ERR_TIMEOUT
+        assert time.time() - t0 < 5.0            # one short wait limit, then the rest of the grid retires at once
+    finally:
+        B.dash_attn_test_hooks()                 # defaults
+    torch.cuda.synchronize()                     # the context is intact: nothing faulted
+    B.dash_attn_reset_status(ws)
+    B.dash_attn_fwd_prefill(p, Q, K, V, O, ws)
+    assert B.dash_attn_last_status(ws) == 0
+    assert torch.equal(O, good)
