@@ -187,6 +187,22 @@ int dash_attn_attend_decode_static(const dash_params* p, const void* Q, const vo
                                    const int32_t* kv_len, const int32_t* count, const int32_t* blk_idx,
                                    const float* blk_bias, void* O, void* stream);
 
+/* Backward of Stage 2 alone, prefill, with the routing held fixed (Section 3.5: the backward pass reuses the forward
+ * pass's bit mask, which the sparse alpha-entmax Jacobian permits -- appendix "The alpha-entmax mapping"; Eq. 7 in the
+ * form of Proposition 1 is what is differentiated).  For L = sum(O * dO) and logits l_j = <q,k_j>/sqrt(d) + bias_c(j):
+ *   dQ     gradient w.r.t. Q, dtype p->dtype, strides p->q_stride (every row is written).
+ *   dK,dV  gradients w.r.t. K and V, fp32, contiguous [batch, seq_kv, h_kv, head_dim]; zeroed, then accumulated
+ *          (tokens no row attends stay zero).
+ *   dbias  gradient w.r.t. every entry of blk_bias, fp32, in the layout of blk_bias (entries outside a row's count
+ *          stay zero): the quantity a backward of Stage 1 continues from.
+ *   dO     incoming gradient of O, dtype p->dtype, strides p->o_stride.
+ * mask / blk_bias as written by dash_attn_select for the same parameters.  This is a correctness path on CUDA cores
+ * (one warp per row and head, fp32 atomics for dK / dV / dbias, so their last bits vary from run to run); it needs
+ * no workspace.  The gradient through the routing itself (Stage 1, Stage 0) is not computed by the library. */
+int dash_attn_bwd_attend_prefill(const dash_params* p, const void* Q, const void* K, const void* V, const void* dO,
+                                 const uint32_t* mask, const float* blk_bias, void* dQ, float* dK, float* dV,
+                                 float* dbias, void* stream);
+
 /* Whole prefill forward: Stage 0 (skipped when Kbar is given), Stage 1, Stage 2.
  *   qbar / qbar_chunk_stride as in dash_attn_block_summaries (used only when Kbar == NULL).
  *   Kbar      NULL: summaries are computed into the workspace; else used as given.

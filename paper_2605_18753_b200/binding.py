@@ -24,7 +24,7 @@ STATUS = {0: "DASH_OK", -1: "DASH_ERR_INVALID_ARG", -2: "DASH_ERR_UNSUPPORTED", 
 EXPORTS = [
     "dash_attn_workspace_bytes", "dash_attn_list_capacity", "dash_attn_list_offset",
     "dash_attn_block_summaries", "dash_attn_select", "dash_attn_attend_prefill", "dash_attn_attend_decode",
-    "dash_attn_attend_decode_static",
+    "dash_attn_attend_decode_static", "dash_attn_bwd_attend_prefill",
     "dash_attn_fwd_prefill", "dash_attn_fwd_decode", "dash_attn_reset_status", "dash_attn_last_status",
     "dash_attn_launch_count", "dash_attn_strerror", "dash_attn_test_hooks",
 ]
@@ -74,6 +74,8 @@ def lib() -> ctypes.CDLL:
         L.dash_attn_attend_decode.argtypes = [P] + [c_void_p] * 9 + [c_size_t, c_void_p]
         L.dash_attn_attend_decode_static.restype = ctypes.c_int
         L.dash_attn_attend_decode_static.argtypes = [P] + [c_void_p] * 9
+        L.dash_attn_bwd_attend_prefill.restype = ctypes.c_int
+        L.dash_attn_bwd_attend_prefill.argtypes = [P] + [c_void_p] * 11
         L.dash_attn_fwd_prefill.restype = ctypes.c_int
         L.dash_attn_fwd_prefill.argtypes = [P, c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_void_p, c_void_p,
                                             c_void_p, c_void_p, c_size_t, c_void_p]
@@ -242,6 +244,13 @@ def dash_attn_attend_decode_static(p, Q, Kc, Vc, kv_len, count, blk_idx, blk_bia
     _check(lib().dash_attn_attend_decode_static(ctypes.byref(p), _ptr(Q), _ptr(Kc), _ptr(Vc), _ptr(kv_len),
                                                 _ptr(count), _ptr(blk_idx), _ptr(blk_bias), _ptr(O), _stream()),
            "dash_attn_attend_decode_static")
+
+
+def dash_attn_bwd_attend_prefill(p, Q, K, V, dO, mask, blk_bias, dQ, dK, dV, dbias):
+    """Backward of Stage 2 (prefill) with the routing held fixed; dK / dV fp32 [b, n, h_kv, d], dbias like blk_bias."""
+    _check(lib().dash_attn_bwd_attend_prefill(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(dO), _ptr(mask),
+                                              _ptr(blk_bias), _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(dbias), _stream()),
+           "dash_attn_bwd_attend_prefill")
 
 
 def dash_attn_fwd_prefill(p, Q, K, V, O, workspace, qbar=None, qbar_chunk_stride=0, Kbar=None, mask_out=None):

@@ -245,6 +245,24 @@ int dash_attn_attend_decode(const dash_params* p, const void* Q, const void* Kca
                                              (cudaStream_t)stream));
 }
 
+int dash_attn_bwd_attend_prefill(const dash_params* p, const void* Q, const void* K, const void* V, const void* dO,
+                                 const uint32_t* mask, const float* blk_bias, void* dQ, float* dK, float* dV,
+                                 float* dbias, void* stream) {
+  Dims dm;
+  int rc = make_dims(p, &dm);
+  if (rc != DASH_OK) return rc;
+  if (dm.decode) return DASH_ERR_INVALID_ARG;
+  if (!Q || !K || !V || !dO || !mask || !dQ || !dK || !dV) return DASH_ERR_INVALID_ARG;
+  if (dm.list_rows > 0 && (!blk_bias || !dbias)) return DASH_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(dO) || !aligned16(dQ) || !aligned16(dK) ||
+      !aligned16(dV))
+    return DASH_ERR_INVALID_ARG;
+  if ((rc = check_device()) != DASH_OK) return rc;
+  StageRange nv("dash_attn: stage 2 prefill attention, backward");
+  return cuda_status(launch_attend_prefill_bwd_generic(dm, Q, K, V, dO, mask, blk_bias, dQ, dK, dV, dbias,
+                                                       (cudaStream_t)stream));
+}
+
 int dash_attn_fwd_prefill(const dash_params* p, const void* Q, const void* K, const void* V, const float* qbar,
                           int64_t qbar_chunk_stride, const float* Kbar, void* O, uint32_t* mask_out, void* workspace,
                           size_t workspace_bytes, void* stream) {

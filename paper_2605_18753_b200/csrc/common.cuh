@@ -204,6 +204,9 @@ cudaError_t launch_select_sm100(const Dims& dm, int token_limit, const void* Q, 
                                 StatusBlock* sb, cudaStream_t st, bool planes_ready = false);
 cudaError_t launch_attend_prefill_generic(const Dims& dm, const void* Q, const void* K, const void* V,
                                           const uint32_t* mask, const float* blk_bias, void* O, cudaStream_t st);
+cudaError_t launch_attend_prefill_bwd_generic(const Dims& dm, const void* Q, const void* K, const void* V,
+                                              const void* dO, const uint32_t* mask, const float* blk_bias, void* dQ,
+                                              float* dK, float* dV, float* dbias, cudaStream_t st);
 int decode_num_splits(const Dims& dm);
 size_t decode_partial_bytes(const Dims& dm);
 cudaError_t launch_attend_decode(const Dims& dm, const void* Q, const void* K, const void* V, const int* kv_len,

@@ -47,11 +47,14 @@ def routing_to_abi(routing: dict, p, list_offset_fn, device="cuda"):
     for (b, r, i), val in routing.items():
         rt = val[0] if isinstance(val, tuple) else val
         own = i // p.block if p.seq_q > 1 else None
-        mask[b, r, i if p.seq_q > 1 else 0] = orc.pack_mask_words(rt.support, own, W)
-        count[b, r, i if p.seq_q > 1 else 0] = rt.support.size
+        # window chunks close the list as ordinary entries with bias 0 (their bits set, counted), as the ABI states
+        members = np.concatenate([rt.support, rt.local]).astype(np.int64)
+        mask[b, r, i if p.seq_q > 1 else 0] = orc.pack_mask_words(members, own, W)
+        count[b, r, i if p.seq_q > 1 else 0] = members.size
         off = int(list_offset_fn(p, b, r, i if p.seq_q > 1 else 0))
-        idx[off:off + rt.support.size] = rt.support
+        idx[off:off + members.size] = members
         bias[off:off + rt.support.size] = rt.bias
+        bias[off + rt.support.size:off + members.size] = 0.0
     dev = lambda a: torch.from_numpy(a.view(np.int32) if a.dtype == np.uint32 else a).to(device)
     return dev(mask), dev(count), dev(idx), dev(bias)
 
