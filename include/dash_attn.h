@@ -218,6 +218,28 @@ int dash_attn_fwd_decode(const dash_params* p, const void* Q, const void* Kcache
                          const float* Kbar, const int32_t* kv_len, void* O, void* workspace,
                          size_t workspace_bytes, void* stream);
 
+/* Paged KV cache (the paper leaves the serving integration open; this is the decode path over a block-table cache as
+ * serving engines keep it, computing exactly what the contiguous calls compute).
+ *   Kpool, Vpool  pools of pages, [num_pages, page_size, h_kv, head_dim]: p->k_stride / p->v_stride are the element
+ *                 strides of (page, token inside the page, head).
+ *   page_table    int32 [batch, max_pages] (device): physical page of every logical page of every sequence; entries
+ *                 behind a sequence's kv_len are never read.
+ *   page_size     tokens per page: a multiple of 64 and of p->block, so that neither a chunk nor a 64-token tile
+ *                 straddles a page;  p->seq_kv must equal max_pages * page_size (the logical capacity).
+ * The summary cache Kbar stays contiguous per sequence ([batch, h_kv, T_s, head_dim], indexed by logical chunk), so
+ * Stage 1 is untouched; dash_attn_block_summaries_paged fills it from the paged keys, dash_attn_fwd_decode_paged is
+ * dash_attn_fwd_decode with the K / V tiles fetched page by page (one TMA box per 64-token tile, its outermost
+ * coordinate the physical page).  Both return DASH_ERR_INVALID_ARG for prefill shapes or a page size that breaks
+ * the rules above. */
+int dash_attn_block_summaries_paged(const dash_params* p, const void* Kpool, const int32_t* page_table,
+                                    int32_t page_size, int32_t max_pages, int32_t num_pages, const float* qbar,
+                                    int64_t qbar_chunk_stride, const int32_t* kv_len, int32_t first_block,
+                                    int32_t num_blocks, float* Kbar, void* stream);
+int dash_attn_fwd_decode_paged(const dash_params* p, const void* Q, const void* Kpool, const void* Vpool,
+                               const int32_t* page_table, int32_t page_size, int32_t max_pages, int32_t num_pages,
+                               const float* Kbar, const int32_t* kv_len, void* O, void* workspace,
+                               size_t workspace_bytes, void* stream);
+
 /* Zeroes the status word (enqueued on stream).  Call once after allocating a workspace, and again after an
  * error: the word is sticky (the first error wins), and while it is non-zero the tensor-core kernels launched
  * on that workspace retire without computing, so that one wait that ran out costs one wait limit, not one per

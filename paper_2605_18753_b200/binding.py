@@ -25,6 +25,7 @@ EXPORTS = [
     "dash_attn_workspace_bytes", "dash_attn_list_capacity", "dash_attn_list_offset",
     "dash_attn_block_summaries", "dash_attn_select", "dash_attn_attend_prefill", "dash_attn_attend_decode",
     "dash_attn_attend_decode_static", "dash_attn_bwd_attend_prefill",
+    "dash_attn_block_summaries_paged", "dash_attn_fwd_decode_paged",
     "dash_attn_fwd_prefill", "dash_attn_fwd_decode", "dash_attn_reset_status", "dash_attn_last_status",
     "dash_attn_launch_count", "dash_attn_strerror", "dash_attn_test_hooks",
 ]
@@ -81,6 +82,12 @@ def lib() -> ctypes.CDLL:
                                             c_void_p, c_void_p, c_size_t, c_void_p]
         L.dash_attn_fwd_decode.restype = ctypes.c_int
         L.dash_attn_fwd_decode.argtypes = [P] + [c_void_p] * 7 + [c_size_t, c_void_p]
+        L.dash_attn_block_summaries_paged.restype = ctypes.c_int
+        L.dash_attn_block_summaries_paged.argtypes = [P, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_void_p, c_int64,
+                                                      c_void_p, c_int32, c_int32, c_void_p, c_void_p]
+        L.dash_attn_fwd_decode_paged.restype = ctypes.c_int
+        L.dash_attn_fwd_decode_paged.argtypes = [P, c_void_p, c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32,
+                                                 c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
         L.dash_attn_reset_status.restype = ctypes.c_int
         L.dash_attn_reset_status.argtypes = [c_void_p, c_void_p]
         L.dash_attn_last_status.restype = ctypes.c_int
@@ -262,6 +269,31 @@ def dash_attn_fwd_prefill(p, Q, K, V, O, workspace, qbar=None, qbar_chunk_stride
 def dash_attn_fwd_decode(p, Q, Kc, Vc, Kbar, kv_len, O, workspace):
     _check(lib().dash_attn_fwd_decode(ctypes.byref(p), _ptr(Q), _ptr(Kc), _ptr(Vc), _ptr(Kbar), _ptr(kv_len),
                                       _ptr(O), _ptr(workspace), workspace.numel(), _stream()), "dash_attn_fwd_decode")
+
+
+def params_for_paged_decode(Q, Kpool, Vpool, O, *, max_pages, block, alpha, gamma=1.0, sigma=10.0, local_blocks=0):
+    """Decode parameters over pools [num_pages, page_size, h_kv, d]: seq_kv is the logical capacity max_pages * page_size
+    and the K / V strides are those of (page, token in page, head)."""
+    b, h_q, d = Q.shape
+    return make_params(batch=b, seq_q=1, seq_kv=max_pages * Kpool.shape[1], h_q=h_q, h_kv=Kpool.shape[2], head_dim=d,
+                       block=block, dtype=Q.dtype, alpha=alpha, gamma=gamma, sigma=sigma, local_blocks=local_blocks,
+                       q_stride=_strides3(Q, True), k_stride=_strides3(Kpool), v_stride=_strides3(Vpool),
+                       o_stride=_strides3(O, True))
+
+
+def dash_attn_block_summaries_paged(p, Kpool, page_table, Kbar, qbar=None, qbar_chunk_stride=0, kv_len=None,
+                                    first_block=0, num_blocks=-1):
+    _check(lib().dash_attn_block_summaries_paged(ctypes.byref(p), _ptr(Kpool), _ptr(page_table), Kpool.shape[1],
+                                                 page_table.shape[1], Kpool.shape[0], _ptr(qbar), qbar_chunk_stride,
+                                                 _ptr(kv_len), first_block, num_blocks, _ptr(Kbar), _stream()),
+           "dash_attn_block_summaries_paged")
+
+
+def dash_attn_fwd_decode_paged(p, Q, Kpool, Vpool, page_table, Kbar, kv_len, O, workspace):
+    _check(lib().dash_attn_fwd_decode_paged(ctypes.byref(p), _ptr(Q), _ptr(Kpool), _ptr(Vpool), _ptr(page_table),
+                                            Kpool.shape[1], page_table.shape[1], Kpool.shape[0], _ptr(Kbar), _ptr(kv_len),
+                                            _ptr(O), _ptr(workspace), workspace.numel(), _stream()),
+           "dash_attn_fwd_decode_paged")
 
 
 def dash_attn_reset_status(workspace):

@@ -133,6 +133,19 @@ static int check_workspace(const Dims& dm, void* ws, size_t bytes, WorkspaceLayo
   return DASH_OK;
 }
 
+// Adds the description of a paged KV cache to a decode problem (see the header for the rules).
+static int add_paging(Dims* dm, const int32_t* page_table, int page_size, int max_pages, int num_pages) {
+  if (!dm->decode) return DASH_ERR_INVALID_ARG;
+  if (!page_table || page_size <= 0 || max_pages <= 0 || num_pages <= 0) return DASH_ERR_INVALID_ARG;
+  if (page_size % 64 != 0 || page_size % dm->B != 0) return DASH_ERR_INVALID_ARG;
+  if ((long long)max_pages * page_size != dm->seq_kv) return DASH_ERR_INVALID_ARG;
+  dm->page_table = page_table;
+  dm->page_size = page_size;
+  dm->max_pages = max_pages;
+  dm->num_pages = num_pages;
+  return DASH_OK;
+}
+
 int validate_params(const dash_params* p, Dims* dm) { return make_dims(p, dm); }
 int validate_device() { return check_device(); }
 
@@ -187,6 +200,26 @@ int dash_attn_block_summaries(const dash_params* p, const void* K, const float* 
   if ((rc = check_device()) != DASH_OK) return rc;
   StageRange nv("dash_attn: stage 0 summaries");
   return cuda_status(launch_summaries(dm, K, qbar, qbar_chunk_stride, kv_len, first_block, num_blocks, Kbar, nullptr,
+                                      (cudaStream_t)stream));
+}
+
+int dash_attn_block_summaries_paged(const dash_params* p, const void* Kpool, const int32_t* page_table,
+                                    int32_t page_size, int32_t max_pages, int32_t num_pages, const float* qbar,
+                                    int64_t qbar_chunk_stride, const int32_t* kv_len, int32_t first_block,
+                                    int32_t num_blocks, float* Kbar, void* stream) {
+  Dims dm;
+  int rc = make_dims(p, &dm);
+  if (rc != DASH_OK) return rc;
+  if ((rc = add_paging(&dm, page_table, page_size, max_pages, num_pages)) != DASH_OK) return rc;
+  if (!Kpool || !aligned16(Kpool)) return DASH_ERR_INVALID_ARG;
+  if (dm.T_s > 0 && (!Kbar || !aligned16(Kbar))) return DASH_ERR_INVALID_ARG;
+  if (qbar && (!aligned16(qbar) || qbar_chunk_stride < 0 || qbar_chunk_stride % 4 != 0)) return DASH_ERR_INVALID_ARG;
+  if (first_block < 0 || first_block > dm.T_s) return DASH_ERR_INVALID_ARG;
+  if (num_blocks < 0) num_blocks = dm.T_s - first_block;
+  if (first_block + num_blocks > dm.T_s) return DASH_ERR_INVALID_ARG;
+  if ((rc = check_device()) != DASH_OK) return rc;
+  StageRange nv("dash_attn: stage 0 summaries");
+  return cuda_status(launch_summaries(dm, Kpool, qbar, qbar_chunk_stride, kv_len, first_block, num_blocks, Kbar, nullptr,
                                       (cudaStream_t)stream));
 }
 
@@ -331,6 +364,37 @@ int dash_attn_fwd_decode(const dash_params* p, const void* Q, const void* Kcache
   }
   StageRange nv("dash_attn: stage 2 decode attention");
   return cuda_status(launch_attend_decode_ex(dm, Q, Kcache, Vcache, kv_len, count, idx, bias, O,
+                                             at<float>(workspace, wl.partials), sb, st));
+}
+
+int dash_attn_fwd_decode_paged(const dash_params* p, const void* Q, const void* Kpool, const void* Vpool,
+                               const int32_t* page_table, int32_t page_size, int32_t max_pages, int32_t num_pages,
+                               const float* Kbar, const int32_t* kv_len, void* O, void* workspace,
+                               size_t workspace_bytes, void* stream) {
+  Dims dm;
+  int rc = make_dims(p, &dm);
+  if (rc != DASH_OK) return rc;
+  if ((rc = add_paging(&dm, page_table, page_size, max_pages, num_pages)) != DASH_OK) return rc;
+  if (!Q || !Kpool || !Vpool || !O) return DASH_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(Kpool) || !aligned16(Vpool) || !aligned16(O)) return DASH_ERR_INVALID_ARG;
+  if (dm.T_s > 0 && (!Kbar || !aligned16(Kbar))) return DASH_ERR_INVALID_ARG;
+  WorkspaceLayout wl;
+  if ((rc = check_workspace(dm, workspace, workspace_bytes, &wl)) != DASH_OK) return rc;
+  if ((rc = check_device()) != DASH_OK) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  StatusBlock* sb = at<StatusBlock>(workspace, wl.status);
+  int* count = at<int>(workspace, wl.count);
+  int* idx = at<int>(workspace, wl.blk_idx);
+  float* bias = at<float>(workspace, wl.blk_bias);
+  {
+    // Stage 1 reads the summary cache only, which is indexed by logical chunk: paging does not reach it
+    StageRange nv("dash_attn: stage 1 routing");
+    if ((rc = cuda_status(launch_select(dm, Q, Kbar, kv_len, at<uint32_t>(workspace, wl.mask), count, idx, bias, nullptr,
+                                        at<void>(workspace, wl.planes), at<float>(workspace, wl.xscratch), sb, st))) != DASH_OK)
+      return rc;
+  }
+  StageRange nv("dash_attn: stage 2 decode attention");
+  return cuda_status(launch_attend_decode_ex(dm, Q, Kpool, Vpool, kv_len, count, idx, bias, O,
                                              at<float>(workspace, wl.partials), sb, st));
 }
 

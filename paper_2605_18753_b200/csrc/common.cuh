@@ -27,7 +27,24 @@ struct Dims {
   float inv_sigma;
   long long qs[3], ks[3], vs[3], os[3];
   long long list_rows;  // list entries per (batch, KV head)
+  // Paged KV cache (decode only): K / V are pools [num_pages, page_size, h_kv, d] (ks / vs = strides of page, token,
+  // head) and logical page lp of sequence b is physical page page_table[b * max_pages + lp].  nullptr: contiguous.
+  const int* page_table;
+  int page_size, max_pages, num_pages;
 };
+
+// Where KV token t of sequence b lives: address = first * stride[0] + tok * stride[1] (+ head * stride[2]).  A chunk
+// and a 64-token sub-block never straddle a page (page_size is a multiple of both).
+__device__ inline void kv_locate(const Dims& dm, int b, int t, int* first, int* tok) {
+  if (dm.page_table) {
+    const int lp = t / dm.page_size;
+    *first = __ldg(dm.page_table + (long long)b * dm.max_pages + lp);
+    *tok = t - lp * dm.page_size;
+  } else {
+    *first = b;
+    *tok = t;
+  }
+}
 
 // Start of row i's list region inside its (batch, KV head) slab.
 __host__ __device__ inline long long list_row_offset(const Dims& dm, int i) {

@@ -91,8 +91,6 @@ decode_split_kernel(Dims dm, int n_split, const T* __restrict__ Q, const T* __re
   }
   __syncthreads();
 
-  const T* kbase = K + (long long)b * dm.ks[0] + (long long)r * dm.ks[2];
-  const T* vbase = V + (long long)b * dm.vs[0] + (long long)r * dm.vs[2];
   const long long loff = grp * dm.list_rows;
 
   float m[G], l[G], acc[G][VPL];
@@ -113,6 +111,11 @@ decode_split_kernel(Dims dm, int n_split, const T* __restrict__ Q, const T* __re
     } else {
       c = c_own; bias = 0.f; t_end = L;
     }
+    // the chunk's rows: token t of the chunk sits at kbase + t * stride (contiguous cache or inside one page)
+    int cfirst, ctok;
+    kv_locate(dm, b, c * dm.B, &cfirst, &ctok);
+    const T* kbase = K + (long long)cfirst * dm.ks[0] + (long long)r * dm.ks[2] + (long long)(ctok - c * dm.B) * dm.ks[1];
+    const T* vbase = V + (long long)cfirst * dm.vs[0] + (long long)r * dm.vs[2] + (long long)(ctok - c * dm.B) * dm.vs[1];
     for (int t0 = c * dm.B; t0 < t_end; t0 += 32) {
       const int t = t0 + lane;
       float s[G];

@@ -53,7 +53,8 @@ struct MiscT {
   float red[2][4][NH];
   float lred[4][NH];
   int is_last;               // this block saw the last arrival of its (batch, KV head)
-  int idx_s[RANGE][CPS];     // first KV token of each chunk slot of each owned sub-block
+  int idx_s[RANGE][CPS];     // first KV token of each chunk slot of each owned sub-block (paged cache: inside its page)
+  int pg_s[RANGE][CPS];      // outermost TMA coordinate of the slot: the sequence, or the physical page
   float bias_s[RANGE][CPS];
   int nval_s[RANGE];         // valid rows of the sub-block
 };
@@ -176,7 +177,7 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
 #pragma unroll
           for (int s = 0; s < CPS; ++s) {
             const int e = e0 + min(s, m - 1);
-            misc->idx_s[k][s] = a.blk_idx[loff + e] * dm.B;
+            kv_locate(dm, b, a.blk_idx[loff + e] * dm.B, &misc->pg_s[k][s], &misc->idx_s[k][s]);
             misc->bias_s[k][s] = a.blk_bias[loff + e];
           }
           misc->nval_s[k] = m * dm.B;
@@ -184,7 +185,7 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
           // the own chunk (shorter than a sub-block): the rows behind it are fetched but marked invalid
 #pragma unroll
           for (int s = 0; s < CPS; ++s) {
-            misc->idx_s[k][s] = c_own * dm.B + s * W;
+            kv_locate(dm, b, c_own * dm.B + s * W, &misc->pg_s[k][s], &misc->idx_s[k][s]);
             misc->bias_s[k][s] = 0.f;
           }
           misc->nval_s[k] = L - c_own * dm.B;
@@ -204,7 +205,8 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         bs = 0.f;
         nv = min(SUB, L - tok0);
       }
-      misc->idx_s[k][0] = tok0; misc->bias_s[k][0] = bs; misc->nval_s[k] = nv;
+      kv_locate(dm, b, tok0, &misc->pg_s[k][0], &misc->idx_s[k][0]);
+      misc->bias_s[k][0] = bs; misc->nval_s[k] = nv;
     }
     __syncwarp();
     if (lane == 0) {
@@ -222,10 +224,10 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             const int k = h ? k1 : k0;
 #pragma unroll
             for (int q = 0; q < CPS; ++q) {
-              const int tok = misc->idx_s[k][q];
+              const int tok = misc->idx_s[k][q], pg = misc->pg_s[k][q];
               const uint32_t d = dst + (h * SUB + q * W) * 128;
-              ptx::tma_load_4d(d, tm, barrier, 0, r, tok, b);
-              if constexpr (HD == 128) ptx::tma_load_4d(d + TILE_BYTES / 2, tm, barrier, 64, r, tok, b);
+              ptx::tma_load_4d(d, tm, barrier, 0, r, tok, pg);
+              if constexpr (HD == 128) ptx::tma_load_4d(d + TILE_BYTES / 2, tm, barrier, 64, r, tok, pg);
             }
           }
         };
@@ -497,7 +499,9 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
 }
 
 bool make_kv_map(CUtensorMap* out, const void* base, const Dims& dm, const long long* s) {
-  cuuint64_t dims[4] = {(cuuint64_t)dm.d, (cuuint64_t)dm.h_kv, (cuuint64_t)dm.seq_kv, (cuuint64_t)dm.batch};
+  // contiguous cache: [batch][seq_kv] tokens; paged cache: [num_pages][page_size]
+  cuuint64_t dims[4] = {(cuuint64_t)dm.d, (cuuint64_t)dm.h_kv, (cuuint64_t)(dm.page_table ? dm.page_size : dm.seq_kv),
+                        (cuuint64_t)(dm.page_table ? dm.num_pages : dm.batch)};
   auto st = [](long long e) { return (cuuint64_t)((e > 0 ? e : 8) * 2); };
   cuuint64_t strides[3] = {st(s[2]), st(s[1]), st(s[0])};
   cuuint32_t box[4] = {64u, 1u, (cuuint32_t)(dm.B < SUB ? dm.B : SUB), 1u};   // chunks below 64 tokens: one box per chunk

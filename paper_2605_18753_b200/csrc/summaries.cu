@@ -30,7 +30,9 @@ summaries_kernel(Dims dm, const T* __restrict__ K, const float* __restrict__ qba
   const int len = kv_len ? min(kv_len[b], dm.seq_kv) : dm.seq_kv;
   if ((long long)(c + 1) * dm.B > len) return;  // chunk not complete: no summary (Algorithm 1 step 1)
 
-  const T* kp = K + (long long)b * dm.ks[0] + (long long)c * dm.B * dm.ks[1] + (long long)r * dm.ks[2] + lane * VPL;
+  int kfirst, ktok;
+  kv_locate(dm, b, c * dm.B, &kfirst, &ktok);       // contiguous cache: (b, c * B); paged: (physical page, offset in it)
+  const T* kp = K + (long long)kfirst * dm.ks[0] + (long long)ktok * dm.ks[1] + (long long)r * dm.ks[2] + lane * VPL;
   float acc[VPL];
 #pragma unroll
   for (int v = 0; v < VPL; ++v) acc[v] = 0.f;
