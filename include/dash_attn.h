@@ -198,10 +198,35 @@ int dash_attn_attend_decode_static(const dash_params* p, const void* Q, const vo
  *   dO     incoming gradient of O, dtype p->dtype, strides p->o_stride.
  * mask / blk_bias as written by dash_attn_select for the same parameters.  This is a correctness path on CUDA cores
  * (one warp per row and head, fp32 atomics for dK / dV / dbias, so their last bits vary from run to run); it needs
- * no workspace.  The gradient through the routing itself (Stage 1, Stage 0) is not computed by the library. */
+ * no workspace.  dash_attn_bwd_select_prefill and dash_attn_bwd_block_summaries carry dbias on through the routing. */
 int dash_attn_bwd_attend_prefill(const dash_params* p, const void* Q, const void* K, const void* V, const void* dO,
                                  const uint32_t* mask, const float* blk_bias, void* dQ, float* dK, float* dV,
                                  float* dbias, void* stream);
+
+/* Backward of Stage 1 (prefill, causal): carries dbias on through the log-prior bias (Proposition 1), the group average
+ * (Section 3.2) and the alpha-entmax of every head (Eq. 2) to the queries and the chunk summaries.  Inside a region
+ * of fixed support the entmax Jacobian is diag(s) - s s^T / sum(s) with s = p^(2 - alpha) on the support and zero
+ * elsewhere (derived from Eq. 2; the appendix "The alpha-entmax mapping" states that such a closed form exists), so
+ * only the routed chunks of a row are visited: the forward pass's list is reused (Section 3.5).
+ *   count, blk_idx, tau   as written by dash_attn_select for the same parameters (blk_idx and tau requested).
+ *   dbias      fp32, layout of blk_bias: gradient w.r.t. every bias entry (dash_attn_bwd_attend_prefill writes it).
+ *   dQ_route   fp32, contiguous [batch, seq_q, h_q, head_dim]: the part of dL/dQ that flows through the routing; the
+ *              caller adds it to the Stage-2 part (every row is written, zeros where nothing is routed).
+ *   dKbar      fp32 [batch, h_kv, T_s, head_dim]: gradient w.r.t. the summaries; zeroed, then accumulated (atomics).
+ * CUDA-core correctness path.  Rows whose support holds a chunk sitting on the threshold have no gradient in the
+ * mathematical sense (the map is piecewise differentiable); the kernel then returns the one-sided value of Eq. 2. */
+int dash_attn_bwd_select_prefill(const dash_params* p, const void* Q, const float* Kbar, const int32_t* count,
+                                 const int32_t* blk_idx, const float* tau, const float* dbias, float* dQ_route,
+                                 float* dKbar, void* stream);
+
+/* Backward of Stage 0 (Eq. 3): adds to dK what reaches the keys through their chunk's summary and returns the gradient
+ * of the summary query.
+ *   qbar / qbar_chunk_stride   as in dash_attn_block_summaries (NULL: mean pooling).
+ *   dKbar   fp32 [batch, h_kv, T_s, head_dim].
+ *   dK      fp32, contiguous [batch, seq_kv, h_kv, head_dim]: ADDED to (it usually already holds the Stage-2 part).
+ *   dqbar   fp32, shape of qbar (zeroed, then accumulated); ignored when qbar is NULL. */
+int dash_attn_bwd_block_summaries(const dash_params* p, const void* K, const float* qbar, int64_t qbar_chunk_stride,
+                                  const float* dKbar, float* dK, float* dqbar, void* stream);
 
 /* Whole prefill forward: Stage 0 (skipped when Kbar is given), Stage 1, Stage 2.
  *   qbar / qbar_chunk_stride as in dash_attn_block_summaries (used only when Kbar == NULL).

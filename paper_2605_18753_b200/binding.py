@@ -26,6 +26,7 @@ EXPORTS = [
     "dash_attn_block_summaries", "dash_attn_select", "dash_attn_attend_prefill", "dash_attn_attend_decode",
     "dash_attn_attend_decode_static", "dash_attn_bwd_attend_prefill",
     "dash_attn_block_summaries_paged", "dash_attn_fwd_decode_paged",
+    "dash_attn_bwd_select_prefill", "dash_attn_bwd_block_summaries",
     "dash_attn_fwd_prefill", "dash_attn_fwd_decode", "dash_attn_reset_status", "dash_attn_last_status",
     "dash_attn_launch_count", "dash_attn_strerror", "dash_attn_test_hooks",
 ]
@@ -77,6 +78,10 @@ def lib() -> ctypes.CDLL:
         L.dash_attn_attend_decode_static.argtypes = [P] + [c_void_p] * 9
         L.dash_attn_bwd_attend_prefill.restype = ctypes.c_int
         L.dash_attn_bwd_attend_prefill.argtypes = [P] + [c_void_p] * 11
+        L.dash_attn_bwd_select_prefill.restype = ctypes.c_int
+        L.dash_attn_bwd_select_prefill.argtypes = [P] + [c_void_p] * 9
+        L.dash_attn_bwd_block_summaries.restype = ctypes.c_int
+        L.dash_attn_bwd_block_summaries.argtypes = [P, c_void_p, c_void_p, c_int64, c_void_p, c_void_p, c_void_p, c_void_p]
         L.dash_attn_fwd_prefill.restype = ctypes.c_int
         L.dash_attn_fwd_prefill.argtypes = [P, c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_void_p, c_void_p,
                                             c_void_p, c_void_p, c_size_t, c_void_p]
@@ -258,6 +263,19 @@ def dash_attn_bwd_attend_prefill(p, Q, K, V, dO, mask, blk_bias, dQ, dK, dV, dbi
     _check(lib().dash_attn_bwd_attend_prefill(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(dO), _ptr(mask),
                                               _ptr(blk_bias), _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(dbias), _stream()),
            "dash_attn_bwd_attend_prefill")
+
+
+def dash_attn_bwd_select_prefill(p, Q, Kbar, count, blk_idx, tau, dbias, dQ_route, dKbar):
+    """Backward of Stage 1 (prefill): dbias -> dQ_route (fp32 [b, n, h_q, d]) and dKbar (fp32 like Kbar)."""
+    _check(lib().dash_attn_bwd_select_prefill(ctypes.byref(p), _ptr(Q), _ptr(Kbar), _ptr(count), _ptr(blk_idx), _ptr(tau),
+                                              _ptr(dbias), _ptr(dQ_route), _ptr(dKbar), _stream()),
+           "dash_attn_bwd_select_prefill")
+
+
+def dash_attn_bwd_block_summaries(p, K, dKbar, dK, qbar=None, qbar_chunk_stride=0, dqbar=None):
+    """Backward of Stage 0: adds the summaries' share to dK (fp32 [b, n, h_kv, d]); dqbar gets the summary query's gradient."""
+    _check(lib().dash_attn_bwd_block_summaries(ctypes.byref(p), _ptr(K), _ptr(qbar), qbar_chunk_stride, _ptr(dKbar),
+                                               _ptr(dK), _ptr(dqbar), _stream()), "dash_attn_bwd_block_summaries")
 
 
 def dash_attn_fwd_prefill(p, Q, K, V, O, workspace, qbar=None, qbar_chunk_stride=0, Kbar=None, mask_out=None):

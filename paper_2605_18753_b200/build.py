@@ -12,7 +12,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libdash_attn.so")
 OBJ_DIR = os.path.join(PKG, "build")
-SOURCES = ["api.cu", "summaries.cu", "select.cu", "select_sm100.cu", "select_decode.cu", "attend_generic.cu", "attend_bwd_generic.cu", "decode.cu", "decode_sm100.cu", "prefill_sm100.cu"]
+SOURCES = ["api.cu", "summaries.cu", "select.cu", "select_sm100.cu", "select_decode.cu", "attend_generic.cu", "attend_bwd_generic.cu", "route_bwd_generic.cu", "decode.cu", "decode_sm100.cu", "prefill_sm100.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "--use_fast_math", "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 

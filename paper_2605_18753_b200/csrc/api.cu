@@ -296,6 +296,37 @@ int dash_attn_bwd_attend_prefill(const dash_params* p, const void* Q, const void
                                                        (cudaStream_t)stream));
 }
 
+int dash_attn_bwd_select_prefill(const dash_params* p, const void* Q, const float* Kbar, const int32_t* count,
+                                 const int32_t* blk_idx, const float* tau, const float* dbias, float* dQ_route,
+                                 float* dKbar, void* stream) {
+  Dims dm;
+  int rc = make_dims(p, &dm);
+  if (rc != DASH_OK) return rc;
+  if (dm.decode || !dm.causal) return DASH_ERR_UNSUPPORTED;
+  if (!Q || !count || !dQ_route || !aligned16(Q)) return DASH_ERR_INVALID_ARG;
+  if (dm.T_s > 0 && (!Kbar || !blk_idx || !tau || !dbias || !dKbar)) return DASH_ERR_INVALID_ARG;
+  if ((rc = check_device()) != DASH_OK) return rc;
+  StageRange nv("dash_attn: stage 1 routing, backward");
+  return cuda_status(launch_route_bwd(dm, Q, Kbar, count, blk_idx, tau, dbias, dQ_route, dKbar, (cudaStream_t)stream));
+}
+
+int dash_attn_bwd_block_summaries(const dash_params* p, const void* K, const float* qbar, int64_t qbar_chunk_stride,
+                                  const float* dKbar, float* dK, float* dqbar, void* stream) {
+  Dims dm;
+  int rc = make_dims(p, &dm);
+  if (rc != DASH_OK) return rc;
+  if (dm.decode) return DASH_ERR_UNSUPPORTED;
+  if (!K || !dK || !aligned16(K)) return DASH_ERR_INVALID_ARG;
+  if (dm.T_s > 0 && !dKbar) return DASH_ERR_INVALID_ARG;
+  if (qbar && (qbar_chunk_stride < 0 || qbar_chunk_stride % 4 != 0)) return DASH_ERR_INVALID_ARG;
+  if ((rc = check_device()) != DASH_OK) return rc;
+  const size_t dq_bytes = !qbar ? 0 : (qbar_chunk_stride == 0 ? (size_t)dm.h_kv * dm.d
+                                                               : (size_t)dm.T_s * (size_t)qbar_chunk_stride) * sizeof(float);
+  StageRange nv("dash_attn: stage 0 summaries, backward");
+  return cuda_status(launch_summaries_bwd(dm, K, qbar, qbar_chunk_stride, dKbar, dK, qbar ? dqbar : nullptr, dq_bytes,
+                                          (cudaStream_t)stream));
+}
+
 int dash_attn_fwd_prefill(const dash_params* p, const void* Q, const void* K, const void* V, const float* qbar,
                           int64_t qbar_chunk_stride, const float* Kbar, void* O, uint32_t* mask_out, void* workspace,
                           size_t workspace_bytes, void* stream) {

@@ -224,6 +224,10 @@ cudaError_t launch_attend_prefill_generic(const Dims& dm, const void* Q, const v
 cudaError_t launch_attend_prefill_bwd_generic(const Dims& dm, const void* Q, const void* K, const void* V,
                                               const void* dO, const uint32_t* mask, const float* blk_bias, void* dQ,
                                               float* dK, float* dV, float* dbias, cudaStream_t st);
+cudaError_t launch_route_bwd(const Dims& dm, const void* Q, const float* Kbar, const int* count, const int* blk_idx,
+                             const float* tau, const float* dbias, float* dQr, float* dKbar, cudaStream_t st);
+cudaError_t launch_summaries_bwd(const Dims& dm, const void* K, const float* qbar, long long qbar_chunk_stride,
+                                 const float* dKbar, float* dK, float* dqbar, size_t dqbar_bytes, cudaStream_t st);
 int decode_num_splits(const Dims& dm);
 size_t decode_partial_bytes(const Dims& dm);
 cudaError_t launch_attend_decode(const Dims& dm, const void* Q, const void* K, const void* V, const int* kv_len,
