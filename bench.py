@@ -272,7 +272,7 @@ def run_paper_protocol(args):
     rows = []
     gen = torch.Generator(device=dev)
     gen.manual_seed(0)
-    for n in (16384, 32768, 65536):
+    for n in (16384, 32768, 65536, 98304):
         Q = torch.randn(1, n, h_q, d, generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
         K = torch.randn(1, n, h_kv, d, generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
         V = torch.randn(1, n, h_kv, d, generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
@@ -308,7 +308,7 @@ def run_paper_protocol(args):
 
     # decode: batch 24, one query per sequence, random routed lists
     bs = 24
-    for n in (16384, 32768, 65536):
+    for n in (16384, 32768, 65536, 98304):
         q1 = torch.randn(bs, h_q, d, generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
         Kc = torch.randn(bs, n, h_kv, d, generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
         Vc = torch.randn(bs, n, h_kv, d, generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
