@@ -489,6 +489,39 @@ def measure_decode(B, synth, wd, dev, peaks, flush, iters=30) -> dict:
     return out
 
 
+def measure_backward(B, synth, w, dev, flush, iters=3) -> dict:
+    """The backward chain (CUDA-core correctness kernels: Stage 2, then routing, then summaries) on one workload:
+    milliseconds only -- these kernels are parity-graded, not tuned."""
+    inp = synth.make_prefill_inputs(w, dev)
+    Q, K, V = inp["Q"], inp["K"], inp["V"]
+    dO = torch.randn(Q.shape, device=dev, dtype=torch.float32).to(Q.dtype)
+    p = B.params_for_prefill(Q, K, V, dO, block=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma)
+    ws, rt, kbar = B.alloc_workspace(p, dev), B.alloc_routing(p, dev, with_tau=True), B.alloc_kbar(p, dev)
+    B.dash_attn_block_summaries(p, K, kbar)
+    B.dash_attn_select(p, Q, kbar, rt["mask"], rt["count"], rt["blk_idx"], rt["blk_bias"], ws, tau=rt["tau"])
+    dQ = torch.empty_like(Q)
+    dK = torch.empty(w.batch, w.seq, w.h_kv, w.head_dim, device=dev)
+    dV = torch.empty_like(dK)
+    dbias = torch.empty_like(rt["blk_bias"])
+    dQr = torch.empty(w.batch, w.seq, w.h_q, w.head_dim, device=dev)
+    dKbar = torch.empty_like(kbar)
+    out = {"workload": f"{w.name} cut to {w.seq} tokens", "kernels": "CUDA-core correctness path (one warp per row and head, fp32 atomics)"}
+    for name, fn in (("stage2_ms", lambda: B.dash_attn_bwd_attend_prefill(p, Q, K, V, dO, rt["mask"], rt["blk_bias"], dQ, dK, dV, dbias)),
+                     ("routing_ms", lambda: B.dash_attn_bwd_select_prefill(p, Q, kbar, rt["count"], rt["blk_idx"], rt["tau"], dbias, dQr, dKbar)),
+                     ("summaries_ms", lambda: B.dash_attn_bwd_block_summaries(p, K, dKbar, dK))):
+        fn()
+        ts = []
+        for k in range(iters):
+            flush.fill_(k)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); fn(); b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        out[name] = float(np.median(ts))
+    assert torch.isfinite(dQ.float()).all() and torch.isfinite(dK).all() and torch.isfinite(dQr).all()
+    return out
+
+
 def all_config_measurements(B, synth, dev, peaks, flush) -> dict:
     """Every other configuration of the task beside the headline: the 64K prefill at two sparsities, the
     (chunk size, alpha) sweep at 32K x batch 2, the 8K prefill with finer chunks, and the decode workload."""
@@ -518,6 +551,7 @@ def all_config_measurements(B, synth, dev, peaks, flush) -> dict:
         guarded(name, lambda name=name: measure_prefill(B, synth, synth.workload(name), dev, peaks, iters=10, flush=flush,
                                                         with_sdpa=False))
     guarded("decode_128k", lambda: measure_decode(B, synth, synth.workload("decode_128k"), dev, peaks, flush))
+    guarded("backward_2k", lambda: measure_backward(B, synth, synth.workload("prefill_8k", seq=2048), dev, flush))
     return out
 
 
