@@ -14,6 +14,7 @@ import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libdash_attn.so")
+DEBUG_LIB_PATH = os.path.join(_PKG, "libdash_attn_debug.so")    # same library with bounds checks compiled in
 
 DASH_F32, DASH_BF16 = 0, 1
 DASH_OK = 0
@@ -105,6 +106,26 @@ def lib() -> ctypes.CDLL:
         L.dash_attn_strerror.argtypes = [ctypes.c_int]
         _lib = L
     return _lib
+
+
+class use_debug_library:
+    """Context manager: inside it every binding call goes to libdash_attn_debug.so (built by
+    `python -m paper_2605_18753_b200.build --debug`), whose kernels check every index they read from device memory
+    and record DASH_ERR_CAPACITY instead of making a bad access.  Raises if that library has not been built."""
+
+    def __enter__(self):
+        global _lib, LIB_PATH
+        if not os.path.exists(DEBUG_LIB_PATH):
+            raise RuntimeError(f"{DEBUG_LIB_PATH} is missing: build it with `python -m paper_2605_18753_b200.build --debug`")
+        self._saved = (_lib, LIB_PATH)
+        _lib, LIB_PATH = None, DEBUG_LIB_PATH
+        lib()
+        return self
+
+    def __exit__(self, *exc):
+        global _lib, LIB_PATH
+        _lib, LIB_PATH = self._saved
+        return False
 
 
 def strerror(code: int) -> str:

@@ -75,6 +75,22 @@ __device__ inline void report_error(StatusBlock* sb, int status, int detail) {
   if (atomicCAS(&sb->status, 0, status) == 0) sb->detail = detail;
 }
 
+// Bounds checks of everything a kernel indexes with values it read from device memory (list entries, counts): compiled
+// in with -DDASH_DEBUG (the debug library), absent from the production build, which trusts the routing outputs it is
+// handed.  A failed check records DASH_ERR_CAPACITY with a site code in the status word (when the call has one) and
+// runs `fallback`, which must avoid the access; it never traps.
+#ifdef DASH_DEBUG
+// no do-while wrapper: `fallback` may be a `continue` or `break` of the loop the check sits in
+#define DASH_CHECK(cond, sb, code, fallback)     \
+  if (!(cond)) {                                 \
+    report_error(sb, DASH_ERR_CAPACITY, code);   \
+    fallback;                                    \
+  } else                                         \
+    ((void)0)
+#else
+#define DASH_CHECK(cond, sb, code, fallback) ((void)0)
+#endif
+
 template <typename T> __device__ inline float to_f32(T v);
 template <> __device__ inline float to_f32<float>(float v) { return v; }
 template <> __device__ inline float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
@@ -232,7 +248,7 @@ int decode_num_splits(const Dims& dm);
 size_t decode_partial_bytes(const Dims& dm);
 cudaError_t launch_attend_decode(const Dims& dm, const void* Q, const void* K, const void* V, const int* kv_len,
                                  const int* count, const int* blk_idx, const float* blk_bias, void* O,
-                                 float* partials, cudaStream_t st);
+                                 float* partials, StatusBlock* sb, cudaStream_t st);
 cudaError_t launch_attend_decode_ex(const Dims& dm, const void* Q, const void* K, const void* V, const int* kv_len,
                                     const int* count, const int* blk_idx, const float* blk_bias, void* O,
                                     float* partials, StatusBlock* sb, cudaStream_t st);

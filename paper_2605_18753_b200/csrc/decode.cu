@@ -63,7 +63,7 @@ __global__ void __launch_bounds__(DEC_WARPS * 32)
 decode_split_kernel(Dims dm, int n_split, const T* __restrict__ Q, const T* __restrict__ K, const T* __restrict__ V,
                     const int* __restrict__ kv_len, const int* __restrict__ count,
                     const int* __restrict__ blk_idx, const float* __restrict__ blk_bias,
-                    float* __restrict__ partials) {
+                    float* __restrict__ partials, StatusBlock* sb) {
   constexpr int VPL = D / 32;
   // the merge buffer reuses the query / probability staging space once the main loop is over
   constexpr int QS_N = G * D, PS_N = DEC_WARPS * 32 * G, RED_N = DEC_WARPS * G * (D + 2);
@@ -80,7 +80,8 @@ decode_split_kernel(Dims dm, int n_split, const T* __restrict__ Q, const T* __re
   L = max(1, min(L, dm.seq_kv));
   const int c_own = (L - 1) / dm.B;
   const long long grp = (long long)b * dm.h_kv + r;
-  const int n_routed = count[grp];
+  int n_routed = count[grp];
+  DASH_CHECK(n_routed >= 0 && n_routed <= min(c_own, dm.T_s), sb, 400, n_routed = 0);
   const int n_items = n_routed + 1;
   const int per = (n_items + n_split - 1) / n_split;
   const int lo = split * per, hi = min(n_items, lo + per);
@@ -107,6 +108,7 @@ decode_split_kernel(Dims dm, int n_split, const T* __restrict__ Q, const T* __re
     if (it < n_routed) {
       c = blk_idx[loff + it];
       bias = blk_bias[loff + it];
+      DASH_CHECK(c >= 0 && c < c_own, sb, 401, continue);       // routed and window chunks precede the own chunk
       t_end = (c + 1) * dm.B;
     } else {
       c = c_own; bias = 0.f; t_end = L;
@@ -114,6 +116,7 @@ decode_split_kernel(Dims dm, int n_split, const T* __restrict__ Q, const T* __re
     // the chunk's rows: token t of the chunk sits at kbase + t * stride (contiguous cache or inside one page)
     int cfirst, ctok;
     kv_locate(dm, b, c * dm.B, &cfirst, &ctok);
+    DASH_CHECK(!dm.page_table || (unsigned)cfirst < (unsigned)dm.num_pages, sb, 402, continue);   // a page id outside the pool
     const T* kbase = K + (long long)cfirst * dm.ks[0] + (long long)r * dm.ks[2] + (long long)(ctok - c * dm.B) * dm.ks[1];
     const T* vbase = V + (long long)cfirst * dm.vs[0] + (long long)r * dm.vs[2] + (long long)(ctok - c * dm.B) * dm.vs[1];
     for (int t0 = c * dm.B; t0 < t_end; t0 += 32) {
@@ -230,13 +233,13 @@ __global__ void decode_merge_kernel(Dims dm, int n_split, const float* __restric
 template <typename T, int D>
 static cudaError_t launch_dec(const Dims& dm, const void* Q, const void* K, const void* V, const int* kv_len,
                               const int* count, const int* blk_idx, const float* blk_bias, void* O,
-                              float* partials, cudaStream_t st) {
+                              float* partials, StatusBlock* sb, cudaStream_t st) {
   const int ns = decode_num_splits(dm);
   dim3 grid(ns, dm.h_kv, dm.batch);
   cudaError_t e = cudaSuccess;
 #define DASH_DEC(G)                                                                                              \
   e = launch_chained(decode_split_kernel<T, D, G>, grid, dim3(DEC_WARPS * 32), 0, st, dm, ns, (const T*)Q,       \
-                     (const T*)K, (const T*)V, kv_len, count, blk_idx, blk_bias, partials)
+                     (const T*)K, (const T*)V, kv_len, count, blk_idx, blk_bias, partials, sb)
   switch (dm.g_q) {
     case 1: DASH_DEC(1); break;
     case 2: DASH_DEC(2); break;
@@ -278,18 +281,18 @@ cudaError_t launch_attend_decode_ex(const Dims& dm, const void* Q, const void* K
     return dm.d == 128 ? launch_merge<__nv_bfloat16, 128>(dm, ns, partials, O, st)
                        : launch_merge<__nv_bfloat16, 64>(dm, ns, partials, O, st);
   }
-  return launch_attend_decode(dm, Q, K, V, kv_len, count, blk_idx, blk_bias, O, partials, st);
+  return launch_attend_decode(dm, Q, K, V, kv_len, count, blk_idx, blk_bias, O, partials, sb, st);
 }
 
 cudaError_t launch_attend_decode(const Dims& dm, const void* Q, const void* K, const void* V, const int* kv_len,
                                  const int* count, const int* blk_idx, const float* blk_bias, void* O,
-                                 float* partials, cudaStream_t st) {
+                                 float* partials, StatusBlock* sb, cudaStream_t st) {
   if (dm.dtype == DASH_BF16) {
-    if (dm.d == 128) return launch_dec<__nv_bfloat16, 128>(dm, Q, K, V, kv_len, count, blk_idx, blk_bias, O, partials, st);
-    return launch_dec<__nv_bfloat16, 64>(dm, Q, K, V, kv_len, count, blk_idx, blk_bias, O, partials, st);
+    if (dm.d == 128) return launch_dec<__nv_bfloat16, 128>(dm, Q, K, V, kv_len, count, blk_idx, blk_bias, O, partials, sb, st);
+    return launch_dec<__nv_bfloat16, 64>(dm, Q, K, V, kv_len, count, blk_idx, blk_bias, O, partials, sb, st);
   }
-  if (dm.d == 128) return launch_dec<float, 128>(dm, Q, K, V, kv_len, count, blk_idx, blk_bias, O, partials, st);
-  return launch_dec<float, 64>(dm, Q, K, V, kv_len, count, blk_idx, blk_bias, O, partials, st);
+  if (dm.d == 128) return launch_dec<float, 128>(dm, Q, K, V, kv_len, count, blk_idx, blk_bias, O, partials, sb, st);
+  return launch_dec<float, 64>(dm, Q, K, V, kv_len, count, blk_idx, blk_bias, O, partials, sb, st);
 }
 
 }  // namespace dash
@@ -343,7 +346,7 @@ extern "C" int dash_attn_attend_decode_static(const dash_params* p, const void* 
   if (decode_static_scratch(&scratch) != cudaSuccess) return DASH_ERR_CUDA;
   // every partial slot that the merge kernel reads is written by the split kernel of the same call,
   // so nothing left over from an earlier call needs clearing
-  return launch_attend_decode(dm, Q, Kcache, Vcache, kv_len, count, blk_idx, blk_bias, O, scratch,
+  return launch_attend_decode(dm, Q, Kcache, Vcache, kv_len, count, blk_idx, blk_bias, O, scratch, nullptr,
                               (cudaStream_t)stream) == cudaSuccess ? DASH_OK : DASH_ERR_CUDA;
 }
 

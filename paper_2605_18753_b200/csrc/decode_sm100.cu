@@ -154,7 +154,8 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   const int c_own = (L - 1) / dm.B;
   const long long grp = (long long)b * dm.h_kv + r;
   const int spb = CPS > 1 ? 1 : dm.B / SUB;                     // sub-blocks per routed chunk (chunks >= 64 tokens)
-  const int n_routed = a.count[grp];
+  int n_routed = a.count[grp];
+  DASH_CHECK(n_routed >= 0 && n_routed <= min(c_own, dm.T_s), a.sb, 310, n_routed = 0);
   const int n_routed_sub = CPS > 1 ? (n_routed + CPS - 1) / CPS : n_routed * spb;
   const int own_tokens = L - c_own * dm.B;                       // 1 .. B
   const int n_items = n_routed_sub + (own_tokens + SUB - 1) / SUB;
@@ -177,7 +178,10 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
 #pragma unroll
           for (int s = 0; s < CPS; ++s) {
             const int e = e0 + min(s, m - 1);
-            kv_locate(dm, b, a.blk_idx[loff + e] * dm.B, &misc->pg_s[k][s], &misc->idx_s[k][s]);
+            int cc = a.blk_idx[loff + e];
+            DASH_CHECK(cc >= 0 && cc < c_own, a.sb, 311, cc = 0);
+            kv_locate(dm, b, cc * dm.B, &misc->pg_s[k][s], &misc->idx_s[k][s]);
+            DASH_CHECK(!dm.page_table || (unsigned)misc->pg_s[k][s] < (unsigned)dm.num_pages, a.sb, 313, misc->pg_s[k][s] = 0);
             misc->bias_s[k][s] = a.blk_bias[loff + e];
           }
           misc->nval_s[k] = m * dm.B;
@@ -186,6 +190,7 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
 #pragma unroll
           for (int s = 0; s < CPS; ++s) {
             kv_locate(dm, b, c_own * dm.B + s * W, &misc->pg_s[k][s], &misc->idx_s[k][s]);
+            DASH_CHECK(!dm.page_table || (unsigned)misc->pg_s[k][s] < (unsigned)dm.num_pages, a.sb, 315, misc->pg_s[k][s] = 0);
             misc->bias_s[k][s] = 0.f;
           }
           misc->nval_s[k] = L - c_own * dm.B;
@@ -196,7 +201,9 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       float bs;
       if (it < n_routed_sub) {
         const int e = it / spb, sub = it % spb;
-        tok0 = a.blk_idx[loff + e] * dm.B + sub * SUB;
+        int cc = a.blk_idx[loff + e];
+        DASH_CHECK(cc >= 0 && cc < c_own, a.sb, 312, cc = 0);
+        tok0 = cc * dm.B + sub * SUB;
         bs = a.blk_bias[loff + e];
         nv = SUB;
       } else {
@@ -206,6 +213,7 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         nv = min(SUB, L - tok0);
       }
       kv_locate(dm, b, tok0, &misc->pg_s[k][0], &misc->idx_s[k][0]);
+      DASH_CHECK(!dm.page_table || (unsigned)misc->pg_s[k][0] < (unsigned)dm.num_pages, a.sb, 314, misc->pg_s[k][0] = 0);
       misc->bias_s[k][0] = bs; misc->nval_s[k] = nv;
     }
     __syncwarp();

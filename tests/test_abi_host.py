@@ -31,6 +31,21 @@ def test_every_declared_symbol_is_exported(lib):
         assert hasattr(lib, n), n
 
 
+def test_debug_library_exports_the_same_symbols_and_swaps_in_and_out(lib):
+    from paper_2605_18753_b200 import build
+    build.build(debug=True)
+    assert os.path.exists(B.DEBUG_LIB_PATH)
+    before = B.LIB_PATH
+    with B.use_debug_library():
+        assert B.LIB_PATH == B.DEBUG_LIB_PATH
+        dbg = B.lib()
+        for n in _declared():
+            assert hasattr(dbg, n), n
+        # host-side validation is the same code
+        assert dbg.dash_attn_workspace_bytes(ctypes.byref(_p())) == lib.dash_attn_workspace_bytes(ctypes.byref(_p()))
+    assert B.LIB_PATH == before and B.lib() is lib
+
+
 def test_params_struct_matches_header_layout():
     assert ctypes.sizeof(B.DashParams) == 4 * 14 + 8 + 8 * 12
     assert B.DashParams.q_stride.offset == 64
