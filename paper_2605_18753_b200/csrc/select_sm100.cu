@@ -8,9 +8,10 @@
 // Q (exact in bf16) times the three planes, accumulated in fp32, carries fp32-class accuracy: the support
 // must match a float64 evaluation except within 1e-4 of the threshold.
 //
-// Each of the 128 solver threads owns one row = one TMEM lane, so the threshold search needs no
-// cross-thread reduction: rows of up to 128 candidates are held in registers over all passes, longer ones
-// stream out of tensor memory 32 columns at a time (loads software-pipelined over two register buffers).
+// A row is one TMEM lane.  Rows of up to 256 candidates have one solver thread each (two blocks per SM), so the
+// threshold search needs no cross-thread reduction: up to 128 candidates are held in registers over all passes, longer
+// rows stream out of tensor memory 32 columns at a time (loads software-pipelined over two register buffers).  Rows of
+// more than 256 candidates (one block per SM) are split over three threads, whose partial sums meet in shared memory.
 // tau is found by Newton's method (f convex and decreasing: monotone from below, finite for alpha = 2).
 // The GQA group's heads sit in adjacent lanes; the group weights come from a halving shuffle exchange, one
 // warp-synchronous step per 32 chunks; log w is parked in tensor memory until mu is known, then the compact
@@ -31,12 +32,17 @@ namespace {
 
 constexpr int SC = 64;               // candidate chunks per MMA block / staged summary tile
 constexpr int HD_MAX = 128;          // the shared-memory layout is the one of head_dim 128; head_dim 64 fills half of each tile
-constexpr int SEL_TC_THREADS = 192;
+// Solver threads per row.  Short rows (<= 256 candidates, two blocks per SM): one, the row lives in the thread.  Long
+// rows (one block per SM holds up to 512 candidates of each row in tensor memory): three threads per row, in three
+// warps that share a quarter of the TMEM lanes, each streaming a third of the row's columns, so that every
+// scheduler of the SM has three solver warps to pick from instead of one; their partial sums meet through shared
+// memory like those of the blocks of a cluster.  (Three, not four: 14 warps leave each thread 128 registers, which
+// the streaming loops fill; 18 warps would leave 96 and spill.)
+__host__ __device__ constexpr int split_of(int nst) { return nst == 1 ? 1 : 3; }
+__host__ __device__ constexpr int sel_threads(int nst) { return (4 * split_of(nst) + 2) * 32; }   // solver warps, producer, MMA issuer
 constexpr uint32_t Q_BYTES = 128 * HD_MAX * 2;        // 32 KiB
 constexpr uint32_t PLANE_BYTES = SC * HD_MAX * 2;     // 16 KiB per plane per stage
 constexpr uint32_t STAGE_BYTES = 3 * PLANE_BYTES;     // hi, mid, lo
-constexpr int XCH_STRIDE = 33;
-constexpr uint32_t XCH_BYTES = 128 * XCH_STRIDE * 4;
 constexpr int MAX_NEWTON = 64, MAX_NEWTON_GENERIC = 400;
 
 struct MiscS {
@@ -46,12 +52,15 @@ struct MiscS {
 };
 enum BarS { Q_FULL = 0, X_FULL = 1, KB_FULL = 2, KB_EMPTY = 4, XBAR = 6 };   // XBAR: [warp 0..3][parity]
 constexpr int CLUSTER_COLS = 512;      // candidates one block of a cluster holds in tensor memory
+constexpr int MAX_CS = 4;              // widest cluster
 
 template <int NST> struct SmemPlan {
   static constexpr uint32_t OFF_Q = 0;
   static constexpr uint32_t OFF_KB = Q_BYTES;
   static constexpr uint32_t OFF_XCH = OFF_KB + NST * STAGE_BYTES;
-  static constexpr uint32_t OFF_MISC = OFF_XCH + ((XCH_BYTES + 127) / 128) * 128;
+  // exchange slots [parity][participant][row] of (float, float); participants = cluster blocks x threads per row
+  static constexpr uint32_t XCH_BYTES = NST == 1 ? 128u : 2u * MAX_CS * split_of(NST) * 128u * 8u;
+  static constexpr uint32_t OFF_MISC = OFF_XCH + XCH_BYTES;
   static constexpr uint32_t TOTAL = OFF_MISC + sizeof(MiscS);
 };
 
@@ -86,12 +95,13 @@ __global__ void kbar_split_kernel(const float* __restrict__ kbar, __nv_bfloat16*
 // SHORT: the tile has fewer than 128 live rows (chunks shorter than 128 / g_q tokens); full tiles compile without
 // any of the padding-row handling.
 template <int NST, int G, int CS, int HD, bool SHORT>
-__global__ void __launch_bounds__(SEL_TC_THREADS, NST == 1 ? 2 : 1)
+__global__ void __launch_bounds__(sel_threads(NST), NST == 1 ? 2 : 1)
 select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKB, SelectTcArgs a) {
   using SP = SmemPlan<NST>;
   extern __shared__ __align__(1024) uint8_t smem[];
   MiscS* misc = reinterpret_cast<MiscS*>(smem + SP::OFF_MISC);
-  float* xch = reinterpret_cast<float*>(smem + SP::OFF_XCH);
+  constexpr int SPLIT = split_of(NST), NSOLVE = 4 * SPLIT, W_PROD = NSOLVE, W_MMA = NSOLVE + 1;
+  constexpr int SEL_TC_THREADS = sel_threads(NST);
   const Dims& dm = a.dm;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t sbase = ptx::smem_u32(smem);
@@ -112,8 +122,9 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   const int c_own = i0 / dm.B;
   // candidates of the tile's rows; with a local window its chunks are not scored (window_rows_kernel lists them)
   const int n_cand = min(max(c_own - dm.local_blocks, 0), dm.T_s);   // (c_own <= T_s in a prefill)
-  const int c_lo = cr * CLUSTER_COLS;                          // first candidate this block holds
-  const int n_loc = CS > 1 ? max(0, min(CLUSTER_COLS, n_cand - c_lo)) : n_cand;
+  constexpr int CCOLS = CLUSTER_COLS;
+  const int c_lo = cr * CCOLS;                                 // first candidate this block holds
+  const int n_loc = CS > 1 ? max(0, min(CCOLS, n_cand - c_lo)) : n_cand;
   const int n_blk = (n_loc + SC - 1) / SC;
 
   if (tid == 0) {
@@ -128,10 +139,10 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       ptx::mbar_init(bar(KB_FULL + s), 1);
       ptx::mbar_init(bar(KB_EMPTY + s), 1);
     }
-    for (int s = 0; s < 8; ++s) ptx::mbar_init(bar(XBAR + s), CS * 32);
+    for (int s = 0; s < 8; ++s) ptx::mbar_init(bar(XBAR + s), CS * SPLIT * 32);
     ptx::fence_barrier_init();
   }
-  if (warp == 5) {
+  if (warp == W_MMA) {
     ptx::tmem_alloc(ptx::smem_u32(&misc->tmem_base), a.tmem_cols);
     ptx::tmem_relinquish();
     ptx::tc_fence_before();
@@ -157,7 +168,7 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   if (a.sb && *reinterpret_cast<volatile int*>(&a.sb->status) != 0) *abort_flag = 1;
   __syncthreads();
 
-  if (warp == 4) {
+  if (warp == W_PROD) {
     // ---------------- producer: Q tile, then the three planes of every 64-chunk block of summaries
     if (lane == 0 && n_loc > 0) {
       ptx::prefetch_tensormap(&tmQ);
@@ -184,7 +195,7 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           for (int k = 0; k < 200000 && !ptx::mbar_try_wait(bar(KB_FULL + s), 0) && !ptx::mbar_try_wait(bar(KB_FULL + s), 1); ++k) {}
       }
     }
-  } else if (warp == 5) {
+  } else if (warp == W_MMA) {
     // ---------------- MMA issuer: X[:, cb*64 .. +64) = Q Kbar_hi^T + Q Kbar_mid^T + Q Kbar_lo^T
     if (lane == 0 && n_loc > 0) {
       constexpr uint32_t IDESC = ptx::idesc_bf16_f32(128, SC, false, false);
@@ -213,15 +224,20 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     }
     __syncwarp();
   } else {
-    // ---------------- solver: thread = row = TMEM lane
-    const int m = tid;
+    // ---------------- solver: row = TMEM lane; SPLIT threads per row (warps q, q + 4, ...: the same quarter of the
+    // lanes), thread `part` of a row owning a contiguous share of the row's 32-column chunks
+    const int q4 = SPLIT == 1 ? warp : (warp & 3), part = SPLIT == 1 ? 0 : (warp >> 2);
+    const int m = q4 * 32 + lane;
     const int t = m / g_q, hh = m % g_q;
     const int i = i0 + t;
     const bool row_valid = SHORT ? (i < dm.seq_q && t < TQ) : i < dm.seq_q;   // (a short tile ends with zero-query rows)
-    const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+    const uint32_t lane_addr = tmem + ((uint32_t)(q4 * 32) << 16);
     const int e_int = dm.e_int;
     const float e = dm.e, xs = dm.x_scale;
     const int n_chunks = (n_loc + 31) / 32;
+    const int per_part = (n_chunks + SPLIT - 1) / SPLIT;
+    const int k_lo = SPLIT == 1 ? 0 : min(part * per_part, n_chunks);                  // this thread's chunks
+    const int k_hi = SPLIT == 1 ? n_chunks : min(k_lo + per_part, n_chunks);
     bool ok = true;
     float tau = 0.f;
     if (n_loc > 0) {
@@ -231,33 +247,50 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     // Cluster all-reduce of two floats per row: every thread writes its pair into slot [parity][its rank][row]
     // of every block, arrives (release, cluster scope) on every block's per-warp barrier, waits on its own and
     // reads the CS pairs back in rank order, so all blocks see bit-identical results and take the same branches.
+    // The participants of a row are ordered by the candidates they hold: rank = cluster rank * SPLIT + part.
+    constexpr int NP = CS * SPLIT;
+    const int my_rank = cr * SPLIT + part;
     int xround = 0;
-    float xa[CS], xb[CS];
+    // what a round leaves behind: sums of both values over all participants (added in rank order, so every
+    // participant holds the same bits and takes the same branches), the maximum of the first, and the sum of the
+    // first over the participants ranked below this one
+    float x_sum_a = 0.f, x_sum_b = 0.f, x_max_a = 0.f, x_below_a = 0.f;
     auto exchange = [&](float va, float vb) -> bool {
-      if constexpr (CS == 1) {
-        xa[0] = va; xb[0] = vb;
+      if constexpr (NP == 1) {
+        x_sum_a = x_max_a = va; x_sum_b = vb; x_below_a = 0.f;
         return true;
       } else {
         const int par = xround & 1;
-        float2* xbuf = reinterpret_cast<float2*>(smem + SP::OFF_XCH);          // [2][CS][128]
-        const uint32_t slot = ptx::smem_u32(&xbuf[(par * CS + cr) * 128 + m]);
-        const uint32_t mybar = bar(XBAR + warp * 2 + par);
+        float2* xbuf = reinterpret_cast<float2*>(smem + SP::OFF_XCH);          // [2][NP][128]
+        float2* mine = &xbuf[(par * NP + my_rank) * 128 + m];
+        const uint32_t mybar = bar(XBAR + q4 * 2 + par);
+        if constexpr (CS == 1) {
+          *mine = make_float2(va, vb);
+          ptx::mbar_arrive(mybar);
+          if (!ptx::mbar_wait(mybar, (xround >> 1) & 1, abort_flag)) return false;
+        } else {
+          const uint32_t slot = ptx::smem_u32(mine);
 #pragma unroll
-        for (int pr = 0; pr < CS; ++pr) ptx::st_cluster_f32x2(ptx::map_to_rank(slot, pr), va, vb);
+          for (int pr = 0; pr < CS; ++pr) ptx::st_cluster_f32x2(ptx::map_to_rank(slot, pr), va, vb);
 #pragma unroll
-        for (int pr = 0; pr < CS; ++pr) ptx::mbar_arrive_cluster(ptx::map_to_rank(mybar, pr));
-        if (!ptx::mbar_wait_cluster(mybar, (xround >> 1) & 1, abort_flag)) return false;
-#pragma unroll
-        for (int pr = 0; pr < CS; ++pr) {
-          const float2 v = xbuf[(par * CS + pr) * 128 + m];
-          xa[pr] = v.x; xb[pr] = v.y;
+          for (int pr = 0; pr < CS; ++pr) ptx::mbar_arrive_cluster(ptx::map_to_rank(mybar, pr));
+          if (!ptx::mbar_wait_cluster(mybar, (xround >> 1) & 1, abort_flag)) return false;
         }
+        float sa = 0.f, sb = 0.f, mxa = -INFINITY, below = 0.f;
+#pragma unroll
+        for (int pr = 0; pr < NP; ++pr) {
+          const float2 v = xbuf[(par * NP + pr) * 128 + m];
+          sa += v.x; sb += v.y;
+          mxa = fmaxf(mxa, v.x);
+          if (pr < my_rank) below += v.x;
+        }
+        x_sum_a = sa; x_sum_b = sb; x_max_a = mxa; x_below_a = below;
         ++xround;
         return true;
       }
     };
-    auto xsum_a = [&]() { float v = xa[0]; for (int pr = 1; pr < CS; ++pr) v += xa[pr]; return v; };
-    auto xsum_b = [&]() { float v = xb[0]; for (int pr = 1; pr < CS; ++pr) v += xb[pr]; return v; };
+    auto xsum_a = [&]() { return x_sum_a; };
+    auto xsum_b = [&]() { return x_sum_b; };
     // Newton on f(tau) = sum [x - tau]_+^e - 1 (steps taken on f^(1/e), see newton_delta), convex and decreasing.
     // From the left of the root the iterates rise monotonically and never pass it; from the right one step lands
     // on the left.  The start is the root
@@ -287,9 +320,10 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       const float nt = tau + newton_delta(f, g, ei, e);
       if (nt == tau) done = true; else tau = nt;
     };
-    float xr[4][32];                               // the whole row, when it has at most 128 candidates
-    const bool in_regs = CS == 1 && n_chunks <= 4;
-    if (ok && n_cand > 0 && in_regs) {
+    constexpr bool CAN_HOLD = CS == 1 && SPLIT == 1;   // one thread per row: a short row can live in its registers
+    float xr[CAN_HOLD ? 4 : 1][32];                // the whole row, when it has at most 128 candidates
+    const bool in_regs = CAN_HOLD && n_chunks <= 4;
+    auto solve_in_regs = [&]() {
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
         if (k < n_chunks) {
@@ -366,20 +400,22 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         newton_step((f[0] + f[1]) + (f[2] + f[3]), (g[0] + g[1]) + (g[2] + g[3]), done);
         if (__all_sync(0xffffffffu, done)) break;
       }
-    } else if (ok && n_cand > 0) {
+    };
+    auto solve_streaming = [&]() {
       // longer rows stream from tensor memory every pass (and, in a cluster, meet the other blocks' partial sums).
       // The 32-column loads are software-pipelined over two register buffers: with one block per SM a solver
       // warp has its scheduler to itself, so an exposed load latency per chunk would be pure idle time.
       auto stream = [&](auto&& body) {
+        if (k_lo >= k_hi) return;                  // a row shorter than the threads it is split over
         uint32_t va[32], vb[32];
-        DASH_TMEM_LD32(va, lane_addr);
-        for (int k = 0; k < n_chunks; k += 2) {
+        DASH_TMEM_LD32(va, lane_addr + k_lo * 32);
+        for (int k = k_lo; k < k_hi; k += 2) {
           DASH_TMEM_WAIT_LD32(va);
-          if (k + 1 < n_chunks) DASH_TMEM_LD32(vb, lane_addr + (k + 1) * 32);
+          if (k + 1 < k_hi) DASH_TMEM_LD32(vb, lane_addr + (k + 1) * 32);
           body(va, k);
-          if (k + 1 < n_chunks) {
+          if (k + 1 < k_hi) {
             DASH_TMEM_WAIT_LD32(vb);
-            if (k + 2 < n_chunks) DASH_TMEM_LD32(va, lane_addr + (k + 2) * 32);
+            if (k + 2 < k_hi) DASH_TMEM_LD32(va, lane_addr + (k + 2) * 32);
             body(vb, k + 1);
           }
         }
@@ -400,7 +436,7 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       });
       float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * xs;
       ok = exchange(mx, 0.f);
-      for (int pr = 0; pr < CS; ++pr) mx = fmaxf(mx, xa[pr]);
+      mx = x_max_a;
       float s1v[4] = {0.f, 0.f, 0.f, 0.f}, s2v[4] = {0.f, 0.f, 0.f, 0.f};
       stream([&](uint32_t (&v)[32], int k) {
         const int lim = n_loc - k * 32;
@@ -451,8 +487,14 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         newton_step(xsum_a(), xsum_b(), done);
         if (__all_sync(0xffffffffu, done)) break;
       }
+    };
+    if constexpr (CAN_HOLD) {
+      if (ok && n_cand > 0 && in_regs) solve_in_regs();
+      else if (ok && n_cand > 0) solve_streaming();
+    } else {
+      if (ok && n_cand > 0) solve_streaming();
     }
-    if (ok && row_valid && a.tau && cr == 0) a.tau[((long long)b * dm.h_q + r * g_q + hh) * dm.seq_q + i] = tau;
+    if (ok && row_valid && a.tau && my_rank == 0) a.tau[((long long)b * dm.h_q + r * g_q + hh) * dm.seq_q + i] = tau;
 
     // ---------------- group weights, mask words, log w, compact lists
     // The g_q heads of a token sit in g_q adjacent lanes.  Per 32-chunk step every lane raises its own margins
@@ -513,13 +555,14 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         for (int o = 1; o < G; o <<= 1) bits |= __shfl_xor_sync(0xffffffffu, bits, o);
         ptx::tmem_st_n<OWN>(lane_addr + k * 32, lwv);            // slot q of this lane = chunk own0 + q of step k
         if (row_valid && hh == 0) {
-          const int wj = cr * (CLUSTER_COLS / 32) + k;         // mask word of this step
+          const int wj = cr * (CCOLS / 32) + k;                // mask word of this step
           mrow[wj] = bits | (((c_own >> 5) == wj) ? (1u << (c_own & 31)) : 0u);
         }
         nsel += __popc(bits);
       };
       if (in_regs) {
         // the register-resident row is spent after this sweep: raise it to the power in place, no second copy
+        if constexpr (CAN_HOLD) {
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
           if (k < n_chunks) {
@@ -528,8 +571,9 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             chunk_step(k, xr[k]);
           }
         }
+        }
       } else {
-        for (int k = 0; k < n_chunks; ++k) {
+        for (int k = k_lo; k < k_hi; ++k) {
           float pe[32];
           uint32_t v[32];
           DASH_TMEM_LD32(v, lane_addr + k * 32);
@@ -548,19 +592,16 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       for (int o = 1; o < G; o <<= 1) slog += __shfl_xor_sync(0xffffffffu, slog, o);
       // counts and sums of log w of the other blocks: total for mu, lower ranks for the list position
       ok = exchange((float)nsel, slog);
-      int nsel_all = 0, base = 0;
-      float slog_all = 0.f;
-      for (int pr = 0; pr < CS; ++pr) {
-        nsel_all += (int)xa[pr];
-        slog_all += xb[pr];
-        if (pr < cr) base += (int)xa[pr];
-      }
-      if (row_valid && hh == 0 && cr == 0) {
+      // (counts are small integers: exact in fp32)
+      const int nsel_all = (int)x_sum_a;
+      int base = (int)x_below_a;
+      const float slog_all = x_sum_b;
+      if (row_valid && hh == 0 && my_rank == 0) {
         for (int j = (n_cand + 31) / 32; j < dm.W; ++j) mrow[j] = ((c_own >> 5) == j) ? (1u << (c_own & 31)) : 0u;
         a.count[row_id] = nsel_all;
       }
       const float mu = nsel_all > 0 ? slog_all / (float)nsel_all : 0.f;
-      for (int k = 0; k < n_chunks && ok; ++k) {
+      for (int k = in_regs ? 0 : k_lo; k < (in_regs ? n_chunks : k_hi) && ok; ++k) {
         uint32_t lwv[OWN];
         ptx::tmem_ld_n<OWN>(lwv, lane_addr + k * 32);
         ptx::tmem_wait_ld();
@@ -590,7 +631,7 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   }
 
   __syncthreads();
-  if (warp == 5) {
+  if (warp == W_MMA) {
     ptx::tc_fence_after();
     ptx::tmem_dealloc(tmem, a.tmem_cols);
   }
@@ -622,7 +663,7 @@ static cudaError_t launch_band(const CUtensorMap& tq, const CUtensorMap& tkb, co
   if (cudaError_t e = allow_dynamic_smem(kern, SmemPlan<NST>::TOTAL, configured); e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(clusters * CS));
-  cfg.blockDim = dim3(SEL_TC_THREADS);
+  cfg.blockDim = dim3(sel_threads(NST));
   cfg.dynamicSmemBytes = SmemPlan<NST>::TOTAL;
   cfg.stream = st;
   cudaLaunchAttribute attr[2];
@@ -751,14 +792,20 @@ cudaError_t launch_select_sm100(const Dims& dm, int token_limit, const void* Q, 
     a.tile_base = t1; a.n_tiles = t2 - t1; a.tmem_cols = 512;
     if ((e = launch_band_g<2, 2>(dm, tq, tkb, a, (long long)a.n_tiles * groups, st)) != cudaSuccess) return e;
   }
+  // one block per tile: rows of 257 .. 512 candidates take the whole tensor memory of an SM (one block per SM, three
+  // solver threads per row); shorter ones leave room for two blocks per SM with the row in one thread
+  const int t0 = tiles_up_to(256);
+  if (t1 > t0) {
+    a.tile_base = t0; a.n_tiles = t1 - t0; a.tmem_cols = 512;
+    if ((e = launch_band_g<2, 1>(dm, tq, tkb, a, (long long)a.n_tiles * groups, st)) != cudaSuccess) return e;
+  }
   {
-    a.tile_base = 0; a.n_tiles = t1;
-    const int max_cand = min(dm.T_s, (int)(((long long)t1 * a.TQ - 1) / dm.B));
+    a.tile_base = 0; a.n_tiles = t0;
+    const int max_cand = min(dm.T_s, (int)(((long long)t0 * a.TQ - 1) / dm.B));
     uint32_t cols = 32;
     while ((int)cols < ((max_cand + SC - 1) / SC) * SC) cols <<= 1;
     a.tmem_cols = cols;
-    if (cols <= 256) e = launch_band_g<1, 1>(dm, tq, tkb, a, (long long)a.n_tiles * groups, st);
-    else e = launch_band_g<2, 1>(dm, tq, tkb, a, (long long)a.n_tiles * groups, st);
+    e = launch_band_g<1, 1>(dm, tq, tkb, a, (long long)a.n_tiles * groups, st);
   }
   if (e == cudaSuccess && dm.local_blocks > 0) {
     const long long rows = (long long)groups * token_limit;
