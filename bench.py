@@ -489,9 +489,10 @@ def measure_decode(B, synth, wd, dev, peaks, flush, iters=30) -> dict:
     return out
 
 
-def measure_backward(B, synth, w, dev, flush, iters=3) -> dict:
-    """The backward chain (CUDA-core correctness kernels: Stage 2, then routing, then summaries) on one workload:
-    milliseconds only -- these kernels are parity-graded, not tuned."""
+def measure_backward(B, synth, w, dev, flush, iters=3, tensor_cores=False, fwd_sel_tflop=None) -> dict:
+    """The backward chain on one workload: Stage 2 (tensor-core kernels or the CUDA-core correctness kernel), then the
+    routing and summary backward kernels (CUDA cores).  Milliseconds; for the tensor-core Stage 2 also TFLOP/s on the
+    selected tokens (2.5 x the forward's selected FLOPs: five products instead of two)."""
     inp = synth.make_prefill_inputs(w, dev)
     Q, K, V = inp["Q"], inp["K"], inp["V"]
     dO = torch.randn(Q.shape, device=dev, dtype=torch.float32).to(Q.dtype)
@@ -505,8 +506,16 @@ def measure_backward(B, synth, w, dev, flush, iters=3) -> dict:
     dbias = torch.empty_like(rt["blk_bias"])
     dQr = torch.empty(w.batch, w.seq, w.h_q, w.head_dim, device=dev)
     dKbar = torch.empty_like(kbar)
-    out = {"workload": f"{w.name} cut to {w.seq} tokens", "kernels": "CUDA-core correctness path (one warp per row and head, fp32 atomics)"}
-    for name, fn in (("stage2_ms", lambda: B.dash_attn_bwd_attend_prefill(p, Q, K, V, dO, rt["mask"], rt["blk_bias"], dQ, dK, dV, dbias)),
+    if tensor_cores:
+        bws = B.alloc_bwd_workspace(p, dev)
+        stage2 = lambda: B.dash_attn_bwd_attend_prefill_tc(p, Q, K, V, dO, rt["mask"], rt["blk_bias"], dQ, dK, dV, dbias, bws)
+        kernels = ("Stage 2 on tensor cores (statistics pass of the forward kernel, dQ / dbias kernel, dK / dV kernel); "
+                   "routing and summaries on CUDA cores")
+    else:
+        stage2 = lambda: B.dash_attn_bwd_attend_prefill(p, Q, K, V, dO, rt["mask"], rt["blk_bias"], dQ, dK, dV, dbias)
+        kernels = "CUDA-core correctness path (one warp per row and head, fp32 atomics)"
+    out = {"workload": w.name if w.seq == synth.workload(w.name).seq else f"{w.name} cut to {w.seq} tokens", "kernels": kernels}
+    for name, fn in (("stage2_ms", stage2),
                      ("routing_ms", lambda: B.dash_attn_bwd_select_prefill(p, Q, kbar, rt["count"], rt["blk_idx"], rt["tau"], dbias, dQr, dKbar)),
                      ("summaries_ms", lambda: B.dash_attn_bwd_block_summaries(p, K, dKbar, dK))):
         fn()
@@ -518,11 +527,16 @@ def measure_backward(B, synth, w, dev, flush, iters=3) -> dict:
             torch.cuda.synchronize()
             ts.append(a.elapsed_time(b))
         out[name] = float(np.median(ts))
+    if tensor_cores:
+        assert B.dash_attn_last_status(bws) == 0
+        if fwd_sel_tflop:
+            out["stage2_selected_tflop"] = 2.5 * fwd_sel_tflop
+            out["stage2_selected_tflops"] = 2.5 * fwd_sel_tflop / (out["stage2_ms"] * 1e-3)
     assert torch.isfinite(dQ.float()).all() and torch.isfinite(dK).all() and torch.isfinite(dQr).all()
     return out
 
 
-def all_config_measurements(B, synth, dev, peaks, flush) -> dict:
+def all_config_measurements(B, synth, dev, peaks, flush, sel_tflop_8k=None) -> dict:
     """Every other configuration of the task beside the headline: the 64K prefill at two sparsities, the
     (chunk size, alpha) sweep at 32K x batch 2, the 8K prefill with finer chunks, and the decode workload."""
     out = {}
@@ -552,6 +566,8 @@ def all_config_measurements(B, synth, dev, peaks, flush) -> dict:
                                                         with_sdpa=False))
     guarded("decode_128k", lambda: measure_decode(B, synth, synth.workload("decode_128k"), dev, peaks, flush))
     guarded("backward_2k", lambda: measure_backward(B, synth, synth.workload("prefill_8k", seq=2048), dev, flush))
+    guarded("backward_8k_tc", lambda: measure_backward(B, synth, synth.workload("prefill_8k"), dev, flush, iters=5,
+                                                       tensor_cores=True, fwd_sel_tflop=sel_tflop_8k))
     return out
 
 
@@ -744,7 +760,8 @@ def main():
             extras["side_error"] = repr(ex)
         del Q, K, V, O, ws, rt, kbar, inp
         torch.cuda.empty_cache()
-        extras["configs"] = all_config_measurements(B, synth, dev, peaks, flush)
+        extras["configs"] = all_config_measurements(B, synth, dev, peaks, flush,
+                                                    sel_tflop_8k=f_sel / 1e12 if w.name == "prefill_8k" else None)
         if "decode_128k" in extras["configs"]:
             extras["decode"] = extras["configs"]["decode_128k"]
 

@@ -203,6 +203,22 @@ int dash_attn_bwd_attend_prefill(const dash_params* p, const void* Q, const void
                                  const uint32_t* mask, const float* blk_bias, void* dQ, float* dK, float* dV,
                                  float* dbias, void* stream);
 
+/* The same gradients on tensor cores (bf16, head_dim 128, chunks of 64 or 128 tokens, at least two query heads per KV
+ * head, causal; anything else returns DASH_ERR_UNSUPPORTED and nothing is enqueued: call dash_attn_bwd_attend_prefill).
+ * Four launches: the forward Stage-2 kernel run for its row statistics (log-sum-exp and delta = <O, dO>; O itself is
+ * not written), the prefix counts of the mask words, a query-tile-stationary kernel for dQ and dbias, and a
+ * key-slice-stationary kernel for dK and dV (no atomics on dQ, dK, dV: every element has one owner and is written
+ * whether or not any row attends it; dbias is zeroed and then receives one or two atomic adds per entry, whose
+ * order cannot change the sum).  P and dS enter the dK / dV products rounded to bf16.
+ *   bwd_workspace   device scratch of at least dash_attn_bwd_workspace_bytes(p) bytes, 256-byte aligned, owned by the
+ *                   caller; it opens with a status word like the forward workspace's (dash_attn_last_status and
+ *                   dash_attn_reset_status accept it): a bounded wait that runs out leaves DASH_ERR_TIMEOUT there.
+ * Other arguments, layouts and dtypes as for dash_attn_bwd_attend_prefill. */
+size_t dash_attn_bwd_workspace_bytes(const dash_params* p);
+int dash_attn_bwd_attend_prefill_tc(const dash_params* p, const void* Q, const void* K, const void* V, const void* dO,
+                                    const uint32_t* mask, const float* blk_bias, void* dQ, float* dK, float* dV,
+                                    float* dbias, void* bwd_workspace, size_t bwd_workspace_bytes, void* stream);
+
 /* Backward of Stage 1 (prefill, causal): carries dbias on through the log-prior bias (Proposition 1), the group average
  * (Section 3.2) and the alpha-entmax of every head (Eq. 2) to the queries and the chunk summaries.  Inside a region
  * of fixed support the entmax Jacobian is diag(s) - s s^T / sum(s) with s = p^(2 - alpha) on the support and zero

@@ -26,6 +26,7 @@ EXPORTS = [
     "dash_attn_workspace_bytes", "dash_attn_list_capacity", "dash_attn_list_offset",
     "dash_attn_block_summaries", "dash_attn_select", "dash_attn_attend_prefill", "dash_attn_attend_decode",
     "dash_attn_attend_decode_static", "dash_attn_bwd_attend_prefill",
+    "dash_attn_bwd_workspace_bytes", "dash_attn_bwd_attend_prefill_tc",
     "dash_attn_block_summaries_paged", "dash_attn_fwd_decode_paged",
     "dash_attn_bwd_select_prefill", "dash_attn_bwd_block_summaries",
     "dash_attn_fwd_prefill", "dash_attn_fwd_decode", "dash_attn_reset_status", "dash_attn_last_status",
@@ -79,6 +80,10 @@ def lib() -> ctypes.CDLL:
         L.dash_attn_attend_decode_static.argtypes = [P] + [c_void_p] * 9
         L.dash_attn_bwd_attend_prefill.restype = ctypes.c_int
         L.dash_attn_bwd_attend_prefill.argtypes = [P] + [c_void_p] * 11
+        L.dash_attn_bwd_workspace_bytes.restype = c_size_t
+        L.dash_attn_bwd_workspace_bytes.argtypes = [P]
+        L.dash_attn_bwd_attend_prefill_tc.restype = ctypes.c_int
+        L.dash_attn_bwd_attend_prefill_tc.argtypes = [P] + [c_void_p] * 11 + [c_size_t, c_void_p]
         L.dash_attn_bwd_select_prefill.restype = ctypes.c_int
         L.dash_attn_bwd_select_prefill.argtypes = [P] + [c_void_p] * 9
         L.dash_attn_bwd_block_summaries.restype = ctypes.c_int
@@ -284,6 +289,25 @@ def dash_attn_bwd_attend_prefill(p, Q, K, V, dO, mask, blk_bias, dQ, dK, dV, dbi
     _check(lib().dash_attn_bwd_attend_prefill(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(dO), _ptr(mask),
                                               _ptr(blk_bias), _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(dbias), _stream()),
            "dash_attn_bwd_attend_prefill")
+
+
+def alloc_bwd_workspace(p: DashParams, device="cuda") -> torch.Tensor:
+    nbytes = int(lib().dash_attn_bwd_workspace_bytes(ctypes.byref(p)))
+    if nbytes == 0:
+        raise DashError(-1, "dash_attn_bwd_workspace_bytes")
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=device)
+    assert ws.data_ptr() % 256 == 0
+    dash_attn_reset_status(ws)
+    return ws
+
+
+def dash_attn_bwd_attend_prefill_tc(p, Q, K, V, dO, mask, blk_bias, dQ, dK, dV, dbias, bwd_workspace):
+    """The same gradients from the tensor-core kernels (bf16, head_dim 128, chunks of 64 / 128); raises DashError with
+    DASH_ERR_UNSUPPORTED for other shapes."""
+    _check(lib().dash_attn_bwd_attend_prefill_tc(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(dO), _ptr(mask),
+                                                 _ptr(blk_bias), _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(dbias),
+                                                 _ptr(bwd_workspace), bwd_workspace.numel(), _stream()),
+           "dash_attn_bwd_attend_prefill_tc")
 
 
 def dash_attn_bwd_select_prefill(p, Q, Kbar, count, blk_idx, tau, dbias, dQ_route, dKbar):

@@ -16,7 +16,7 @@ LIB_DEBUG = os.path.join(PKG, "libdash_attn_debug.so")
 # (bounds checks that record DASH_ERR_CAPACITY instead of making the access) for the debug library
 DEBUG_SOURCES = ["decode.cu", "decode_sm100.cu"]
 OBJ_DIR = os.path.join(PKG, "build")
-SOURCES = ["api.cu", "summaries.cu", "select.cu", "select_sm100.cu", "select_decode.cu", "attend_generic.cu", "attend_bwd_generic.cu", "route_bwd_generic.cu", "decode.cu", "decode_sm100.cu", "prefill_sm100.cu"]
+SOURCES = ["api.cu", "summaries.cu", "select.cu", "select_sm100.cu", "select_decode.cu", "attend_generic.cu", "attend_bwd_generic.cu", "route_bwd_generic.cu", "decode.cu", "decode_sm100.cu", "prefill_sm100.cu", "prefill_bwd_sm100.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "--use_fast_math", "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 

@@ -296,6 +296,58 @@ int dash_attn_bwd_attend_prefill(const dash_params* p, const void* Q, const void
                                                        (cudaStream_t)stream));
 }
 
+// Layout of the backward scratch: status region, then lse2 and delta [batch][token][query head], then the routed-chunk
+// prefix counts [batch * h_kv * seq_q][W].
+struct BwdLayout {
+  size_t status, lse2, delta, prefix, total;
+};
+static BwdLayout bwd_layout(const Dims& dm) {
+  auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
+  BwdLayout l;
+  l.status = 0;
+  size_t at = up(STATUS_REGION_BYTES);
+  const size_t rows = (size_t)dm.batch * dm.seq_q * dm.h_q;
+  l.lse2 = at; at = up(at + rows * sizeof(float));
+  l.delta = at; at = up(at + rows * sizeof(float));
+  l.prefix = at; at = up(at + (size_t)dm.batch * dm.h_kv * dm.seq_q * (size_t)dm.W * sizeof(int));
+  l.total = at;
+  return l;
+}
+
+size_t dash_attn_bwd_workspace_bytes(const dash_params* p) {
+  Dims dm;
+  if (make_dims(p, &dm) != DASH_OK || dm.decode) return 0;
+  return bwd_layout(dm).total;
+}
+
+int dash_attn_bwd_attend_prefill_tc(const dash_params* p, const void* Q, const void* K, const void* V, const void* dO,
+                                    const uint32_t* mask, const float* blk_bias, void* dQ, float* dK, float* dV,
+                                    float* dbias, void* bwd_workspace, size_t bwd_workspace_bytes, void* stream) {
+  Dims dm;
+  int rc = make_dims(p, &dm);
+  if (rc != DASH_OK) return rc;
+  if (dm.decode) return DASH_ERR_INVALID_ARG;
+  if (!Q || !K || !V || !dO || !mask || !dQ || !dK || !dV) return DASH_ERR_INVALID_ARG;
+  if (dm.list_rows > 0 && (!blk_bias || !dbias)) return DASH_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(dO) || !aligned16(dQ) || !aligned16(dK) ||
+      !aligned16(dV))
+    return DASH_ERR_INVALID_ARG;
+  const BwdLayout l = bwd_layout(dm);
+  if (!bwd_workspace || (reinterpret_cast<uintptr_t>(bwd_workspace) & 255) != 0) return DASH_ERR_WORKSPACE;
+  if (bwd_workspace_bytes < l.total) return DASH_ERR_WORKSPACE;
+  if ((rc = check_device()) != DASH_OK) return rc;
+  if (!prefill_bwd_sm100_supported(dm)) return DASH_ERR_UNSUPPORTED;
+  cudaStream_t st = (cudaStream_t)stream;
+  StageRange nv("dash_attn: stage 2 prefill attention, backward (tensor cores)");
+  const size_t list_bytes = (size_t)dm.batch * dm.h_kv * (size_t)dm.list_rows * sizeof(float);
+  if (list_bytes > 0) {
+    if ((rc = cuda_status(cudaMemsetAsync(dbias, 0, list_bytes, st))) != DASH_OK) return rc;
+  }
+  return cuda_status(launch_attend_prefill_bwd_sm100(dm, Q, K, V, dO, mask, blk_bias, at<float>(bwd_workspace, l.lse2),
+                                                     at<float>(bwd_workspace, l.delta), at<int>(bwd_workspace, l.prefix),
+                                                     dQ, dK, dV, dbias, at<StatusBlock>(bwd_workspace, l.status), st));
+}
+
 int dash_attn_bwd_select_prefill(const dash_params* p, const void* Q, const float* Kbar, const int32_t* count,
                                  const int32_t* blk_idx, const float* tau, const float* dbias, float* dQ_route,
                                  float* dKbar, void* stream) {

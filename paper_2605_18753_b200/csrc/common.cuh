@@ -261,6 +261,14 @@ bool prefill_sm100_supported(const Dims& dm);
 // inputs_stable: Q, K, V were not written by the kernel launched just before on the stream
 cudaError_t launch_attend_prefill_sm100(const Dims& dm, const void* Q, const void* K, const void* V,
                                         const uint32_t* mask, const float* blk_bias, void* O, StatusBlock* sb,
-                                        bool inputs_stable, cudaStream_t st);
+                                        bool inputs_stable, cudaStream_t st, float* lse2 = nullptr,
+                                        float* delta = nullptr, const void* dO = nullptr);
+// Stage 2 backward on tensor cores (bf16, head_dim 128, chunks of 64 or 128 tokens, g_q >= 2); scratch: lse2 and delta
+// [batch][token][query head] floats, prefix [batch * h_kv * seq_q][W] ints.
+bool prefill_bwd_sm100_supported(const Dims& dm);
+cudaError_t launch_attend_prefill_bwd_sm100(const Dims& dm, const void* Q, const void* K, const void* V, const void* dO,
+                                            const uint32_t* mask, const float* blk_bias, float* lse2, float* delta,
+                                            int* prefix, void* dQ, float* dK, float* dV, float* dbias, StatusBlock* sb,
+                                            cudaStream_t st);
 
 }  // namespace dash

@@ -87,7 +87,12 @@ struct PrefillArgs {
   long long wait_limit;   // cycles a bounded wait may spin
   const uint32_t* mask;
   const float* blk_bias;
-  __nv_bfloat16* O;
+  __nv_bfloat16* O;          // may be null when only the row statistics are wanted
+  // Row statistics for the backward pass, [batch][token][query head] (null: not wanted): the log-sum-exp of the row's
+  // logits in the log2 domain, and delta = <O_row, dO_row> (dO: strides of O), both from the fp32 accumulator.
+  float* lse2;
+  float* delta;
+  const __nv_bfloat16* dO;
   StatusBlock* sb;
 };
 
@@ -592,13 +597,30 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
     if (ok && n_steps > 0) {
       ptx::tc_fence_after();
       const float inv = l > 0.f ? 1.f / l : 0.f;
-      __nv_bfloat16* op = a.O + (long long)b * dm.os[0] + (long long)i_row * dm.os[1] + (long long)(r * g_q + hh) * dm.os[2];
+      const long long o_off = (long long)b * dm.os[0] + (long long)i_row * dm.os[1] + (long long)(r * g_q + hh) * dm.os[2];
+      __nv_bfloat16* op = a.O + o_off;
+      const bool row_out = i_row < dm.seq_q && (!SHORT || row_live);
+      float dot = 0.f;
 #pragma unroll 1
       for (int q = 0; q < HD / 32; ++q) {
         uint32_t o[32];
         DASH_TMEM_LD32(o, lane_addr + 2 * NKV + q * 32);
         ptx::tmem_wait_ld();
-        if (i_row < dm.seq_q && (!SHORT || row_live)) {
+        if (a.lse2 && row_out) {
+          const __nv_bfloat16* gp = a.dO + o_off + q * 32;
+#pragma unroll
+          for (int c = 0; c < 32; c += 8) {
+            const uint4 gv = *reinterpret_cast<const uint4*>(gp + c);
+            const __nv_bfloat162* g2 = reinterpret_cast<const __nv_bfloat162*>(&gv);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              const float2 gf = __bfloat1622float2(g2[u]);
+              dot = fmaf(__uint_as_float(o[c + 2 * u]), gf.x, dot);
+              dot = fmaf(__uint_as_float(o[c + 2 * u + 1]), gf.y, dot);
+            }
+          }
+        }
+        if (a.O && row_out) {
 #pragma unroll
           for (int c = 0; c < 32; c += 8) {
             uint4 v;
@@ -611,6 +633,11 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
             *reinterpret_cast<uint4*>(op + q * 32 + c) = v;
           }
         }
+      }
+      if (a.lse2 && row_out) {
+        const long long row = ((long long)b * dm.seq_q + i_row) * dm.h_q + r * g_q + hh;
+        a.lse2[row] = m_used + log2f(l);
+        a.delta[row] = dot * inv;
       }
     }
     ptx::tc_fence_before();
@@ -649,8 +676,11 @@ bool prefill_sm100_supported(const Dims& dm) {
 
 cudaError_t launch_attend_prefill_sm100(const Dims& dm, const void* Q, const void* K, const void* V,
                                         const uint32_t* mask, const float* blk_bias, void* O, StatusBlock* sb,
-                                        bool inputs_stable, cudaStream_t st) {
+                                        bool inputs_stable, cudaStream_t st, float* lse2, float* delta, const void* dO) {
   PrefillArgs a;
+  a.lse2 = lse2;
+  a.delta = delta;
+  a.dO = (const __nv_bfloat16*)dO;
   a.dm = dm;
   a.TQ = 128 / dm.g_q < dm.B ? 128 / dm.g_q : dm.B;     // a tile stays inside one chunk
   a.n_tiles = (dm.seq_q + a.TQ - 1) / a.TQ;

@@ -1,0 +1,109 @@
+"""GPU parity of the tensor-core Stage-2 backward (dash_attn_bwd_attend_prefill_tc): against the float64 backward oracle
+on the oracle's own routing lists (every row, every gradient), and against the CUDA-core backward kernel on a larger
+case with the library's routing.  P and dS enter the dK / dV products rounded to bf16, dQ is stored as bf16, and delta
+= <O, dO> comes from the forward kernel's accumulator, whose P V product also takes P in bf16: all four gradients carry
+the bf16 tolerance (1e-2 of the largest reference value)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import dash_oracle_bwd as bwd
+from paper_2605_18753_b200 import binding as B
+from paper_2605_18753_b200 import synth
+from tests import helpers as H
+from tests.test_gpu_backward import _close
+from tests.test_gpu_parity import _wl
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _run_tc(p, Q, K, V, dO, mask, bias, w):
+    dQ = torch.full_like(Q, float("nan"))
+    dK = torch.full((w.batch, w.seq, w.h_kv, w.head_dim), float("nan"), device=DEV)
+    dV = torch.full_like(dK, float("nan"))
+    dbias = torch.full((max(B.dash_attn_list_capacity(p), 1),), float("nan"), device=DEV)
+    bws = B.alloc_bwd_workspace(p)
+    B.dash_attn_bwd_attend_prefill_tc(p, Q, K, V, dO, mask, bias, dQ, dK, dV, dbias, bws)
+    torch.cuda.synchronize()
+    assert B.dash_attn_last_status(bws) == 0
+    return dQ, dK, dV, dbias
+
+
+@pytest.mark.parametrize("kw,L", [
+    (dict(seq=400, h_q=8, h_kv=2, head_dim=128, block=64, sigma=1.0), 0),
+    (dict(seq=700, h_q=4, h_kv=2, head_dim=128, block=128, seed=21, sigma=2.0), 0),      # two steps per chunk, g_q = 2
+    (dict(seq=333, h_q=8, h_kv=1, head_dim=128, block=64, alpha=2.0, seed=22), 0),        # g_q = 8, ragged length
+    (dict(seq=520, h_q=8, h_kv=2, head_dim=128, block=64, batch=2, seed=23, gamma=2.0), 0),
+    (dict(seq=420, h_q=4, h_kv=1, head_dim=128, block=64, seed=24), 1),                   # local window
+    (dict(seq=64, h_q=4, h_kv=2, head_dim=128, block=64, seed=25), 0),                    # one chunk: nothing routed
+    (dict(seq=5, h_q=4, h_kv=2, head_dim=128, block=64, seed=26), 0),
+])
+def test_tensor_core_stage2_backward_matches_oracle(kw, L):
+    w = _wl(**kw)
+    inp = synth.make_prefill_inputs(w, DEV)
+    Q, K, V = inp["Q"], inp["K"], inp["V"]
+    dO = torch.randn(Q.shape, device=DEV, generator=torch.Generator(DEV).manual_seed(w.seed + 190)).to(Q.dtype)
+    p = B.params_for_prefill(Q, K, V, dO, block=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma, local_blocks=L)
+    Qn, Kn, Vn, Gn = (H.to_np64(t) for t in (Q, K, V, dO))
+    kwo = dict(B=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma, local_blocks=L)
+    ora = H.oracle_prefill_rows(Q, K, V, rows=range(w.seq), **kwo)
+    mask, count, idx, bias = H.routing_to_abi(ora, p, B.dash_attn_list_offset)
+    ref = bwd.backward_prefill(Qn, Kn, Vn, Gn, through_routing=False, **kwo)
+    dQ, dK, dV, dbias = _run_tc(p, Q, K, V, dO, mask, bias, w)
+    _close(dQ.float().cpu().double().numpy(), ref["dQ"], 1e-2, "dQ")
+    _close(dK.cpu().double().numpy(), ref["dK"], 1e-2, "dK")
+    _close(dV.cpu().double().numpy(), ref["dV"], 1e-2, "dV")
+    db = dbias.cpu().double().numpy()
+    n_entries = 0
+    scale = max([1.0] + [float(np.abs(v).max()) for v in ref["dbias"].values() if v.size])
+    for (b, r, i), want in ref["dbias"].items():
+        off = B.dash_attn_list_offset(p, b, r, i)
+        if want.size:
+            err = float(np.abs(db[off:off + want.size] - want).max())
+            assert err <= 1e-2 * scale, f"dbias row {(b, r, i)}: {err:.3e} vs scale {scale:.3g}"
+            n_entries += want.size
+    if w.seq > 4 * w.block:
+        assert n_entries > 0
+    # entries outside every row's count are zeroed as well
+    if B.dash_attn_list_capacity(p) > 0:
+        assert np.isfinite(db).all()
+
+
+def test_tensor_core_backward_equals_cuda_core_backward_on_library_routing():
+    w = _wl(seq=2048 + 37, h_q=8, h_kv=2, head_dim=128, block=64, seed=31, batch=2)
+    inp = synth.make_prefill_inputs(w, DEV)
+    Q, K, V = inp["Q"], inp["K"], inp["V"]
+    dO = torch.randn(Q.shape, device=DEV, generator=torch.Generator(DEV).manual_seed(131)).to(Q.dtype)
+    p = B.params_for_prefill(Q, K, V, dO, block=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma)
+    kbar = B.alloc_kbar(p)
+    B.dash_attn_block_summaries(p, K, kbar)
+    ws = B.alloc_workspace(p)
+    rt = B.alloc_routing(p)
+    B.dash_attn_select(p, Q, kbar, rt["mask"], rt["count"], rt["blk_idx"], rt["blk_bias"], ws)
+    assert int(rt["count"].max()) > 0
+    dQ0 = torch.empty_like(Q)
+    dK0 = torch.empty(w.batch, w.seq, w.h_kv, w.head_dim, device=DEV)
+    dV0 = torch.empty_like(dK0)
+    db0 = torch.empty_like(rt["blk_bias"])
+    B.dash_attn_bwd_attend_prefill(p, Q, K, V, dO, rt["mask"], rt["blk_bias"], dQ0, dK0, dV0, db0)
+    dQ, dK, dV, db = _run_tc(p, Q, K, V, dO, rt["mask"], rt["blk_bias"], w)
+    for got, want, what, rel in ((dQ, dQ0, "dQ", 1e-2), (dK, dK0, "dK", 1e-2), (dV, dV0, "dV", 1e-2), (db, db0, "dbias", 1e-2)):
+        _close(got.float().cpu().double().numpy(), want.float().cpu().double().numpy(), rel, what)
+    # a second run gives the same bits (no atomics on dQ, dK, dV; one or two commutative adds per dbias entry)
+    dQ2, dK2, dV2, db2 = _run_tc(p, Q, K, V, dO, rt["mask"], rt["blk_bias"], w)
+    assert torch.equal(dQ, dQ2) and torch.equal(dK, dK2) and torch.equal(dV, dV2) and torch.equal(db, db2)
+
+
+def test_tensor_core_backward_refuses_other_shapes():
+    w = _wl(seq=300, h_q=4, h_kv=2, head_dim=128, block=32, seed=5)
+    inp = synth.make_prefill_inputs(w, DEV)
+    Q, K, V = inp["Q"], inp["K"], inp["V"]
+    p = B.params_for_prefill(Q, K, V, Q, block=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma)
+    rt = B.alloc_routing(p)
+    bws = B.alloc_bwd_workspace(p)
+    dK = torch.empty(w.batch, w.seq, w.h_kv, w.head_dim, device=DEV)
+    with pytest.raises(B.DashError) as ei:
+        B.dash_attn_bwd_attend_prefill_tc(p, Q, K, V, Q, rt["mask"], rt["blk_bias"], torch.empty_like(Q), dK,
+                                          torch.empty_like(dK), torch.empty_like(rt["blk_bias"]), bws)
+    assert ei.value.code == -2
