@@ -205,11 +205,13 @@ int dash_attn_bwd_attend_prefill(const dash_params* p, const void* Q, const void
 
 /* The same gradients on tensor cores (bf16, head_dim 128, chunks of 64 or 128 tokens, at least two query heads per KV
  * head, causal; anything else returns DASH_ERR_UNSUPPORTED and nothing is enqueued: call dash_attn_bwd_attend_prefill).
- * Four launches: the forward Stage-2 kernel run for its row statistics (log-sum-exp and delta = <O, dO>; O itself is
- * not written), the prefix counts of the mask words, a query-tile-stationary kernel for dQ and dbias, and a
- * key-slice-stationary kernel for dK and dV (no atomics on dQ, dK, dV: every element has one owner and is written
- * whether or not any row attends it; dbias is zeroed and then receives one or two atomic adds per entry, whose
- * order cannot change the sum).  P and dS enter the dK / dV products rounded to bf16.
+ * Five launches: the forward Stage-2 kernel run for its row statistics (log-sum-exp and delta = <O, dO>; O itself is
+ * not written, and P enters its P V product as two bf16 terms, so that delta, which the routing's backward amplifies,
+ * is accurate to fp32 class), two small kernels over the mask (routed-chunk counts before every mask word; the union
+ * of every query tile's mask words), a query-tile-stationary kernel for dQ and dbias, and a key-slice-stationary
+ * kernel for dK and dV (no atomics on dQ, dK, dV: every element has one owner and is written whether or not any
+ * row attends it; dbias is zeroed and then receives a few atomic adds per entry, whose order cannot change the
+ * sum beyond the last bit).  P and dS enter the dQ / dK / dV products rounded to bf16.
  *   bwd_workspace   device scratch of at least dash_attn_bwd_workspace_bytes(p) bytes, 256-byte aligned, owned by the
  *                   caller; it opens with a status word like the forward workspace's (dash_attn_last_status and
  *                   dash_attn_reset_status accept it): a bounded wait that runs out leaves DASH_ERR_TIMEOUT there.

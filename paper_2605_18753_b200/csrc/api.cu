@@ -1,5 +1,6 @@
 // C ABI of the DashAttention library: argument validation, workspace carving and stage dispatch.
 // Every operation is defined in include/dash_attn.h; kernels live in the sibling translation units.
+#include <algorithm>
 #include <atomic>
 #include <cmath>
 #include <cstring>
@@ -296,8 +297,8 @@ int dash_attn_bwd_attend_prefill(const dash_params* p, const void* Q, const void
                                                        (cudaStream_t)stream));
 }
 
-// Layout of the backward scratch: status region, then lse2 and delta [batch][token][query head], then the routed-chunk
-// prefix counts [batch * h_kv * seq_q][W].
+// Layout of the backward scratch: status region, then lse2 and delta [batch][KV head][query tile][128 rows], then the
+// routed-chunk prefix counts [batch * h_kv * seq_q][W].
 struct BwdLayout {
   size_t status, lse2, delta, prefix, total;
 };
@@ -306,10 +307,13 @@ static BwdLayout bwd_layout(const Dims& dm) {
   BwdLayout l;
   l.status = 0;
   size_t at = up(STATUS_REGION_BYTES);
-  const size_t rows = (size_t)dm.batch * dm.seq_q * dm.h_q;
+  const int tq = std::max(1, std::min(128 / std::max(dm.g_q, 1), dm.B));
+  const size_t rows = (size_t)dm.batch * dm.h_kv * (size_t)((dm.seq_q + tq - 1) / tq) * 128;
   l.lse2 = at; at = up(at + rows * sizeof(float));
   l.delta = at; at = up(at + rows * sizeof(float));
-  l.prefix = at; at = up(at + (size_t)dm.batch * dm.h_kv * dm.seq_q * (size_t)dm.W * sizeof(int));
+  // prefix counts [batch * h_kv * seq_q][W], then the tiles' mask unions [batch * h_kv][query tile][W]
+  l.prefix = at; at = up(at + ((size_t)dm.batch * dm.h_kv * dm.seq_q + (size_t)dm.batch * dm.h_kv * ((dm.seq_q + tq - 1) / tq)) *
+                                  (size_t)dm.W * sizeof(int));
   l.total = at;
   return l;
 }

@@ -264,7 +264,7 @@ cudaError_t launch_attend_prefill_sm100(const Dims& dm, const void* Q, const voi
                                         bool inputs_stable, cudaStream_t st, float* lse2 = nullptr,
                                         float* delta = nullptr, const void* dO = nullptr);
 // Stage 2 backward on tensor cores (bf16, head_dim 128, chunks of 64 or 128 tokens, g_q >= 2); scratch: lse2 and delta
-// [batch][token][query head] floats, prefix [batch * h_kv * seq_q][W] ints.
+// [batch][KV head][query tile][128] floats, prefix [batch * h_kv * seq_q][W] ints.
 bool prefill_bwd_sm100_supported(const Dims& dm);
 cudaError_t launch_attend_prefill_bwd_sm100(const Dims& dm, const void* Q, const void* K, const void* V, const void* dO,
                                             const uint32_t* mask, const float* blk_bias, float* lse2, float* delta,

@@ -18,6 +18,8 @@
 // bf16 operands, fp32 accumulation; head_dim 128; chunks of 64 or 128 tokens; g_q >= 2.  Every wait is bounded.
 #include <cuda.h>
 
+#include <type_traits>
+
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 #include "tensor_map.cuh"
@@ -44,6 +46,7 @@ struct BwdArgs {
   const float* lse2;
   const float* delta;
   const int* prefix;
+  const uint32_t* tile_union;   // [batch * h_kv][query tile][W]: OR of the tile's rows' mask words
   __nv_bfloat16* dQ;
   float* dK;
   float* dV;
@@ -72,26 +75,53 @@ mask_prefix_kernel(Dims dm, const uint32_t* __restrict__ mask, int* __restrict__
   }
 }
 
+// tile_union[group][tile][w] = OR over the tile's rows of mask word w: which chunks any row of the tile attends
+__global__ void __launch_bounds__(256)
+tile_union_kernel(Dims dm, int TQ, int n_tiles, const uint32_t* __restrict__ mask, uint32_t* __restrict__ tile_union) {
+  chain_wait();
+  chain_release();
+  const long long warp_id = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  const long long total = (long long)dm.batch * dm.h_kv * n_tiles;
+  if (warp_id >= total) return;
+  const long long grp = warp_id / n_tiles;
+  const int tile = (int)(warp_id % n_tiles);
+  for (int w = 0; w < dm.W; ++w) {
+    uint32_t u = 0u;
+    for (int t = lane; t < TQ; t += 32) {
+      const int i = tile * TQ + t;
+      if (i < dm.seq_q) u |= mask[(grp * dm.seq_q + i) * dm.W + w];
+    }
+    u = __reduce_or_sync(0xffffffffu, u);
+    if (lane == 0) tile_union[warp_id * dm.W + w] = u;
+  }
+}
+
 // ===================================================================================================================
 // dQ and dbias: query-tile stationary
 // ===================================================================================================================
 namespace dq {
 
-constexpr int THREADS = 224;            // 4 softmax warps, K producer, MMA issuer, V / bias producer
-constexpr uint32_t TMEM_COLS = 512;     // S0 [0,64) S1 [64,128) dP0 [128,192) dP1 [192,256) dQ [256,384)
-constexpr uint32_t COL_DP = 128, COL_DQ = 256;
-enum Bar { QD_FULL = 0, META, SD_FULL = 2, DQ_DONE = 4, DS_FULL = 6, V_FULL = 8, K_FULL = 10, N_BARS = 12 };
+// Two warpgroups form dS, each for half of a step's 64 columns (no row maximum is needed: the log-sum-exp is known), so
+// a step's exponentials take half as long.  One issuing thread per product (S, dP, dQ): a thread issues an MMA every
+// 60-80 clocks whatever its size, and 20 per step through one thread would be the kernel's pace.
+constexpr int W_KPROD = 8, W_S = 9, W_VPROD = 10, W_DP = 11, W_DQ = 12;
+constexpr int THREADS = 416;
+constexpr int KST = 3;                  // K / V ring and S / dP ring: stage = step mod 3, held until the step's dQ product is done
+constexpr uint32_t TMEM_COLS = 512;     // S [0,192) dP [192,384) dQ [384,512)
+constexpr uint32_t COL_DP = 192, COL_DQ = 384;
+enum Bar { QD_FULL = 0, META, S_FULL = 2, DP_FULL = 5, DS_FULL = 8, V_FULL = 11, K_FULL = 14, KV_FREE = 17, N_BARS = 20 };
 struct Misc {
   unsigned long long bar[N_BARS];
   uint32_t tmem_base;
   int n_steps;
   int abort_flag;
-  int kvbase[2];
-  float bias[2][MAX_TQ];
-  long long entry[2][MAX_TQ];           // list entry of the token for the step's chunk (-1: none: own chunk or not routed)
+  int kvbase[KST];
+  float bias[KST][MAX_TQ];
+  long long entry[KST][MAX_TQ];         // list entry of the token for the step's chunk (-1: none: own chunk or not routed)
 };
-constexpr uint32_t OFF_Q = 0, OFF_DO = OFF_Q + Q_BYTES, OFF_K = OFF_DO + Q_BYTES, OFF_V = OFF_K + 2 * KV_TILE_BYTES,
-                   OFF_MISC = OFF_V + 2 * KV_TILE_BYTES, SMEM = OFF_MISC + sizeof(Misc);
+constexpr uint32_t OFF_Q = 0, OFF_DO = OFF_Q + Q_BYTES, OFF_K = OFF_DO + Q_BYTES, OFF_V = OFF_K + KST * KV_TILE_BYTES,
+                   OFF_MISC = OFF_V + KST * KV_TILE_BYTES, SMEM = OFF_MISC + sizeof(Misc);
 static_assert(SMEM <= 232448, "one block per SM");
 
 __global__ void __launch_bounds__(THREADS, 1)
@@ -122,16 +152,17 @@ attend_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     if (misc->abort_flag) report_error(a.sb, DASH_ERR_CUDA, 110);
     ptx::mbar_init(bar(QD_FULL), 1);
     ptx::mbar_init(bar(META), 1);
-    for (int s = 0; s < 2; ++s) {
-      ptx::mbar_init(bar(SD_FULL + s), 1);
-      ptx::mbar_init(bar(DQ_DONE + s), 1);
+    for (int s = 0; s < KST; ++s) {
+      ptx::mbar_init(bar(S_FULL + s), 1);
+      ptx::mbar_init(bar(DP_FULL + s), 1);
+      ptx::mbar_init(bar(DS_FULL + s), 256);
       ptx::mbar_init(bar(K_FULL + s), 1);
       ptx::mbar_init(bar(V_FULL + s), 1);
-      ptx::mbar_init(bar(DS_FULL + s), 128);
+      ptx::mbar_init(bar(KV_FREE + s), 1);
     }
     ptx::fence_barrier_init();
   }
-  if (warp == 5) {
+  if (warp == W_S) {
     ptx::tmem_alloc(ptx::smem_u32(&misc->tmem_base), TMEM_COLS);
     ptx::tmem_relinquish();
     ptx::tc_fence_before();
@@ -150,9 +181,9 @@ attend_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     ptx::tma_load_4d(dst + KV_TILE_BYTES / 2, tm, barrier, 64, r, kv0, b);
   };
 
-  if (warp == 4 || warp == 6) {
+  if (warp == W_KPROD || warp == W_VPROD) {
     // =========================== producers: the forward kernel's walk ===========================
-    const bool do_k = (warp == 4), do_v = (warp == 6);
+    const bool do_k = (warp == W_KPROD), do_v = (warp == W_VPROD);
     if (lane == 0 && do_k) {
       ptx::prefetch_tensormap(&tmQ);
       ptx::prefetch_tensormap(&tmDO);
@@ -164,7 +195,7 @@ attend_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
       ptx::tma_load_4d(sbase + OFF_DO, &tmDO, bar(QD_FULL), 0, r * g_q, i0, b);
       ptx::tma_load_4d(sbase + OFF_DO + Q_BYTES / 2, &tmDO, bar(QD_FULL), 64, r * g_q, i0, b);
     }
-    // own chunk first (steps 0 .. own_steps-1 go to stages 0 / 1, which are free)
+    // own chunk first (steps 0 .. own_steps-1 <= 2 go to stages 0 / 1, which are free)
     for (int sub = 0; sub < own_steps; ++sub) {
       const int kv0 = c_own * dm.B + sub * NKV;
       if (do_k) {
@@ -209,12 +240,13 @@ attend_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     }
     int j = own_steps;
     bool ok = true;
-    int last_j[2] = {-1, -1};
-    for (int sub = 0; sub < own_steps; ++sub) last_j[sub] = sub;
+    int last_j[KST];
+    for (int s = 0; s < KST; ++s) last_j[s] = s < own_steps ? s : -1;
     int seen[2] = {0, 0};
+    uint32_t rw[2], rw_n[2] = {0u, 0u};
+    load_rows(0, rw);
+    if (n_words > 1) load_rows(1, rw_n);
     for (int w = 0; w < n_words && ok; ++w) {
-      uint32_t rw[2];
-      load_rows(w, rw);
       uint32_t u = union_of(w, rw);
       uint32_t rb[2];
       for (int q = 0; q < 2; ++q) rb[q] = w == n_words - 1 ? rw[q] & own_word_keep & ~(1u << (c_own & 31)) : rw[q];
@@ -233,15 +265,15 @@ attend_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         }
         for (int sub = 0; sub < sub_per_blk && ok; ++sub, ++j) {
           const int kv0 = c * dm.B + sub * NKV;
-          const int st = j & 1, prev_ph = ((j >> 1) - 1) & 1;
-          if (j >= 2) ok = wait_on(bar(DQ_DONE + st), prev_ph);     // every product of step j-2 has read the stage
+          const int st = j % KST;
+          if (j >= KST) ok = wait_on(bar(KV_FREE + st), (uint32_t)(j / KST - 1) & 1u);   // every product of step j-3 has read the stage
           if (!ok) break;
           if (do_k) {
             if (lane == 0) load_kv(&tmK, sbase + OFF_K + st * KV_TILE_BYTES, bar(K_FULL + st), kv0);
           } else {
             for (int q = 0; q < 2; ++q) {
               const int t = lane + 32 * q;
-              if (t < TQ) { misc->bias[st][t] = bv[q]; misc->entry[st][t] = sub == 0 ? en[q] : en[q]; }
+              if (t < TQ) { misc->bias[st][t] = bv[q]; misc->entry[st][t] = en[q]; }
             }
             if (lane == 0) misc->kvbase[st] = kv0;
             __syncwarp();
@@ -252,105 +284,101 @@ attend_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
       }
       seen[0] += __popc(rb[0]);
       seen[1] += __popc(rb[1]);
+      rw[0] = rw_n[0]; rw[1] = rw_n[1];
+      if (w + 2 < n_words) load_rows(w + 2, rw_n);
     }
     if (!ok && lane == 0) {
-      for (int s = 0; s < 2; ++s) {
+      for (int s = 0; s < KST; ++s) {
         if (last_j[s] < 0) continue;
-        const uint32_t full = bar((do_k ? K_FULL : V_FULL) + s), parity = (uint32_t)(last_j[s] >> 1) & 1u;
+        const uint32_t full = bar((do_k ? K_FULL : V_FULL) + s), parity = (uint32_t)(last_j[s] / KST) & 1u;
         for (int k = 0; k < 200000 && !ptx::mbar_try_wait(full, parity); ++k) {}
       }
       if (do_k)
         for (int k = 0; k < 200000 && !ptx::mbar_try_wait(bar(QD_FULL), 0); ++k) {}
     }
-  } else if (warp == 5) {
-    // =========================== MMA issuer ===========================
+  } else if (warp == W_S || warp == W_DP) {
+    // =========================== issuers of S = Q K^T (warp W_S) and dP = dO V^T (warp W_DP) ===========================
+    // Ring slot j mod 3 of S / dP is free when the K / V stage of the same index is: both wait for the dQ product of
+    // step j-3 (the producers do, before they refill the stage).
     if (lane == 0) {
-      bool ok = wait_on(bar(QD_FULL), 0);
-      constexpr uint32_t IDESC_S = ptx::idesc_bf16_f32(128, NKV, false, false);
-      constexpr uint32_t IDESC_DQ = ptx::idesc_bf16_f32(128, HD, false, true);
-      const uint64_t qd0 = ptx::smem_desc_sw128(sbase + OFF_Q, 16, 1024);
-      const uint64_t gd0 = ptx::smem_desc_sw128(sbase + OFF_DO, 16, 1024);
-      const uint64_t kd0 = ptx::smem_desc_sw128(sbase + OFF_K, 16, 1024);
-      const uint64_t vd0 = ptx::smem_desc_sw128(sbase + OFF_V, 16, 1024);
-      const uint64_t kmn0 = ptx::smem_desc_sw128(sbase + OFF_K, KV_TILE_BYTES / 2, 1024);   // K as MN-major B of dQ += dS K
-      auto issue_sd = [&](int j) -> bool {
-        const int buf = j & 1;
-        if (!wait_on(bar(K_FULL + buf), (j >> 1) & 1)) return false;
-        if (!wait_on(bar(V_FULL + buf), (j >> 1) & 1)) return false;
-        ptx::tc_fence_after();
-        const uint64_t kd = kd0 + (uint64_t)((buf * KV_TILE_BYTES) >> 4);
-        const uint64_t vd = vd0 + (uint64_t)((buf * KV_TILE_BYTES) >> 4);
-#pragma unroll
-        for (int k = 0; k < HD / 16; ++k) {
-          const uint64_t off_a = (uint64_t)(((k >> 2) * (Q_BYTES / 2) + (k & 3) * 32) >> 4);
-          const uint64_t off_b = (uint64_t)(((k >> 2) * (KV_TILE_BYTES / 2) + (k & 3) * 32) >> 4);
-          ptx::mma_bf16_ss(tmem + buf * NKV, qd0 + off_a, kd + off_b, IDESC_S, k > 0 ? 1u : 0u);
-        }
-#pragma unroll
-        for (int k = 0; k < HD / 16; ++k) {
-          const uint64_t off_a = (uint64_t)(((k >> 2) * (Q_BYTES / 2) + (k & 3) * 32) >> 4);
-          const uint64_t off_b = (uint64_t)(((k >> 2) * (KV_TILE_BYTES / 2) + (k & 3) * 32) >> 4);
-          ptx::mma_bf16_ss(tmem + COL_DP + buf * NKV, gd0 + off_a, vd + off_b, IDESC_S, k > 0 ? 1u : 0u);
-        }
-        ptx::mma_commit(bar(SD_FULL + buf));
-        return true;
-      };
-      if (ok) ok = issue_sd(0);
-      ok = ok && wait_on(bar(META), 0);
+      const bool is_s = warp == W_S;
+      bool ok = wait_on(bar(QD_FULL), 0) && wait_on(bar(META), 0);
       const int n_steps = ok ? misc->n_steps : 0;
+      constexpr uint32_t IDESC_S = ptx::idesc_bf16_f32(128, NKV, false, false);
+      const uint64_t ad0 = ptx::smem_desc_sw128(sbase + (is_s ? OFF_Q : OFF_DO), 16, 1024);
+      const uint64_t bd0 = ptx::smem_desc_sw128(sbase + (is_s ? OFF_K : OFF_V), 16, 1024);
+      const uint32_t col0 = is_s ? 0u : COL_DP;
       for (int j = 0; j < n_steps && ok; ++j) {
-        if (j + 1 < n_steps) ok = issue_sd(j + 1);
-        if (!ok) break;
-        const int buf = j & 1;
-        ok = wait_on(bar(DS_FULL + buf), (j >> 1) & 1);
+        const int st = j % KST;
+        ok = wait_on(bar((is_s ? K_FULL : V_FULL) + st), (uint32_t)(j / KST) & 1u);
         if (!ok) break;
         ptx::tc_fence_after();
-        const uint64_t kmn = kmn0 + (uint64_t)((buf * KV_TILE_BYTES) >> 4);
+        const uint64_t bd = bd0 + (uint64_t)((st * KV_TILE_BYTES) >> 4);
+#pragma unroll
+        for (int k = 0; k < HD / 16; ++k) {
+          const uint64_t off_a = (uint64_t)(((k >> 2) * (Q_BYTES / 2) + (k & 3) * 32) >> 4);
+          const uint64_t off_b = (uint64_t)(((k >> 2) * (KV_TILE_BYTES / 2) + (k & 3) * 32) >> 4);
+          ptx::mma_bf16_ss(tmem + col0 + st * NKV, ad0 + off_a, bd + off_b, IDESC_S, k > 0 ? 1u : 0u);
+        }
+        ptx::mma_commit(bar((is_s ? S_FULL : DP_FULL) + st));
+      }
+    }
+    __syncwarp();
+  } else if (warp == W_DQ) {
+    // =========================== issuer of dQ += dS K ===========================
+    if (lane == 0) {
+      bool ok = wait_on(bar(META), 0);
+      const int n_steps = ok ? misc->n_steps : 0;
+      constexpr uint32_t IDESC_DQ = ptx::idesc_bf16_f32(128, HD, false, true);
+      const uint64_t kmn0 = ptx::smem_desc_sw128(sbase + OFF_K, KV_TILE_BYTES / 2, 1024);   // K as MN-major B
+      for (int j = 0; j < n_steps && ok; ++j) {
+        const int st = j % KST;
+        ok = wait_on(bar(DS_FULL + st), (uint32_t)(j / KST) & 1u);
+        if (!ok) break;
+        ptx::tc_fence_after();
+        const uint64_t kmn = kmn0 + (uint64_t)((st * KV_TILE_BYTES) >> 4);
 #pragma unroll
         for (int k = 0; k < NKV / 16; ++k)
-          ptx::mma_bf16_ts(tmem + COL_DQ, tmem + buf * NKV + k * 8, kmn + (uint64_t)((k * 16 * 128) >> 4), IDESC_DQ,
-                           (j > 0 || k > 0) ? 1u : 0u);
-        ptx::mma_commit(bar(DQ_DONE + buf));
+          // dS of keys 16k .. 16k+15: eight packed columns, keys 0-31 at columns 0-15 and keys 32-63 at columns 32-47
+          ptx::mma_bf16_ts(tmem + COL_DQ, tmem + st * NKV + (k >> 1) * 32 + (k & 1) * 8, kmn + (uint64_t)((k * 16 * 128) >> 4),
+                           IDESC_DQ, (j > 0 || k > 0) ? 1u : 0u);
+        ptx::mma_commit(bar(KV_FREE + st));
       }
     }
     __syncwarp();
   } else {
-    // =========================== dS / epilogue: thread = tile row ===========================
-    const int m = tid;
+    // =========================== dS / epilogue: thread = tile row, warpgroup = column half ===========================
+    const int wg = warp >> 2;
+    const int m = (warp & 3) * 32 + lane;
     const int t = m / g_q, hh = m % g_q;
     const int i_row = i0 + t;
     const bool row_ok = i_row < dm.seq_q;
-    const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+    const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
     const float c1 = dm.sm_scale * LOG2E;
-    const long long srow = ((long long)b * dm.seq_q + min(i_row, dm.seq_q - 1)) * dm.h_q + r * g_q + hh;
+    const long long srow = (((long long)b * dm.h_kv + r) * a.n_tiles + tile) * 128 + m;
     const float lse2 = row_ok ? a.lse2[srow] : 0.f;
     const float delta = row_ok ? a.delta[srow] : 0.f;
-    bool ok = true;
-    int n_steps = 0x7fffffff;
-    for (int j = 0; ok; ++j) {
-      if (j == 1) {
-        ok = wait_on(bar(META), 0);
-        if (!ok) break;
-        n_steps = misc->n_steps;
-      }
-      if (j >= n_steps) break;
-      const int buf = j & 1;
-      ok = wait_on(bar(V_FULL + buf), (j >> 1) & 1);       // bias / entry / kvbase of the step visible
+    bool ok = wait_on(bar(META), 0);
+    const int n_steps = ok ? misc->n_steps : 0;
+    for (int j = 0; j < n_steps && ok; ++j) {
+      const int st = j % KST;
+      const uint32_t ph = (uint32_t)(j / KST) & 1u;
+      ok = wait_on(bar(V_FULL + st), ph);                  // bias / entry / kvbase of the step visible
       if (!ok) break;
-      const float bias = row_ok ? misc->bias[buf][t] : -INFINITY;
-      const long long entry = misc->entry[buf][t];
-      const int kv0 = misc->kvbase[buf];
-      ok = wait_on(bar(SD_FULL + buf), (j >> 1) & 1);
+      const float bias = row_ok ? misc->bias[st][t] : -INFINITY;
+      const long long entry = misc->entry[st][t];
+      const int kv0 = misc->kvbase[st];
+      ok = wait_on(bar(S_FULL + st), ph) && wait_on(bar(DP_FULL + st), ph);
       if (!ok) break;
       ptx::tc_fence_after();
       const int n_vis = i_row - kv0 + 1;                   // causal: column c visible iff c < n_vis
       const float off = bias * LOG2E - lse2;               // -inf: the row did not route the chunk
       float rowsum = 0.f;
-#pragma unroll 1
-      for (int half = 0; half < 2; ++half) {
+      {
+        const int half = wg;
         uint32_t sv[32], gv[32];
-        DASH_TMEM_LD32(sv, lane_addr + buf * NKV + half * 32);
-        DASH_TMEM_LD32(gv, lane_addr + COL_DP + buf * NKV + half * 32);
+        DASH_TMEM_LD32(sv, lane_addr + st * NKV + half * 32);
+        DASH_TMEM_LD32(gv, lane_addr + COL_DP + st * NKV + half * 32);
         ptx::tmem_wait_ld();
         uint32_t packed[16];
 #pragma unroll
@@ -366,24 +394,25 @@ attend_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
           __nv_bfloat162 h = __floats2bfloat162_rn(ds[0], ds[1]);
           packed[c >> 1] = *reinterpret_cast<uint32_t*>(&h);
         }
-        // dS row -> columns [half*16, half*16 + 16) of the step's S buffer (two bf16 per column)
-        ptx::tmem_st_n<16>(lane_addr + buf * NKV + half * 16, packed);
+        // dS row -> the first 16 columns of this warpgroup's own half of the step's S buffer (two bf16 per column):
+        // the other warpgroup's scores, in the other 32 columns, are never touched
+        ptx::tmem_st_n<16>(lane_addr + st * NKV + half * 32, packed);
       }
       ptx::tmem_wait_st();
       ptx::tc_fence_before();
-      ptx::mbar_arrive(bar(DS_FULL + buf));
+      ptx::mbar_arrive(bar(DS_FULL + st));
       // dbias of the (token, chunk): the row sums of the group's heads (adjacent lanes) added up
       for (int o = 1; o < g_q; o <<= 1) rowsum += __shfl_xor_sync(0xffffffffu, rowsum, o);
       if (hh == 0 && entry >= 0 && row_ok) atomicAdd(a.dbias + entry, rowsum);
     }
-    // epilogue: dQ / sqrt(d) -> global
-    if (ok && n_steps > 0) ok = wait_on(bar(DQ_DONE + ((n_steps - 1) & 1)), ((n_steps - 1) >> 1) & 1);
+    // epilogue: dQ / sqrt(d) -> global; each warpgroup takes half of the row's columns
+    if (ok && n_steps > 0) ok = wait_on(bar(KV_FREE + ((n_steps - 1) % KST)), (uint32_t)((n_steps - 1) / KST) & 1u);
     if (ok && n_steps > 0) {
       ptx::tc_fence_after();
       __nv_bfloat16* op = a.dQ + (long long)b * dm.qs[0] + (long long)i_row * dm.qs[1] + (long long)(r * g_q + hh) * dm.qs[2];
       const float sc = dm.sm_scale;
 #pragma unroll 1
-      for (int q = 0; q < HD / 32; ++q) {
+      for (int q = wg * 2; q < wg * 2 + 2; ++q) {
         uint32_t o[32];
         DASH_TMEM_LD32(o, lane_addr + COL_DQ + q * 32);
         ptx::tmem_wait_ld();
@@ -406,7 +435,7 @@ attend_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
   }
 
   __syncthreads();
-  if (warp == 5) {
+  if (warp == W_S) {
     ptx::tc_fence_after();
     ptx::tmem_dealloc(tmem, TMEM_COLS);
   }
@@ -420,17 +449,24 @@ attend_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
 // ===================================================================================================================
 namespace dkv {
 
-constexpr int THREADS = 192;            // 4 softmax warps, producer, MMA issuer
+// Two warpgroups form P and dS (even / odd steps, one S / dP buffer each); producer; one issuer for the score products
+// (S, dP) and one for the accumulating products (dV^T, dK^T): 32 MMAs per step are too many for one issuing thread.
+// W_PROD loads the tiles, W_META the per-token biases of each step; W_SD issues S, W_DP dP, W_ACC dV^T, W_DK dK^T
+constexpr int W_PROD = 8, W_SD = 9, W_ACC = 10, W_DP = 11, W_DK = 12, W_META = 13;
+constexpr int THREADS = 448;
 constexpr uint32_t TMEM_COLS = 512;     // S0 S1 [0,128) dP0 dP1 [128,256) dV^T [256,320) dK^T [320,384)
 constexpr uint32_t COL_DP = 128, COL_DV = 256, COL_DK = 320;
 constexpr uint32_t PS_BYTES = 128 * NKV * 2;       // 16 KiB: P (or dS) of a step, 128 rows of 128 bytes
-enum Bar { KV_FULL = 0, QD_FULL = 1, SD_FULL = 3, ACC_DONE = 5, PDS_FULL = 7, N_BARS = 8 };
+enum Bar { KV_FULL = 0, QD_FULL = 1, SD_FULL = 3, ACC_DONE = 5, PDS_FULL = 7, N_BARS = 9 };   // SD_FULL, ACC_DONE: two arrivals (one per issuer)
 struct Misc {
   unsigned long long bar[N_BARS];
   uint32_t tmem_base;
   int abort_flag;
+  int total;                            // number of steps, written with the end markers
   int tile[2];                          // query tile of the stage's step (-1: no more steps)
   float bias[2][MAX_TQ];                // per token of the tile: the chunk's bias (-inf: the token does not attend it)
+  alignas(16) float lse2[2][128];       // the tile's row statistics (bulk copies)
+  alignas(16) float delta[2][128];
 };
 constexpr uint32_t OFF_K = 0, OFF_V = OFF_K + KV_TILE_BYTES, OFF_Q = OFF_V + KV_TILE_BYTES,   // Q stage s at OFF_Q + s * 2 * Q_BYTES,
                    OFF_P = OFF_Q + 4 * Q_BYTES, OFF_DS = OFF_P + PS_BYTES,                   //   its dO tile Q_BYTES behind
@@ -463,14 +499,14 @@ attend_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     if (misc->abort_flag) report_error(a.sb, DASH_ERR_CUDA, 120);
     ptx::mbar_init(bar(KV_FULL), 1);
     for (int s = 0; s < 2; ++s) {
-      ptx::mbar_init(bar(QD_FULL + s), 1);
-      ptx::mbar_init(bar(SD_FULL + s), 1);
-      ptx::mbar_init(bar(ACC_DONE + s), 1);
+      ptx::mbar_init(bar(QD_FULL + s), 2);     // the loader's arrival (with the byte count) and the bias warp's
+      ptx::mbar_init(bar(SD_FULL + s), 2);
+      ptx::mbar_init(bar(ACC_DONE + s), 2);
+      ptx::mbar_init(bar(PDS_FULL + s), 128);
     }
-    ptx::mbar_init(bar(PDS_FULL), 128);
     ptx::fence_barrier_init();
   }
-  if (warp == 5) {
+  if (warp == W_SD) {
     ptx::tmem_alloc(ptx::smem_u32(&misc->tmem_base), TMEM_COLS);
     ptx::tmem_relinquish();
     ptx::tc_fence_before();
@@ -483,9 +519,15 @@ attend_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   if (a.sb && *reinterpret_cast<volatile int*>(&a.sb->status) != 0) *abort_flag = 1;
   __syncthreads();
 
-  if (warp == 4) {
-    // =========================== producer: K / V slice, then the query tiles that attend it ===========================
-    if (lane == 0) {
+  if (warp == W_PROD || warp == W_META) {
+    // =========================== producers ===========================
+    // Both warps enumerate the slice's steps in the same order: (i) the tiles of the slice's own chunk that can see it
+    // (tokens from k0 on: bias 0, causal mask in the kernel), (ii) the later tiles one of whose rows routed the chunk,
+    // read 32 tiles at a time from the tile unions.  W_PROD fetches K / V once and the Q / dO tiles and row
+    // statistics of every step; W_META looks up the per-token biases.  A step's stage is free once both accumulating
+    // products of step j-2 have completed.
+    const bool loader = warp == W_PROD;
+    if (lane == 0 && loader) {
       ptx::prefetch_tensormap(&tmQ);
       ptx::prefetch_tensormap(&tmDO);
       ptx::prefetch_tensormap(&tmK);
@@ -496,74 +538,130 @@ attend_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       ptx::tma_load_4d(sbase + OFF_V, &tmV, bar(KV_FULL), 0, r, k0, b);
       ptx::tma_load_4d(sbase + OFF_V + KV_TILE_BYTES / 2, &tmV, bar(KV_FULL), 64, r, k0, b);
     }
-    const long long row0 = ((long long)b * dm.h_kv + r) * dm.seq_q;
+    const long long grp_l = (long long)b * dm.h_kv + r;
+    const long long row0 = grp_l * dm.seq_q;
+    const long long list0 = grp_l * dm.list_rows;
+    const long long stat0 = grp_l * a.n_tiles * 128;
+    const uint32_t* tu = a.tile_union + grp_l * a.n_tiles * dm.W;
     const int wc = c >> 5, bit = c & 31;
     int j = 0;
     bool ok = true;
-    // one step: the stage is free once both accumulating products of step j-2 have completed
-    auto push = [&](int tile_idx, const float* bv) {
+    auto stage_free = [&]() {
+      if (j >= 2) ok = wait_on(bar(ACC_DONE + (j & 1)), (uint32_t)((j >> 1) - 1) & 1u);
+      return ok;
+    };
+    // ---- the loader's step
+    auto load_step = [&](int tile_idx) {
+      if (!stage_free()) return;
       const int st = j & 1;
-      if (j >= 2) ok = wait_on(bar(ACC_DONE + st), (uint32_t)((j >> 1) - 1) & 1u);
-      if (!ok) return;
-      if (tile_idx >= 0) {
-        for (int q = 0; q < 2; ++q) {
-          const int t = lane + 32 * q;
-          if (t < TQ) misc->bias[st][t] = bv[q];
-        }
-      }
-      if (lane == 0) misc->tile[st] = tile_idx;
-      __syncwarp();
       if (lane == 0) {
+        misc->tile[st] = tile_idx;
         if (tile_idx >= 0) {
           const int i0 = tile_idx * TQ;
           const uint32_t dst = sbase + OFF_Q + st * 2 * Q_BYTES;
-          ptx::mbar_arrive_expect_tx(bar(QD_FULL + st), 2 * Q_BYTES);
+          ptx::mbar_arrive_expect_tx(bar(QD_FULL + st), 2 * Q_BYTES + 2 * 512);
           ptx::tma_load_4d(dst, &tmQ, bar(QD_FULL + st), 0, r * g_q, i0, b);
           ptx::tma_load_4d(dst + Q_BYTES / 2, &tmQ, bar(QD_FULL + st), 64, r * g_q, i0, b);
           ptx::tma_load_4d(dst + Q_BYTES, &tmDO, bar(QD_FULL + st), 0, r * g_q, i0, b);
           ptx::tma_load_4d(dst + Q_BYTES + Q_BYTES / 2, &tmDO, bar(QD_FULL + st), 64, r * g_q, i0, b);
+          ptx::bulk_load(ptx::smem_u32(&misc->lse2[st][0]), a.lse2 + stat0 + (long long)tile_idx * 128, 512, bar(QD_FULL + st));
+          ptx::bulk_load(ptx::smem_u32(&misc->delta[st][0]), a.delta + stat0 + (long long)tile_idx * 128, 512, bar(QD_FULL + st));
         } else {
           ptx::mbar_arrive(bar(QD_FULL + st));
         }
       }
       ++j;
     };
-    // (i) the tiles of the slice's own chunk that can see it (tokens from k0 on): bias 0, causal mask in the kernel
-    const int t_own_lo = k0 / TQ, t_first_routed = min(((c + 1) * dm.B + TQ - 1) / TQ, a.n_tiles);
-    for (int tl = t_own_lo; tl < t_first_routed && ok; ++tl) {
-      float bv[2];
-      for (int q = 0; q < 2; ++q) bv[q] = (tl * TQ + lane + 32 * q < dm.seq_q) ? 0.f : -INFINITY;
-      push(tl, bv);
-    }
-    // (ii) later tiles whose rows routed the chunk; four tiles' mask words are fetched per round
-    for (int tl0 = t_first_routed; tl0 < a.n_tiles && ok; tl0 += 4) {
-      uint32_t wd[4][2];
+    // ---- the bias warp's steps, four at a time: the mask words and prefix counts of all four, then their biases,
+    // then the four hand-overs (lane t owns tokens t and t + 32 of a tile)
+    int pend[4], n_pend = 0;
+    bool pend_own = false;
+    auto flush = [&]() {
+      float bv[4][2];
+      if (pend_own) {
 #pragma unroll
-      for (int u = 0; u < 4; ++u)
-        for (int q = 0; q < 2; ++q) {
-          const int t = lane + 32 * q, i = (tl0 + u) * TQ + t;
-          wd[u][q] = (tl0 + u < a.n_tiles && t < TQ && i < dm.seq_q) ? a.mask[(row0 + i) * dm.W + wc] : 0u;
-        }
+        for (int u = 0; u < 4; ++u)
+          for (int q = 0; q < 2; ++q) bv[u][q] = (u < n_pend && pend[u] * TQ + lane + 32 * q < dm.seq_q) ? 0.f : -INFINITY;
+      } else {
+        uint32_t wd[4][2];
+        int pf[4][2];
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+#pragma unroll
+          for (int q = 0; q < 2; ++q) {
+            const int t = lane + 32 * q, i = (u < n_pend ? pend[u] : 0) * TQ + t;
+            const bool live = u < n_pend && t < TQ && i < dm.seq_q;
+            wd[u][q] = live ? a.mask[(row0 + i) * dm.W + wc] : 0u;
+            pf[u][q] = live ? a.prefix[(row0 + i) * dm.W + wc] : 0;
+          }
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+#pragma unroll
+          for (int q = 0; q < 2; ++q) {
+            bv[u][q] = -INFINITY;
+            if ((wd[u][q] >> bit) & 1u) {
+              const int i = pend[u] * TQ + lane + 32 * q;
+              bv[u][q] = __ldg(a.blk_bias + list0 + list_row_offset(dm, i) + pf[u][q] + __popc(wd[u][q] & ((1u << bit) - 1u)));
+            }
+          }
+      }
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
-        const bool mine = (((wd[u][0] | wd[u][1]) >> bit) & 1u) != 0u;
-        if (!__any_sync(0xffffffffu, mine) || !ok) continue;
-        float bv[2];
-        for (int q = 0; q < 2; ++q) {
-          const int t = lane + 32 * q, i = (tl0 + u) * TQ + t;
-          bv[q] = -INFINITY;
-          if ((wd[u][q] >> bit) & 1u) {
-            const long long row = row0 + i;
-            const long long e = ((long long)b * dm.h_kv + r) * dm.list_rows + list_row_offset(dm, i) +
-                                a.prefix[row * dm.W + wc] + __popc(wd[u][q] & ((1u << bit) - 1u));
-            bv[q] = __ldg(a.blk_bias + e);
+        if (u < n_pend && stage_free()) {
+          const int st = j & 1;
+          for (int q = 0; q < 2; ++q) {
+            const int t = lane + 32 * q;
+            if (t < TQ) misc->bias[st][t] = bv[u][q];
           }
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(bar(QD_FULL + st));
+          ++j;
         }
-        push(tl0 + u, bv);
+      }
+      n_pend = 0;
+    };
+    auto meta_step = [&](int tile_idx, bool own) {
+      if (n_pend > 0 && own != pend_own) flush();
+      pend_own = own;
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (u == n_pend) pend[u] = tile_idx;
+      if (++n_pend == 4) flush();
+    };
+    auto step = [&](int tile_idx, bool own) {
+      if (loader) load_step(tile_idx); else meta_step(tile_idx, own);
+    };
+    const int t_own_lo = k0 / TQ, t_first_routed = min(((c + 1) * dm.B + TQ - 1) / TQ, a.n_tiles);
+    for (int tl = t_own_lo; tl < t_first_routed && ok; ++tl) step(tl, true);
+    auto union_word = [&](int tl0) -> uint32_t {
+      const int tl = tl0 + lane;
+      return tl < a.n_tiles ? __ldg(tu + (long long)tl * dm.W + wc) : 0u;
+    };
+    uint32_t uw = t_first_routed < a.n_tiles ? union_word(t_first_routed) : 0u, uw_n = 0u;
+    for (int tl0 = t_first_routed; tl0 < a.n_tiles && ok; tl0 += 32) {
+      if (tl0 + 32 < a.n_tiles) uw_n = union_word(tl0 + 32);
+      uint32_t hits = __ballot_sync(0xffffffffu, ((uw >> bit) & 1u) != 0u);
+      while (hits != 0u && ok) {
+        const int k = __ffs(hits) - 1;
+        hits &= hits - 1;
+        step(tl0 + k, false);
+      }
+      uw = uw_n;
+    }
+    if (!loader && ok && n_pend > 0) flush();
+    // two end markers: one for each step parity (each warpgroup meets one)
+    if (ok && loader) {
+      if (lane == 0) misc->total = j;
+      __syncwarp();
+      load_step(-1);
+      if (ok) load_step(-1);
+    } else if (ok) {
+      for (int e = 0; e < 2 && stage_free(); ++e) {
+        if (lane == 0) ptx::mbar_arrive(bar(QD_FULL + (j & 1)));
+        ++j;
       }
     }
-    if (ok) push(-1, nullptr);         // end marker
-    if (!ok && lane == 0) {
+    if (!ok && lane == 0 && loader) {
       // a wait ran out: let the copies already issued land (bounded) before the block retires
       for (int k = 0; k < 200000 && !ptx::mbar_try_wait(bar(KV_FULL), 0); ++k) {}
       for (int s = 0; s < 2; ++s) {
@@ -572,85 +670,96 @@ attend_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         for (int k = 0; k < 200000 && !ptx::mbar_try_wait(bar(QD_FULL + (lj & 1)), (uint32_t)(lj >> 1) & 1u); ++k) {}
       }
     }
-  } else if (warp == 5) {
-    // =========================== MMA issuer ===========================
+  } else if (warp == W_SD || warp == W_DP) {
+    // =========================== issuers of the score products: S = Q K^T (W_SD), dP = dO V^T (W_DP) ===========================
     if (lane == 0) {
+      const bool is_s = warp == W_SD;
       bool ok = wait_on(bar(KV_FULL), 0);
       constexpr uint32_t IDESC_S = ptx::idesc_bf16_f32(128, NKV, false, false);
-      constexpr uint32_t IDESC_ACC = ptx::idesc_bf16_f32(128, NKV, true, true);     // A = (Q | dO)^T, B = (dS | P): both MN-major
       const uint64_t kd0 = ptx::smem_desc_sw128(sbase + OFF_K, 16, 1024);
       const uint64_t vd0 = ptx::smem_desc_sw128(sbase + OFF_V, 16, 1024);
-      const uint64_t pd0 = ptx::smem_desc_sw128(sbase + OFF_P, PS_BYTES, 1024);
-      const uint64_t sd0 = ptx::smem_desc_sw128(sbase + OFF_DS, PS_BYTES, 1024);
-      auto stage_tile = [&](int j) -> int {                  // waits for the stage; -1: end marker, -2: gave up
-        if (!wait_on(bar(QD_FULL + (j & 1)), (uint32_t)(j >> 1) & 1u)) return -2;
-        return *reinterpret_cast<volatile int*>(&misc->tile[j & 1]);
-      };
-      auto issue_sd = [&](int j) {
+      for (int j = 0; ok; ++j) {
         const int buf = j & 1;
+        ok = wait_on(bar(QD_FULL + buf), (uint32_t)(j >> 1) & 1u);
+        if (!ok || *reinterpret_cast<volatile int*>(&misc->tile[buf]) < 0) break;
+        // the warpgroup of this parity has read S / dP of step j-2
+        if (j >= 2) ok = wait_on(bar(PDS_FULL + buf), (uint32_t)((j >> 1) - 1) & 1u);
+        if (!ok) break;
         ptx::tc_fence_after();
         const uint64_t qd = ptx::smem_desc_sw128(sbase + OFF_Q + buf * 2 * Q_BYTES, 16, 1024);
         const uint64_t gd = ptx::smem_desc_sw128(sbase + OFF_Q + buf * 2 * Q_BYTES + Q_BYTES, 16, 1024);
+        if (is_s) {
 #pragma unroll
-        for (int k = 0; k < HD / 16; ++k) {
-          const uint64_t off_a = (uint64_t)(((k >> 2) * (Q_BYTES / 2) + (k & 3) * 32) >> 4);
-          const uint64_t off_b = (uint64_t)(((k >> 2) * (KV_TILE_BYTES / 2) + (k & 3) * 32) >> 4);
-          ptx::mma_bf16_ss(tmem + buf * NKV, qd + off_a, kd0 + off_b, IDESC_S, k > 0 ? 1u : 0u);
-        }
+          for (int k = 0; k < HD / 16; ++k) {
+            const uint64_t off_a = (uint64_t)(((k >> 2) * (Q_BYTES / 2) + (k & 3) * 32) >> 4);
+            const uint64_t off_b = (uint64_t)(((k >> 2) * (KV_TILE_BYTES / 2) + (k & 3) * 32) >> 4);
+            ptx::mma_bf16_ss(tmem + buf * NKV, qd + off_a, kd0 + off_b, IDESC_S, k > 0 ? 1u : 0u);
+          }
+        } else {
 #pragma unroll
-        for (int k = 0; k < HD / 16; ++k) {
-          const uint64_t off_a = (uint64_t)(((k >> 2) * (Q_BYTES / 2) + (k & 3) * 32) >> 4);
-          const uint64_t off_b = (uint64_t)(((k >> 2) * (KV_TILE_BYTES / 2) + (k & 3) * 32) >> 4);
-          ptx::mma_bf16_ss(tmem + COL_DP + buf * NKV, gd + off_a, vd0 + off_b, IDESC_S, k > 0 ? 1u : 0u);
+          for (int k = 0; k < HD / 16; ++k) {
+            const uint64_t off_a = (uint64_t)(((k >> 2) * (Q_BYTES / 2) + (k & 3) * 32) >> 4);
+            const uint64_t off_b = (uint64_t)(((k >> 2) * (KV_TILE_BYTES / 2) + (k & 3) * 32) >> 4);
+            ptx::mma_bf16_ss(tmem + COL_DP + buf * NKV, gd + off_a, vd0 + off_b, IDESC_S, k > 0 ? 1u : 0u);
+          }
         }
         ptx::mma_commit(bar(SD_FULL + buf));
-      };
-      int cur = ok ? stage_tile(0) : -2;
-      if (cur >= 0) issue_sd(0);
-      for (int j = 0; cur >= 0; ++j) {
-        const int nxt = stage_tile(j + 1);
-        if (nxt >= 0) issue_sd(j + 1);
-        if (nxt == -2) break;
-        if (!wait_on(bar(PDS_FULL), (uint32_t)j & 1u)) break;
-        ptx::tc_fence_after();
+      }
+    }
+    __syncwarp();
+  } else if (warp == W_ACC || warp == W_DK) {
+    // =========================== issuers of the accumulating products: dV^T += dO^T P (W_ACC), dK^T += Q^T dS (W_DK) ===========================
+    if (lane == 0) {
+      const bool is_v = warp == W_ACC;
+      constexpr uint32_t IDESC_ACC = ptx::idesc_bf16_f32(128, NKV, true, true);     // A = (Q | dO)^T, B = (dS | P): both MN-major
+      const uint64_t pd0 = ptx::smem_desc_sw128(sbase + OFF_P, PS_BYTES, 1024);
+      const uint64_t sd0 = ptx::smem_desc_sw128(sbase + OFF_DS, PS_BYTES, 1024);
+      bool ok = true;
+      for (int j = 0; ok; ++j) {
         const int buf = j & 1;
+        ok = wait_on(bar(QD_FULL + buf), (uint32_t)(j >> 1) & 1u);
+        if (!ok || *reinterpret_cast<volatile int*>(&misc->tile[buf]) < 0) break;
+        ok = wait_on(bar(PDS_FULL + buf), (uint32_t)(j >> 1) & 1u);
+        if (!ok) break;
+        ptx::tc_fence_after();
         // (Q | dO) tile [row][d] read as MN-major A: M = d (two blocks of 64, Q_BYTES / 2 apart), K = rows (16 rows = 2048 B)
         const uint64_t qmn = ptx::smem_desc_sw128(sbase + OFF_Q + buf * 2 * Q_BYTES, Q_BYTES / 2, 1024);
         const uint64_t gmn = ptx::smem_desc_sw128(sbase + OFF_Q + buf * 2 * Q_BYTES + Q_BYTES, Q_BYTES / 2, 1024);
+        if (is_v) {
 #pragma unroll
-        for (int k = 0; k < 128 / 16; ++k) {
-          const uint64_t adv = (uint64_t)((k * 16 * 128) >> 4);
-          ptx::mma_bf16_ss(tmem + COL_DV, gmn + adv, pd0 + adv, IDESC_ACC, (j > 0 || k > 0) ? 1u : 0u);
-        }
+          for (int k = 0; k < 128 / 16; ++k) {
+            const uint64_t adv = (uint64_t)((k * 16 * 128) >> 4);
+            ptx::mma_bf16_ss(tmem + COL_DV, gmn + adv, pd0 + adv, IDESC_ACC, (j > 0 || k > 0) ? 1u : 0u);
+          }
+        } else {
 #pragma unroll
-        for (int k = 0; k < 128 / 16; ++k) {
-          const uint64_t adv = (uint64_t)((k * 16 * 128) >> 4);
-          ptx::mma_bf16_ss(tmem + COL_DK, qmn + adv, sd0 + adv, IDESC_ACC, (j > 0 || k > 0) ? 1u : 0u);
+          for (int k = 0; k < 128 / 16; ++k) {
+            const uint64_t adv = (uint64_t)((k * 16 * 128) >> 4);
+            ptx::mma_bf16_ss(tmem + COL_DK, qmn + adv, sd0 + adv, IDESC_ACC, (j > 0 || k > 0) ? 1u : 0u);
+          }
         }
         ptx::mma_commit(bar(ACC_DONE + buf));
-        cur = nxt;
       }
     }
     __syncwarp();
   } else {
-    // =========================== P, dS: thread = tile row; epilogue: thread = d ===========================
-    const int m = tid;
-    const int t = m / g_q, hh = m % g_q;
-    const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+    // =========================== P, dS: thread = tile row, warpgroup = step parity; epilogue: thread = d ===========================
+    const int wg = warp >> 2;
+    const int m = (warp & 3) * 32 + lane;
+    const int t = m / g_q;
+    const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
     const float c1 = dm.sm_scale * LOG2E;
+    const int buf = wg;
     bool ok = true;
-    int n_done = 0;
-    for (int j = 0; ok; ++j) {
-      const int buf = j & 1;
+    for (int j = wg; ok; j += 2) {
       ok = wait_on(bar(QD_FULL + buf), (uint32_t)(j >> 1) & 1u);
       if (!ok) break;
       const int tile_idx = *reinterpret_cast<volatile int*>(&misc->tile[buf]);
       if (tile_idx < 0) break;
       const int i_row = tile_idx * TQ + t;
       const bool row_ok = i_row < dm.seq_q;
-      const long long srow = ((long long)b * dm.seq_q + min(i_row, dm.seq_q - 1)) * dm.h_q + r * g_q + hh;
-      const float lse2 = row_ok ? __ldg(a.lse2 + srow) : 0.f;
-      const float delta = row_ok ? __ldg(a.delta + srow) : 0.f;
+      const float lse2 = row_ok ? misc->lse2[buf][m] : 0.f;
+      const float delta = row_ok ? misc->delta[buf][m] : 0.f;
       const float bias = row_ok ? misc->bias[buf][t] : -INFINITY;
       const float off = bias * LOG2E - lse2;
       const int n_vis = i_row - k0 + 1;
@@ -679,49 +788,45 @@ attend_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           dd[half * 16 + (cc >> 1)] = *reinterpret_cast<uint32_t*>(&hd);
         }
       }
-      // the accumulating products of the step before have read P / dS
-      if (j >= 1) ok = wait_on(bar(ACC_DONE + ((j - 1) & 1)), (uint32_t)((j - 1) >> 1) & 1u);
+      // the accumulating products of the step before (the other warpgroup's) have read P / dS
+      if (j >= 1) ok = wait_on(bar(ACC_DONE + (buf ^ 1)), (uint32_t)((j - 1) >> 1) & 1u);
       if (!ok) break;
       // row m of the [128 rows][64 keys] tiles: 128 bytes, 16-byte pieces swizzled with the row (128-byte swizzle)
       uint8_t* prow = smem + OFF_P + m * 128;
-      uint8_t* srow_p = smem + OFF_DS + m * 128;
+      uint8_t* drow = smem + OFF_DS + m * 128;
 #pragma unroll
       for (int ch = 0; ch < 8; ++ch) {
         const int phys = (ch ^ (m & 7)) << 4;
         *reinterpret_cast<uint4*>(prow + phys) = make_uint4(pp[ch * 4], pp[ch * 4 + 1], pp[ch * 4 + 2], pp[ch * 4 + 3]);
-        *reinterpret_cast<uint4*>(srow_p + phys) = make_uint4(dd[ch * 4], dd[ch * 4 + 1], dd[ch * 4 + 2], dd[ch * 4 + 3]);
+        *reinterpret_cast<uint4*>(drow + phys) = make_uint4(dd[ch * 4], dd[ch * 4 + 1], dd[ch * 4 + 2], dd[ch * 4 + 3]);
       }
       ptx::fence_proxy_async_smem();
       ptx::tc_fence_before();
-      ptx::mbar_arrive(bar(PDS_FULL));
-      n_done = j + 1;
+      ptx::mbar_arrive(bar(PDS_FULL + buf));
     }
-    // epilogue: dV^T, dK^T [d = TMEM lane][key = column] -> dV, dK [batch][key][KV head][d]
+    // epilogue: dV^T, dK^T [d = TMEM lane][key = column] -> dV, dK [batch][key][KV head][d]; one warpgroup each
+    const int n_done = ok ? *reinterpret_cast<volatile int*>(&misc->total) : 0;
     if (ok && n_done > 0) ok = wait_on(bar(ACC_DONE + ((n_done - 1) & 1)), (uint32_t)((n_done - 1) >> 1) & 1u);
     if (ok) {
       ptx::tc_fence_after();
-      const int d = tid;
-      const float sc = dm.sm_scale;
+      const int d = m;
+      float* out = wg == 0 ? a.dV : a.dK;
+      const float mul = wg == 0 ? 1.f : dm.sm_scale;
 #pragma unroll 1
-      for (int which = 0; which < 2; ++which) {
-        float* out = which == 0 ? a.dV : a.dK;
-        const float mul = which == 0 ? 1.f : sc;
-#pragma unroll 1
-        for (int half = 0; half < 2; ++half) {
-          uint32_t v[32];
-          if (n_done > 0) {
-            DASH_TMEM_LD32(v, lane_addr + (which == 0 ? COL_DV : COL_DK) + half * 32);
-            ptx::tmem_wait_ld();
-          } else {
+      for (int half = 0; half < 2; ++half) {
+        uint32_t v[32];
+        if (n_done > 0) {
+          DASH_TMEM_LD32(v, lane_addr + (wg == 0 ? COL_DV : COL_DK) + half * 32);
+          ptx::tmem_wait_ld();
+        } else {
 #pragma unroll
-            for (int cc = 0; cc < 32; ++cc) v[cc] = 0u;
-          }
+          for (int cc = 0; cc < 32; ++cc) v[cc] = 0u;
+        }
 #pragma unroll
-          for (int cc = 0; cc < 32; ++cc) {
-            const int key = k0 + half * 32 + cc;
-            if (key < dm.seq_kv)
-              out[(((long long)b * dm.seq_kv + key) * dm.h_kv + r) * HD + d] = __uint_as_float(v[cc]) * mul;
-          }
+        for (int cc = 0; cc < 32; ++cc) {
+          const int key = k0 + half * 32 + cc;
+          if (key < dm.seq_kv)
+            out[(((long long)b * dm.seq_kv + key) * dm.h_kv + r) * HD + d] = __uint_as_float(v[cc]) * mul;
         }
       }
     }
@@ -729,7 +834,7 @@ attend_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   }
 
   __syncthreads();
-  if (warp == 5) {
+  if (warp == W_SD) {
     ptx::tc_fence_after();
     ptx::tmem_dealloc(tmem, TMEM_COLS);
   }
@@ -777,6 +882,16 @@ cudaError_t launch_attend_prefill_bwd_sm100(const Dims& dm, const void* Q, const
   a.n_slices = (dm.seq_kv + NKV - 1) / NKV;
   a.wait_limit = test_hooks().wait_limit_cycles;
   a.mask = mask; a.blk_bias = blk_bias; a.lse2 = lse2; a.delta = delta; a.prefix = prefix;
+  // the tile unions sit behind the prefix counts in the same scratch region
+  uint32_t* tile_union = reinterpret_cast<uint32_t*>(prefix + rows * dm.W);
+  a.tile_union = tile_union;
+  {
+    const long long warps = (long long)dm.batch * dm.h_kv * a.n_tiles;
+    e = launch_chained(tile_union_kernel, dim3((unsigned)((warps * 32 + 255) / 256)), dim3(256), 0, st, dm, a.TQ, a.n_tiles,
+                       mask, tile_union);
+    count_launch();
+    if (e != cudaSuccess) return e;
+  }
   a.dQ = (__nv_bfloat16*)dQ; a.dK = dK; a.dV = dV; a.dbias = dbias; a.sb = sb;
   CUtensorMap tq, tg, tk, tv;
   if (!make_map(&tq, Q, dm.seq_q, dm.h_q, dm.batch, dm.qs, dm.g_q, a.TQ)) return cudaErrorInvalidValue;

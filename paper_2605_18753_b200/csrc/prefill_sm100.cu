@@ -88,8 +88,9 @@ struct PrefillArgs {
   const uint32_t* mask;
   const float* blk_bias;
   __nv_bfloat16* O;          // may be null when only the row statistics are wanted
-  // Row statistics for the backward pass, [batch][token][query head] (null: not wanted): the log-sum-exp of the row's
-  // logits in the log2 domain, and delta = <O_row, dO_row> (dO: strides of O), both from the fp32 accumulator.
+  // Row statistics for the backward pass, [batch][KV head][tile][row of the tile (128)] (null: not wanted): the
+  // log-sum-exp of the row's logits in the log2 domain, and delta = <O_row, dO_row> (dO: strides of O), both from the
+  // fp32 accumulator.
   float* lse2;
   float* delta;
   const __nv_bfloat16* dO;
@@ -98,7 +99,11 @@ struct PrefillArgs {
 
 // SHORT: the tile has fewer than 128 live rows (chunks shorter than 128 / g_q tokens); full tiles compile without
 // any of the padding-row handling.
-template <int HD, int CPS, bool SHORT>
+// STATS: the kernel also leaves the row statistics the backward pass starts from (a.lse2, a.delta).  delta = <O, dO> feeds
+// the gradient of the routing, which amplifies its error, so in this mode P enters the P V product as two bf16 terms
+// (P = hi + lo, the remainder in the second half of the step's S columns): O, and with it delta, is then accurate to
+// fp32 class instead of bf16 class.
+template <int HD, int CPS, bool SHORT, bool STATS = false>
 __global__ void __launch_bounds__(PF_THREADS, 2)
 attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                             const __grid_constant__ CUtensorMap tmV, PrefillArgs a) {
@@ -441,6 +446,13 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
           // A = P from tensor memory: 16 bf16 per K step = 8 packed columns
           ptx::mma_bf16_ts(tmem + 2 * NKV, p_tmem + k * 8, bd, IDESC_PV, (j > 0 || k > 0) ? 1u : 0u);
         }
+        if constexpr (STATS) {
+#pragma unroll
+          for (int k = 0; k < NKV / 16; ++k) {
+            const uint64_t bd = vd + (uint64_t)((k * 16 * 128) >> 4);
+            ptx::mma_bf16_ts(tmem + 2 * NKV, p_tmem + 32 + k * 8, bd, IDESC_PV, 1u);      // the remainders
+          }
+        }
         ptx::mma_commit(bar(PV_DONE + buf));
       }
     }
@@ -544,6 +556,7 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
       }
       l *= corr;
       uint32_t packed[32];
+      [[maybe_unused]] uint32_t packed_lo[STATS ? 32 : 1];
       if (selected) {
         // scale-and-shift and the row sum on packed pairs (one instruction per two scores); a slot that is not
         // routed has offset -inf, so its probabilities come out as exactly 0
@@ -560,12 +573,21 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
           lsum[(c >> 1) & 3] = __fadd2_rn(lsum[(c >> 1) & 3], pp);
           __nv_bfloat162 h = __floats2bfloat162_rn(pp.x, pp.y);
           packed[c >> 1] = *reinterpret_cast<uint32_t*>(&h);
+          if constexpr (STATS) {
+            const float2 hf = __bfloat1622float2(h);
+            __nv_bfloat162 lo = __floats2bfloat162_rn(pp.x - hf.x, pp.y - hf.y);
+            packed_lo[c >> 1] = *reinterpret_cast<uint32_t*>(&lo);
+          }
         }
         const float2 ls = __fadd2_rn(__fadd2_rn(lsum[0], lsum[1]), __fadd2_rn(lsum[2], lsum[3]));
         l += ls.x + ls.y;
       } else {
 #pragma unroll
         for (int c = 0; c < 32; ++c) packed[c] = 0u;
+        if constexpr (STATS) {
+#pragma unroll
+          for (int c = 0; c < 32; ++c) packed_lo[c] = 0u;
+        }
       }
 
       // O is stable once the previous step's PV has completed
@@ -587,6 +609,7 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
       }
       // P row -> the first 32 columns of this step's S buffer (two bf16 per column)
       DASH_TMEM_ST32(lane_addr + buf * NKV, packed);
+      if constexpr (STATS) DASH_TMEM_ST32(lane_addr + buf * NKV + 32, packed_lo);
       ptx::tmem_wait_st();
       ptx::tc_fence_before();
       ptx::mbar_arrive(bar(P_FULL + (j & 1)));
@@ -606,7 +629,7 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
         uint32_t o[32];
         DASH_TMEM_LD32(o, lane_addr + 2 * NKV + q * 32);
         ptx::tmem_wait_ld();
-        if (a.lse2 && row_out) {
+        if (STATS && row_out) {
           const __nv_bfloat16* gp = a.dO + o_off + q * 32;
 #pragma unroll
           for (int c = 0; c < 32; c += 8) {
@@ -634,8 +657,8 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
           }
         }
       }
-      if (a.lse2 && row_out) {
-        const long long row = ((long long)b * dm.seq_q + i_row) * dm.h_q + r * g_q + hh;
+      if (STATS && row_out) {
+        const long long row = (((long long)b * dm.h_kv + r) * a.n_tiles + tile) * 128 + m;
         a.lse2[row] = m_used + log2f(l);
         a.delta[row] = dot * inv;
       }
@@ -714,6 +737,18 @@ cudaError_t launch_attend_prefill_sm100(const Dims& dm, const void* Q, const voi
   else { if (short_tile) DASH_PF(HDV, 4, true) else DASH_PF(HDV, 4, false) }
   const int cps = NKV / box_kv;
   const bool short_tile = a.TQ * dm.g_q < 128;      // only with chunks below 64 tokens
+  if (lse2) {
+    // statistics mode: the shapes the tensor-core backward takes (head_dim 128, chunks of 64 / 128, full tiles)
+    if (dm.d != 128 || cps != 1 || short_tile || !delta || !dO) return cudaErrorInvalidValue;
+    static std::atomic<unsigned long long> configured{0};
+    if (cudaError_t e = allow_dynamic_smem(attend_prefill_sm100_kernel<128, 1, false, true>, PfLayout<128, 1>::SMEM, configured);
+        e != cudaSuccess)
+      return e;
+    le = launch_chained(attend_prefill_sm100_kernel<128, 1, false, true>, dim3((unsigned)blocks), dim3(PF_THREADS),
+                        PfLayout<128, 1>::SMEM, st, tq, tk, tv, a);
+    count_launch();
+    return le;
+  }
   if (dm.d == 128) { DASH_PF_HD(128) } else { DASH_PF_HD(64) }
 #undef DASH_PF_HD
 #undef DASH_PF

@@ -1,8 +1,9 @@
 """GPU parity of the tensor-core Stage-2 backward (dash_attn_bwd_attend_prefill_tc): against the float64 backward oracle
 on the oracle's own routing lists (every row, every gradient), and against the CUDA-core backward kernel on a larger
-case with the library's routing.  P and dS enter the dK / dV products rounded to bf16, dQ is stored as bf16, and delta
-= <O, dO> comes from the forward kernel's accumulator, whose P V product also takes P in bf16: all four gradients carry
-the bf16 tolerance (1e-2 of the largest reference value)."""
+case with the library's routing.  P and dS enter the dK / dV products rounded to bf16 and dQ is stored as bf16: those
+three carry the bf16 tolerance (1e-2 of the largest reference value).  dbias is formed from fp32 values (delta comes
+from a statistics pass that feeds P to its P V product as two bf16 terms), because the routing's backward amplifies its
+error: 2e-3 of the largest reference value, and the whole chain through the routing is checked as well."""
 import numpy as np
 import pytest
 import torch
@@ -11,7 +12,7 @@ from oracle import dash_oracle_bwd as bwd
 from paper_2605_18753_b200 import binding as B
 from paper_2605_18753_b200 import synth
 from tests import helpers as H
-from tests.test_gpu_backward import _close
+from tests.test_gpu_backward import _close, whole_chain_case
 from tests.test_gpu_parity import _wl
 
 pytestmark = pytest.mark.gpu
@@ -61,7 +62,7 @@ def test_tensor_core_stage2_backward_matches_oracle(kw, L):
         off = B.dash_attn_list_offset(p, b, r, i)
         if want.size:
             err = float(np.abs(db[off:off + want.size] - want).max())
-            assert err <= 1e-2 * scale, f"dbias row {(b, r, i)}: {err:.3e} vs scale {scale:.3g}"
+            assert err <= 2e-3 * scale, f"dbias row {(b, r, i)}: {err:.3e} vs scale {scale:.3g}"
             n_entries += want.size
     if w.seq > 4 * w.block:
         assert n_entries > 0
@@ -107,3 +108,13 @@ def test_tensor_core_backward_refuses_other_shapes():
         B.dash_attn_bwd_attend_prefill_tc(p, Q, K, V, Q, rt["mask"], rt["blk_bias"], torch.empty_like(Q), dK,
                                           torch.empty_like(dK), torch.empty_like(rt["blk_bias"]), bws)
     assert ei.value.code == -2
+
+
+@pytest.mark.parametrize("kw,qbar_mode,L", [
+    (dict(seq=400, h_q=8, h_kv=2, head_dim=128, block=64, sigma=1.0, seed=14), "none", 0),
+    (dict(seq=520, h_q=4, h_kv=2, head_dim=128, block=128, sigma=2.0, seed=41), "head", 0),
+    (dict(seq=420, h_q=4, h_kv=2, head_dim=128, block=64, seed=17, sigma=2.0), "chunk", 1),
+])
+def test_whole_backward_chain_with_tensor_core_stage2(kw, qbar_mode, L):
+    """The whole gradient chain of the method with Stage 2 on tensor cores (its dbias feeds the routing backward)."""
+    whole_chain_case(kw, qbar_mode, L, tensor_cores=True)
