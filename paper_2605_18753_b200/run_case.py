@@ -2,6 +2,7 @@
 
     python -m paper_2605_18753_b200.run_case prefill_8k --iters 5
     python -m paper_2605_18753_b200.run_case decode_128k --batch 4 --iters 3      # 2 GiB of KV cache instead of 8
+    python -m paper_2605_18753_b200.run_case prefill_8k --backward --iters 2       # Stage-2 backward on tensor cores
 
 A quick way to see the path work on a given shape (overrides: --batch, --seq, --block, --alpha, --head-dim, --local-blocks), and a small,
 self-terminating command to put under a profiler.  Inputs are the seeded synthetic tensors of `synth`."""
@@ -25,6 +26,7 @@ def main() -> None:
     ap.add_argument("--alpha", type=float)
     ap.add_argument("--head-dim", type=int, dest="head_dim")
     ap.add_argument("--local-blocks", type=int, default=0, help="window chunks before the own chunk (0 = none)")
+    ap.add_argument("--backward", action="store_true", help="prefill only: time the tensor-core Stage-2 backward instead")
     args = ap.parse_args()
     over = {k: getattr(args, k) for k in ("batch", "seq", "block", "alpha", "head_dim") if getattr(args, k) is not None}
     w = synth.workload(args.workload, **over)
@@ -39,6 +41,19 @@ def main() -> None:
                                  local_blocks=args.local_blocks)
         ws = B.alloc_workspace(p)
         step = lambda: B.dash_attn_fwd_prefill(p, Q, K, V, O, ws)
+        if args.backward:
+            # routing from one forward pass, then the gradients of Stage 2 for a random dO
+            rt, kbar = B.alloc_routing(p), B.alloc_kbar(p)
+            B.dash_attn_block_summaries(p, K, kbar)
+            B.dash_attn_select(p, Q, kbar, rt["mask"], rt["count"], rt["blk_idx"], rt["blk_bias"], ws)
+            dO = torch.randn(Q.shape, device=dev, dtype=torch.float32).to(Q.dtype)
+            dQ = torch.empty_like(Q)
+            dK = torch.empty(w.batch, w.seq, w.h_kv, w.head_dim, device=dev)
+            dV = torch.empty_like(dK)
+            dbias = torch.empty_like(rt["blk_bias"])
+            ws = B.alloc_bwd_workspace(p)        # its status word is the one checked below
+            O = dQ
+            step = lambda: B.dash_attn_bwd_attend_prefill_tc(p, Q, K, V, dO, rt["mask"], rt["blk_bias"], dQ, dK, dV, dbias, ws)
     else:
         di = synth.make_decode_inputs(w, dev)
         q, Kc, Vc, kl = di["Q"], di["K"], di["V"], di["kv_len"]
@@ -62,7 +77,7 @@ def main() -> None:
         if it > 0:
             times.append(a.elapsed_time(b))
     status = B.dash_attn_last_status(ws)
-    print(f"{w.name} {over or ''}: forward ms {['%.4f' % t for t in times]}  status {B.STATUS.get(status, status)}  "
+    print(f"{w.name} {over or ''}: {'backward' if args.backward else 'forward'} ms {['%.4f' % t for t in times]}  status {B.STATUS.get(status, status)}  "
           f"output finite {bool(torch.isfinite(O.float()).all())}")
     if status != 0:
         raise SystemExit(1)
