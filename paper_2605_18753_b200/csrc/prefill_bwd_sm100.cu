@@ -502,7 +502,7 @@ attend_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       ptx::mbar_init(bar(QD_FULL + s), 2);     // the loader's arrival (with the byte count) and the bias warp's
       ptx::mbar_init(bar(SD_FULL + s), 2);
       ptx::mbar_init(bar(ACC_DONE + s), 2);
-      ptx::mbar_init(bar(PDS_FULL + s), 128);
+      ptx::mbar_init(bar(PDS_FULL + s), 256);
     }
     ptx::fence_barrier_init();
   }
@@ -743,16 +743,17 @@ attend_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     }
     __syncwarp();
   } else {
-    // =========================== P, dS: thread = tile row, warpgroup = step parity; epilogue: thread = d ===========================
+    // =========================== P, dS: thread = tile row, warpgroup = half of the keys; epilogue: thread = d ===========================
     const int wg = warp >> 2;
     const int m = (warp & 3) * 32 + lane;
     const int t = m / g_q;
     const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
     const float c1 = dm.sm_scale * LOG2E;
-    const int buf = wg;
     bool ok = true;
-    for (int j = wg; ok; j += 2) {
-      ok = wait_on(bar(QD_FULL + buf), (uint32_t)(j >> 1) & 1u);
+    for (int j = 0; ok; ++j) {
+      const int buf = j & 1;
+      const uint32_t ph = (uint32_t)(j >> 1) & 1u;
+      ok = wait_on(bar(QD_FULL + buf), ph);
       if (!ok) break;
       const int tile_idx = *reinterpret_cast<volatile int*>(&misc->tile[buf]);
       if (tile_idx < 0) break;
@@ -762,41 +763,41 @@ attend_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       const float delta = row_ok ? misc->delta[buf][m] : 0.f;
       const float bias = row_ok ? misc->bias[buf][t] : -INFINITY;
       const float off = bias * LOG2E - lse2;
-      const int n_vis = i_row - k0 + 1;
-      ok = wait_on(bar(SD_FULL + buf), (uint32_t)(j >> 1) & 1u);
+      const int n_vis = i_row - k0 + 1 - wg * 32;            // visible columns of this warpgroup's half
+      ok = wait_on(bar(SD_FULL + buf), ph);
       if (!ok) break;
       ptx::tc_fence_after();
-      uint32_t pp[32], dd[32];                             // the row's 64 P and 64 dS values as bf16 pairs
-#pragma unroll
-      for (int half = 0; half < 2; ++half) {
+      uint32_t pp[16], dd[16];                               // the row's 32 P and 32 dS values of this half as bf16 pairs
+      {
         uint32_t sv[32], gv[32];
-        DASH_TMEM_LD32(sv, lane_addr + buf * NKV + half * 32);
-        DASH_TMEM_LD32(gv, lane_addr + COL_DP + buf * NKV + half * 32);
+        DASH_TMEM_LD32(sv, lane_addr + buf * NKV + wg * 32);
+        DASH_TMEM_LD32(gv, lane_addr + COL_DP + buf * NKV + wg * 32);
         ptx::tmem_wait_ld();
 #pragma unroll
         for (int cc = 0; cc < 32; cc += 2) {
           float p[2], ds[2];
 #pragma unroll
           for (int u = 0; u < 2; ++u) {
-            const bool vis = half * 32 + cc + u < n_vis;
+            const bool vis = cc + u < n_vis;
             p[u] = vis ? exp2f(fmaf(__uint_as_float(sv[cc + u]), c1, off)) : 0.f;
             ds[u] = p[u] * (__uint_as_float(gv[cc + u]) - delta);
           }
           __nv_bfloat162 hp = __floats2bfloat162_rn(p[0], p[1]);
           __nv_bfloat162 hd = __floats2bfloat162_rn(ds[0], ds[1]);
-          pp[half * 16 + (cc >> 1)] = *reinterpret_cast<uint32_t*>(&hp);
-          dd[half * 16 + (cc >> 1)] = *reinterpret_cast<uint32_t*>(&hd);
+          pp[cc >> 1] = *reinterpret_cast<uint32_t*>(&hp);
+          dd[cc >> 1] = *reinterpret_cast<uint32_t*>(&hd);
         }
       }
-      // the accumulating products of the step before (the other warpgroup's) have read P / dS
+      // the accumulating products of the step before have read P / dS
       if (j >= 1) ok = wait_on(bar(ACC_DONE + (buf ^ 1)), (uint32_t)((j - 1) >> 1) & 1u);
       if (!ok) break;
-      // row m of the [128 rows][64 keys] tiles: 128 bytes, 16-byte pieces swizzled with the row (128-byte swizzle)
+      // row m of the [128 rows][64 keys] tiles: 128 bytes, 16-byte pieces swizzled with the row (128-byte swizzle); this
+      // warpgroup's keys are pieces 4 wg .. 4 wg + 3
       uint8_t* prow = smem + OFF_P + m * 128;
       uint8_t* drow = smem + OFF_DS + m * 128;
 #pragma unroll
-      for (int ch = 0; ch < 8; ++ch) {
-        const int phys = (ch ^ (m & 7)) << 4;
+      for (int ch = 0; ch < 4; ++ch) {
+        const int phys = ((wg * 4 + ch) ^ (m & 7)) << 4;
         *reinterpret_cast<uint4*>(prow + phys) = make_uint4(pp[ch * 4], pp[ch * 4 + 1], pp[ch * 4 + 2], pp[ch * 4 + 3]);
         *reinterpret_cast<uint4*>(drow + phys) = make_uint4(dd[ch * 4], dd[ch * 4 + 1], dd[ch * 4 + 2], dd[ch * 4 + 3]);
       }
