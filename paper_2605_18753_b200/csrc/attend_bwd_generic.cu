@@ -157,11 +157,20 @@ attend_prefill_bwd_generic_kernel(Dims dm, const T* __restrict__ Q, const T* __r
           const T* kp = kbase + (long long)(t0 + u) * dm.ks[1] + lane * VPL;
           float* dkp = dkbase + (long long)(t0 + u) * gtok + lane * VPL;
           float* dvp = dvbase + (long long)(t0 + u) * gtok + lane * VPL;
+          float ak[VPL], av[VPL];
 #pragma unroll
           for (int v = 0; v < VPL; ++v) {
             dq[v] = fmaf(du, to_f32<T>(kp[v]), dq[v]);
-            atomicAdd(dkp + v, du * qs[warp][lane * VPL + v]);          // qs already carries 1/sqrt(d)
-            atomicAdd(dvp + v, pu * gs[warp][lane * VPL + v]);
+            ak[v] = du * qs[warp][lane * VPL + v];          // qs already carries 1/sqrt(d)
+            av[v] = pu * gs[warp][lane * VPL + v];
+          }
+          // one vector reduction per lane and tensor: the L2 atomic units count requests, not bytes
+          if constexpr (VPL == 4) {
+            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dkp), "f"(ak[0]), "f"(ak[1]), "f"(ak[2]), "f"(ak[3]) : "memory");
+            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dvp), "f"(av[0]), "f"(av[1]), "f"(av[2]), "f"(av[3]) : "memory");
+          } else {
+            asm volatile("red.global.add.v2.f32 [%0], {%1, %2};" ::"l"(dkp), "f"(ak[0]), "f"(ak[1]) : "memory");
+            asm volatile("red.global.add.v2.f32 [%0], {%1, %2};" ::"l"(dvp), "f"(av[0]), "f"(av[1]) : "memory");
           }
         }
         __syncwarp();

@@ -13,7 +13,8 @@
 //   w_c = mean_h p_hc                        =>  dp_hc = dw_c / g_q
 //   p_h = entmax(z_h), z_hc = gamma <q_h, kbar_c>/sqrt(d)   =>  dz_h by the Jacobian above
 //   dq_h = gamma/sqrt(d) sum_c dz_hc kbar_c (written, fp32);   dkbar_c += gamma/sqrt(d) sum_h dz_hc q_h (atomic, fp32)
-// Only routed chunks are touched (two sweeps over the row's list; the chunk logits are recomputed from Q and Kbar).
+// Only routed chunks are touched (two sweeps over the row's list, four entries at a time; the chunk logits are
+// recomputed from Q and Kbar).
 //
 // summaries_bwd_kernel: one warp per (batch, KV head, chunk): Eq. 3, kbar_c = sum_t a_t k_t with
 // a = softmax(<qbar, k_t>/sqrt(d)) (a_t = 1/B without a summary query): dk_t += a_t dkbar_c + ds_t qbar/sqrt(d),
@@ -24,13 +25,46 @@ namespace dash {
 
 constexpr int RB_WARPS = 4;
 
-template <typename T, int D>
+// Sums V values that every lane holds across the warp with the halving exchange (V - 1 + log2(32 / V) ... shuffles
+// instead of 5 V): value v ends up complete in lane v * (32 / V) as x[0]; then every value is broadcast, so that all
+// lanes hold all V sums (another V shuffles).  V must be a power of two <= 32.
+template <int V>
+__device__ __forceinline__ void warp_sum_all(float (&x)[V], int lane) {
+  float y[V];
+#pragma unroll
+  for (int k = 0; k < V; ++k) y[k] = x[k];
+#pragma unroll
+  for (int width = 16, live = V; width >= 1; width >>= 1) {
+    if (live > 1) {
+      const bool upper = (lane & width) != 0;
+      const int half = live / 2;
+#pragma unroll
+      for (int k = 0; k < V / 2; ++k) {
+        if (k < half) {
+          const float mine = upper ? y[k + half] : y[k];
+          const float give = upper ? y[k] : y[k + half];
+          y[k] = mine + __shfl_xor_sync(0xffffffffu, give, width);
+        }
+      }
+      live = half;
+    } else {
+      y[0] += __shfl_xor_sync(0xffffffffu, y[0], width);
+    }
+  }
+  // the lane bits were consumed from the top: value v sits in the lane whose top log2(V) bits spell v
+#pragma unroll
+  for (int v = 0; v < V; ++v) x[v] = __shfl_sync(0xffffffffu, y[0], v * (32 / V));
+}
+
+// G (heads per KV head) is a template parameter so that the per-head arrays live in registers; the row's routed chunks
+// are taken NB at a time: their summary rows are fetched together and the NB * G dot products are reduced together.
+template <typename T, int D, int G>
 __global__ void __launch_bounds__(RB_WARPS * 32)
 route_bwd_kernel(Dims dm, const T* __restrict__ Q, const float* __restrict__ Kbar, const int* __restrict__ count,
                  const int* __restrict__ blk_idx, const float* __restrict__ tau, const float* __restrict__ dbias,
                  float* __restrict__ dQr, float* __restrict__ dKbar) {
   constexpr int VPL = D / 32;
-  constexpr int MAXG = 16;
+  constexpr int NB = G <= 8 ? 4 : 2;           // entries per batch: NB * G <= 32 values per reduction
   const int lane = threadIdx.x & 31;
   const long long gw = (long long)blockIdx.x * RB_WARPS + (threadIdx.x >> 5);
   const long long total = (long long)dm.batch * dm.h_kv * dm.seq_q;
@@ -38,21 +72,22 @@ route_bwd_kernel(Dims dm, const T* __restrict__ Q, const float* __restrict__ Kba
   const int i = (int)(gw % dm.seq_q);
   const int r = (int)((gw / dm.seq_q) % dm.h_kv);
   const int b = (int)(gw / ((long long)dm.seq_q * dm.h_kv));
-  const int G = dm.g_q;
   const long long grp = (long long)b * dm.h_kv + r;
   // fp32 gradient of Q from the routing: [batch, seq_q, h_q, d], every row written (zeros where nothing is routed)
   float* dq_out = dQr + (((long long)b * dm.seq_q + i) * dm.h_q + (long long)r * G) * D + lane * VPL;
   const int c_own = i / dm.B;
   const int n_local = min(dm.local_blocks, c_own);              // window chunks close the list and carry no gradient
   const int n_routed = count[grp * dm.seq_q + i] - n_local;
-  float q[MAXG][VPL], dq[MAXG][VPL];
+  float q[G][VPL], dq[G][VPL];
+#pragma unroll
   for (int h = 0; h < G; ++h)
 #pragma unroll
     for (int v = 0; v < VPL; ++v) dq[h][v] = 0.f;
   if (n_routed > 0) {
     const long long loff = grp * dm.list_rows + list_row_offset(dm, i);
     const float* kb = Kbar + grp * dm.T_s * D + lane * VPL;
-    float th[MAXG];
+    float th[G];
+#pragma unroll
     for (int h = 0; h < G; ++h) {
       const T* qp = Q + (long long)b * dm.qs[0] + (long long)i * dm.qs[1] + (long long)(r * G + h) * dm.qs[2] + lane * VPL;
 #pragma unroll
@@ -64,65 +99,103 @@ route_bwd_kernel(Dims dm, const T* __restrict__ Q, const float* __restrict__ Kba
     dmean = warp_sum(dmean) / (float)n_routed;
     const float e = dm.e;
     const int e_int = dm.e_int;
-    // margins of one routed chunk for all heads of the group: m_h = x_scale <q_h, kbar_c> - tau_h (clamped at 0)
-    auto margins = [&](int c, float* m) {
-      float kv[VPL];
+    // One batch: entries k0 .. k0 + NB - 1 (those beyond the list repeat the last one and are ignored by the caller).
+    // kv: their summary rows; m: the margins m_h = x_scale <q_h, kbar_c> - tau_h (clamped at 0) of every entry and head;
+    // dw: the gradient w.r.t. the entry's group weight.
+    auto batch = [&](int k0, int (&c)[NB], float (&kv)[NB][VPL], float (&m)[NB][G], float (&dw)[NB]) {
+      float db[NB];
 #pragma unroll
-      for (int v = 0; v < VPL; ++v) kv[v] = kb[(long long)c * D + v];
-      for (int h = 0; h < G; ++h) {
-        float s = 0.f;
+      for (int u = 0; u < NB; ++u) {
+        const int k = min(k0 + u, n_routed - 1);
+        c[u] = blk_idx[loff + k];
+        db[u] = dbias[loff + k];
+      }
 #pragma unroll
-        for (int v = 0; v < VPL; ++v) s = fmaf(q[h][v], kv[v], s);
-        m[h] = fmaxf(warp_sum(s) * dm.x_scale - th[h], 0.f);
+      for (int u = 0; u < NB; ++u)
+#pragma unroll
+        for (int v = 0; v < VPL; ++v) kv[u][v] = kb[(long long)c[u] * D + v];
+      float part[NB * G];
+#pragma unroll
+      for (int u = 0; u < NB; ++u)
+#pragma unroll
+        for (int h = 0; h < G; ++h) {
+          float s = 0.f;
+#pragma unroll
+          for (int v = 0; v < VPL; ++v) s = fmaf(q[h][v], kv[u][v], s);
+          part[u * G + h] = s;
+        }
+      warp_sum_all<NB * G>(part, lane);
+#pragma unroll
+      for (int u = 0; u < NB; ++u) {
+        float w = 0.f;
+#pragma unroll
+        for (int h = 0; h < G; ++h) {
+          m[u][h] = fmaxf(part[u * G + h] * dm.x_scale - th[h], 0.f);
+          w += pow_e(m[u][h], e_int, e);
+        }
+        w /= (float)G;
+        dw[u] = w > 0.f ? (db[u] - dmean) * dm.inv_sigma / w : 0.f;
       }
     };
     // sweep 1: per head A_h = sum_c s_hc dw_c / g_q and S_h = sum_c s_hc
-    float A[MAXG], S[MAXG];
+    float A[G], S[G];
+#pragma unroll
     for (int h = 0; h < G; ++h) A[h] = S[h] = 0.f;
-    for (int k = 0; k < n_routed; ++k) {
-      const int c = blk_idx[loff + k];
-      float m[MAXG];
-      margins(c, m);
-      float w = 0.f;
-      for (int h = 0; h < G; ++h) w += pow_e(m[h], e_int, e);
-      w /= (float)G;
-      const float dw = w > 0.f ? (dbias[loff + k] - dmean) * dm.inv_sigma / w : 0.f;
-      for (int h = 0; h < G; ++h) {
-        const float s = pow_em1(m[h], e_int, e);
-        A[h] += s * dw / (float)G;
-        S[h] += s;
+    for (int k0 = 0; k0 < n_routed; k0 += NB) {
+      int c[NB];
+      float kv[NB][VPL], m[NB][G], dw[NB];
+      batch(k0, c, kv, m, dw);
+#pragma unroll
+      for (int u = 0; u < NB; ++u) {
+        if (k0 + u < n_routed) {
+#pragma unroll
+          for (int h = 0; h < G; ++h) {
+            const float s = pow_em1(m[u][h], e_int, e);
+            A[h] += s * dw[u] / (float)G;
+            S[h] += s;
+          }
+        }
       }
     }
     // sweep 2: dz_hc, then dq_h and dkbar_c
     const float zscale = dm.x_scale / (1.f / e);       // gamma / sqrt(d) = x_scale / (alpha - 1)
-    for (int k = 0; k < n_routed; ++k) {
-      const int c = blk_idx[loff + k];
-      float m[MAXG];
-      margins(c, m);
-      float w = 0.f;
-      for (int h = 0; h < G; ++h) w += pow_e(m[h], e_int, e);
-      w /= (float)G;
-      const float dw = w > 0.f ? (dbias[loff + k] - dmean) * dm.inv_sigma / w : 0.f;
-      float kv[VPL], dkb[VPL];
+    for (int k0 = 0; k0 < n_routed; k0 += NB) {
+      int c[NB];
+      float kv[NB][VPL], m[NB][G], dw[NB];
+      batch(k0, c, kv, m, dw);
 #pragma unroll
-      for (int v = 0; v < VPL; ++v) { kv[v] = kb[(long long)c * D + v]; dkb[v] = 0.f; }
-      for (int h = 0; h < G; ++h) {
-        const float s = pow_em1(m[h], e_int, e);
-        const float dz = S[h] > 0.f ? s * (dw / (float)G - A[h] / S[h]) : 0.f;
+      for (int u = 0; u < NB; ++u) {
+        if (k0 + u < n_routed) {
+          float dkb[VPL];
 #pragma unroll
-        for (int v = 0; v < VPL; ++v) {
-          dq[h][v] = fmaf(dz, kv[v], dq[h][v]);
-          dkb[v] = fmaf(dz, q[h][v], dkb[v]);
+          for (int v = 0; v < VPL; ++v) dkb[v] = 0.f;
+#pragma unroll
+          for (int h = 0; h < G; ++h) {
+            const float s = pow_em1(m[u][h], e_int, e);
+            const float dz = S[h] > 0.f ? s * (dw[u] / (float)G - A[h] / S[h]) : 0.f;
+#pragma unroll
+            for (int v = 0; v < VPL; ++v) {
+              dq[h][v] = fmaf(dz, kv[u][v], dq[h][v]);
+              dkb[v] = fmaf(dz, q[h][v], dkb[v]);
+            }
+          }
+          float* dst = dKbar + (grp * dm.T_s + c[u]) * D + lane * VPL;
+          // one vector reduction per lane (16 or 8 bytes): a quarter / half of the requests of scalar atomic adds, and
+          // the requests, not the bytes, are what the L2 atomic units count
+          if constexpr (VPL == 4)
+            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "f"(dkb[0] * zscale), "f"(dkb[1] * zscale),
+                         "f"(dkb[2] * zscale), "f"(dkb[3] * zscale) : "memory");
+          else
+            asm volatile("red.global.add.v2.f32 [%0], {%1, %2};" ::"l"(dst), "f"(dkb[0] * zscale), "f"(dkb[1] * zscale) : "memory");
         }
       }
-      float* dst = dKbar + (grp * dm.T_s + c) * D + lane * VPL;
-#pragma unroll
-      for (int v = 0; v < VPL; ++v) atomicAdd(dst + v, dkb[v] * zscale);
     }
+#pragma unroll
     for (int h = 0; h < G; ++h)
 #pragma unroll
       for (int v = 0; v < VPL; ++v) dq[h][v] *= zscale;
   }
+#pragma unroll
   for (int h = 0; h < G; ++h)
 #pragma unroll
     for (int v = 0; v < VPL; ++v) dq_out[(long long)h * D + v] = dq[h][v];
@@ -215,13 +288,23 @@ cudaError_t launch_route_bwd(const Dims& dm, const void* Q, const float* Kbar, c
   }
   const long long total = (long long)dm.batch * dm.h_kv * dm.seq_q;
   const unsigned grid = (unsigned)((total + RB_WARPS - 1) / RB_WARPS);
-#define DASH_RB(T, D) \
-  route_bwd_kernel<T, D><<<grid, RB_WARPS * 32, 0, st>>>(dm, (const T*)Q, Kbar, count, blk_idx, tau, dbias, dQr, dKbar)
-  if (dm.dtype == DASH_BF16) {
-    if (dm.d == 128) DASH_RB(__nv_bfloat16, 128); else DASH_RB(__nv_bfloat16, 64);
-  } else {
-    if (dm.d == 128) DASH_RB(float, 128); else DASH_RB(float, 64);
+#define DASH_RB(T, D, GV) \
+  route_bwd_kernel<T, D, GV><<<grid, RB_WARPS * 32, 0, st>>>(dm, (const T*)Q, Kbar, count, blk_idx, tau, dbias, dQr, dKbar)
+#define DASH_RB_G(T, D)                   \
+  switch (dm.g_q) {                       \
+    case 1: DASH_RB(T, D, 1); break;      \
+    case 2: DASH_RB(T, D, 2); break;      \
+    case 4: DASH_RB(T, D, 4); break;      \
+    case 8: DASH_RB(T, D, 8); break;      \
+    case 16: DASH_RB(T, D, 16); break;    \
+    default: return cudaErrorInvalidValue; \
   }
+  if (dm.dtype == DASH_BF16) {
+    if (dm.d == 128) { DASH_RB_G(__nv_bfloat16, 128) } else { DASH_RB_G(__nv_bfloat16, 64) }
+  } else {
+    if (dm.d == 128) { DASH_RB_G(float, 128) } else { DASH_RB_G(float, 64) }
+  }
+#undef DASH_RB_G
 #undef DASH_RB
   count_launch();
   return cudaGetLastError();
