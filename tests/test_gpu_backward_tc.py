@@ -37,6 +37,7 @@ def _run_tc(p, Q, K, V, dO, mask, bias, w):
     (dict(seq=333, h_q=8, h_kv=1, head_dim=128, block=64, alpha=2.0, seed=22), 0),        # g_q = 8, ragged length
     (dict(seq=520, h_q=8, h_kv=2, head_dim=128, block=64, batch=2, seed=23, gamma=2.0), 0),
     (dict(seq=420, h_q=4, h_kv=1, head_dim=128, block=64, seed=24), 1),                   # local window
+    (dict(seq=300, h_q=16, h_kv=1, head_dim=128, block=64, seed=27, gamma=2.0), 0),       # g_q = 16: tiles of 8 tokens
     (dict(seq=64, h_q=4, h_kv=2, head_dim=128, block=64, seed=25), 0),                    # one chunk: nothing routed
     (dict(seq=5, h_q=4, h_kv=2, head_dim=128, block=64, seed=26), 0),
 ])
@@ -118,3 +119,42 @@ def test_tensor_core_backward_refuses_other_shapes():
 def test_whole_backward_chain_with_tensor_core_stage2(kw, qbar_mode, L):
     """The whole gradient chain of the method with Stage 2 on tensor cores (its dbias feeds the routing backward)."""
     whole_chain_case(kw, qbar_mode, L, tensor_cores=True)
+
+
+def test_tensor_core_backward_gives_up_cleanly_when_a_wait_runs_out():
+    """The statistics pass is the forward kernel: with the test hooks its first K tile never arrives and its waits give
+    up after 2e5 cycles.  The status word of the backward scratch then holds DASH_ERR_TIMEOUT, the kernels behind it
+    (launched on the same status word) retire at their first wait, nothing hangs or faults, and after a reset the same
+    scratch serves a correct backward pass."""
+    import time
+    w = _wl(seq=900, h_q=8, h_kv=2, head_dim=128, block=64, seed=33)
+    inp = synth.make_prefill_inputs(w, DEV)
+    Q, K, V = inp["Q"], inp["K"], inp["V"]
+    dO = torch.randn(Q.shape, device=DEV, generator=torch.Generator(DEV).manual_seed(133)).to(Q.dtype)
+    p = B.params_for_prefill(Q, K, V, dO, block=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma)
+    kbar = B.alloc_kbar(p)
+    B.dash_attn_block_summaries(p, K, kbar)
+    ws = B.alloc_workspace(p)
+    rt = B.alloc_routing(p)
+    B.dash_attn_select(p, Q, kbar, rt["mask"], rt["count"], rt["blk_idx"], rt["blk_bias"], ws)
+    bws = B.alloc_bwd_workspace(p)
+    outs = lambda: (torch.full_like(Q, float("nan")), torch.empty(w.batch, w.seq, w.h_kv, w.head_dim, device=DEV),
+                    torch.empty(w.batch, w.seq, w.h_kv, w.head_dim, device=DEV), torch.empty_like(rt["blk_bias"]))
+    good = outs()
+    B.dash_attn_bwd_attend_prefill_tc(p, Q, K, V, dO, rt["mask"], rt["blk_bias"], *good, bws)
+    assert B.dash_attn_last_status(bws) == 0
+    try:
+        B.dash_attn_test_hooks(wait_limit_cycles=200_000, skip_own_k_load=1)
+        t0 = time.time()
+        B.dash_attn_bwd_attend_prefill_tc(p, Q, K, V, dO, rt["mask"], rt["blk_bias"], *outs(), bws)
+        assert B.dash_attn_last_status(bws) == -7          # DASH_ERR_TIMEOUT
+        assert time.time() - t0 < 5.0
+    finally:
+        B.dash_attn_test_hooks()
+    torch.cuda.synchronize()
+    B.dash_attn_reset_status(bws)
+    again = outs()
+    B.dash_attn_bwd_attend_prefill_tc(p, Q, K, V, dO, rt["mask"], rt["blk_bias"], *again, bws)
+    assert B.dash_attn_last_status(bws) == 0
+    for g, a_ in zip(good, again):
+        assert torch.equal(g, a_)
