@@ -158,3 +158,38 @@ def test_tensor_core_backward_gives_up_cleanly_when_a_wait_runs_out():
     assert B.dash_attn_last_status(bws) == 0
     for g, a_ in zip(good, again):
         assert torch.equal(g, a_)
+
+
+def test_tensor_core_backward_on_random_shapes_against_the_cuda_core_kernel():
+    """Seeded random shapes inside the tensor-core path's domain (lengths that end inside a tile or a chunk, every group
+    size, both chunk sizes, windows, batches), library routing, CUDA-core kernel as the reference (itself checked
+    against the oracle above and in test_gpu_backward.py)."""
+    rng = np.random.default_rng(20261125)
+    for draw in range(14):
+        g_q = int(rng.choice([2, 4, 8, 16]))
+        h_kv = int(rng.choice([1, 2, 3]))
+        kw = dict(seq=int(rng.integers(65, 1400)), h_q=g_q * h_kv, h_kv=h_kv, head_dim=128, block=int(rng.choice([64, 128])),
+                  batch=int(rng.choice([1, 2])), alpha=float(rng.choice([1.25, 1.5, 2.0])), gamma=float(rng.choice([1.0, 2.0, 4.0])),
+                  sigma=float(rng.choice([1.0, 10.0])), seed=100 + draw)
+        L = int(rng.choice([0, 0, 1]))
+        w = _wl(**kw)
+        inp = synth.make_prefill_inputs(w, DEV)
+        Q, K, V = inp["Q"], inp["K"], inp["V"]
+        dO = torch.randn(Q.shape, device=DEV, generator=torch.Generator(DEV).manual_seed(500 + draw)).to(Q.dtype)
+        p = B.params_for_prefill(Q, K, V, dO, block=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma, local_blocks=L)
+        kbar = B.alloc_kbar(p)
+        B.dash_attn_block_summaries(p, K, kbar)
+        ws = B.alloc_workspace(p)
+        rt = B.alloc_routing(p)
+        B.dash_attn_select(p, Q, kbar, rt["mask"], rt["count"], rt["blk_idx"], rt["blk_bias"], ws)
+        assert B.dash_attn_last_status(ws) == 0
+        dQ0 = torch.empty_like(Q)
+        dK0 = torch.empty(w.batch, w.seq, w.h_kv, w.head_dim, device=DEV)
+        dV0 = torch.empty_like(dK0)
+        db0 = torch.empty_like(rt["blk_bias"])
+        B.dash_attn_bwd_attend_prefill(p, Q, K, V, dO, rt["mask"], rt["blk_bias"], dQ0, dK0, dV0, db0)
+        dQ, dK, dV, db = _run_tc(p, Q, K, V, dO, rt["mask"], rt["blk_bias"], w)
+        what = f"draw {draw} {kw} L={L}"
+        for got, want, name, rel in ((dQ, dQ0, "dQ", 1e-2), (dK, dK0, "dK", 1e-2), (dV, dV0, "dV", 1e-2), (db, db0, "dbias", 3e-3)):
+            if want.numel():
+                _close(got.float().cpu().double().numpy(), want.float().cpu().double().numpy(), rel, f"{name} ({what})")
