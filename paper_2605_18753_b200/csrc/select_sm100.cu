@@ -39,7 +39,11 @@ constexpr int HD_MAX = 128;          // the shared-memory layout is the one of h
 // memory like those of the blocks of a cluster.  (Three, not four: 14 warps leave each thread 128 registers, which
 // the streaming loops fill; 18 warps would leave 96 and spill.)
 __host__ __device__ constexpr int split_of(int nst) { return nst == 1 ? 1 : 3; }
-__host__ __device__ constexpr int sel_threads(int nst) { return (4 * split_of(nst) + 2) * 32; }   // solver warps, producer, MMA issuer
+// MMA issuers: one for the short-row kernel (a single stage of summaries); two for long rows (even and odd 64-chunk
+// blocks), fed by a three-stage ring of summary tiles: 192 products through one thread, each stage waiting a full L2
+// round trip behind the product that freed it, take longer than the tensor pipe needs.
+__host__ __device__ constexpr int issuers_of(int nst) { return nst == 1 ? 1 : 2; }
+__host__ __device__ constexpr int sel_threads(int nst) { return (4 * split_of(nst) + 1 + issuers_of(nst)) * 32; }   // solver warps, producer, issuers
 constexpr uint32_t Q_BYTES = 128 * HD_MAX * 2;        // 32 KiB
 constexpr uint32_t PLANE_BYTES = SC * HD_MAX * 2;     // 16 KiB per plane per stage
 constexpr uint32_t STAGE_BYTES = 3 * PLANE_BYTES;     // hi, mid, lo
@@ -50,7 +54,7 @@ struct MiscS {
   uint32_t tmem_base;
   int abort_flag;
 };
-enum BarS { Q_FULL = 0, X_FULL = 1, KB_FULL = 2, KB_EMPTY = 4, XBAR = 6 };   // XBAR: [warp 0..3][parity]
+enum BarS { Q_FULL = 0, X_FULL = 1, KB_FULL = 2, KB_EMPTY = 5, XBAR = 8 };   // KB_*: up to three stages; XBAR: [warp 0..3][parity]
 constexpr int CLUSTER_COLS = 512;      // candidates one block of a cluster holds in tensor memory
 constexpr int MAX_CS = 4;              // widest cluster
 
@@ -101,6 +105,7 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   extern __shared__ __align__(1024) uint8_t smem[];
   MiscS* misc = reinterpret_cast<MiscS*>(smem + SP::OFF_MISC);
   constexpr int SPLIT = split_of(NST), NSOLVE = 4 * SPLIT, W_PROD = NSOLVE, W_MMA = NSOLVE + 1;
+  constexpr int N_ISSUE = issuers_of(NST);      // issuing warps W_MMA .. W_MMA + N_ISSUE - 1; the first owns the TMEM allocation
   constexpr int SEL_TC_THREADS = sel_threads(NST);
   const Dims& dm = a.dm;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -134,8 +139,8 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       misc->abort_flag = 1;
     }
     ptx::mbar_init(bar(Q_FULL), 1);
-    ptx::mbar_init(bar(X_FULL), 1);
-    for (int s = 0; s < 2; ++s) {
+    ptx::mbar_init(bar(X_FULL), N_ISSUE);
+    for (int s = 0; s < NST; ++s) {
       ptx::mbar_init(bar(KB_FULL + s), 1);
       ptx::mbar_init(bar(KB_EMPTY + s), 1);
     }
@@ -195,8 +200,11 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           for (int k = 0; k < 200000 && !ptx::mbar_try_wait(bar(KB_FULL + s), 0) && !ptx::mbar_try_wait(bar(KB_FULL + s), 1); ++k) {}
       }
     }
-  } else if (warp == W_MMA) {
-    // ---------------- MMA issuer: X[:, cb*64 .. +64) = Q Kbar_hi^T + Q Kbar_mid^T + Q Kbar_lo^T
+  } else if (warp >= W_MMA) {
+    // ---------------- MMA issuers: X[:, cb*64 .. +64) = Q Kbar_hi^T + Q Kbar_mid^T + Q Kbar_lo^T; with two issuers,
+    // issuer k takes the blocks cb = k, k + 2, ...  Every issuer waits for EVERY block's tile, also those it leaves to
+    // the other one: a parity wait only tells a phase from its neighbour, so a thread must see a barrier's phases in
+    // order (an issuer that skipped a phase could take the stage's previous fill for the one it waits for).
     if (lane == 0 && n_loc > 0) {
       constexpr uint32_t IDESC = ptx::idesc_bf16_f32(128, SC, false, false);
       bool ok = ptx::mbar_wait(bar(Q_FULL), 0, abort_flag);
@@ -204,6 +212,7 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         const int s = cb % NST;
         ok = ptx::mbar_wait(bar(KB_FULL + s), (cb / NST) & 1, abort_flag);
         if (!ok) break;
+        if (cb % N_ISSUE != warp - W_MMA) continue;
         ptx::tc_fence_after();
         // descriptors differ only in the start-address field (16-byte units, no carry into the next field): built once
         // per stage, then one add per MMA keeps the issuing thread's instruction stream short
@@ -786,18 +795,18 @@ cudaError_t launch_select_sm100(const Dims& dm, int token_limit, const void* Q, 
   // widest bands first: they are the long-running ones
   if (t3 > t2) {
     a.tile_base = t2; a.n_tiles = t3 - t2; a.tmem_cols = 512;
-    if ((e = launch_band_g<2, 4>(dm, tq, tkb, a, (long long)a.n_tiles * groups, st)) != cudaSuccess) return e;
+    if ((e = launch_band_g<3, 4>(dm, tq, tkb, a, (long long)a.n_tiles * groups, st)) != cudaSuccess) return e;
   }
   if (t2 > t1) {
     a.tile_base = t1; a.n_tiles = t2 - t1; a.tmem_cols = 512;
-    if ((e = launch_band_g<2, 2>(dm, tq, tkb, a, (long long)a.n_tiles * groups, st)) != cudaSuccess) return e;
+    if ((e = launch_band_g<3, 2>(dm, tq, tkb, a, (long long)a.n_tiles * groups, st)) != cudaSuccess) return e;
   }
   // one block per tile: rows of 257 .. 512 candidates take the whole tensor memory of an SM (one block per SM, three
   // solver threads per row); shorter ones leave room for two blocks per SM with the row in one thread
   const int t0 = tiles_up_to(256);
   if (t1 > t0) {
     a.tile_base = t0; a.n_tiles = t1 - t0; a.tmem_cols = 512;
-    if ((e = launch_band_g<2, 1>(dm, tq, tkb, a, (long long)a.n_tiles * groups, st)) != cudaSuccess) return e;
+    if ((e = launch_band_g<3, 1>(dm, tq, tkb, a, (long long)a.n_tiles * groups, st)) != cudaSuccess) return e;
   }
   {
     a.tile_base = 0; a.n_tiles = t0;
