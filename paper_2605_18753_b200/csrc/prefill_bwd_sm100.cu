@@ -4,9 +4,10 @@
 // With P = softmax of the row's logits l_j = <q,k_j>/sqrt(d) + bias_c(j) over its selected tokens, dP = dO V^T,
 // delta = <O, dO> per row and dS = P o (dP - delta):
 //     dQ = dS K / sqrt(d),   dK = dS^T Q / sqrt(d),   dV = P^T dO,   dbias_c = sum of dS over the chunk's tokens.
-// Three launches behind the forward kernel run in "statistics" mode (it leaves the log-sum-exp and delta of every row):
+// Four launches behind the forward kernel run in "statistics" mode (it leaves the log-sum-exp and delta of every row):
 //   mask_prefix_kernel      per row, the number of routed chunks in the mask words before each word (so that a row's
 //                           list entry for a chunk can be found from one word of its mask);
+//   tile_union_kernel       per query tile, the OR of its rows' mask words (which chunks any of its rows attends);
 //   attend_bwd_dq_kernel    query-tile stationary, the forward kernel's walk over the union of the tile's routed
 //                           chunks: S = Q K^T and dP = dO V^T into tensor memory, dS (bf16) back into tensor memory,
 //                           dQ += dS K accumulated in tensor memory; dbias from the row sums of dS;
@@ -449,9 +450,10 @@ attend_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
 // ===================================================================================================================
 namespace dkv {
 
-// Two warpgroups form P and dS (even / odd steps, one S / dP buffer each); producer; one issuer for the score products
-// (S, dP) and one for the accumulating products (dV^T, dK^T): 32 MMAs per step are too many for one issuing thread.
-// W_PROD loads the tiles, W_META the per-token biases of each step; W_SD issues S, W_DP dP, W_ACC dV^T, W_DK dK^T
+// Two warpgroups form P and dS, each for half of the slice's keys on every step (no row maximum is needed, so the halves
+// are independent and a step's P / dS stretch takes half as long); one issuing thread per product: 32 MMAs per step
+// are too many for one.  W_PROD loads the tiles, W_META looks up the per-token biases of each step; W_SD issues S,
+// W_DP dP, W_ACC dV^T, W_DK dK^T.
 constexpr int W_PROD = 8, W_SD = 9, W_ACC = 10, W_DP = 11, W_DK = 12, W_META = 13;
 constexpr int THREADS = 448;
 constexpr uint32_t TMEM_COLS = 512;     // S0 S1 [0,128) dP0 dP1 [128,256) dV^T [256,320) dK^T [320,384)
@@ -462,7 +464,7 @@ struct Misc {
   unsigned long long bar[N_BARS];
   uint32_t tmem_base;
   int abort_flag;
-  int total;                            // number of steps, written with the end markers
+  int total;                            // number of steps, written with the end marker
   int tile[2];                          // query tile of the stage's step (-1: no more steps)
   float bias[2][MAX_TQ];                // per token of the tile: the chunk's bias (-inf: the token does not attend it)
   alignas(16) float lse2[2][128];       // the tile's row statistics (bulk copies)
@@ -649,17 +651,14 @@ attend_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       uw = uw_n;
     }
     if (!loader && ok && n_pend > 0) flush();
-    // two end markers: one for each step parity (each warpgroup meets one)
+    // the end marker (every role visits every step, so one is enough): both producers arrive on its stage
     if (ok && loader) {
       if (lane == 0) misc->total = j;
       __syncwarp();
       load_step(-1);
-      if (ok) load_step(-1);
-    } else if (ok) {
-      for (int e = 0; e < 2 && stage_free(); ++e) {
-        if (lane == 0) ptx::mbar_arrive(bar(QD_FULL + (j & 1)));
-        ++j;
-      }
+    } else if (ok && stage_free()) {
+      if (lane == 0) ptx::mbar_arrive(bar(QD_FULL + (j & 1)));
+      ++j;
     }
     if (!ok && lane == 0 && loader) {
       // a wait ran out: let the copies already issued land (bounded) before the block retires
