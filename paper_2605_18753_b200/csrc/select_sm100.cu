@@ -48,13 +48,17 @@ constexpr uint32_t Q_BYTES = 128 * HD_MAX * 2;        // 32 KiB
 constexpr uint32_t PLANE_BYTES = SC * HD_MAX * 2;     // 16 KiB per plane per stage
 constexpr uint32_t STAGE_BYTES = 3 * PLANE_BYTES;     // hi, mid, lo
 constexpr int MAX_NEWTON = 64, MAX_NEWTON_GENERIC = 400;
+constexpr int CLUSTER_COLS_FOR_BARRIERS = 512;     // = CLUSTER_COLS below: columns of one block's score tile
 
 struct MiscS {
-  unsigned long long bar[16];
+  unsigned long long bar[24];
   uint32_t tmem_base;
   int abort_flag;
 };
-enum BarS { Q_FULL = 0, X_FULL = 1, KB_FULL = 2, KB_EMPTY = 5, XBAR = 8 };   // KB_*: up to three stages; XBAR: [warp 0..3][parity]
+// KB_*: up to three stages; XBAR: [warp 0..3][parity]; CB_DONE: one per 64-chunk block of the score tile (each completes
+// exactly once, so a late waiter cannot mistake one completion for another)
+enum BarS { Q_FULL = 0, X_FULL = 1, KB_FULL = 2, KB_EMPTY = 5, XBAR = 8, CB_DONE = 16 };
+constexpr int MAX_CB = CLUSTER_COLS_FOR_BARRIERS / 64;
 constexpr int CLUSTER_COLS = 512;      // candidates one block of a cluster holds in tensor memory
 constexpr int MAX_CS = 4;              // widest cluster
 
@@ -63,7 +67,7 @@ template <int NST> struct SmemPlan {
   static constexpr uint32_t OFF_KB = Q_BYTES;
   static constexpr uint32_t OFF_XCH = OFF_KB + NST * STAGE_BYTES;
   // exchange slots [parity][participant][row] of (float, float); participants = cluster blocks x threads per row
-  static constexpr uint32_t XCH_BYTES = NST == 1 ? 128u : 2u * MAX_CS * split_of(NST) * 128u * 8u;
+  static constexpr uint32_t XCH_BYTES = NST == 1 ? 128u : 2u * MAX_CS * split_of(NST) * 128u * 16u;
   static constexpr uint32_t OFF_MISC = OFF_XCH + XCH_BYTES;
   static constexpr uint32_t TOTAL = OFF_MISC + sizeof(MiscS);
 };
@@ -145,6 +149,7 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       ptx::mbar_init(bar(KB_EMPTY + s), 1);
     }
     for (int s = 0; s < 8; ++s) ptx::mbar_init(bar(XBAR + s), CS * SPLIT * 32);
+    for (int s = 0; s < MAX_CB; ++s) ptx::mbar_init(bar(CB_DONE + s), 1);
     ptx::fence_barrier_init();
   }
   if (warp == W_MMA) {
@@ -228,6 +233,7 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           }
         }
         ptx::mma_commit(bar(KB_EMPTY + s));
+        ptx::mma_commit(bar(CB_DONE + cb));
       }
       if (ok) ptx::mma_commit(bar(X_FULL));
     }
@@ -249,7 +255,10 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const int k_hi = SPLIT == 1 ? n_chunks : min(k_lo + per_part, n_chunks);
     bool ok = true;
     float tau = 0.f;
-    if (n_loc > 0) {
+    // rows that are held in registers wait for the whole score tile here; streamed rows start on the tile's first
+    // 64-chunk blocks while the later ones are still being produced (see solve_streaming)
+    const bool row_in_regs = CS == 1 && SPLIT == 1 && n_chunks <= 4;
+    if (n_loc > 0 && (row_in_regs || n_cand == 0)) {
       ok = ptx::mbar_wait(bar(X_FULL), 0, abort_flag);
       ptx::tc_fence_after();
     }
@@ -263,37 +272,37 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     // what a round leaves behind: sums of both values over all participants (added in rank order, so every
     // participant holds the same bits and takes the same branches), the maximum of the first, and the sum of the
     // first over the participants ranked below this one
-    float x_sum_a = 0.f, x_sum_b = 0.f, x_max_a = 0.f, x_below_a = 0.f;
-    auto exchange = [&](float va, float vb) -> bool {
+    float x_sum_a = 0.f, x_sum_b = 0.f, x_sum_c = 0.f, x_max_a = 0.f, x_below_a = 0.f;
+    auto exchange = [&](float va, float vb, float vc = 0.f) -> bool {
       if constexpr (NP == 1) {
-        x_sum_a = x_max_a = va; x_sum_b = vb; x_below_a = 0.f;
+        x_sum_a = x_max_a = va; x_sum_b = vb; x_sum_c = vc; x_below_a = 0.f;
         return true;
       } else {
         const int par = xround & 1;
-        float2* xbuf = reinterpret_cast<float2*>(smem + SP::OFF_XCH);          // [2][NP][128]
-        float2* mine = &xbuf[(par * NP + my_rank) * 128 + m];
+        float4* xbuf = reinterpret_cast<float4*>(smem + SP::OFF_XCH);          // [2][NP][128]
+        float4* mine = &xbuf[(par * NP + my_rank) * 128 + m];
         const uint32_t mybar = bar(XBAR + q4 * 2 + par);
         if constexpr (CS == 1) {
-          *mine = make_float2(va, vb);
+          *mine = make_float4(va, vb, vc, 0.f);
           ptx::mbar_arrive(mybar);
           if (!ptx::mbar_wait(mybar, (xround >> 1) & 1, abort_flag)) return false;
         } else {
           const uint32_t slot = ptx::smem_u32(mine);
 #pragma unroll
-          for (int pr = 0; pr < CS; ++pr) ptx::st_cluster_f32x2(ptx::map_to_rank(slot, pr), va, vb);
+          for (int pr = 0; pr < CS; ++pr) ptx::st_cluster_f32x4(ptx::map_to_rank(slot, pr), va, vb, vc, 0.f);
 #pragma unroll
           for (int pr = 0; pr < CS; ++pr) ptx::mbar_arrive_cluster(ptx::map_to_rank(mybar, pr));
           if (!ptx::mbar_wait_cluster(mybar, (xround >> 1) & 1, abort_flag)) return false;
         }
-        float sa = 0.f, sb = 0.f, mxa = -INFINITY, below = 0.f;
+        float sa = 0.f, sb = 0.f, sc = 0.f, mxa = -INFINITY, below = 0.f;
 #pragma unroll
         for (int pr = 0; pr < NP; ++pr) {
-          const float2 v = xbuf[(par * NP + pr) * 128 + m];
-          sa += v.x; sb += v.y;
+          const float4 v = xbuf[(par * NP + pr) * 128 + m];
+          sa += v.x; sb += v.y; sc += v.z;
           mxa = fmaxf(mxa, v.x);
           if (pr < my_rank) below += v.x;
         }
-        x_sum_a = sa; x_sum_b = sb; x_max_a = mxa; x_below_a = below;
+        x_sum_a = sa; x_sum_b = sb; x_sum_c = sc; x_max_a = mxa; x_below_a = below;
         ++xround;
         return true;
       }
@@ -437,27 +446,42 @@ select_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           for (int c = 0; c < 32; ++c) v[c] = c < lim ? v[c] : 0xff800000u;
         }
       };
+      // First pass, while the tile is still being produced: a 32-column chunk is read as soon as its 64-chunk block is
+      // complete (CB_DONE), and gives the row's maximum and the raw moments sum x, sum x^2 in one sweep; the moments
+      // about the maximum, which the start value needs, follow from them after the one exchange.
       float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-      stream([&](uint32_t (&v)[32], int k) {
-        cut_tail(v, k);
-#pragma unroll
-        for (int c = 0; c < 32; ++c) mx4[c & 3] = fmaxf(mx4[c & 3], __uint_as_float(v[c]));
-      });
-      float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * xs;
-      ok = exchange(mx, 0.f);
-      mx = x_max_a;
       float s1v[4] = {0.f, 0.f, 0.f, 0.f}, s2v[4] = {0.f, 0.f, 0.f, 0.f};
-      stream([&](uint32_t (&v)[32], int k) {
+      for (int k = k_lo; k < k_hi && ok; ++k) {
+        ok = ptx::mbar_wait(bar(CB_DONE + (k >> 1)), 0, abort_flag);
+        if (!ok) break;
+        ptx::tc_fence_after();
+        uint32_t v[32];
+        DASH_TMEM_LD32(v, lane_addr + k * 32);
+        ptx::tmem_wait_ld();
         const int lim = n_loc - k * 32;
 #pragma unroll
         for (int c = 0; c < 32; ++c) {
-          const float y = c < lim ? fmaf(__uint_as_float(v[c]), xs, -mx) : 0.f;
-          s1v[c & 3] += y;
-          s2v[c & 3] = fmaf(y, y, s2v[c & 3]);
+          if (c < lim) {
+            const float y = __uint_as_float(v[c]) * xs;
+            mx4[c & 3] = fmaxf(mx4[c & 3], y);
+            s1v[c & 3] += y;
+            s2v[c & 3] = fmaf(y, y, s2v[c & 3]);
+          }
         }
-      });
-      ok = ok && exchange((s1v[0] + s1v[1]) + (s1v[2] + s1v[3]), (s2v[0] + s2v[1]) + (s2v[2] + s2v[3]));
-      tau = start_tau(mx, xsum_a(), xsum_b());
+      }
+      // the later passes read all of this thread's columns at will: the whole tile must be there
+      if (ok && n_loc > 0) {
+        ok = ptx::mbar_wait(bar(X_FULL), 0, abort_flag);
+        ptx::tc_fence_after();
+      }
+      float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+      ok = ok && exchange(mx, (s1v[0] + s1v[1]) + (s1v[2] + s1v[3]), (s2v[0] + s2v[1]) + (s2v[2] + s2v[3]));
+      mx = x_max_a;
+      {
+        // sum (x - mx) = S1 - n mx,  sum (x - mx)^2 = S2 - 2 mx S1 + n mx^2  (only the start value depends on them)
+        const float n = (float)n_cand, S1 = x_sum_b, S2 = x_sum_c;
+        tau = start_tau(mx, S1 - n * mx, fmaxf(fmaf(n * mx, mx, fmaf(-2.f * mx, S1, S2)), 0.f));
+      }
       bool done = false;
       for (int it = 0; it < max_it && ok; ++it) {
         float f[4] = {0.f, 0.f, 0.f, 0.f}, g[4] = {0.f, 0.f, 0.f, 0.f};
