@@ -193,3 +193,47 @@ def test_tensor_core_backward_on_random_shapes_against_the_cuda_core_kernel():
         for got, want, name, rel in ((dQ, dQ0, "dQ", 1e-2), (dK, dK0, "dK", 1e-2), (dV, dV0, "dV", 1e-2), (db, db0, "dbias", 3e-3)):
             if want.numel():
                 _close(got.float().cpu().double().numpy(), want.float().cpu().double().numpy(), rel, f"{name} ({what})")
+
+
+def test_tensor_core_backward_at_the_full_8k_workload():
+    """The workload bench.py times (prefill_8k, library routing): dQ rows and dbias entries of sampled rows against the
+    float64 oracle's row-wise Stage-2 backward on the GPU's own lists, and all four gradients against the CUDA-core
+    kernel."""
+    w = synth.workload("prefill_8k")
+    inp = synth.make_prefill_inputs(w, DEV)
+    Q, K, V = inp["Q"], inp["K"], inp["V"]
+    dO = torch.randn(Q.shape, device=DEV, generator=torch.Generator(DEV).manual_seed(777)).to(Q.dtype)
+    p = B.params_for_prefill(Q, K, V, dO, block=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma)
+    kbar = B.alloc_kbar(p)
+    B.dash_attn_block_summaries(p, K, kbar)
+    ws = B.alloc_workspace(p)
+    rt = B.alloc_routing(p)
+    B.dash_attn_select(p, Q, kbar, rt["mask"], rt["count"], rt["blk_idx"], rt["blk_bias"], ws)
+    dQ, dK, dV, db = _run_tc(p, Q, K, V, dO, rt["mask"], rt["blk_bias"], w)
+    dQ0 = torch.empty_like(Q)
+    dK0 = torch.empty(w.batch, w.seq, w.h_kv, w.head_dim, device=DEV)
+    dV0 = torch.empty_like(dK0)
+    db0 = torch.empty_like(rt["blk_bias"])
+    B.dash_attn_bwd_attend_prefill(p, Q, K, V, dO, rt["mask"], rt["blk_bias"], dQ0, dK0, dV0, db0)
+    for got, want, name, rel in ((dQ, dQ0, "dQ", 1e-2), (dK, dK0, "dK", 1e-2), (dV, dV0, "dV", 1e-2), (db, db0, "dbias", 3e-3)):
+        _close(got.float().cpu().double().numpy(), want.float().cpu().double().numpy(), rel, f"{name} vs the CUDA-core kernel")
+    # sampled rows against the oracle
+    Qn, Kn, Vn, Gn = (H.to_np64(t) for t in (Q, K, V, dO))
+    cnt = rt["count"].cpu().numpy(); idx = rt["blk_idx"].cpu().numpy(); bias = rt["blk_bias"].cpu().numpy().astype(np.float64)
+    dbn = db.cpu().double().numpy()
+    dQn = dQ.float().cpu().double().numpy()
+    g_q = w.h_q // w.h_kv
+    rng = np.random.default_rng(5)
+    scale_q = float(np.abs(dQn).max())
+    for _ in range(48):
+        r = int(rng.integers(0, w.h_kv)); i = int(rng.integers(0, w.seq))
+        off = B.dash_attn_list_offset(p, 0, r, i)
+        c = int(cnt[0, r, i])
+        dq, tok, dk, dv, dbr = bwd.attend_row_vjp(Qn[0, i, r * g_q:(r + 1) * g_q], Kn[0, :, r], Vn[0, :, r], w.block,
+                                                  idx[off:off + c], bias[off:off + c], (i // w.block) * w.block, i + 1,
+                                                  Gn[0, i, r * g_q:(r + 1) * g_q])
+        err = float(np.abs(dQn[0, i, r * g_q:(r + 1) * g_q] - dq).max())
+        assert err <= 1e-2 * max(1.0, scale_q), f"dQ row {(r, i)}: {err:.3e}"
+        if c:
+            errb = float(np.abs(dbn[off:off + c] - dbr).max())
+            assert errb <= 2e-3 * max(1.0, float(np.abs(dbr).max())), f"dbias row {(r, i)}: {errb:.3e}"
