@@ -598,6 +598,9 @@ def all_config_measurements(B, synth, dev, peaks, flush, sel_tflop_8k=None) -> d
     guarded("backward_2k", lambda: measure_backward(B, synth, synth.workload("prefill_8k", seq=2048), dev, flush))
     guarded("backward_8k_tc", lambda: measure_backward(B, synth, synth.workload("prefill_8k"), dev, flush, iters=5,
                                                        tensor_cores=True, fwd_sel_tflop=sel_tflop_8k))
+    guarded("backward_64k_s90_tc", lambda: measure_backward(
+        B, synth, synth.workload("prefill_64k_s90"), dev, flush, iters=3, tensor_cores=True,
+        fwd_sel_tflop=out.get("prefill_64k_s90", {}).get("selected_tflop")))
     return out
 
 
