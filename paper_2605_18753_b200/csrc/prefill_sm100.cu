@@ -555,9 +555,39 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
         moved = true;
       }
       l *= corr;
-      uint32_t packed[32];
-      [[maybe_unused]] uint32_t packed_lo[STATS ? 32 : 1];
-      if (selected) {
+      [[maybe_unused]] uint32_t packed[STATS ? 1 : 32];
+      if constexpr (STATS) {
+        // P = hi + lo as two bf16 terms, 32 scores at a time, stored as they are formed (the scores are all in registers
+        // already): hi into the first 32 columns of the step's S buffer, lo into the second 32
+        float2 lsum[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+        const float2 c1v = make_float2(c1, c1);
+        const float2 offv = make_float2(b2s[0] - m_used, b2s[0] - m_used);
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          uint32_t hi16[16], lo16[16];
+          if (selected) {
+#pragma unroll
+            for (int c = 0; c < 32; c += 2) {
+              const int cc = half * 32 + c;
+              const float2 t = __ffma2_rn(make_float2(__uint_as_float(sreg[cc]), __uint_as_float(sreg[cc + 1])), c1v, offv);
+              const float2 pp = make_float2(exp2f(t.x), exp2f(t.y));
+              lsum[(c >> 1) & 1] = __fadd2_rn(lsum[(c >> 1) & 1], pp);
+              __nv_bfloat162 h = __floats2bfloat162_rn(pp.x, pp.y);
+              const float2 hf = __bfloat1622float2(h);
+              __nv_bfloat162 lo = __floats2bfloat162_rn(pp.x - hf.x, pp.y - hf.y);
+              hi16[c >> 1] = *reinterpret_cast<uint32_t*>(&h);
+              lo16[c >> 1] = *reinterpret_cast<uint32_t*>(&lo);
+            }
+          } else {
+#pragma unroll
+            for (int c = 0; c < 16; ++c) hi16[c] = lo16[c] = 0u;
+          }
+          ptx::tmem_st_n<16>(lane_addr + buf * NKV + half * 16, hi16);
+          ptx::tmem_st_n<16>(lane_addr + buf * NKV + 32 + half * 16, lo16);
+        }
+        const float2 ls = __fadd2_rn(lsum[0], lsum[1]);
+        l += ls.x + ls.y;
+      } else if (selected) {
         // scale-and-shift and the row sum on packed pairs (one instruction per two scores); a slot that is not
         // routed has offset -inf, so its probabilities come out as exactly 0
         const float2 c1v = make_float2(c1, c1);
@@ -573,21 +603,12 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
           lsum[(c >> 1) & 3] = __fadd2_rn(lsum[(c >> 1) & 3], pp);
           __nv_bfloat162 h = __floats2bfloat162_rn(pp.x, pp.y);
           packed[c >> 1] = *reinterpret_cast<uint32_t*>(&h);
-          if constexpr (STATS) {
-            const float2 hf = __bfloat1622float2(h);
-            __nv_bfloat162 lo = __floats2bfloat162_rn(pp.x - hf.x, pp.y - hf.y);
-            packed_lo[c >> 1] = *reinterpret_cast<uint32_t*>(&lo);
-          }
         }
         const float2 ls = __fadd2_rn(__fadd2_rn(lsum[0], lsum[1]), __fadd2_rn(lsum[2], lsum[3]));
         l += ls.x + ls.y;
       } else {
 #pragma unroll
         for (int c = 0; c < 32; ++c) packed[c] = 0u;
-        if constexpr (STATS) {
-#pragma unroll
-          for (int c = 0; c < 32; ++c) packed_lo[c] = 0u;
-        }
       }
 
       // O is stable once the previous step's PV has completed
@@ -608,8 +629,7 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
         }
       }
       // P row -> the first 32 columns of this step's S buffer (two bf16 per column)
-      DASH_TMEM_ST32(lane_addr + buf * NKV, packed);
-      if constexpr (STATS) DASH_TMEM_ST32(lane_addr + buf * NKV + 32, packed_lo);
+      if constexpr (!STATS) DASH_TMEM_ST32(lane_addr + buf * NKV, packed);
       ptx::tmem_wait_st();
       ptx::tc_fence_before();
       ptx::mbar_arrive(bar(P_FULL + (j & 1)));
