@@ -303,13 +303,19 @@ attend_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     // step j-3 (the producers do, before they refill the stage).
     if (lane == 0) {
       const bool is_s = warp == W_S;
-      bool ok = wait_on(bar(QD_FULL), 0) && wait_on(bar(META), 0);
-      const int n_steps = ok ? misc->n_steps : 0;
+      bool ok = wait_on(bar(QD_FULL), 0);
+      int n_steps = 0x7fffffff;            // known from step 1 on; step 0 (the own chunk) always exists
       constexpr uint32_t IDESC_S = ptx::idesc_bf16_f32(128, NKV, false, false);
       const uint64_t ad0 = ptx::smem_desc_sw128(sbase + (is_s ? OFF_Q : OFF_DO), 16, 1024);
       const uint64_t bd0 = ptx::smem_desc_sw128(sbase + (is_s ? OFF_K : OFF_V), 16, 1024);
       const uint32_t col0 = is_s ? 0u : COL_DP;
       for (int j = 0; j < n_steps && ok; ++j) {
+        if (j == 1) {
+          ok = wait_on(bar(META), 0);
+          if (!ok) break;
+          n_steps = misc->n_steps;
+          if (j >= n_steps) break;
+        }
         const int st = j % KST;
         ok = wait_on(bar((is_s ? K_FULL : V_FULL) + st), (uint32_t)(j / KST) & 1u);
         if (!ok) break;
@@ -328,11 +334,17 @@ attend_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
   } else if (warp == W_DQ) {
     // =========================== issuer of dQ += dS K ===========================
     if (lane == 0) {
-      bool ok = wait_on(bar(META), 0);
-      const int n_steps = ok ? misc->n_steps : 0;
+      bool ok = true;
+      int n_steps = 0x7fffffff;
       constexpr uint32_t IDESC_DQ = ptx::idesc_bf16_f32(128, HD, false, true);
       const uint64_t kmn0 = ptx::smem_desc_sw128(sbase + OFF_K, KV_TILE_BYTES / 2, 1024);   // K as MN-major B
       for (int j = 0; j < n_steps && ok; ++j) {
+        if (j == 1) {
+          ok = wait_on(bar(META), 0);
+          if (!ok) break;
+          n_steps = misc->n_steps;
+          if (j >= n_steps) break;
+        }
         const int st = j % KST;
         ok = wait_on(bar(DS_FULL + st), (uint32_t)(j / KST) & 1u);
         if (!ok) break;
@@ -359,9 +371,15 @@ attend_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     const long long srow = (((long long)b * dm.h_kv + r) * a.n_tiles + tile) * 128 + m;
     const float lse2 = row_ok ? a.lse2[srow] : 0.f;
     const float delta = row_ok ? a.delta[srow] : 0.f;
-    bool ok = wait_on(bar(META), 0);
-    const int n_steps = ok ? misc->n_steps : 0;
+    bool ok = true;
+    int n_steps = 0x7fffffff;              // known from step 1 on; step 0 (the own chunk) always exists
     for (int j = 0; j < n_steps && ok; ++j) {
+      if (j == 1) {
+        ok = wait_on(bar(META), 0);
+        if (!ok) break;
+        n_steps = misc->n_steps;
+        if (j >= n_steps) break;
+      }
       const int st = j % KST;
       const uint32_t ph = (uint32_t)(j / KST) & 1u;
       ok = wait_on(bar(V_FULL + st), ph);                  // bias / entry / kvbase of the step visible
