@@ -35,7 +35,12 @@ namespace {
 constexpr int NKV = 64;           // KV tokens per step
 constexpr int KST = 2, VST = 2;   // ring depths: stage = step parity, like the S/P buffers, so that the two
                                   // MMA completion barriers of a step also release its K and V stages
-constexpr int PF_THREADS = 224;   // 4 softmax warps, K producer, MMA issuer, V/bias producer
+constexpr int PF_THREADS = 256;   // 4 softmax warps, K producer, MMA issuer, V/bias producer and an idle warp: two whole
+                                  // warpgroups, because a warpgroup changes its register budget only when all four of
+                                  // its warps ask (a block of seven warps waits for the eighth for ever)
+// Registers per thread after the re-division (two blocks per SM start with 128 each): 128 * (200 - 128) taken by the
+// softmax warpgroup = 128 * (128 - 56) given up by the other one; the block's own pool is all that it can draw from.
+constexpr int PF_REGS_SERVICE = 56, PF_REGS_SOFTMAX = 200;
 constexpr uint32_t TMEM_COLS = 256;  // S0 [0,64), S1 [64,128), O [128,256)
 constexpr float RESCALE_LOG2 = 8.f;  // the running maximum is moved only when it grew by more than this
 
@@ -244,6 +249,10 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
   if (a.sb && *reinterpret_cast<volatile int*>(&a.sb->status) != 0) *abort_flag = 1;
   __syncthreads();
 
+  if (warp >= 4) {
+  // the register file of the block is re-divided between its two warpgroups: this one gives up what the softmax
+  // warpgroup takes (each side opens with its own instruction, so the allocator knows the budget of each)
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(PF_REGS_SERVICE));
   if (warp == 4 || warp == 6) {
     // =========================== producers ===========================
     // Two warps walk the same union list: warp 4 feeds the K ring (and loads Q), warp 6 feeds the V ring and
@@ -457,8 +466,10 @@ attend_prefill_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __gri
       }
     }
     __syncwarp();
+  }
   } else {
     // =========================== softmax / epilogue ===========================
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(PF_REGS_SOFTMAX));
     const int m = tid;                       // tile row = TMEM lane
     const int t = m / g_q, hh = m % g_q;     // token in tile, head in group
     const int i_row = i0 + t;
