@@ -107,7 +107,8 @@ namespace dq {
 // a step's exponentials take half as long.  One issuing thread per product (S, dP, dQ): a thread issues an MMA every
 // 60-80 clocks whatever its size, and 20 per step through one thread would be the kernel's pace.
 constexpr int W_KPROD = 8, W_S = 9, W_VPROD = 10, W_DP = 11, W_DQ = 12;
-constexpr int THREADS = 416;
+constexpr int THREADS = 512;              // 8 dS warps, 5 service warps, 3 idle: whole warpgroups, so that the registers can be re-divided
+constexpr int REGS_SERVICE = 56, REGS_SOFTMAX = 200;   // per thread after the re-division (128 each at launch)
 constexpr int KST = 3;                  // K / V ring and S / dP ring: stage = step mod 3, held until the step's dQ product is done
 constexpr uint32_t TMEM_COLS = 512;     // S [0,192) dP [192,384) dQ [384,512)
 constexpr uint32_t COL_DP = 192, COL_DQ = 384;
@@ -182,6 +183,8 @@ attend_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     ptx::tma_load_4d(dst + KV_TILE_BYTES / 2, tm, barrier, 64, r, kv0, b);
   };
 
+  if (warp >= 8) {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS_SERVICE));
   if (warp == W_KPROD || warp == W_VPROD) {
     // =========================== producers: the forward kernel's walk ===========================
     const bool do_k = (warp == W_KPROD), do_v = (warp == W_VPROD);
@@ -359,8 +362,10 @@ attend_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
       }
     }
     __syncwarp();
+  }
   } else {
     // =========================== dS / epilogue: thread = tile row, warpgroup = column half ===========================
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS_SOFTMAX));
     const int wg = warp >> 2;
     const int m = (warp & 3) * 32 + lane;
     const int t = m / g_q, hh = m % g_q;
@@ -473,7 +478,8 @@ namespace dkv {
 // are too many for one.  W_PROD loads the tiles, W_META looks up the per-token biases of each step; W_SD issues S,
 // W_DP dP, W_ACC dV^T, W_DK dK^T.
 constexpr int W_PROD = 8, W_SD = 9, W_ACC = 10, W_DP = 11, W_DK = 12, W_META = 13;
-constexpr int THREADS = 448;
+constexpr int THREADS = 512;              // 8 P / dS warps, 6 service warps, 2 idle: whole warpgroups
+constexpr int REGS_SERVICE = 80, REGS_SOFTMAX = 176;     // (the bias and loader warps need more than the issuers)
 constexpr uint32_t TMEM_COLS = 512;     // S0 S1 [0,128) dP0 dP1 [128,256) dV^T [256,320) dK^T [320,384)
 constexpr uint32_t COL_DP = 128, COL_DV = 256, COL_DK = 320;
 constexpr uint32_t PS_BYTES = 128 * NKV * 2;       // 16 KiB: P (or dS) of a step, 128 rows of 128 bytes
@@ -539,6 +545,8 @@ attend_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   if (a.sb && *reinterpret_cast<volatile int*>(&a.sb->status) != 0) *abort_flag = 1;
   __syncthreads();
 
+  if (warp >= 8) {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS_SERVICE));
   if (warp == W_PROD || warp == W_META) {
     // =========================== producers ===========================
     // Both warps enumerate the slice's steps in the same order: (i) the tiles of the slice's own chunk that can see it
@@ -759,8 +767,10 @@ attend_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       }
     }
     __syncwarp();
+  }
   } else {
     // =========================== P, dS: thread = tile row, warpgroup = half of the keys; epilogue: thread = d ===========================
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS_SOFTMAX));
     const int wg = warp >> 2;
     const int m = (warp & 3) * 32 + lane;
     const int t = m / g_q;
