@@ -109,6 +109,8 @@ namespace dq {
 constexpr int W_KPROD = 8, W_S = 9, W_VPROD = 10, W_DP = 11, W_DQ = 12;
 constexpr int THREADS = 512;              // 8 dS warps, 5 service warps, 3 idle: whole warpgroups, so that the registers can be re-divided
 constexpr int REGS_SERVICE = 56, REGS_SOFTMAX = 200;   // per thread after the re-division (128 each at launch)
+static_assert(THREADS == 512 && 256 * (REGS_SOFTMAX - 128) <= 256 * (128 - REGS_SERVICE),
+              "the dS warpgroups can only take what the service warpgroups released: a larger request never completes");
 constexpr int KST = 3;                  // K / V ring and S / dP ring: stage = step mod 3, held until the step's dQ product is done
 constexpr uint32_t TMEM_COLS = 512;     // S [0,192) dP [192,384) dQ [384,512)
 constexpr uint32_t COL_DP = 192, COL_DQ = 384;
@@ -480,6 +482,7 @@ namespace dkv {
 constexpr int W_PROD = 8, W_SD = 9, W_ACC = 10, W_DP = 11, W_DK = 12, W_META = 13;
 constexpr int THREADS = 512;              // 8 P / dS warps, 6 service warps, 2 idle: whole warpgroups
 constexpr int REGS_SERVICE = 80, REGS_SOFTMAX = 176;     // (the bias and loader warps need more than the issuers)
+static_assert(THREADS == 512 && 256 * (REGS_SOFTMAX - 128) <= 256 * (128 - REGS_SERVICE), "see the dQ kernel");
 constexpr uint32_t TMEM_COLS = 512;     // S0 S1 [0,128) dP0 dP1 [128,256) dV^T [256,320) dK^T [320,384)
 constexpr uint32_t COL_DP = 128, COL_DV = 256, COL_DK = 320;
 constexpr uint32_t PS_BYTES = 128 * NKV * 2;       // 16 KiB: P (or dS) of a step, 128 rows of 128 bytes

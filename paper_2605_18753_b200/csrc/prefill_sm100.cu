@@ -41,6 +41,8 @@ constexpr int PF_THREADS = 256;   // 4 softmax warps, K producer, MMA issuer, V/
 // Registers per thread after the re-division (two blocks per SM start with 128 each): 128 * (200 - 128) taken by the
 // softmax warpgroup = 128 * (128 - 56) given up by the other one; the block's own pool is all that it can draw from.
 constexpr int PF_REGS_SERVICE = 56, PF_REGS_SOFTMAX = 200;
+static_assert(PF_THREADS == 256 && 128 * (PF_REGS_SOFTMAX - 128) <= 128 * (128 - PF_REGS_SERVICE),
+              "the softmax warpgroup can only take what the service warpgroup released: a larger request never completes");
 constexpr uint32_t TMEM_COLS = 256;  // S0 [0,64), S1 [64,128), O [128,256)
 constexpr float RESCALE_LOG2 = 8.f;  // the running maximum is moved only when it grew by more than this
 
