@@ -8,7 +8,8 @@
 // a chunk gets bias -inf for that step (probability exactly 0), so every row still attends to its own
 // selection only.
 //
-// Warp roles (224 threads, two blocks per SM so one block's softmax overlaps the other's MMAs):
+// Warp roles (256 threads = two warpgroups, two blocks per SM so one block's softmax overlaps the other's MMAs; after
+// set-up the second warpgroup hands most of its registers to the first with setmaxnreg):
 //   warps 0-3  softmax: S (TMEM) -> registers, logit = S/sqrt(d) + bias, causal mask inside the own chunk,
 //              online softmax with a lazily moved row maximum, P (bf16) -> TMEM over the S columns, rescale of
 //              the O accumulator in TMEM when the maximum moved, final O / l -> global.
@@ -20,6 +21,7 @@
 //   warp 5     MMA issuer: S_{j+1} = Q K_{j+1}^T (M128 N64 K128) into one of two TMEM buffers, then O += P_j V_j
 //              (M128 N128 K64, P from TMEM); one tcgen05.commit per product, to the mbarrier that the softmax
 //              warps and the producer of the stage both listen to; owns the TMEM allocation.
+//   warp 7     idle (it completes the second warpgroup: registers are re-divided per whole warpgroup).
 // Every wait is bounded; a wait that runs out raises DASH_ERR_TIMEOUT in the status word and every role
 // leaves its loop, frees TMEM and returns.
 #include <cuda.h>
