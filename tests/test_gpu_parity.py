@@ -188,6 +188,43 @@ def test_attend_prefill_with_oracle_lists(kw):
     H.check_outputs(_gather_O(O, keys, w.h_q // w.h_kv), want, Q.dtype, "attend_prefill")
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_attend_prefill_running_maximum_moves_late(dtype):
+    """Keys whose magnitude rises from chunk to chunk in periods of five: along a row's walk (own chunk first, then its
+    routed chunks in ascending order) the row maximum grows by more than the lazy-rescale threshold several times, so
+    the accumulator is rescaled in tensor memory well after its first products.  Stage 2 alone on the oracle's lists,
+    every row compared."""
+    w = _wl(seq=900, h_q=8, h_kv=2, head_dim=128, block=64, gamma=0.1, dtype=dtype)
+    inp = synth.make_prefill_inputs(w, DEV)
+    Q, K, V = inp["Q"], inp["K"], inp["V"]
+    fac = 1.0 + 2.5 * ((torch.arange(w.seq, device=DEV) // w.block) % 5).float()
+    K = (K.float() * fac[None, :, None, None]).to(K.dtype)
+    O = torch.full_like(Q, float("nan"))
+    p = B.params_for_prefill(Q, K, V, O, block=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma)
+    ora = H.oracle_prefill_rows(Q, K, V, B=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma, rows=range(w.seq))
+    # the premise: on a sample of rows, count the steps at which the maximum grows by more than 2^8
+    Qn, Kn = H.to_np64(Q), H.to_np64(K)
+    g_q, c1 = w.h_q // w.h_kv, 1.4426950408889634 / np.sqrt(w.head_dim)
+    moves = []
+    for (b, r, i), (rt, _) in list(ora.items())[::9]:
+        q = Qn[b, i, r * g_q]
+        m = (Kn[b, (i // w.block) * w.block:i + 1, r] @ q).max() * c1
+        k = 0
+        for c, bias in zip(rt.support, rt.bias):
+            mm = (Kn[b, int(c) * w.block:(int(c) + 1) * w.block, r] @ q).max() * c1 + bias * 1.4426950408889634
+            if mm > m + 8.0:
+                m, k = mm, k + 1
+        moves.append(k)
+    assert np.mean(np.array(moves) >= 2) > 0.2, np.bincount(moves)
+    mask, count, idx, bias = H.routing_to_abi(ora, p, B.dash_attn_list_offset)
+    ws = B.alloc_workspace(p)
+    B.dash_attn_attend_prefill(p, Q, K, V, mask, bias, O, ws)
+    assert B.dash_attn_last_status(ws) == 0
+    keys = list(ora.keys())
+    want = np.stack([ora[k][1] for k in keys])
+    H.check_outputs(_gather_O(O, keys, g_q), want, Q.dtype, "attend_prefill, late maxima")
+
+
 @pytest.mark.parametrize("name,sigmas", [("tiny", (10.0, 1.0, 1e8)), ("tiny_g512", (10.0, 1e8))])
 def test_fwd_prefill_tiny_fp32(name, sigmas):
     for sigma in sigmas:
@@ -345,9 +382,12 @@ def test_fwd_prefill_8k_config_sampled_rows(seed):
 
 # ------------------------------------------------------------------ decode
 
-def _decode_case(w, kv_len, use_lists_from_oracle=False, local_blocks=0):
+def _decode_case(w, kv_len, use_lists_from_oracle=False, local_blocks=0, key_ramp=False):
     inp = synth.make_decode_inputs(w, DEV, kv_len=kv_len)
     Q, Kc, Vc, lens = inp["Q"], inp["K"], inp["V"], inp["kv_len"]
+    if key_ramp:      # key magnitudes rise from chunk to chunk in periods of five: partial maxima far apart
+        fac = 1.0 + 2.5 * ((torch.arange(Kc.shape[1], device=DEV) // w.block) % 5).float()
+        Kc = (Kc.float() * fac[None, :, None, None]).to(Kc.dtype)
     O = torch.full_like(Q, float("nan"))
     p = B.params_for_decode(Q, Kc, Vc, O, block=w.block, alpha=w.alpha, gamma=w.gamma, sigma=w.sigma,
                             local_blocks=local_blocks)
@@ -405,6 +445,16 @@ def test_decode_matches_oracle(kw, kv_len):
     w = _wl(**kw)
     _decode_case(w, kv_len, use_lists_from_oracle=True)
     _decode_case(w, kv_len)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_decode_partial_maxima_far_apart(dtype):
+    """Key magnitudes that rise from chunk to chunk: the running maximum of a split moves by more than the lazy-rescale
+    threshold several times and the splits of a (batch, KV head) end with maxima tens of units apart, which the merge
+    has to bring onto one scale."""
+    w = _wl(kind="decode", batch=2, seq=6000, h_q=8, h_kv=2, head_dim=128, block=64, gamma=0.1, dtype=dtype)
+    _decode_case(w, [6000, 3100], use_lists_from_oracle=True, key_ramp=True)
+    _decode_case(w, [6000, 3100], key_ramp=True)
 
 
 def test_decode_equals_last_prefill_row_on_gpu():
