@@ -568,7 +568,8 @@ def measure_backward(B, synth, w, dev, flush, iters=3, tensor_cores=False, fwd_s
 
 def all_config_measurements(B, synth, dev, peaks, flush, sel_tflop_8k=None) -> dict:
     """Every other configuration of the task beside the headline: the 64K prefill at two sparsities, the
-    (chunk size, alpha) sweep at 32K x batch 2, the 8K prefill with finer chunks, and the decode workload."""
+    (chunk size, alpha) sweep and a gamma sweep at 32K x batch 2, the 8K prefill with finer chunks, the decode workload
+    and the backward chains."""
     out = {}
 
     def guarded(name, fn):
@@ -591,6 +592,10 @@ def all_config_measurements(B, synth, dev, peaks, flush, sel_tflop_8k=None) -> d
                 sdpa.setdefault("ms", r.get("sdpa_dense_ms"))        # the dense baseline does not depend on B or alpha
                 return r
             guarded(key, run)
+    for gamma in (0.5, 2.0):                       # the routing temperature around its default (the gamma = 1 row is above)
+        guarded(f"sweep_32k_b64_a1.5_g{gamma}", lambda gamma=gamma: measure_prefill(
+            B, synth, synth.workload("sweep_32k", block=64, alpha=1.5, gamma=gamma), dev, peaks, iters=4, flush=flush,
+            sdpa_ms=sdpa.get("ms")))
     for name in ("prefill_8k_b32", "prefill_8k_b16"):
         guarded(name, lambda name=name: measure_prefill(B, synth, synth.workload(name), dev, peaks, iters=10, flush=flush,
                                                         with_sdpa=False))

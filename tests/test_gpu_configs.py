@@ -83,6 +83,13 @@ def test_alpha_sweep_32k(alpha, block):
     _prefill_sampled(w, _sample_rows(w.seq, w.block, 1024, 2), kv_heads=[3], batches=(1,))
 
 
+@pytest.mark.parametrize("gamma", [0.5, 2.0])
+def test_gamma_sweep_32k(gamma):
+    """The routing temperature around its default, at the sweep's size (the rows bench.py prints as ..._g0.5 / _g2.0)."""
+    w = synth.workload("sweep_32k", alpha=1.5, block=64, gamma=gamma)
+    _prefill_sampled(w, _sample_rows(w.seq, w.block, 1024, 3), kv_heads=[5], batches=(0,))
+
+
 def test_decode_128k():
     w = synth.workload("decode_128k")
     lens = [w.seq] * w.batch
