@@ -6,10 +6,10 @@
 //                         row reads (one warp per row, four rows in flight per warp) and write the scaled
 //                         chunk logits x = gamma(alpha-1) <q, kbar_c>/sqrt(d) of the g_q heads to a small
 //                         fp32 scratch (b * h_q * T_s floats, stays in L2);
-//   decode_route_kernel   one thread block of 32 warps per (batch, KV head) loads its g_q logit rows into shared
-//                         memory, finds tau per head (Newton from max - 1: monotone from below; eight
-//                         warps in all, a team of 8 / g_q per head), then forms the group weights, mask words, log w, mu and
-//                         the compact (chunk, bias) list.
+//   decode_route_kernel   one thread block of 16 warps per (batch, KV head) loads its g_q logit rows into shared
+//                         memory, finds tau per head (Newton; one warp per head with its share of the row in
+//                         registers, no barrier inside the iteration), then forms the group weights, mask words, log w,
+//                         mu and the compact (chunk, bias) list.
 // With a local window of L chunks the last L chunks before the own one are not scored; the routing kernel sets
 // their bits and appends them to the list with bias 0.
 #include <type_traits>
@@ -22,7 +22,7 @@ namespace {
 
 constexpr int SC_WARPS = 8;
 constexpr int SC_ROWS_PER_BLOCK = 256;   // summary rows one thread block scores
-constexpr int RT_THREADS = 1024;
+constexpr int RT_THREADS = 512;      // 128 registers per thread: a Newton warp keeps 64 logits per lane in registers
 constexpr int RT_MAX_NEWTON = 64, RT_MAX_NEWTON_GENERIC = 400;
 
 // Sum V values held by every lane across the warp with V-1+... shuffles (halving exchange): after the
@@ -121,7 +121,7 @@ decode_route_kernel(Dims dm, const float* __restrict__ xs, const int* __restrict
                     float* __restrict__ tau_out) {
   extern __shared__ __align__(16) float sm[];
   constexpr int NW = RT_THREADS / 32;
-  static_assert(NW == 32, "one lane per warp segment in the Newton phase");
+  static_assert(NW <= 32 && G <= NW, "a lane per warp in the reduction of the maxima; a warp per head in the iteration");
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int r = blockIdx.x, b = blockIdx.y;
   int L = kv_len ? kv_len[b] : dm.seq_kv;     // the caller's input, not a product of the chain: read it before the wait
@@ -134,9 +134,7 @@ decode_route_kernel(Dims dm, const float* __restrict__ xs, const int* __restrict
   const int stride = route_stride(n_vis);
   float* X = sm;                                 // [G][stride] all logits of the group
   float* taus = X + (size_t)G * stride;          // [G] (32 floats reserved)
-  float2* part = reinterpret_cast<float2*>(taus + 32);   // [RT_THREADS] per-lane (F, G) partials + [G] control words;
-                                                 // 8-byte aligned: the offset G * stride + 32 is a multiple of 32 floats
-  float* wsum = taus + 32 + 2 * RT_THREADS + 32; // per-word sum of log w   [W]
+  float* wsum = taus + 32;                       // per-word sum of log w   [W]
   int* wcnt = reinterpret_cast<int*>(wsum + dm.W);   // per-word popcount / exclusive prefix [W + 1]
   float* red = reinterpret_cast<float*>(wcnt + dm.W + 1);   // [NW][G] per-warp maxima
   const long long grp = (long long)b * dm.h_kv + r;
@@ -176,109 +174,94 @@ decode_route_kernel(Dims dm, const float* __restrict__ xs, const int* __restrict
   }
   __syncthreads();
 #pragma unroll
-  for (int g = 0; g < G; ++g) mx[g] = ord2f(__reduce_max_sync(0xffffffffu, f2ord(red[lane * G + g])));
+  for (int g = 0; g < G; ++g) mx[g] = ord2f(__reduce_max_sync(0xffffffffu, f2ord(lane < NW ? red[lane * G + g] : -INFINITY)));
 
-  // ---- tau per head (Newton from max - 1, monotone from below).  Shuffles retire one warp per clock per SM, so
-  // warp sums in all 32 warps would dominate a pass.  Instead the warps form g_q teams, one per head: every lane
-  // sums its few logits and stores the pair (F, G) unreduced; after the team's named barrier the team's first
-  // warp adds the columns, does the one warp sum, takes the Newton step and publishes (tau, done).
+  // ---- tau per head.  One warp per head, no barrier inside the iteration: a lane keeps its share of the row (up to
+  // 64 logits, i.e. rows of up to 2048 candidates; anything beyond is re-read from shared memory) in registers over all
+  // passes, a pass is the lane's sums, two warp sums and the step.  The start is the larger of the all-active root and
+  // the normal-tail estimate from the row's mean and variance (closed forms for alpha = 2 and 1.5, as in the prefill
+  // kernel); either side of the root is a valid start: from the left the iterates rise monotonically, from the right
+  // one step lands on the left.
   const int e_int = dm.e_int;
   const float e = dm.e;
-  {
-    constexpr int NWH = G < 8 ? 8 / G : 1;        // warps per team: eight Newton warps in all (named barriers 1..4)
-    constexpr int TEAM = NWH * 32;
-    const int g = min(warp / NWH, G - 1), sw = warp % NWH;
-    const bool in_team = warp < G * NWH;
-    float2* pt = part + (size_t)g * TEAM;         // this team's [TEAM] lane partials
-    float2* ctrl = part + (size_t)G * TEAM + g;   // (tau, continue?) of this team
-    const float* x = X + (size_t)g * stride;
+  if (warp < G) {
+    const int g = warp;
     float tau = 0.f;
+    if (n_cand > 0) {
+      const float* x = X + (size_t)g * stride;
+      float mxg = 0.f;
 #pragma unroll
-    for (int k = 0; k < G; ++k) if (k == g) tau = mx[k] - 1.f;
-    // the exponent is a compile-time constant inside the loop (alpha = 2, 1.5, 1.25 -> 1, 2, 4; 0 = powf)
-    auto newton = [&](auto ei_tag) {
-      constexpr int EI = decltype(ei_tag)::value;
-      const int max_it = EI ? RT_MAX_NEWTON : RT_MAX_NEWTON_GENERIC;
-      // a lane's first eight logits stay in registers over the passes (all of them up to 8 * TEAM candidates)
-      float xr[8];
+      for (int k = 0; k < G; ++k) if (k == g) mxg = mx[k];
+      constexpr int RPL = 64;                       // logits a lane holds
+      float xr[RPL];
 #pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const int c = sw * 32 + lane + u * TEAM;
+      for (int u = 0; u < RPL; ++u) {
+        const int c = lane + 32 * u;
         xr[u] = c < n_cand ? x[c] : -INFINITY;
       }
-      for (int it = 0; it < max_it; ++it) {
-        float F[8], Gs[8];
+      // moments about the maximum
+      float s1 = 0.f, s2 = 0.f;
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          const float m = fmaxf(xr[u] - tau, 0.f);
-          F[u] = pow_e(m, EI, e);
-          Gs[u] = pow_em1(m, EI, e);
-        }
-        int c = sw * 32 + lane + 8 * TEAM;
-        for (; c + 7 * TEAM < n_cand; c += 8 * TEAM) {
-#pragma unroll
-          for (int u = 0; u < 8; ++u) {
-            const float m = fmaxf(x[c + u * TEAM] - tau, 0.f);
-            F[u] += pow_e(m, EI, e);
-            Gs[u] += pow_em1(m, EI, e);
-          }
-        }
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          if (c < n_cand) {
-            const float m = fmaxf(x[c] - tau, 0.f);
-            F[u] += pow_e(m, EI, e);
-            Gs[u] += pow_em1(m, EI, e);
-          }
-          c += TEAM;
-        }
-        float2 t = make_float2(((F[0] + F[1]) + (F[2] + F[3])) + ((F[4] + F[5]) + (F[6] + F[7])),
-                               ((Gs[0] + Gs[1]) + (Gs[2] + Gs[3])) + ((Gs[4] + Gs[5]) + (Gs[6] + Gs[7])));
-        bool go = true;
-        if constexpr (NWH > 1) {
-          pt[sw * 32 + lane] = t;
-          asm volatile("bar.sync %0, %1;" ::"r"(1 + g), "r"(TEAM) : "memory");
-          if (sw == 0) {
-#pragma unroll
-            for (int k = 1; k < NWH; ++k) {
-              const float2 o = pt[k * 32 + lane];
-              t.x += o.x;
-              t.y += o.y;
-            }
-          }
-        }
-        if (NWH == 1 || sw == 0) {
-          t.x = warp_sum(t.x);
-          t.y = warp_sum(t.y);
-          go = t.x - 1.f > NEWTON_F_TOL;
-          if (go) {
-            const float nt = tau + newton_delta(t.x, t.y, EI, e);
-            go = nt > tau;
-            if (go) tau = nt;
-          }
-          if (NWH > 1 && lane == 0) *ctrl = make_float2(tau, go ? 1.f : 0.f);
-        }
-        if constexpr (NWH > 1) {
-          // the partials are rewritten only after this barrier, the control word only after the next pass's first
-          asm volatile("bar.sync %0, %1;" ::"r"(1 + g), "r"(TEAM) : "memory");
-          const float2 cw = *ctrl;
-          tau = cw.x;
-          go = cw.y != 0.f;
-        }
-        if (!go) break;
+      for (int u = 0; u < RPL; ++u) {
+        const float y = xr[u] > -INFINITY ? xr[u] - mxg : 0.f;
+        s1 += y;
+        s2 = fmaf(y, y, s2);
       }
-    };
-    if (n_cand > 0 && in_team) {
+      for (int c = lane + 32 * RPL; c < n_cand; c += 32) {
+        const float y = x[c] - mxg;
+        s1 += y;
+        s2 = fmaf(y, y, s2);
+      }
+      s1 = warp_sum(s1);
+      s2 = warp_sum(s2);
+      {
+        const float n = (float)n_cand;
+        float t = -1.f;
+        if (e_int == 1) {
+          t = (s1 - 1.f) / n;
+        } else if (e_int == 2) {
+          const float mean = s1 / n, ss = s2 - s1 * mean;
+          if (ss < 1.f) t = mean - sqrtf((1.f - ss) / n);
+          if (n_cand >= 8 && ss > 0.f) {
+            const float L = -__logf(fminf(fmaxf(ss, 0.3334f), 1e7f));
+            const float z = fmaf(fmaf(fmaf(fmaf(-8.93074e-05f, L, -0.0037117f), L, -0.0612527f), L, -0.717421f), L, -0.499476f);
+            t = fmaxf(t, fmaf(z, sqrtf(ss / n), mean));
+          }
+        }
+        tau = mxg + fminf(fmaxf(t, -1.f), -1e-6f);
+      }
+      auto newton = [&](auto ei_tag) {
+        constexpr int EI = decltype(ei_tag)::value;
+        const int max_it = EI ? RT_MAX_NEWTON : RT_MAX_NEWTON_GENERIC;
+        for (int it = 0; it < max_it; ++it) {
+          float F[4] = {0.f, 0.f, 0.f, 0.f}, Gs[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+          for (int u = 0; u < RPL; ++u) {
+            const float m = fmaxf(xr[u] - tau, 0.f);
+            F[u & 3] += pow_e(m, EI, e);
+            Gs[u & 3] += pow_em1(m, EI, e);
+          }
+          for (int c = lane + 32 * RPL; c < n_cand; c += 32) {
+            const float m = fmaxf(x[c] - tau, 0.f);
+            F[0] += pow_e(m, EI, e);
+            Gs[0] += pow_em1(m, EI, e);
+          }
+          const float f = warp_sum((F[0] + F[1]) + (F[2] + F[3]));
+          const float gs = warp_sum((Gs[0] + Gs[1]) + (Gs[2] + Gs[3]));
+          if (fabsf(f - 1.f) <= NEWTON_F_TOL || !(gs > 0.f)) break;
+          const float nt = tau + newton_delta(f, gs, EI, e);
+          if (nt == tau) break;
+          tau = nt;
+        }
+      };
       switch (e_int) {
         case 1: newton(std::integral_constant<int, 1>{}); break;
         case 2: newton(std::integral_constant<int, 2>{}); break;
         case 4: newton(std::integral_constant<int, 4>{}); break;
         default: newton(std::integral_constant<int, 0>{}); break;
       }
-    } else {
-      tau = 0.f;
     }
-    if (in_team && sw == 0 && lane == 0) {
+    if (lane == 0) {
       taus[g] = tau;
       if (tau_out) tau_out[(long long)b * dm.h_q + r * G + g] = tau;
     }
@@ -368,8 +351,8 @@ size_t select_decode_scratch_bytes(const Dims& dm) {
 }
 
 static size_t route_smem(const Dims& dm) {
-  // logits, taus, per-lane (F, G) partials and control words, per-word sums and counts, per-warp maxima
-  return ((size_t)dm.g_q * route_stride(dm.T_s) + 32 + 2 * RT_THREADS + 32 + dm.W + dm.W + 1 + 8 +
+  // logits, taus, per-word sums and counts, per-warp maxima
+  return ((size_t)dm.g_q * route_stride(dm.T_s) + 32 + dm.W + dm.W + 1 + 8 +
           (size_t)(RT_THREADS / 32) * dm.g_q) * sizeof(float);
 }
 
