@@ -23,6 +23,7 @@ namespace {
 constexpr int SC_WARPS = 8;
 constexpr int SC_ROWS_PER_BLOCK = 256;   // summary rows one thread block scores
 constexpr int RT_THREADS = 512;      // 128 registers per thread: a Newton warp keeps 64 logits per lane in registers
+constexpr int RT_LOADS = 4;           // logits per head a thread requests per sweep (2048 candidates: one sweep)
 constexpr int RT_MAX_NEWTON = 64, RT_MAX_NEWTON_GENERIC = 400;
 
 // Sum V values held by every lane across the warp with V-1+... shuffles (halving exchange): after the
@@ -145,19 +146,19 @@ decode_route_kernel(Dims dm, const float* __restrict__ xs, const int* __restrict
 #pragma unroll
   for (int g = 0; g < G; ++g) mx[g] = -INFINITY;
   // all of a thread's loads of one sweep are issued before the first is used (one L2 round trip per sweep)
-  for (int c0 = 0; c0 < n_cand; c0 += 2 * RT_THREADS) {
-    float v[G][2];
+  for (int c0 = 0; c0 < n_cand; c0 += RT_LOADS * RT_THREADS) {
+    float v[G][RT_LOADS];
 #pragma unroll
     for (int g = 0; g < G; ++g)
 #pragma unroll
-      for (int u = 0; u < 2; ++u) {
+      for (int u = 0; u < RT_LOADS; ++u) {
         const int c = c0 + u * RT_THREADS + tid;
         v[g][u] = c < n_cand ? __ldcg(xg + (long long)g * dm.T_s + c) : -INFINITY;
       }
 #pragma unroll
     for (int g = 0; g < G; ++g)
 #pragma unroll
-      for (int u = 0; u < 2; ++u) {
+      for (int u = 0; u < RT_LOADS; ++u) {
         const int c = c0 + u * RT_THREADS + tid;
         if (c < n_cand) X[(size_t)g * stride + c] = v[g][u];
         mx[g] = fmaxf(mx[g], v[g][u]);
