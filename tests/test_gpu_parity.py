@@ -440,6 +440,8 @@ def _decode_case(w, kv_len, use_lists_from_oracle=False, local_blocks=0, key_ram
     (dict(kind="decode", batch=3, seq=4000, h_q=16, h_kv=2, head_dim=64, block=64), [4000, 1, 2049]),   # head_dim 64: stacked sub-blocks
     (dict(kind="decode", batch=2, seq=3000, h_q=8, h_kv=2, head_dim=64, block=128, alpha=2.0), [2999, 130]),
     (dict(kind="decode", batch=2, seq=2500, h_q=2, h_kv=1, head_dim=64, block=32), [2500, 1777]),
+    # more than 2048 candidates: the routing warp keeps 64 logits per lane and re-reads the rest from shared memory
+    (dict(kind="decode", batch=2, seq=40000, h_q=4, h_kv=1, head_dim=64, block=16), [40000, 33000]),
 ])
 def test_decode_matches_oracle(kw, kv_len):
     w = _wl(**kw)
